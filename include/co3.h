@@ -1,0 +1,174 @@
+/*
+ * co3.h -- C ABI of the B200 (sm_100a) CO3 gradient pipeline.
+ *
+ * CO3 ("convert, compress, correct") is the per-iteration gradient processing of Algorithm 1 of
+ * the paper: at every user u, ghat = Q_fp(g + gamma m) (line 8), b = h_Hf(ghat) (line 9),
+ * m <- gamma m + g - ghat (line 10); at the parameter server, decode every user's stream
+ * (line 13) and average (line 14, Eq. "aggregate").  Q_fp is the conversion to a float with 1
+ * sign, `exp_bits` exponent and `mant_bits` mantissa bits and an exponent bias b_t chosen per
+ * layer from a generalized-normal fit (Sec. III (i), Eq. "exp bias", Eq. "approximate"); h_Hf is
+ * an element-wise Huffman code, one per layer and shared by all users, designed from the same
+ * fitted model (Sec. III (ii)).
+ *
+ * Conventions
+ *  - Every pointer marked "device" is CUDA device memory owned by the caller; "host" is host
+ *    memory.  The plan owns its scratch, tables and status word; no call after co3_plan_create
+ *    allocates memory.
+ *  - co3_encode / co3_decode_aggregate only enqueue work on `cuda_stream` (a cudaStream_t cast
+ *    to void*, NULL = default stream) and return without synchronising.  Calls on one plan must
+ *    be issued on one stream (or be ordered by the caller).
+ *  - Return value: 0, or a negative CO3_E* code for errors detected on the host.  Conditions
+ *    detected on the device (non-finite inputs, payload capacity, corrupt stream) set sticky
+ *    flags read with co3_status.  Nothing throws, prints or exits.
+ *  - Row layout: user u's vectors start at element u*ld of `grad` / `residual`; ld >= d,
+ *    ld % 4 == 0 and the base pointers are 16-byte aligned.  A "segment" is a layer: a range
+ *    [seg_offsets[l], seg_offsets[l+1]) of every user's row with its own bias and code.
+ *
+ * Container (what co3_encode writes and co3_decode_aggregate reads).  A row is cut into chunks
+ * at every multiple of 4096 elements and at every segment boundary, and each chunk into
+ * sub-chunks at every multiple of 128 elements.  Chunk c of user u is the 32-bit words
+ * [chunk_off[u][c], chunk_off[u][c+1]) of bitstream row u; its word count is its bit count
+ * rounded up to a multiple of 128 bits.  Codewords are packed without gaps, stream bit p is bit
+ * (p & 31) of word (p >> 5), a codeword's root bit first, pad bits zero.  sub_bits[u][k] is the
+ * bit length of sub-chunk k (numbered along the row).  The per-segment header (bias and the two
+ * indices that name the code model) is shared by all users.
+ */
+#ifndef CO3_H
+#define CO3_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CO3_OK 0
+#define CO3_EINVAL (-1)     /* bad argument or unsupported configuration            */
+#define CO3_ENOMEM (-2)     /* device or host allocation failed in co3_plan_create  */
+#define CO3_ECUDA (-3)      /* a CUDA runtime call failed                            */
+#define CO3_ECAPACITY (-4)  /* a user's payload does not fit cap_words               */
+#define CO3_ECORRUPT (-5)   /* a stream did not decode to its recorded lengths       */
+#define CO3_ENONFINITE (-6) /* NaN/Inf met in g + gamma m (coded as 0, memory reset) */
+
+#define CO3_FLAG_CAPACITY 1u
+#define CO3_FLAG_CORRUPT 2u
+#define CO3_FLAG_NONFINITE 4u
+
+#define CO3_BIAS_CURRENT 0 /* b_t from the moments of g_t + gamma m_{t-1} itself: one extra read pass */
+#define CO3_BIAS_LAGGED 1  /* that pass at t = 0 only; b_t (t >= 1) from the fit of iteration t-1      */
+
+typedef struct co3_plan co3_plan; /* opaque, library-owned */
+
+/* Sec. III (i): one sign bit is implied.  Supported: 1 <= exp_bits <= 4, 1 <= mant_bits,
+ * exp_bits + mant_bits <= 7; (4,3), (3,2) and (1,2) are the 8-, 6- and 4-bit formats. */
+typedef struct {
+    int32_t exp_bits, mant_bits;
+} co3_format;
+
+/* What the parameter server needs per segment to rebuild grid and code: the integer exponent
+ * bias b (grid value = +-K(j) * 2^(b + 1 - bias_F - mant_bits)), and the fitted GenNorm shape
+ * and scale on a 1/8-octave grid: beta_q = 2^(ibeta/8), alpha_q = 2^(b + ir/8). */
+typedef struct {
+    int8_t bias;
+    int8_t ibeta;
+    int16_t ir;
+} co3_seg_header;
+
+typedef struct {
+    int64_t d;                  /* elements per user                                              */
+    int64_t ld;                 /* row pitch of grad/residual in elements, >= d, multiple of 4    */
+    int32_t n_users;            /* U; n_users * K_max < 2^24 (K_max: largest integer magnitude)    */
+    co3_format fmt;
+    int32_t n_segments;         /* S >= 1                                                          */
+    const int64_t* seg_offsets; /* host, S+1 non-decreasing entries, [0] = 0, [S] = d; NULL: S = 1 */
+    float gamma;                /* memory decay of Algorithm 1 line 8; 0: no feedback, 1: plain EF */
+    int32_t bias_mode;          /* CO3_BIAS_CURRENT or CO3_BIAS_LAGGED                             */
+    int64_t cap_words;          /* row pitch of `bitstream` in 32-bit words, multiple of 4         */
+} co3_config;
+
+/* Algorithm 1 line 2 and Table I: fixes d, U, the format, the layers, gamma.  Validates the
+ * configuration, computes the static chunk partition, builds the GenNorm model-weight table on
+ * the host and allocates all device scratch on the current device.  The iteration counter
+ * starts at 0 (memory m_0 = 0 is the caller's zero-filled `residual`). */
+int co3_plan_create(co3_plan** out, const co3_config* cfg);
+void co3_plan_destroy(co3_plan* plan);
+
+/* Sizes of the side-information arrays and the worst-case payload (16 bits per symbol plus
+ * chunk padding) in words per user.  Any pointer may be NULL. */
+int co3_sizes(const co3_plan* plan, int64_t* n_chunks, int64_t* n_sub, int64_t* worst_case_words);
+
+/* Algorithm 1 lines 8-10 for all users (one iteration t, then t <- t + 1):
+ *   grad      device, const, [U][ld] fp32   g_t^(u)
+ *   residual  device, in/out, [U][ld] fp32  m_{t-1}^(u) -> m_t^(u)
+ *   bitstream device, out, [U][cap_words]   h_Hf(ghat_t^(u)), container as described above
+ *   sub_bits  device, out, [U][n_sub] u16
+ *   chunk_off device, out, [U][n_chunks+1] u32, in words
+ *   user_bits device, out, [U] u64          r_t^(u): code bits of user u
+ *   hdr       device, out, [n_segments]
+ * If a user's payload would exceed cap_words, CO3_FLAG_CAPACITY is raised and that user's
+ * bitstream row is left untouched; chunk_off, sub_bits and user_bits are still written.
+ * Non-finite g + gamma m: counted, coded as +0, memory reset to 0, CO3_FLAG_NONFINITE raised. */
+int co3_encode(co3_plan* plan, const float* grad, float* residual, uint32_t* bitstream,
+               uint16_t* sub_bits, uint32_t* chunk_off, uint64_t* user_bits, co3_seg_header* hdr,
+               void* cuda_stream);
+
+/* Algorithm 1 lines 13-14 without the model update: decode all U streams and write
+ * avg_grad[i] = (1/U) sum_u ghat^(u)[i] (Eq. "aggregate"), device [d] fp32.  Depends only on
+ * its arguments and the plan's static configuration, never on encoder scratch.  The integer
+ * magnitudes are summed exactly and scaled once, so the result does not depend on the order of
+ * the users.  A stream that does not decode to its recorded lengths raises CO3_FLAG_CORRUPT;
+ * no out-of-bounds access is made for any input bytes. */
+int co3_decode_aggregate(co3_plan* plan, const uint32_t* bitstream, const uint16_t* sub_bits,
+                         const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
+                         void* cuda_stream);
+
+/* One whole iteration from host memory (what a training loop that keeps gradients on the host
+ * would call): copies h_grad (host, [U][ld], pinned for full speed) to d_grad, runs co3_encode
+ * and co3_decode_aggregate with the given device buffers, and copies the average back to h_avg
+ * (host, [d]).  Everything is enqueued on cuda_stream; the caller synchronises. */
+int co3_iteration_host(co3_plan* plan, const float* h_grad, float* d_grad, float* d_residual,
+                       uint32_t* d_bitstream, uint16_t* d_sub_bits, uint32_t* d_chunk_off,
+                       uint64_t* d_user_bits, co3_seg_header* d_hdr, float* d_avg, float* h_avg,
+                       void* cuda_stream);
+
+/* Synchronises the stream last used by the plan and reports the sticky flags and the running
+ * count of non-finite inputs.  clear != 0 resets both.  Returns CO3_OK or CO3_ECUDA. */
+int co3_status(co3_plan* plan, uint32_t* flags, uint64_t* nonfinite_count, int32_t clear);
+
+/* Fit of the last encoded iteration for one segment (synchronises): GenNorm shape and scale by
+ * moment matching, and the pooled moments N, sum|a|, sum a^2 of a = g + gamma m. */
+int co3_get_fit(co3_plan* plan, int32_t seg, double* beta, double* alpha, double* N, double* S1,
+                double* S2);
+
+/* Checkpoint/resume of what the method carries between iterations besides the caller's
+ * residual: the iteration counter and the next bias per segment (host int32 [n_segments]). */
+int co3_state_export(co3_plan* plan, int64_t* iteration, int32_t* next_bias);
+int co3_state_import(co3_plan* plan, int64_t iteration, const int32_t* next_bias);
+
+/* Inspection hooks (synchronise; used by the parity tests).
+ * symbols: device out [U][d] u8, the converted symbols of the last iteration
+ *          (sign << (E+M) | exponent << M | mantissa).
+ * hist:    host out [n_segments][2^(1+E+M)] u64, symbol counts pooled over users.
+ * code:    host out, lengths [n_segments][2^B] u8 and codewords [n_segments][2^B] u32 (root bit
+ *          = most significant of `length` bits) of the last encode. */
+int co3_debug_symbols(co3_plan* plan, uint8_t* symbols, void* cuda_stream);
+int co3_debug_hist(co3_plan* plan, uint64_t* hist);
+int co3_debug_code(co3_plan* plan, uint8_t* lengths, uint32_t* codewords);
+
+/* Host only, no GPU needed: integer model weights of the quantised GenNorm source for header
+ * indices (ibeta in [-14, 8], ir in [-96, 31]), one per symbol byte, 2^(1+E+M) entries.  The
+ * Huffman code of a segment is built from exactly these numbers (Sec. III (ii)). */
+int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint32_t* weights);
+
+/* Host only: the static partition for (d, segments), as co3_plan_create computes it.  Arrays
+ * are host, sized by a first call with NULL arrays that returns the chunk count. */
+int64_t co3_partition(int64_t d, int32_t n_segments, const int64_t* seg_offsets,
+                      int32_t* chunk_seg, int64_t* chunk_start, int64_t* chunk_end,
+                      int64_t* sub_base, int64_t* n_sub);
+
+const char* co3_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CO3_H */

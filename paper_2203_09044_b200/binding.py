@@ -1,0 +1,265 @@
+"""ctypes binding of the CO3 CUDA library (include/co3.h): argument marshalling only.
+
+Every step of the pipeline runs in the library's CUDA kernels.  There is no CPU fallback: if the
+library has not been built (python -m paper_2203_09044_b200.build, or __graft_entry__.build())
+loading raises.  torch is used for device memory and streams only.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libco3.so")
+
+OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ECORRUPT, ENONFINITE = 0, -1, -2, -3, -4, -5, -6
+FLAG_CAPACITY, FLAG_CORRUPT, FLAG_NONFINITE = 1, 2, 4
+BIAS_CURRENT, BIAS_LAGGED = 0, 1
+
+EXPORTS = [
+    "co3_plan_create", "co3_plan_destroy", "co3_sizes", "co3_encode", "co3_decode_aggregate",
+    "co3_iteration_host", "co3_status", "co3_get_fit", "co3_state_export", "co3_state_import",
+    "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
+    "co3_strerror",
+]
+
+
+class Format(C.Structure):
+    _fields_ = [("exp_bits", C.c_int32), ("mant_bits", C.c_int32)]
+
+
+class Config(C.Structure):
+    _fields_ = [("d", C.c_int64), ("ld", C.c_int64), ("n_users", C.c_int32), ("fmt", Format),
+                ("n_segments", C.c_int32), ("seg_offsets", C.POINTER(C.c_int64)),
+                ("gamma", C.c_float), ("bias_mode", C.c_int32), ("cap_words", C.c_int64)]
+
+
+HDR_DTYPE = np.dtype([("bias", np.int8), ("ibeta", np.int8), ("ir", np.int16)])
+
+_lib = None
+
+
+class Co3Error(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {lib().co3_strerror(code).decode()} ({code})")
+
+
+def lib():
+    """Load csrc/libco3.so; raises if it is missing (there is no other implementation)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not built: run `python -m paper_2203_09044_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    vp, i64p = C.c_void_p, C.POINTER(C.c_int64)
+    L.co3_plan_create.restype = C.c_int
+    L.co3_plan_create.argtypes = [C.POINTER(vp), C.POINTER(Config)]
+    L.co3_plan_destroy.restype = None
+    L.co3_plan_destroy.argtypes = [vp]
+    L.co3_sizes.restype = C.c_int
+    L.co3_sizes.argtypes = [vp, i64p, i64p, i64p]
+    L.co3_encode.restype = C.c_int
+    L.co3_encode.argtypes = [vp] * 9
+    L.co3_decode_aggregate.restype = C.c_int
+    L.co3_decode_aggregate.argtypes = [vp] * 7
+    L.co3_iteration_host.restype = C.c_int
+    L.co3_iteration_host.argtypes = [vp] * 12
+    L.co3_status.restype = C.c_int
+    L.co3_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_uint64), C.c_int32]
+    L.co3_get_fit.restype = C.c_int
+    L.co3_get_fit.argtypes = [vp, C.c_int32] + [C.POINTER(C.c_double)] * 5
+    L.co3_state_export.restype = C.c_int
+    L.co3_state_export.argtypes = [vp, i64p, vp]
+    L.co3_state_import.restype = C.c_int
+    L.co3_state_import.argtypes = [vp, C.c_int64, vp]
+    L.co3_debug_symbols.restype = C.c_int
+    L.co3_debug_symbols.argtypes = [vp, vp, vp]
+    L.co3_debug_hist.restype = C.c_int
+    L.co3_debug_hist.argtypes = [vp, vp]
+    L.co3_debug_code.restype = C.c_int
+    L.co3_debug_code.argtypes = [vp, vp, vp]
+    L.co3_model_weights.restype = C.c_int
+    L.co3_model_weights.argtypes = [Format, C.c_int32, C.c_int32, vp]
+    L.co3_partition.restype = C.c_int64
+    L.co3_partition.argtypes = [C.c_int64, C.c_int32, vp, vp, vp, vp, vp, i64p]
+    L.co3_strerror.restype = C.c_char_p
+    L.co3_strerror.argtypes = [C.c_int]
+    _lib = L
+    return L
+
+
+def model_weights(exp_bits, mant_bits, ibeta, ir):
+    """Host only: integer model weights per symbol byte for header indices (ibeta, ir)."""
+    w = np.zeros(1 << (1 + exp_bits + mant_bits), np.uint32)
+    rc = lib().co3_model_weights(Format(exp_bits, mant_bits), ibeta, ir, w.ctypes.data)
+    if rc != OK:
+        raise Co3Error(rc, "co3_model_weights")
+    return w
+
+
+def partition(d, seg_offsets):
+    """Host only: (chunk_seg, chunk_start, chunk_end, sub_base, n_sub) of the static partition."""
+    off = np.ascontiguousarray(seg_offsets, np.int64)
+    ns = C.c_int64()
+    nc = lib().co3_partition(d, len(off) - 1, off.ctypes.data, None, None, None, None, C.byref(ns))
+    if nc < 0:
+        raise Co3Error(int(nc), "co3_partition")
+    seg = np.zeros(nc, np.int32)
+    st, en, sb = (np.zeros(nc, np.int64) for _ in range(3))
+    lib().co3_partition(d, len(off) - 1, off.ctypes.data, seg.ctypes.data, st.ctypes.data,
+                        en.ctypes.data, sb.ctypes.data, C.byref(ns))
+    return seg, st, en, sb, int(ns.value)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class Plan:
+    """co3_plan plus the torch buffers of one pipeline instance on the current CUDA device."""
+
+    def __init__(self, d, n_users, exp_bits, mant_bits, seg_offsets=None, gamma=0.9,
+                 bias_mode=BIAS_LAGGED, cap_words=None, ld=None):
+        import torch
+        self.torch = torch
+        L = lib()
+        self.d, self.U, self.E, self.M = int(d), int(n_users), int(exp_bits), int(mant_bits)
+        self.ld = int(ld) if ld is not None else (self.d + 3) // 4 * 4
+        self.nsym = 1 << (1 + self.E + self.M)
+        off = np.ascontiguousarray([0, d] if seg_offsets is None else seg_offsets, np.int64)
+        self.S = len(off) - 1
+        self._off = off
+        # worst case needs the partition; compute it on the host first
+        _, st, en, _, _ = partition(self.d, off)
+        worst = int(sum(4 * ((16 * int(e - s) + 127) // 128) for s, e in zip(st, en)))
+        self.cap_words = int(cap_words) if cap_words is not None else worst
+        cfg = Config(self.d, self.ld, self.U, Format(self.E, self.M), self.S,
+                     off.ctypes.data_as(C.POINTER(C.c_int64)), float(gamma), int(bias_mode),
+                     self.cap_words)
+        h = C.c_void_p()
+        rc = L.co3_plan_create(C.byref(h), C.byref(cfg))
+        if rc != OK:
+            raise Co3Error(rc, "co3_plan_create")
+        self.handle = h
+        nc, ns, wc = C.c_int64(), C.c_int64(), C.c_int64()
+        L.co3_sizes(h, C.byref(nc), C.byref(ns), C.byref(wc))
+        self.n_chunks, self.n_sub, self.worst_case_words = nc.value, ns.value, wc.value
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().co3_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- buffers ---------------------------------------------------------------------------
+    def alloc_outputs(self, device="cuda"):
+        t = self.torch
+        return dict(
+            bitstream=t.zeros((self.U, self.cap_words), dtype=t.int32, device=device),
+            sub_bits=t.zeros((self.U, max(self.n_sub, 1)), dtype=t.int16, device=device),
+            chunk_off=t.zeros((self.U, self.n_chunks + 1), dtype=t.int32, device=device),
+            user_bits=t.zeros((self.U,), dtype=t.int64, device=device),
+            hdr=t.zeros((self.S,), dtype=t.int32, device=device),
+            avg=t.zeros((self.d,), dtype=t.float32, device=device),
+        )
+
+    def _stream(self, stream):
+        s = self.torch.cuda.current_stream() if stream is None else stream
+        return C.c_void_p(s.cuda_stream)
+
+    # ---- the C-ABI calls -------------------------------------------------------------------
+    def encode(self, grad, residual, out, stream=None):
+        rc = lib().co3_encode(self.handle, _ptr(grad), _ptr(residual), _ptr(out["bitstream"]),
+                              _ptr(out["sub_bits"]), _ptr(out["chunk_off"]), _ptr(out["user_bits"]),
+                              _ptr(out["hdr"]), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_encode")
+
+    def decode_aggregate(self, out, avg=None, stream=None):
+        avg = out["avg"] if avg is None else avg
+        rc = lib().co3_decode_aggregate(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
+                                        _ptr(out["chunk_off"]), _ptr(out["hdr"]), _ptr(avg),
+                                        self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_decode_aggregate")
+        return avg
+
+    def iteration_host(self, h_grad, d_grad, residual, out, h_avg, stream=None):
+        rc = lib().co3_iteration_host(self.handle, _ptr(h_grad), _ptr(d_grad), _ptr(residual),
+                                      _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
+                                      _ptr(out["chunk_off"]), _ptr(out["user_bits"]), _ptr(out["hdr"]),
+                                      _ptr(out["avg"]), _ptr(h_avg), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_iteration_host")
+
+    def status(self, clear=False):
+        f, n = C.c_uint32(), C.c_uint64()
+        rc = lib().co3_status(self.handle, C.byref(f), C.byref(n), int(clear))
+        if rc != OK:
+            raise Co3Error(rc, "co3_status")
+        return int(f.value), int(n.value)
+
+    def get_fit(self, seg):
+        v = [C.c_double() for _ in range(5)]
+        rc = lib().co3_get_fit(self.handle, seg, *[C.byref(x) for x in v])
+        if rc != OK:
+            raise Co3Error(rc, "co3_get_fit")
+        return tuple(x.value for x in v)        # beta, alpha, N, S1, S2
+
+    def state_export(self):
+        it = C.c_int64()
+        nb = np.zeros(self.S, np.int32)
+        rc = lib().co3_state_export(self.handle, C.byref(it), nb.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_state_export")
+        return int(it.value), nb
+
+    def state_import(self, iteration, next_bias):
+        nb = np.ascontiguousarray(next_bias, np.int32)
+        rc = lib().co3_state_import(self.handle, int(iteration), nb.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_state_import")
+
+    def debug_symbols(self, stream=None):
+        t = self.torch
+        sym = t.zeros((self.U, self.d), dtype=t.uint8, device="cuda")
+        rc = lib().co3_debug_symbols(self.handle, _ptr(sym), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_debug_symbols")
+        return sym
+
+    def debug_hist(self):
+        h = np.zeros((self.S, self.nsym), np.uint64)
+        rc = lib().co3_debug_hist(self.handle, h.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_debug_hist")
+        return h
+
+    def debug_code(self):
+        ln = np.zeros((self.S, self.nsym), np.uint8)
+        cw = np.zeros((self.S, self.nsym), np.uint32)
+        rc = lib().co3_debug_code(self.handle, ln.ctypes.data, cw.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_debug_code")
+        return ln, cw
+
+
+def hdr_to_numpy(hdr_tensor):
+    """[S] int32 device tensor of packed headers -> [S][3] int32 (bias, ibeta, ir)."""
+    raw = hdr_tensor.cpu().numpy().view(HDR_DTYPE)
+    return np.stack([raw["bias"].astype(np.int32), raw["ibeta"].astype(np.int32),
+                     raw["ir"].astype(np.int32)], axis=1)
+
+
+def hdr_from_numpy(hdr3, device="cuda"):
+    import torch
+    raw = np.zeros(len(hdr3), HDR_DTYPE)
+    raw["bias"], raw["ibeta"], raw["ir"] = hdr3[:, 0], hdr3[:, 1], hdr3[:, 2]
+    return torch.from_numpy(raw.view(np.int32).copy()).to(device)

@@ -1,0 +1,343 @@
+// C ABI of the CO3 library: plan management and the kernel sequences of one iteration of
+// Algorithm 1 (lines 8-10 at the users: co3_encode; lines 13-14 at the server:
+// co3_decode_aggregate).  Everything is enqueued on the caller's stream; nothing here allocates
+// after co3_plan_create and nothing synchronises except the inspection calls.
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+#include "co3_internal.h"
+
+cudaError_t co3_setup_decode_kernels(void);
+
+namespace {
+
+template <typename T>
+int dev_alloc(co3_plan* pl, T** out, size_t count) {
+    void* ptr = nullptr;
+    if (pl->n_allocs >= 64) return CO3_ENOMEM;
+    if (cudaMalloc(&ptr, (count ? count : 1) * sizeof(T)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CO3_ENOMEM;
+    }
+    pl->allocs[pl->n_allocs++] = ptr;
+    *out = (T*)ptr;
+    return CO3_OK;
+}
+
+int alloc_codebook(co3_plan* pl, Co3CodeBook& cb, int S) {
+    int rc = 0;
+    rc |= dev_alloc(pl, &cb.cand_len, (size_t)S * CO3_NCAND * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.cand_max, (size_t)S * CO3_NCAND);
+    rc |= dev_alloc(pl, &cb.len8, (size_t)S * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.enc, (size_t)S * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.code_msb, (size_t)S * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.lut, (size_t)S * CO3_LUT_SIZE);
+    rc |= dev_alloc(pl, &cb.first, (size_t)S * (CO3_MAXLEN + 1));
+    rc |= dev_alloc(pl, &cb.count, (size_t)S * (CO3_MAXLEN + 1));
+    rc |= dev_alloc(pl, &cb.offs, (size_t)S * (CO3_MAXLEN + 1));
+    rc |= dev_alloc(pl, &cb.perm, (size_t)S * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.ksign, (size_t)S * CO3_MAXSYM);
+    return rc ? CO3_ENOMEM : CO3_OK;
+}
+
+inline cudaStream_t as_stream(void* s) { return (cudaStream_t)s; }
+
+bool g_kernels_ready = false;
+
+}  // namespace
+
+extern "C" const char* co3_strerror(int code) {
+    switch (code) {
+        case CO3_OK: return "ok";
+        case CO3_EINVAL: return "invalid argument or unsupported configuration";
+        case CO3_ENOMEM: return "out of memory";
+        case CO3_ECUDA: return "CUDA runtime error";
+        case CO3_ECAPACITY: return "payload exceeds cap_words";
+        case CO3_ECORRUPT: return "stream does not decode to its recorded lengths";
+        case CO3_ENONFINITE: return "non-finite value in g + gamma*m";
+        default: return "unknown error";
+    }
+}
+
+extern "C" void co3_plan_destroy(co3_plan* pl) {
+    if (!pl) return;
+    for (int i = 0; i < pl->n_allocs; ++i) cudaFree(pl->allocs[i]);
+    free(pl->h_seg_off);
+    delete pl;
+}
+
+extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
+    if (!out || !cfg) return CO3_EINVAL;
+    *out = nullptr;
+    const int E = cfg->fmt.exp_bits, M = cfg->fmt.mant_bits;
+    if (!co3_host_fmt_ok(cfg->fmt)) return CO3_EINVAL;
+    if (cfg->d < 1 || cfg->ld < cfg->d || (cfg->ld & 3) || cfg->n_users < 1) return CO3_EINVAL;
+    if (cfg->cap_words < 4 || (cfg->cap_words & 3) || cfg->cap_words > 0xFFFFFFFFLL) return CO3_EINVAL;
+    if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED) return CO3_EINVAL;
+    if (!(cfg->gamma >= 0.0f) || !(cfg->gamma <= 1.0f)) return CO3_EINVAL;
+    if (cfg->d > ((int64_t)1 << 31)) return CO3_EINVAL;
+    const int nm = E + M, J = 1 << nm, nsym = 2 * J;
+    const int64_t Kmax = co3_host_K(M, J - 1);
+    if ((int64_t)cfg->n_users * Kmax >= ((int64_t)1 << 24)) return CO3_EINVAL;   // exact integer sums
+    const int S = cfg->seg_offsets ? cfg->n_segments : 1;
+    if (S < 1 || S > (1 << 20)) return CO3_EINVAL;
+
+    co3_plan* pl = new (std::nothrow) co3_plan();
+    if (!pl) return CO3_ENOMEM;
+    memset(pl, 0, sizeof(*pl));
+    pl->cfg = *cfg;
+    pl->h_seg_off = (int64_t*)malloc(sizeof(int64_t) * (size_t)(S + 1));
+    if (!pl->h_seg_off) { delete pl; return CO3_ENOMEM; }
+    if (cfg->seg_offsets) memcpy(pl->h_seg_off, cfg->seg_offsets, sizeof(int64_t) * (size_t)(S + 1));
+    else { pl->h_seg_off[0] = 0; pl->h_seg_off[1] = cfg->d; }
+    pl->cfg.seg_offsets = pl->h_seg_off;
+    pl->cfg.n_segments = S;
+
+    int64_t n_sub = 0;
+    const int64_t nc = co3_partition(cfg->d, S, pl->h_seg_off, nullptr, nullptr, nullptr, nullptr, &n_sub);
+    if (nc < 1) { co3_plan_destroy(pl); return CO3_EINVAL; }
+
+    int rc = CO3_OK;
+    Co3Chunk* h_chunks = (Co3Chunk*)calloc((size_t)nc, sizeof(Co3Chunk));
+    int32_t* h_seg = (int32_t*)malloc(sizeof(int32_t) * (size_t)nc);
+    int64_t* h_start = (int64_t*)malloc(sizeof(int64_t) * (size_t)nc);
+    int64_t* h_end = (int64_t*)malloc(sizeof(int64_t) * (size_t)nc);
+    int64_t* h_sub = (int64_t*)malloc(sizeof(int64_t) * (size_t)nc);
+    int32_t* h_seg_chunk0 = (int32_t*)malloc(sizeof(int32_t) * (size_t)(S + 1));
+    Co3Group* h_groups = (Co3Group*)calloc((size_t)nc, sizeof(Co3Group));
+    const uint32_t* wtab = co3_host_weight_table(E, M);
+    if (!h_chunks || !h_seg || !h_start || !h_end || !h_sub || !h_seg_chunk0 || !h_groups || !wtab) rc = CO3_ENOMEM;
+
+    int64_t n_groups = 0, worst = 0;
+    if (rc == CO3_OK) {
+        co3_partition(cfg->d, S, pl->h_seg_off, h_seg, h_start, h_end, h_sub, &n_sub);
+        int seg_cursor = 0;
+        for (int64_t c = 0; c < nc; ++c) {
+            h_chunks[c].start = h_start[c];
+            h_chunks[c].len = (int32_t)(h_end[c] - h_start[c]);
+            h_chunks[c].seg = h_seg[c];
+            h_chunks[c].sub0 = (int32_t)h_sub[c];
+            worst += 4 * ((16 * (int64_t)h_chunks[c].len + 127) / 128);
+            while (seg_cursor <= h_seg[c]) h_seg_chunk0[seg_cursor++] = (int32_t)c;
+        }
+        while (seg_cursor <= S) h_seg_chunk0[seg_cursor++] = (int32_t)nc;
+        const int cpg = cfg->n_users <= 8 ? 8 / cfg->n_users : 1;
+        for (int64_t c = 0; c < nc;) {
+            int cnt = 1;
+            while (cnt < cpg && c + cnt < nc && h_seg[c + cnt] == h_seg[c]) ++cnt;
+            h_groups[n_groups].chunk0 = (int32_t)c;
+            h_groups[n_groups].count = cnt;
+            h_groups[n_groups].seg = h_seg[c];
+            ++n_groups;
+            c += cnt;
+        }
+    }
+
+    Co3Dev& dv = pl->dev;
+    if (rc == CO3_OK) {
+        cudaGetDevice(&pl->device);
+        cudaDeviceGetAttribute(&pl->num_sms, cudaDevAttrMultiProcessorCount, pl->device);
+        if (pl->num_sms < 1) rc = CO3_ECUDA;
+    }
+    if (rc == CO3_OK) {
+        dv.E = E; dv.M = M; dv.nm = nm; dv.nsym = nsym; dv.J = J; dv.cF = co3_host_cF(E, M);
+        dv.Kmax = (uint32_t)Kmax;
+        dv.b_lo = -120 - dv.cF;
+        int bl = 0;
+        while ((Kmax >> bl) != 0) ++bl;
+        dv.b_hi = (100 - bl) - dv.cF;
+        dv.U = cfg->n_users; dv.S = S; dv.d = cfg->d; dv.ld = cfg->ld;
+        dv.sld = (cfg->d + CO3_TILE - 1) / CO3_TILE * CO3_TILE;
+        dv.n_chunks = nc; dv.n_sub = n_sub; dv.n_groups = n_groups; dv.cap_words = cfg->cap_words;
+        dv.gamma = cfg->gamma;
+        pl->worst_case_words = worst;
+
+        Co3Chunk* d_chunks = nullptr; Co3Group* d_groups = nullptr; int64_t* d_seg_off = nullptr;
+        int32_t* d_seg_chunk0 = nullptr; uint32_t* d_wtab = nullptr;
+        const size_t items = (size_t)nc * (size_t)dv.U;
+        int a = 0;
+        a |= dev_alloc(pl, &d_chunks, (size_t)nc);
+        a |= dev_alloc(pl, &d_groups, (size_t)n_groups);
+        a |= dev_alloc(pl, &d_seg_off, (size_t)S + 1);
+        a |= dev_alloc(pl, &d_seg_chunk0, (size_t)S + 1);
+        a |= dev_alloc(pl, &d_wtab, (size_t)CO3_NIBETA * CO3_NIR * J);
+        a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
+        a |= dev_alloc(pl, &dv.hist, (size_t)S * CO3_MAXSYM);
+        a |= dev_alloc(pl, &dv.part_s1, items);
+        a |= dev_alloc(pl, &dv.part_s2, items);
+        a |= dev_alloc(pl, &dv.part_nf, items);
+        a |= dev_alloc(pl, &dv.fit, (size_t)S * 5);
+        a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
+        a |= dev_alloc(pl, &dv.chunk_words, items);
+        a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
+        a |= dev_alloc(pl, &dv.flags, 1);
+        a |= dev_alloc(pl, &dv.nonfinite_total, 1);
+        a |= alloc_codebook(pl, pl->cb_enc, S);
+        a |= alloc_codebook(pl, pl->cb_dec, S);
+        if (a) rc = CO3_ENOMEM;
+        if (rc == CO3_OK) {
+            cudaError_t e = cudaSuccess;
+            auto up = [&](void* dst, const void* src, size_t bytes) {
+                if (e == cudaSuccess) e = cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice);
+            };
+            up(d_chunks, h_chunks, sizeof(Co3Chunk) * (size_t)nc);
+            up(d_groups, h_groups, sizeof(Co3Group) * (size_t)n_groups);
+            up(d_seg_off, pl->h_seg_off, sizeof(int64_t) * (size_t)(S + 1));
+            up(d_seg_chunk0, h_seg_chunk0, sizeof(int32_t) * (size_t)(S + 1));
+            up(d_wtab, wtab, sizeof(uint32_t) * (size_t)CO3_NIBETA * CO3_NIR * J);
+            if (e == cudaSuccess) e = cudaMemset(dv.flags, 0, sizeof(uint32_t));
+            if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
+            if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);
+            if (e == cudaSuccess) e = cudaMemset(dv.fit, 0, sizeof(double) * (size_t)S * 5);
+            if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * (size_t)S * CO3_MAXSYM);
+            if (e == cudaSuccess) e = cudaMemset(dv.sym, 0, (size_t)dv.U * (size_t)dv.sld);
+            if (e == cudaSuccess && !g_kernels_ready) {
+                e = co3_setup_kernels();
+                if (e == cudaSuccess) e = co3_setup_decode_kernels();
+                g_kernels_ready = (e == cudaSuccess);
+            }
+            if (e != cudaSuccess) { (void)cudaGetLastError(); rc = CO3_ECUDA; }
+            dv.chunks = d_chunks; dv.groups = d_groups; dv.seg_off = d_seg_off;
+            dv.seg_chunk0 = d_seg_chunk0; dv.wtab = d_wtab;
+        }
+    }
+    free(h_chunks); free(h_seg); free(h_start); free(h_end); free(h_sub); free(h_seg_chunk0); free(h_groups);
+    if (rc != CO3_OK) { co3_plan_destroy(pl); return rc; }
+    *out = pl;
+    return CO3_OK;
+}
+
+extern "C" int co3_sizes(const co3_plan* pl, int64_t* n_chunks, int64_t* n_sub, int64_t* worst_case_words) {
+    if (!pl) return CO3_EINVAL;
+    if (n_chunks) *n_chunks = pl->dev.n_chunks;
+    if (n_sub) *n_sub = pl->dev.n_sub;
+    if (worst_case_words) *worst_case_words = pl->worst_case_words;
+    return CO3_OK;
+}
+
+#define CO3_TRY(call) do { if ((call) != cudaSuccess) { (void)cudaGetLastError(); return CO3_ECUDA; } } while (0)
+
+extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint32_t* bitstream,
+                          uint16_t* sub_bits, uint32_t* chunk_off, uint64_t* user_bits,
+                          co3_seg_header* hdr, void* cuda_stream) {
+    if (!pl || !grad || !residual || !bitstream || !sub_bits || !chunk_off || !user_bits || !hdr) return CO3_EINVAL;
+    if (((uintptr_t)grad | (uintptr_t)residual | (uintptr_t)bitstream) & 15) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    if (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) {
+        CO3_TRY(co3_launch_stats(pl, grad, residual, st));
+        CO3_TRY(co3_launch_fit(pl, 0, hdr, st));
+    }
+    CO3_TRY(co3_launch_convert(pl, grad, residual, st));
+    CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
+    CO3_TRY(co3_launch_codebook(pl, pl->cb_enc, hdr, 0, st));
+    CO3_TRY(co3_launch_encode(pl, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
+    pl->iteration++;
+    return CO3_OK;
+}
+
+extern "C" int co3_decode_aggregate(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+                                    const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
+                                    void* cuda_stream) {
+    if (!pl || !bitstream || !sub_bits || !chunk_off || !hdr || !avg_grad) return CO3_EINVAL;
+    if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    CO3_TRY(co3_launch_codebook(pl, pl->cb_dec, hdr, 1, st));
+    CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, st));
+    return CO3_OK;
+}
+
+extern "C" int co3_iteration_host(co3_plan* pl, const float* h_grad, float* d_grad, float* d_residual,
+                                  uint32_t* d_bitstream, uint16_t* d_sub_bits, uint32_t* d_chunk_off,
+                                  uint64_t* d_user_bits, co3_seg_header* d_hdr, float* d_avg, float* h_avg,
+                                  void* cuda_stream) {
+    if (!pl || !h_grad || !d_grad || !h_avg || !d_avg) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    CO3_TRY(cudaMemcpyAsync(d_grad, h_grad, sizeof(float) * (size_t)pl->dev.U * (size_t)pl->dev.ld,
+                            cudaMemcpyHostToDevice, st));
+    int rc = co3_encode(pl, d_grad, d_residual, d_bitstream, d_sub_bits, d_chunk_off, d_user_bits, d_hdr, cuda_stream);
+    if (rc != CO3_OK) return rc;
+    rc = co3_decode_aggregate(pl, d_bitstream, d_sub_bits, d_chunk_off, d_hdr, d_avg, cuda_stream);
+    if (rc != CO3_OK) return rc;
+    CO3_TRY(cudaMemcpyAsync(h_avg, d_avg, sizeof(float) * (size_t)pl->dev.d, cudaMemcpyDeviceToHost, st));
+    return CO3_OK;
+}
+
+extern "C" int co3_status(co3_plan* pl, uint32_t* flags, uint64_t* nonfinite_count, int32_t clear) {
+    if (!pl) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    uint32_t f = 0;
+    unsigned long long n = 0;
+    CO3_TRY(cudaMemcpy(&f, pl->dev.flags, sizeof(f), cudaMemcpyDeviceToHost));
+    CO3_TRY(cudaMemcpy(&n, pl->dev.nonfinite_total, sizeof(n), cudaMemcpyDeviceToHost));
+    if (flags) *flags = f;
+    if (nonfinite_count) *nonfinite_count = n;
+    if (clear) {
+        CO3_TRY(cudaMemset(pl->dev.flags, 0, sizeof(uint32_t)));
+        CO3_TRY(cudaMemset(pl->dev.nonfinite_total, 0, sizeof(unsigned long long)));
+    }
+    return CO3_OK;
+}
+
+extern "C" int co3_get_fit(co3_plan* pl, int32_t seg, double* beta, double* alpha, double* N, double* S1,
+                           double* S2) {
+    if (!pl || seg < 0 || seg >= pl->dev.S) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    double f[5];
+    CO3_TRY(cudaMemcpy(f, pl->dev.fit + 5 * (size_t)seg, sizeof(f), cudaMemcpyDeviceToHost));
+    if (beta) *beta = f[0];
+    if (alpha) *alpha = f[1];
+    if (N) *N = f[2];
+    if (S1) *S1 = f[3];
+    if (S2) *S2 = f[4];
+    return CO3_OK;
+}
+
+extern "C" int co3_state_export(co3_plan* pl, int64_t* iteration, int32_t* next_bias) {
+    if (!pl || !iteration || !next_bias) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    CO3_TRY(cudaMemcpy(next_bias, pl->dev.bias_cur, sizeof(int32_t) * (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
+    *iteration = pl->iteration;
+    return CO3_OK;
+}
+
+extern "C" int co3_state_import(co3_plan* pl, int64_t iteration, const int32_t* next_bias) {
+    if (!pl || !next_bias || iteration < 0) return CO3_EINVAL;
+    for (int l = 0; l < pl->dev.S; ++l)
+        if (next_bias[l] < pl->dev.b_lo || next_bias[l] > pl->dev.b_hi) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    CO3_TRY(cudaMemcpy(pl->dev.bias_cur, next_bias, sizeof(int32_t) * (size_t)pl->dev.S, cudaMemcpyHostToDevice));
+    pl->iteration = iteration;
+    return CO3_OK;
+}
+
+extern "C" int co3_debug_symbols(co3_plan* pl, uint8_t* symbols, void* cuda_stream) {
+    if (!pl || !symbols) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    CO3_TRY(cudaMemcpy2DAsync(symbols, (size_t)pl->dev.d, pl->dev.sym, (size_t)pl->dev.sld, (size_t)pl->dev.d,
+                              (size_t)pl->dev.U, cudaMemcpyDeviceToDevice, st));
+    CO3_TRY(cudaStreamSynchronize(st));
+    return CO3_OK;
+}
+
+extern "C" int co3_debug_hist(co3_plan* pl, uint64_t* hist) {
+    if (!pl || !hist) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    CO3_TRY(cudaMemcpy2D(hist, sizeof(uint64_t) * (size_t)pl->dev.nsym, pl->dev.hist,
+                         sizeof(uint64_t) * CO3_MAXSYM, sizeof(uint64_t) * (size_t)pl->dev.nsym,
+                         (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
+    return CO3_OK;
+}
+
+extern "C" int co3_debug_code(co3_plan* pl, uint8_t* lengths, uint32_t* codewords) {
+    if (!pl || !lengths || !codewords) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    CO3_TRY(cudaMemcpy2D(lengths, (size_t)pl->dev.nsym, pl->cb_enc.len8, CO3_MAXSYM, (size_t)pl->dev.nsym,
+                         (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
+    CO3_TRY(cudaMemcpy2D(codewords, sizeof(uint32_t) * (size_t)pl->dev.nsym, pl->cb_enc.code_msb,
+                         sizeof(uint32_t) * CO3_MAXSYM, sizeof(uint32_t) * (size_t)pl->dev.nsym,
+                         (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
+    return CO3_OK;
+}

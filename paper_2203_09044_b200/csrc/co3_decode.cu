@@ -1,0 +1,330 @@
+// Parameter-server side (Algorithm 1 lines 13-14 up to the model update, Eq. "aggregate"):
+// decode every user's stream and write the average of the reconstructed gradients.
+//
+// A lane decodes one sub-chunk (<= 128 codewords) serially with an 11-bit primary table whose
+// entries already hold the signed integer magnitude; the 32 sub-chunks of a chunk are the 32
+// lanes of a warp, so a warp is one (chunk, user) stream.  The integer magnitudes of all users
+// are accumulated with shared-memory atomics into a transposed, padded tile (conflict-free both
+// for the per-lane scattered adds and for the coalesced read-out), scaled once by 2^lambda and
+// divided by U.  The stream words are staged in shared memory with 128-bit loads, so global
+// traffic is fully coalesced.
+//
+// Two variants: U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
+// per sub-chunk (small accumulator, several chunks per block when U < 8); U > 8 keeps a whole
+// chunk accumulator and loops over user groups.
+//
+// Bound: HBM for U = 1 (4 B written per element); for U >= 4 the serial decode (issue slots and
+// shared-memory look-ups per symbol) dominates.
+#include "co3_internal.h"
+
+namespace {
+
+constexpr int NW = CO3_THREADS / 32;              // warps = concurrent streams per block
+constexpr int PADW = 33;                          // row stride of the transposed accumulator
+
+struct Tables {                                   // per-segment decoder tables in shared memory
+    uint32_t lut[CO3_LUT_SIZE];
+    uint32_t first[CO3_MAXLEN + 1], count[CO3_MAXLEN + 1], offs[CO3_MAXLEN + 1];
+    int32_t ksign[CO3_MAXSYM];
+    uint8_t perm[CO3_MAXSYM];
+};
+
+__device__ void load_tables(Tables& t, const Co3CodeBook& cb, int seg, int nsym, int tid) {
+    const uint32_t* lut = cb.lut + (size_t)seg * CO3_LUT_SIZE;
+    for (int i = tid; i < CO3_LUT_SIZE; i += CO3_THREADS) t.lut[i] = lut[i];
+    if (tid <= CO3_MAXLEN) {
+        const size_t o = (size_t)seg * (CO3_MAXLEN + 1) + tid;
+        t.first[tid] = cb.first[o]; t.count[tid] = cb.count[o]; t.offs[tid] = cb.offs[o];
+    }
+    if (tid < nsym) {
+        t.ksign[tid] = cb.ksign[(size_t)seg * CO3_MAXSYM + tid];
+        t.perm[tid] = cb.perm[(size_t)seg * CO3_MAXSYM + tid];
+    }
+}
+
+__device__ __forceinline__ float pow2_clamped(int e) {   // 2^e; a corrupt header cannot make a NaN
+    e = min(max(e, -126), 127);
+    return __uint_as_float((uint32_t)(e + 127) << 23);
+}
+
+struct Reader {                                   // LSB-first bit reader over a bounded word array
+    unsigned long long buf;
+    int nb;                                       // valid bits in buf
+    uint32_t wp;                                  // next word to fetch
+};
+
+__device__ __forceinline__ uint32_t fetch(const uint32_t* src, uint32_t nwords, uint32_t i) {
+    return i < nwords ? src[i] : 0u;
+}
+
+__device__ __forceinline__ void reader_init(Reader& r, const uint32_t* src, uint32_t nwords, uint32_t bitpos) {
+    r.wp = bitpos >> 5;
+    const uint32_t sh = bitpos & 31u;
+    r.buf = (unsigned long long)(fetch(src, nwords, r.wp) >> sh);
+    r.nb = 32 - (int)sh;
+    r.wp++;
+    r.buf |= (unsigned long long)fetch(src, nwords, r.wp) << r.nb;
+    r.nb += 32;
+    r.wp++;
+}
+
+// Decode one codeword; returns its signed integer magnitude.  bad is set if no codeword matches
+// (cannot happen for a complete code; kept so that corrupt tables cannot loop or read outside).
+__device__ __forceinline__ int32_t decode_one(Reader& r, const Tables& t, const uint32_t* src,
+                                              uint32_t nwords, bool& bad) {
+    const uint32_t window = (uint32_t)r.buf;
+    uint32_t e = t.lut[window & (CO3_LUT_SIZE - 1)];
+    int32_t k;
+    uint32_t len = e & 0xFFu;
+    if (len != 0) {
+        k = (int32_t)e >> 8;
+    } else {                                      // codeword longer than 11 bits: canonical search
+        const uint32_t v = __brev(window) >> 16;  // 16 stream bits, root bit on top
+        k = 0;
+        len = CO3_MAXLEN;
+        bool found = false;
+        for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
+            const uint32_t dd = (v >> (CO3_MAXLEN - L)) - t.first[L];
+            if (dd < t.count[L]) {
+                k = t.ksign[t.perm[(t.offs[L] + dd) & (CO3_MAXSYM - 1)]];
+                len = (uint32_t)L;
+                found = true;
+                break;
+            }
+        }
+        bad |= !found;
+    }
+    r.buf >>= len;
+    r.nb -= (int)len;
+    if (r.nb < 32) {
+        r.buf |= (unsigned long long)fetch(src, nwords, r.wp) << r.nb;
+        r.nb += 32;
+        r.wp++;
+    }
+    return k;
+}
+
+struct Stream {                                   // one (chunk, user) stream as seen by a lane
+    const uint32_t* src;                          // staged or global words of the chunk
+    uint32_t nwords;
+    uint32_t bitpos;                              // start of this lane's sub-chunk
+    uint32_t sub_len_bits;                        // recorded length of this lane's sub-chunk
+    int i_lo, i_hi;                               // this lane's symbols within its 128-window
+    bool active;
+};
+
+// Stage the words of (chunk c, user u) into `stage` (or point at global memory if they do not
+// fit) and give every lane the start of its sub-chunk.  Called by one whole warp.
+__device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co3Chunk& cd, int64_t c, int u,
+                                            const uint32_t* __restrict__ bitstream,
+                                            const uint16_t* __restrict__ sub_bits,
+                                            const uint32_t* __restrict__ chunk_off,
+                                            uint32_t* stage, int lane, bool& bad) {
+    const uint32_t* co = chunk_off + (size_t)u * (p.n_chunks + 1) + c;
+    const uint32_t w0 = co[0], w1 = co[1];
+    uint32_t nwords = 0;
+    if ((w0 & 3u) || w1 < w0 || (int64_t)w1 > p.cap_words) bad = true;   // offsets must be sane
+    else nwords = w1 - w0;
+    const uint32_t* g = bitstream + (size_t)u * p.cap_words + w0;
+    if (nwords <= CO3_STAGE_WORDS) {
+        const uint4* gv = reinterpret_cast<const uint4*>(g);
+        uint4* sv = reinterpret_cast<uint4*>(stage);
+        for (uint32_t i = lane; i < nwords / 4; i += 32) sv[i] = __ldg(gv + i);
+        for (uint32_t i = (nwords & ~3u) + lane; i < nwords; i += 32) stage[i] = __ldg(g + i);
+        s.src = stage;
+    } else {
+        s.src = g;
+    }
+    s.nwords = nwords;
+    const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+    const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+    const int sub_first = lo / CO3_SUB, sub_last = (hi - 1) / CO3_SUB;
+    s.active = lane >= sub_first && lane <= sub_last;
+    s.i_lo = max(lo - lane * CO3_SUB, 0);
+    s.i_hi = min(hi - lane * CO3_SUB, CO3_SUB);
+    uint32_t sb = s.active ? sub_bits[(size_t)u * p.n_sub + cd.sub0 + (lane - sub_first)] : 0u;
+    uint32_t x = sb;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+    }
+    s.bitpos = x - sb;
+    s.sub_len_bits = sb;
+    __syncwarp();
+}
+
+__device__ __forceinline__ void write_out(const Co3Dev& p, float* __restrict__ avg, const int32_t* acc,
+                                          const Co3Chunk& cd, int i0, int ni, float scale, float fu,
+                                          int t, int nt) {
+    // acc holds symbols i0 .. i0+ni-1 of every sub-chunk: acc[(i - i0) * PADW + kk]
+    const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+    const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+    for (int x = t; x < 32 * ni; x += nt) {
+        const int kk = x / ni, il = x - kk * ni;
+        const int e = kk * CO3_SUB + i0 + il;
+        if (e >= lo && e < hi)
+            avg[tb + e] = __fdiv_rn(__fmul_rn((float)acc[il * PADW + kk], scale), fu);
+    }
+}
+
+// ---- U <= 8: one stream per warp, quarter batches ------------------------------------------
+static_assert(CO3_STAGE_WORDS % 4 == 0, "stage rows must keep 16-byte alignment");
+constexpr int QB = 32;                            // symbols per lane per batch
+
+struct SmemA {
+    Tables t;
+    alignas(16) uint32_t stage[NW][CO3_STAGE_WORDS];   // filled with 128-bit stores
+    int32_t acc[1][QB * PADW];                    // one accumulator per chunk of the group:
+};                                                // really [chunks per group], sized at launch
+
+__host__ __device__ inline size_t smem_a_bytes(int U) {
+    return sizeof(SmemA) + (size_t)(NW / U - 1) * QB * PADW * sizeof(int32_t);
+}
+
+__global__ void __launch_bounds__(CO3_THREADS)
+decode_small_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bitstream,
+                      const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
+                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    SmemA& sm = *reinterpret_cast<SmemA*>(s_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int U = p.U;
+    const int cpg = NW / U;                        // chunks per group (>= 1)
+    const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
+    const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
+    const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
+    const float fu = (float)U;
+    int cur_seg = -1;
+    bool bad = false;
+    for (int64_t gi = g0; gi < g1; ++gi) {
+        const Co3Group grp = p.groups[gi];
+        if (grp.seg != cur_seg) {
+            __syncthreads();
+            load_tables(sm.t, cb, grp.seg, p.nsym, tid);
+            cur_seg = grp.seg;
+            __syncthreads();
+        }
+        const bool mine = ci < cpg && ci < grp.count;
+        Stream s;
+        s.active = false;
+        Co3Chunk cd;
+        cd.start = 0; cd.len = 0; cd.seg = 0; cd.sub0 = 0;
+        Reader r;
+        r.buf = 0; r.nb = 0; r.wp = 0;
+        if (mine) {
+            cd = p.chunks[grp.chunk0 + ci];
+            open_stream(s, p, cd, grp.chunk0 + ci, us, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
+            if (s.active) reader_init(r, s.src, s.nwords, s.bitpos);
+        }
+        const float scale = pow2_clamped((int)hdr[grp.seg].bias + p.cF);
+        for (int q = 0; q < CO3_SUB / QB; ++q) {
+            for (int i = tid; i < grp.count * QB * PADW; i += CO3_THREADS) (&sm.acc[0][0])[i] = 0;
+            __syncthreads();
+            if (mine && s.active) {
+                const int a = max(s.i_lo, q * QB), b = min(s.i_hi, (q + 1) * QB);
+                int32_t* acc = sm.acc[ci];
+                for (int i = a; i < b; ++i) {
+                    const int32_t k = decode_one(r, sm.t, s.src, s.nwords, bad);
+                    atomicAdd(&acc[(i - q * QB) * PADW + lane], k);
+                }
+            }
+            __syncthreads();
+            for (int cc = 0; cc < grp.count; ++cc)
+                write_out(p, avg, sm.acc[cc], p.chunks[grp.chunk0 + cc], q * QB, QB, scale, fu, tid, CO3_THREADS);
+            __syncthreads();
+        }
+        if (mine && s.active) {
+            const uint32_t endpos = r.wp * 32u - (uint32_t)r.nb;
+            if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
+        }
+    }
+    if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
+}
+
+// ---- U > 8: whole-chunk accumulator, user groups of 8 --------------------------------------
+struct SmemB {
+    Tables t;
+    int32_t acc[CO3_SUB * PADW];
+    alignas(16) uint32_t stage[NW][CO3_STAGE_WORDS];   // filled with 128-bit stores
+};
+
+__global__ void __launch_bounds__(CO3_THREADS)
+decode_large_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bitstream,
+                      const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
+                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    SmemB& sm = *reinterpret_cast<SmemB*>(s_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t per = (p.n_chunks + gridDim.x - 1) / gridDim.x;
+    const int64_t c0 = (int64_t)blockIdx.x * per, c1 = min(p.n_chunks, c0 + per);
+    const float fu = (float)p.U;
+    int cur_seg = -1;
+    bool bad = false;
+    for (int64_t c = c0; c < c1; ++c) {
+        const Co3Chunk cd = p.chunks[c];
+        if (cd.seg != cur_seg) {
+            __syncthreads();
+            load_tables(sm.t, cb, cd.seg, p.nsym, tid);
+            cur_seg = cd.seg;
+        }
+        for (int i = tid; i < CO3_SUB * PADW; i += CO3_THREADS) sm.acc[i] = 0;
+        __syncthreads();
+        for (int u = warp; u < p.U; u += NW) {
+            Stream s;
+            open_stream(s, p, cd, c, u, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
+            if (s.active) {
+                Reader r;
+                reader_init(r, s.src, s.nwords, s.bitpos);
+                for (int i = s.i_lo; i < s.i_hi; ++i) {
+                    const int32_t k = decode_one(r, sm.t, s.src, s.nwords, bad);
+                    atomicAdd(&sm.acc[i * PADW + lane], k);
+                }
+                const uint32_t endpos = r.wp * 32u - (uint32_t)r.nb;
+                if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
+            }
+            __syncwarp();                          // the stage is reused by this warp's next user
+        }
+        __syncthreads();
+        const float scale = pow2_clamped((int)hdr[cd.seg].bias + p.cF);
+        write_out(p, avg, sm.acc, cd, 0, CO3_SUB, scale, fu, tid, CO3_THREADS);
+        __syncthreads();
+    }
+    if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
+}
+
+int g_bpsm_b = 0;
+
+}  // namespace
+
+cudaError_t co3_setup_decode_kernels(void) {
+    cudaError_t e = cudaFuncSetAttribute(decode_small_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem_a_bytes(1));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_large_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)sizeof(SmemB));
+}
+
+cudaError_t co3_launch_decode(const co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+                              const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
+                              cudaStream_t st) {
+    const Co3Dev& p = pl->dev;
+    if (p.U <= NW) {
+        const size_t smem = smem_a_bytes(p.U);
+        int bpsm = 0;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bpsm, decode_small_u_kernel, CO3_THREADS, smem);
+        if (bpsm < 1) bpsm = 1;
+        const int64_t grid = (int64_t)pl->num_sms * bpsm;
+        decode_small_u_kernel<<<(int)(p.n_groups < grid ? p.n_groups : grid), CO3_THREADS, smem, st>>>(
+            p, pl->cb_dec, bitstream, sub_bits, chunk_off, hdr, avg);
+    } else {
+        if (!g_bpsm_b) {
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_bpsm_b, decode_large_u_kernel, CO3_THREADS, sizeof(SmemB));
+            if (g_bpsm_b < 1) g_bpsm_b = 1;
+        }
+        const int64_t grid = (int64_t)pl->num_sms * g_bpsm_b;
+        decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), CO3_THREADS, sizeof(SmemB), st>>>(
+            p, pl->cb_dec, bitstream, sub_bits, chunk_off, hdr, avg);
+    }
+    return cudaGetLastError();
+}

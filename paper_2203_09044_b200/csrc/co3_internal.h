@@ -1,0 +1,119 @@
+// Internal declarations of the CO3 CUDA library (sm_100a).  Not part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "co3.h"
+
+constexpr int CO3_TILE = 4096;      // chunk grid (elements)
+constexpr int CO3_SUB = 128;        // sub-chunk grid (elements)
+constexpr int CO3_MAXLEN = 16;      // longest codeword
+constexpr int CO3_LUT_BITS = 11;    // primary decode table index width
+constexpr int CO3_LUT_SIZE = 1 << CO3_LUT_BITS;
+constexpr int CO3_NCAND = 10;       // weight floors 2^0 .. 2^9 tried in parallel (2^9 always passes)
+constexpr int CO3_NIBETA = 23;      // ibeta in [-14, 8]
+constexpr int CO3_NIR = 128;        // ir in [-96, 31]
+constexpr int CO3_IBETA_MIN = -14, CO3_IBETA_MAX = 8, CO3_IR_MIN = -96, CO3_IR_MAX = 31;
+constexpr int CO3_MAXSYM = 256;     // alphabet rows are padded to 256 entries
+constexpr int CO3_STAGE_WORDS = 1024;  // shared-memory staging per (chunk, user) stream in decode
+constexpr int CO3_THREADS = 256;
+
+// One chunk of the static partition: elements [start, start+len) of every user's row, all in
+// segment `seg`, inside one 4096-aligned tile.  sub0 = index of its first sub-chunk.
+struct Co3Chunk {
+    int64_t start;
+    int32_t len;
+    int32_t seg;
+    int32_t sub0;
+    int32_t pad_;
+};
+
+// A group of consecutive chunks of one segment decoded together by one block (U <= 8).
+struct Co3Group {
+    int32_t chunk0;
+    int32_t count;
+    int32_t seg;
+    int32_t pad_;
+};
+
+// Per-segment code tables built on the device from the header (one instance for the encoder,
+// one for the decoder; rows are CO3_MAXSYM / CO3_LUT_SIZE wide).
+struct Co3CodeBook {
+    uint8_t* cand_len;   // [S][NCAND][256] code lengths per weight-floor candidate
+    int32_t* cand_max;   // [S][NCAND]      longest codeword per candidate
+    uint8_t* len8;       // [S][256]        chosen lengths
+    uint32_t* enc;       // [S][256]        bit-reversed codeword | length << 16
+    uint32_t* code_msb;  // [S][256]        canonical codeword, root bit most significant
+    uint32_t* lut;       // [S][2048]       (signed magnitude << 8) | length, 0 = longer than 11 bits
+    uint32_t* first;     // [S][17]         first canonical code of each length
+    uint32_t* count;     // [S][17]
+    uint32_t* offs;      // [S][17]         start of each length in perm
+    uint8_t* perm;       // [S][256]        symbols ordered by (length, symbol)
+    int32_t* ksign;      // [S][256]        signed integer magnitude of each symbol
+};
+
+// Everything the kernels need, passed by value.
+struct Co3Dev {
+    int E, M, nm, nsym, J, cF, b_lo, b_hi;
+    uint32_t Kmax;
+    int U, S;
+    int64_t d, ld, sld, n_chunks, n_sub, n_groups, cap_words;
+    float gamma;
+    const Co3Chunk* chunks;       // [n_chunks]
+    const Co3Group* groups;       // [n_groups]
+    const int64_t* seg_off;       // [S+1]
+    const int32_t* seg_chunk0;    // [S+1] first chunk of each segment
+    uint8_t* sym;                 // [U][sld]
+    unsigned long long* hist;     // [S][256]
+    double* part_s1;              // [U*n_chunks] per-(user,chunk) partial sums of |a|
+    double* part_s2;              //              ... of a^2
+    uint32_t* part_nf;            //              ... count of non-finite a
+    double* fit;                  // [S][5] beta, alpha, N, S1, S2
+    int32_t* bias_cur;            // [S] bias used by the next convert pass
+    const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
+    uint32_t* chunk_words;        // [U][n_chunks]
+    uint32_t* user_ovf;           // [U] 1 if the user's payload exceeds cap_words
+    uint32_t* flags;              // sticky status flags
+    unsigned long long* nonfinite_total;
+};
+
+struct co3_plan {
+    co3_config cfg;
+    Co3Dev dev;
+    Co3CodeBook cb_enc, cb_dec;
+    int64_t iteration;
+    int64_t worst_case_words;
+    int device;
+    int num_sms;
+    cudaStream_t last_stream;
+    void* allocs[64];
+    int n_allocs;
+    int64_t* h_seg_off;
+};
+
+// host-side helpers (co3_model.cu)
+int co3_host_fmt_ok(co3_format f);
+int co3_host_cF(int E, int M);
+int64_t co3_host_K(int M, int j);
+const uint32_t* co3_host_weight_table(int E, int M);   // [NIBETA][NIR][J], cached per format
+
+// kernel launchers (each returns a cudaError_t from the launch)
+cudaError_t co3_launch_stats(const co3_plan* pl, const float* g, const float* m, cudaStream_t st);
+cudaError_t co3_launch_convert(const co3_plan* pl, const float* g, float* m, cudaStream_t st);
+cudaError_t co3_launch_fit(const co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
+cudaError_t co3_launch_codebook(const co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
+                                int want_decode_tables, cudaStream_t st);
+cudaError_t co3_launch_encode(const co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
+                              uint32_t* chunk_off, unsigned long long* user_bits, cudaStream_t st);
+cudaError_t co3_launch_decode(const co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+                              const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
+                              cudaStream_t st);
+cudaError_t co3_setup_kernels(void);
+
+// Signed integer magnitude of a symbol byte: K(j) = f (e = 0) or (2^M + f) << (e - 1).
+__host__ __device__ inline int32_t co3_ksigned(int sym, int M, int nm) {
+    int j = sym & ((1 << nm) - 1);
+    int e = j >> M, f = j & ((1 << M) - 1);
+    int32_t k = (e == 0) ? f : (((1 << M) + f) << (e - 1));
+    return (sym >> nm) ? -k : k;
+}

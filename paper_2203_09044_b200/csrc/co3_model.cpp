@@ -1,0 +1,164 @@
+// Host side of the code model: format arithmetic and the table of integer symbol weights of the
+// quantised generalized-normal source (Sec. III (ii): the Huffman code is designed from the
+// GenNorm model of the converted gradient; Sec. IV-B "Huffman coding").
+//
+// The table T[ibeta][ir][j] is a pure function of the format.  For shape beta_q = 2^(ibeta/8)
+// and scale (relative to the bias) r_q = ir/8, the cell of magnitude code j is bounded by the
+// midpoints to its neighbours; its probability is a difference of the GenNorm CDF
+// Pr(|X| <= t) = P(1/beta, (t/alpha)^beta) (regularised lower incomplete gamma).
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "co3_internal.h"
+
+int co3_host_fmt_ok(co3_format f) {
+    return f.exp_bits >= 1 && f.exp_bits <= 4 && f.mant_bits >= 1 && f.exp_bits + f.mant_bits <= 7;
+}
+
+int co3_host_cF(int E, int M) { return 1 - ((1 << (E - 1)) - 1) - M; }
+
+int64_t co3_host_K(int M, int j) {
+    int e = j >> M, f = j & ((1 << M) - 1);
+    return e == 0 ? (int64_t)f : ((int64_t)((1 << M) + f) << (e - 1));
+}
+
+namespace {
+
+// lower series: gamma(a,x) = x^a e^-x sum_{n>=0} x^n / (a (a+1) ... (a+n))
+double lower_series(double a, double x, double log_pref) {
+    double denom = a, term = 1.0 / a, total = term;
+    for (int n = 1; n < 200000; ++n) {
+        denom += 1.0;
+        term = term * x / denom;
+        total += term;
+        if (term <= total * 5e-18) break;
+    }
+    return total * exp(log_pref);
+}
+
+// upper continued fraction, evaluated with the forward (Wallis) recurrence and rescaling:
+// Gamma(a,x) = x^a e^-x * 1/(x+1-a - 1(1-a)/(x+3-a - 2(2-a)/(x+5-a - ...)))
+double upper_fraction(double a, double x, double log_pref) {
+    // Write the fraction as 1/f, f = b0 + a1/(b1 + a2/(b2 + ...)); convergents A_i/B_i of f with
+    // A_{-1} = 1, A_0 = b0, B_{-1} = 0, B_0 = 1.
+    const double b0 = x + 1.0 - a;
+    double Am1 = 1.0, A0 = b0, Bm1 = 0.0, B0 = 1.0;
+    double prev = A0 / B0;
+    for (int i = 1; i < 200000; ++i) {
+        double ai = -(double)i * ((double)i - a);
+        double bi = x + (double)(2 * i + 1) - a;
+        double A1 = bi * A0 + ai * Am1;
+        double B1 = bi * B0 + ai * Bm1;
+        Am1 = A0; A0 = A1; Bm1 = B0; B0 = B1;
+        if (fabs(A0) > 1e200 || fabs(B0) > 1e200) {
+            Am1 *= 1e-200; A0 *= 1e-200; Bm1 *= 1e-200; B0 *= 1e-200;
+        }
+        if (B0 != 0.0) {
+            double cur = A0 / B0;
+            if (fabs(cur - prev) <= fabs(cur) * 1e-16) { prev = cur; break; }
+            prev = cur;
+        }
+    }
+    return exp(log_pref) / prev;
+}
+
+double reg_lower_gamma(double a, double x) {
+    if (!(x > 0.0)) return 0.0;
+    if (isinf(x)) return 1.0;
+    double log_pref = a * log(x) - x - lgamma(a);
+    if (x < a + 1.0) {
+        double p = lower_series(a, x, log_pref);
+        return p > 1.0 ? 1.0 : p;
+    }
+    double q = upper_fraction(a, x, log_pref);
+    if (q < 0.0) q = 0.0;
+    if (q > 1.0) q = 1.0;
+    return 1.0 - q;
+}
+
+void weight_row(int E, int M, int ibeta, int ir, uint32_t* half /* J entries */) {
+    const int J = 1 << (E + M);
+    const double beta_q = exp2((double)ibeta / 8.0), r_q = (double)ir / 8.0;
+    const double unit = exp2((double)co3_host_cF(E, M) - r_q);
+    const double scale = 1048576.0;
+    double below = 0.0;
+    for (int j = 0; j < J; ++j) {
+        double cdf = 1.0;
+        if (j < J - 1) {
+            double tau = 0.5 * (double)(co3_host_K(M, j) + co3_host_K(M, j + 1)) * unit;
+            cdf = reg_lower_gamma(1.0 / beta_q, pow(tau, beta_q));
+        }
+        double mass = cdf - below;
+        below = cdf;
+        double x = (j == 0) ? floor(scale * mass + 0.5) : floor(scale * mass / 2.0 + 0.5);
+        half[j] = x < 1.0 ? 1u : (uint32_t)x;
+    }
+}
+
+struct TableCache {
+    int E, M;
+    uint32_t* data;
+};
+TableCache g_cache[16];
+int g_ncache = 0;
+std::mutex g_mu;
+
+}  // namespace
+
+const uint32_t* co3_host_weight_table(int E, int M) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (int i = 0; i < g_ncache; ++i)
+        if (g_cache[i].E == E && g_cache[i].M == M) return g_cache[i].data;
+    if (g_ncache == 16) return nullptr;
+    const int J = 1 << (E + M);
+    uint32_t* t = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)CO3_NIBETA * CO3_NIR * J);
+    if (!t) return nullptr;
+    for (int ib = 0; ib < CO3_NIBETA; ++ib)
+        for (int r = 0; r < CO3_NIR; ++r)
+            weight_row(E, M, ib + CO3_IBETA_MIN, r + CO3_IR_MIN, t + ((size_t)ib * CO3_NIR + r) * J);
+    g_cache[g_ncache++] = TableCache{E, M, t};
+    return t;
+}
+
+extern "C" int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint32_t* weights) {
+    if (!co3_host_fmt_ok(fmt) || !weights || ibeta < CO3_IBETA_MIN || ibeta > CO3_IBETA_MAX ||
+        ir < CO3_IR_MIN || ir > CO3_IR_MAX)
+        return CO3_EINVAL;
+    const int E = fmt.exp_bits, M = fmt.mant_bits, J = 1 << (E + M);
+    uint32_t half[128];
+    weight_row(E, M, ibeta, ir, half);
+    for (int j = 0; j < J; ++j) {
+        weights[j] = half[j];
+        weights[J + j] = (j == 0) ? 1u : half[j];   // "-0" is never emitted
+    }
+    return CO3_OK;
+}
+
+extern "C" int64_t co3_partition(int64_t d, int32_t n_segments, const int64_t* seg_offsets,
+                                 int32_t* chunk_seg, int64_t* chunk_start, int64_t* chunk_end,
+                                 int64_t* sub_base, int64_t* n_sub) {
+    const int64_t one_seg[2] = {0, d};
+    if (!seg_offsets) { seg_offsets = one_seg; n_segments = 1; }
+    if (d < 1 || n_segments < 1 || seg_offsets[0] != 0 || seg_offsets[n_segments] != d) return CO3_EINVAL;
+    int64_t nc = 0, ns = 0;
+    for (int l = 0; l < n_segments; ++l) {
+        int64_t lo = seg_offsets[l], hi = seg_offsets[l + 1];
+        if (hi < lo) return CO3_EINVAL;
+        while (lo < hi) {
+            int64_t cut = (lo / CO3_TILE + 1) * CO3_TILE;
+            if (cut > hi) cut = hi;
+            if (chunk_seg) chunk_seg[nc] = l;
+            if (chunk_start) chunk_start[nc] = lo;
+            if (chunk_end) chunk_end[nc] = cut;
+            if (sub_base) sub_base[nc] = ns;
+            ns += (cut - 1) / CO3_SUB - lo / CO3_SUB + 1;
+            ++nc;
+            lo = cut;
+        }
+    }
+    if (n_sub) *n_sub = ns;
+    return nc;
+}

@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded
+inputs.  Bit-exact on symbols, residuals, histograms, headers, code tables, bitstreams, side
+information and averaged gradients; GenNorm fit parameters within 1e-5 relative."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+FORMATS = [(1, 2), (3, 2), (4, 3)]
+
+
+@pytest.fixture(scope="module")
+def binding():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2203_09044_b200 import binding as b
+    b.lib()          # raises if the CUDA library is not built: there is no fallback
+    return b
+
+
+def _bits(x):
+    return np.ascontiguousarray(x).view(np.uint32)
+
+
+def compare_iteration(b, plan, out, r, m_gpu, m_cpu, tag=""):
+    """One encoded iteration: everything co3_encode produced vs the oracle's IterationResult."""
+    U, d = plan.U, plan.d
+    sym = plan.debug_symbols().cpu().numpy()
+    assert np.array_equal(sym, r.sym), f"{tag} symbols"
+    assert np.array_equal(_bits(m_gpu.cpu().numpy()[:, :d]), _bits(m_cpu[:, :d])), f"{tag} residual"
+    assert np.array_equal(plan.debug_hist(), r.hist), f"{tag} histogram"
+    for l in range(plan.S):
+        beta, alpha, N, S1, S2 = plan.get_fit(l)
+        assert N == r.moments[l, 0], f"{tag} N"
+        np.testing.assert_allclose([S1, S2], r.moments[l, 1:], rtol=1e-12, err_msg=f"{tag} moments")
+        np.testing.assert_allclose([beta, alpha], r.fit[l], rtol=1e-5, err_msg=f"{tag} fit")
+    hdr = b.hdr_to_numpy(out["hdr"])
+    assert np.array_equal(hdr, r.hdr), f"{tag} header {hdr[hdr != r.hdr]} vs {r.hdr[hdr != r.hdr]}"
+    lens, codes = plan.debug_code()
+    assert np.array_equal(lens, r.lens), f"{tag} code lengths"
+    assert np.array_equal(codes, r.codes), f"{tag} codewords"
+    co = out["chunk_off"].cpu().numpy().view(np.uint32)
+    assert np.array_equal(co, r.chunk_off), f"{tag} chunk offsets"
+    assert np.array_equal(out["sub_bits"].cpu().numpy().view(np.uint16)[:, :plan.n_sub],
+                          r.sub_bits[:, :plan.n_sub]), f"{tag} sub_bits"
+    assert np.array_equal(out["user_bits"].cpu().numpy().view(np.uint64), r.user_bits), f"{tag} user_bits"
+    pay = out["bitstream"].cpu().numpy().view(np.uint32)
+    for u in range(U):
+        n = int(co[u, -1])
+        if n <= plan.cap_words:
+            assert np.array_equal(pay[u, :n], r.payload[u, :n]), f"{tag} bitstream user {u}"
+
+
+def run_case(b, oracle, d, U, E, M, off, grads, gamma=0.9, mode=1, cap=None, decode_plan=None):
+    """grads: list of [U][ld] float32 cuda tensors, one per iteration."""
+    plan = b.Plan(d, U, E, M, off, gamma=gamma, bias_mode=mode, cap_words=cap)
+    orc = oracle.OracleCO3(d, U, E, M, off, gamma=gamma, mode=mode, cap_words=plan.cap_words)
+    assert plan.worst_case_words == orc.worst_case_words
+    assert (plan.n_chunks, plan.n_sub) == (orc.part.n_chunks, orc.part.n_sub)
+    out = plan.alloc_outputs()
+    m_gpu = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+    m_cpu = np.zeros((U, plan.ld), np.float32)
+    dec = decode_plan or plan
+    results = []
+    for t, g in enumerate(grads):
+        g_cpu = g.cpu().numpy()
+        plan.encode(g, m_gpu, out)
+        r = orc.encode(g_cpu, m_cpu)
+        compare_iteration(b, plan, out, r, m_gpu, m_cpu, tag=f"t={t}")
+        flags, nf = plan.status()
+        assert nf == r.nonfinite or t > 0
+        if r.status == oracle.OK:
+            avg = dec.decode_aggregate(out).cpu().numpy()
+            rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+            assert rc == oracle.OK
+            assert np.array_equal(_bits(avg), _bits(avg_o)), f"t={t} averaged gradient"
+            assert not (dec.status()[0] & b.FLAG_CORRUPT)
+        results.append((r, flags))
+    return plan, orc, out, results
+
+
+def _grads(wl, iters, device="cuda"):
+    return [wl.gradient(t, device=device).to("cuda") for t in range(iters)]
+
+
+# --------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_configs_scaled_down(binding, oracle, idx):
+    """The four benchmark configurations at a size the oracle finishes in seconds: several
+    tiles, ragged tails, all their segments/users/formats, error feedback over iterations."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(idx, d={0: 70_001, 1: 200_000, 2: 150_010, 3: 300_007}[idx])
+    run_case(binding, oracle, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.seg_offsets,
+             _grads(wl, 4), gamma=wl.gamma)
+
+
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("U", [1, 2, 3, 5, 8, 9, 16])
+def test_users_and_formats(binding, oracle, E, M, U):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(20_000 + 37 * U, U, 1.0, E, M)
+    run_case(binding, oracle, wl.d, U, E, M, wl.seg_offsets, _grads(wl, 2, "cpu"))
+
+
+@pytest.mark.parametrize("beta", [0.5, 1.0, 2.0])
+def test_shapes_fp4(binding, oracle, beta):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 16, 8, beta, 1, 2)
+    run_case(binding, oracle, wl.d, 8, 1, 2, wl.seg_offsets, _grads(wl, 3, "cpu"))
+
+
+@pytest.mark.parametrize("gamma", [0.0, 1.0])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_gamma_and_bias_modes(binding, oracle, gamma, mode):
+    gen = torch.Generator().manual_seed(5)
+    d, U = 30_001, 3
+    ld = (d + 3) // 4 * 4
+    grads = []
+    for t in range(4):                                   # scale drifts: the modes differ for t >= 1
+        g = torch.zeros((U, ld))
+        g[:, :d] = torch.randn((U, d), generator=gen) * (1e-3 * 3.0 ** t)
+        grads.append(g.cuda())
+    run_case(binding, oracle, d, U, 3, 2, [0, 12_345, d], grads, gamma=gamma, mode=mode)
+
+
+def test_ragged_segments_and_tiny_inputs(binding, oracle):
+    gen = torch.Generator().manual_seed(6)
+    for d, off in ((1, [0, 1]), (5, [0, 2, 2, 5]), (130, [0, 1, 130]), (4097, [0, 4096, 4097]),
+                   (9000, [0, 5, 5, 4101, 8192, 9000]), (12_289, [0, 3, 127, 128, 129, 4095, 4097, 12_289])):
+        ld = (d + 3) // 4 * 4
+        grads = []
+        for t in range(2):
+            g = torch.zeros((2, ld))
+            g[:, :d] = torch.randn((2, d), generator=gen) * 1e-2
+            grads.append(g.cuda())
+        run_case(binding, oracle, d, 2, 4, 3, off, grads)
+
+
+def test_degenerate_values(binding, oracle):
+    """All-zero gradient, a constant segment, huge and subnormal values, signed zeros, ties."""
+    d = 6000
+    g = torch.zeros((2, d))
+    g[:, 1000:2000] = 3e-4                               # single-symbol histogram in segment 1
+    g[0, 2000:2008] = torch.tensor([1e30, -1e30, 2.0 ** -140, -0.0, 2.0 ** -127, 1e-38, -3e38, 1.0])
+    g[1, 2008:4000] = torch.linspace(-1, 1, 1992)
+    g[:, 4000:] = torch.arange(2000, dtype=torch.float32) * 2.0 ** -12   # many exact ties
+    off = [0, 1000, 2000, 4000, d]
+    for E, M in FORMATS:
+        run_case(binding, oracle, d, 2, E, M, off, [g.cuda(), (g * -0.5).cuda(), torch.zeros((2, d)).cuda()], gamma=1.0)
+
+
+def test_nonfinite_inputs(binding, oracle):
+    d = 5000
+    gen = torch.Generator().manual_seed(3)
+    g = torch.randn((2, d), generator=gen) * 1e-3
+    g[0, 7] = float("nan"); g[1, 4500] = float("inf"); g[1, 4501] = float("-inf")
+    plan, orc, out, res = run_case(binding, oracle, d, 2, 4, 3, [0, 4096, d], [g.cuda(), torch.zeros((2, d)).cuda()])
+    flags, nf = plan.status(clear=True)
+    assert flags & binding.FLAG_NONFINITE and nf == 3
+    assert plan.status() == (0, 0)
+
+
+def test_capacity_overflow_is_flagged_and_nothing_written(binding, oracle):
+    d, U = 20_000, 2
+    gen = torch.Generator().manual_seed(4)
+    g = (torch.randn((U, d), generator=gen) * 1e-3).cuda()
+    plan, orc, out, res = run_case(binding, oracle, d, U, 4, 3, None, [g], cap=1024)
+    r, flags = res[0]
+    assert r.status == oracle.ECAPACITY and flags & binding.FLAG_CAPACITY
+    assert not out["bitstream"].any().item()
+    assert int(out["chunk_off"][0, -1]) > 1024
+
+
+def test_corrupt_streams_are_flagged_not_faulting(binding, oracle):
+    d, U = 30_000, 3
+    gen = torch.Generator().manual_seed(8)
+    g = (torch.randn((U, d), generator=gen) * 1e-3).cuda()
+    plan, orc, out, res = run_case(binding, oracle, d, U, 4, 3, [0, 10_000, d], [g])
+    good = {k: v.clone() for k, v in out.items()}
+
+    def flagged(mut):
+        o = {k: v.clone() for k, v in good.items()}
+        mut(o)
+        plan.status(clear=True)
+        plan.decode_aggregate(o)
+        return bool(plan.status(clear=True)[0] & binding.FLAG_CORRUPT)
+
+    assert not flagged(lambda o: None)
+    assert flagged(lambda o: o["sub_bits"][1, 5].add_(1))
+    assert flagged(lambda o: o["chunk_off"][2, 3].add_(2))             # not a multiple of 4
+    assert flagged(lambda o: o["chunk_off"][0, 1:].fill_(2 ** 31 - 4))  # far outside the payload
+    assert flagged(lambda o: o["hdr"].copy_(binding.hdr_from_numpy(
+        binding.hdr_to_numpy(good["hdr"]) + np.array([0, 3, 0]))))      # another code model
+    assert flagged(lambda o: o["hdr"].fill_(0x7FFF7F7F))                # indices out of range
+    o = {k: v.clone() for k, v in good.items()}                        # random bytes: any outcome but a fault
+    o["bitstream"].random_(-2 ** 31, 2 ** 31 - 1)
+    plan.decode_aggregate(o)
+    torch.cuda.synchronize()
+    plan.status(clear=True)
+    assert np.array_equal(_bits(plan.decode_aggregate(good).cpu().numpy()),
+                          _bits(orc.decode_aggregate(res[0][0].payload, res[0][0].sub_bits,
+                                                     res[0][0].chunk_off, res[0][0].hdr)[1]))
+
+
+def test_decoder_depends_only_on_the_stream(binding, oracle):
+    """A second plan that never encoded anything (the parameter server) decodes the outputs."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=120_000, n_users=4)
+    server = binding.Plan(wl.d, 4, wl.exp_bits, wl.mant_bits, wl.seg_offsets)
+    run_case(binding, oracle, wl.d, 4, wl.exp_bits, wl.mant_bits, wl.seg_offsets, _grads(wl, 2),
+             decode_plan=server)
+
+
+def test_run_to_run_determinism_and_state_resume(binding, oracle):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(2, d=100_003, n_users=4)
+    grads = _grads(wl, 4)
+
+    def run(plan, m, ts):
+        outs = []
+        for t in ts:
+            out = plan.alloc_outputs()
+            plan.encode(grads[t], m, out)
+            plan.decode_aggregate(out)
+            outs.append({k: v.clone() for k, v in out.items()})
+        return outs
+
+    mk = lambda: binding.Plan(wl.d, 4, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma)
+    z = lambda p: torch.zeros((4, p.ld), device="cuda")
+    p1, p2 = mk(), mk()
+    m1, m2 = z(p1), z(p2)
+    a = run(p1, m1, range(4))
+    b2 = run(p2, m2, range(2))
+    it, nb = p2.state_export()
+    assert it == 2
+    p3 = mk()
+    p3.state_import(it, nb)                              # resume on a fresh plan with the saved memory
+    b2 += run(p3, m2, range(2, 4))
+    for x, y in zip(a, b2):
+        for k in x:
+            assert torch.equal(x[k], y[k]), k
+    assert torch.equal(m1, m2)
+
+
+def test_host_iteration_entry_point(binding, oracle):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(0, d=50_000, n_users=2)
+    plan = binding.Plan(wl.d, 2, 4, 3)
+    orc = oracle.OracleCO3(wl.d, 2, 4, 3, cap_words=plan.cap_words)
+    out = plan.alloc_outputs()
+    m = torch.zeros((2, plan.ld), device="cuda")
+    m_cpu = np.zeros((2, plan.ld), np.float32)
+    d_grad = torch.empty((2, plan.ld), device="cuda")
+    h_avg = torch.empty(wl.d).pin_memory()
+    for t in range(2):
+        h_grad = wl.gradient(t).pin_memory()
+        plan.iteration_host(h_grad, d_grad, m, out, h_avg)
+        torch.cuda.synchronize()
+        r = orc.encode(h_grad.numpy().copy(), m_cpu)
+        rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+        assert np.array_equal(_bits(h_avg.numpy()), _bits(avg_o))
+
+
+# ---- full sizes, in the launch configuration the benchmark times ---------------------------
+@pytest.mark.slow
+def test_config0_full(binding, oracle):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(0)
+    run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, wl.iters), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+def test_config1_full_two_iterations(binding, oracle):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1)
+    run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma)

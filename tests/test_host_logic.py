@@ -1,0 +1,93 @@
+"""CPU-only checks of the CUDA library's host side: it loads, exports what include/co3.h
+declares, rejects bad configurations before touching CUDA, and its two host-computed tables (the
+static partition and the GenNorm model-weight table) are identical to the oracle's own."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2203_09044_b200 import build, binding as b
+    build.build()
+    b.lib()
+    return b
+
+
+def test_library_exports_every_declared_symbol(binding):
+    header = open(os.path.join(ROOT, "include", "co3.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(co3_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    L = binding.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+    assert L.co3_strerror(0) == b"ok" and b"capacity" not in L.co3_strerror(-1)
+
+
+def test_bad_configurations_are_rejected_on_the_host(binding):
+    L = binding.lib()
+
+    def create(**kw):
+        base = dict(d=1000, ld=1000, n_users=2, E=4, M=3, gamma=0.9, mode=1, cap=4000, off=None)
+        base.update(kw)
+        off = None if base["off"] is None else np.asarray(base["off"], np.int64)
+        cfg = binding.Config(base["d"], base["ld"], base["n_users"], binding.Format(base["E"], base["M"]),
+                             0 if off is None else len(off) - 1,
+                             None if off is None else off.ctypes.data_as(C.POINTER(C.c_int64)),
+                             base["gamma"], base["mode"], base["cap"])
+        h = C.c_void_p()
+        rc = L.co3_plan_create(C.byref(h), C.byref(cfg))
+        if rc == 0:
+            L.co3_plan_destroy(h)
+        return rc
+
+    assert create(d=0) == binding.EINVAL
+    assert create(ld=998) == binding.EINVAL and create(ld=1002) == binding.EINVAL
+    assert create(E=5) == binding.EINVAL and create(M=0) == binding.EINVAL and create(E=4, M=4) == binding.EINVAL
+    assert create(n_users=0) == binding.EINVAL
+    assert create(n_users=69) == binding.EINVAL          # 69 * 245760 >= 2^24: sums not exact
+    assert create(cap=4001) == binding.EINVAL and create(cap=0) == binding.EINVAL
+    assert create(gamma=1.5) == binding.EINVAL and create(mode=7) == binding.EINVAL
+    assert create(off=[0, 600, 500, 1000]) == binding.EINVAL
+    assert create(off=[0, 500, 900]) == binding.EINVAL
+    try:
+        import torch
+        has_gpu = torch.cuda.is_available()
+    except Exception:
+        has_gpu = False
+    if not has_gpu:                                      # a valid plan needs a device: clean error
+        assert create() in (binding.ENOMEM, binding.ECUDA)
+
+
+@pytest.mark.parametrize("E,M", [(1, 2), (3, 2), (4, 3)])
+def test_model_weight_table_identical_to_oracle(binding, oracle, E, M):
+    """The code tables of both sides are built from these integers: they must agree exactly for
+    every header index pair."""
+    for ib in range(-14, 9):
+        for ir in range(-96, 32):
+            a = binding.model_weights(E, M, ib, ir)
+            b = oracle.model_weights(E, M, ib, ir)
+            assert np.array_equal(a, b), (ib, ir, np.nonzero(a != b))
+    with pytest.raises(binding.Co3Error):
+        binding.model_weights(E, M, 9, 0)
+
+
+def test_partition_identical_to_oracle(binding, oracle):
+    from paper_2203_09044_b200 import inputs
+    cases = [(10000, [0, 10000]), (9000, [0, 5, 5, 4101, 8192, 9000]), (130, [0, 1, 130]),
+             (1, [0, 1]), (4096, [0, 4096])]
+    w1, w2 = inputs.workload(1), inputs.workload(2)
+    cases += [(w1.d, w1.seg_offsets), (w2.d, w2.seg_offsets)]
+    for d, off in cases:
+        seg, st, en, sb, ns = binding.partition(d, off)
+        p = oracle.Partition(d, off)
+        assert ns == p.n_sub and len(seg) == p.n_chunks
+        n = p.n_chunks
+        assert np.array_equal(seg, p.chunk_seg[:n]) and np.array_equal(st, p.chunk_start[:n])
+        assert np.array_equal(en, p.chunk_end[:n]) and np.array_equal(sb, p.sub_base[:n])
