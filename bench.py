@@ -1,0 +1,337 @@
+#!/usr/bin/env python
+"""Benchmark of the CO3 gradient pipeline on B200.
+
+A step is one CO3 iteration of Algorithm 1 over one batch of synthetic gradients: co3_encode
+(error-feedback add, float conversion, residual update, histogram and moments, GenNorm fit,
+Huffman code build, bit packing) followed by co3_decode_aggregate (code rebuild from the header,
+decode of all users, average).  The workload is the 8-user ResNet-18-sized configuration
+(d = 11,173,962 per user, 62 layers, 8-bit format, gamma = 0.9, lagged bias).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Metric: GB/s of fp32 gradient consumed = 4 * d * U * steps / time, inputs resident in HBM.
+With N > 1 (torchrun) every rank runs an independent replica of the workload: the path has no
+exchange step, so there is no collective on the data path.
+"""
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "co3_encode_decode_fp32_gradient_throughput"
+UNIT = "GB/s"
+POOL = 4                      # distinct gradient batches cycled through (each > L2)
+# algorithmic bytes per user-element of the fused convert pass: read g, m (8), write m (4), symbol (1)
+CONVERT_BYTES_PER_ELEMENT = 13.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel on this workload,
+# from the ncu capture summarised in profiles/ (None until one has been taken)
+CONVERT_DRAM_TRAFFIC_BYTES = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (earlier pool measurement)"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake", 0x2: "applications_clocks_setting",
+               0x100: "display_clock_setting", 0x10: "sync_boost"}
+
+    def __init__(self, index, period=0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2203_09044_b200 import binding, inputs
+
+    binding.lib()                                      # no CUDA library -> raise, never fall back
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    wl = inputs.workload(1, n_users=args.users)
+    U, d = wl.n_users, wl.d
+    plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
+                        bias_mode=binding.BIAS_LAGGED)
+    out = plan.alloc_outputs()
+    residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+    # every rank draws its own users' gradients (seed offset by rank): a weak-scaling replica
+    wl.index = wl.index + 100 * rank
+    pool = [wl.gradient(t, device="cuda") for t in range(POOL)]
+    torch.cuda.synchronize()
+
+    def step(t):
+        plan.encode(pool[t % POOL], residual, out)
+        plan.decode_aggregate(out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        step(t)
+    barrier()
+    flags, _ = plan.status(clear=True)
+    assert flags == 0, f"status flags {flags} after warm-up"
+
+    # ---- timed region: K steps, the dominant kernel traced with CUDA events --------------------
+    plan.profile_enable(["convert"], max_records=args.steps)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    launches0 = plan.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    for t in range(args.steps):
+        step(args.warmup + t)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    elapsed_ms = e0.elapsed_time(e1)
+    launches = plan.launch_count() - launches0
+    conv_ms, conv_n = plan.profile_collect()["convert"]
+    flags, _ = plan.status(clear=True)
+    assert flags == 0, f"status flags {flags} in the timed region"
+    code_bits = float(out["user_bits"].sum().item()) / (U * d)
+    container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
+                      + 32.0 * U * (plan.n_chunks + 1) + 32.0 * plan.S) / (U * d)
+
+    if world > 1:
+        tmax = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tmax.item())
+
+    # ---- per-kernel breakdown: the same steps again with every kernel class traced -----------
+    nb = min(args.steps, 50)
+    plan.profile_enable(None, max_records=2 * nb + 4)
+    for t in range(nb):
+        step(args.warmup + args.steps + t)
+    breakdown = {k: {"ms_per_step": v[0] / nb, "launches_per_step": v[1] / nb}
+                 for k, v in plan.profile_collect().items() if v[1]}
+    plan.profile_enable([], 0)
+
+    # ---- end to end: host gradients in, host average out, through co3_iteration_host ---------
+    ne = min(args.steps, 20)
+    h_pool = [g.cpu().pin_memory() for g in pool[:2]]
+    h_avg = torch.empty(d, dtype=torch.float32).pin_memory()
+    d_grad = torch.empty((U, plan.ld), dtype=torch.float32, device="cuda")
+    for t in range(3):
+        plan.iteration_host(h_pool[t % 2], d_grad, residual, out, h_avg)
+    barrier()
+    e0.record()
+    for t in range(ne):
+        plan.iteration_host(h_pool[t % 2], d_grad, residual, out, h_avg)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        tmax = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+    flags, _ = plan.status(clear=True)
+    assert flags == 0
+
+    in_bytes = 4.0 * d * U
+    value = world * in_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9
+    e2e_value = world * in_bytes * ne / (e2e_ms * 1e-3) / 1e9
+    peak, peak_src = measured_peaks()
+    conv_avg_ms = conv_ms / max(conv_n, 1)
+    achieved = CONVERT_BYTES_PER_ELEMENT * U * d / (conv_avg_ms * 1e-3) / 1e9
+    step_bytes = (15.9 * U + 4.0) * d                 # all passes of one LAGGED iteration, E4M3
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "configs[1]: %d users x ResNet-18 (10-class head) gradient, d=11173962, "
+                               "62 layers, iid GenNorm(beta=0.8) per layer, E4M3, gamma=0.9, lagged bias" % U,
+                   "d": d, "n_users": U, "n_segments": plan.S, "format": "E4M3", "gamma": wl.gamma,
+                   "bias_mode": "lagged", "replicas": world,
+                   "l2": "inputs larger than L2: %d MB of gradient+memory read per step, %d gradient "
+                         "batches cycled" % (8 * U * d // 1000000, POOL)},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(4 * U * plan.ld),
+                "d2h_bytes_per_step": int(4 * d), "steps": ne, "ms_per_step": e2e_ms / ne,
+                "call": "co3_iteration_host (pinned host gradients in, host average out)"},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "ef_kernel<convert> (fused EF-add/convert/residual/histogram/moments)",
+                     "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src,
+                     "traffic": CONVERT_DRAM_TRAFFIC_BYTES,
+                     "algorithmic_bytes_per_launch": CONVERT_BYTES_PER_ELEMENT * U * d,
+                     "avg_launch_ms": conv_avg_ms, "launches_timed": conv_n,
+                     "timing": "cudaEvent pair around each launch on the launching stream, inside the timed region"},
+        "elements_per_s": world * U * d * args.steps / (elapsed_ms * 1e-3),
+        "bits_per_element": {"code": code_bits, "container": container_bits},
+        "whole_step_hbm": {"algorithmic_bytes_per_step": step_bytes,
+                           "achieved_GBps": step_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9,
+                           "frac_of_peak": step_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9 / peak},
+        "kernels": breakdown,
+    }
+    if rank == 0:
+        if not args.no_cpu_baseline:
+            result["cpu_baseline"] = cpu_baseline(wl_index=1, budget_s=25.0)
+        print(json.dumps(result), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def oracle_sample_step(orc, wl, g, m):
+    """One CO3 iteration of the oracle (encode + decode-aggregate) on host arrays."""
+    r = orc.encode(g, m)
+    rc, avg, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+    assert rc == 0
+    return r
+
+
+def cpu_baseline(wl_index, budget_s):
+    """The oracle as it stands, single-threaded, on a bounded sample of the same workload."""
+    import numpy as np
+    from oracle import co3_oracle
+    from paper_2203_09044_b200 import inputs
+    full = inputs.workload(wl_index)
+    per_elem = 2.0e-7                                   # rough oracle cost per user-element
+    users = max(1, min(full.n_users, int(budget_s / (per_elem * full.d))))
+    wl = inputs.workload(wl_index, n_users=users)
+    g = wl.gradient(0).numpy()
+    m = np.zeros_like(g)
+    orc = co3_oracle.OracleCO3(wl.d, users, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma)
+    t0 = time.perf_counter()
+    oracle_sample_step(orc, wl, g, m)
+    dt = time.perf_counter() - t0
+    return {"value": 4.0 * wl.d * users / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"1 iteration (encode + decode-aggregate) of {users} of the {full.n_users} users "
+                      f"at full d={wl.d}, {dt:.1f} s",
+            "host_cores_available": os.cpu_count()}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle timed on this machine's host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import co3_oracle
+    from paper_2203_09044_b200 import inputs
+    full = inputs.workload(1)
+    total = max(1, args.steps + args.warmup)
+    per_elem = 2.0e-7
+    n = int(min(full.n_users * full.d, max(65536, 150.0 / (total * per_elem))))   # user-elements per step
+    users = max(1, min(full.n_users, n // 65536, 8))
+    d_s = max(4096, min(full.d, n // users))
+    wl = inputs.workload(1, d=None if d_s >= full.d else d_s, n_users=users)
+    orc = co3_oracle.OracleCO3(wl.d, users, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma)
+    grads = [wl.gradient(t).numpy() for t in range(2)]
+    m = np.zeros_like(grads[0])
+    for t in range(args.warmup):
+        oracle_sample_step(orc, wl, grads[t % 2], m)
+    t0 = time.perf_counter()
+    for t in range(args.steps):
+        oracle_sample_step(orc, wl, grads[t % 2], m)
+    dt = time.perf_counter() - t0
+    value = 4.0 * wl.d * users * args.steps / dt / 1e9
+    sample = (f"each step = 1 iteration (encode + decode-aggregate) on {users} users x d={wl.d} of the "
+              f"workload's {full.n_users} x {full.d} (same 62-layer size mix)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "configs[1] (8 users x ResNet-18 gradient, E4M3, gamma=0.9), sampled",
+                   "d": wl.d, "n_users": users},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--users", type=int, default=None,
+                    help="override the number of simulated users (profiling a smaller case); default 8")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -145,6 +145,26 @@ int co3_get_fit(co3_plan* plan, int32_t seg, double* beta, double* alpha, double
 int co3_state_export(co3_plan* plan, int64_t* iteration, int32_t* next_bias);
 int co3_state_import(co3_plan* plan, int64_t iteration, const int32_t* next_bias);
 
+/* Tracing: per-kernel device time measured with CUDA events recorded on the caller's stream
+ * around the launches of the selected kernel classes.  co3_profile_enable creates the events
+ * (max_records launches per class between two collects; mask 0 frees them);
+ * co3_profile_collect synchronises, adds up the recorded launches of each class since the last
+ * collect (total_ms and launches are host arrays of CO3_NUM_KERNELS entries) and starts over.
+ * co3_launch_count: number of the library's kernels launched on this plan so far. */
+#define CO3_K_STATS 0        /* moments of g + gamma m (t = 0, or every t in CURRENT mode) */
+#define CO3_K_FIT 1          /* GenNorm fit, bias, header                                   */
+#define CO3_K_CONVERT 2      /* fused EF-add / convert / residual / histogram / moments      */
+#define CO3_K_CODE_ENC 3     /* Huffman code build, user side                                */
+#define CO3_K_ENC_LEN 4      /* code lengths -> sub-chunk bits, chunk words                  */
+#define CO3_K_ENC_SCAN 5     /* chunk offsets                                                */
+#define CO3_K_ENC_PACK 6     /* bit packing                                                  */
+#define CO3_K_CODE_DEC 7     /* Huffman code + decode tables, server side                    */
+#define CO3_K_DECODE 8       /* decode + aggregate                                           */
+#define CO3_NUM_KERNELS 9
+int co3_profile_enable(co3_plan* plan, uint32_t kernel_mask, int32_t max_records);
+int co3_profile_collect(co3_plan* plan, double* total_ms, int64_t* launches);
+int64_t co3_launch_count(const co3_plan* plan);
+
 /* Inspection hooks (synchronise; used by the parity tests).
  * symbols: device out [U][d] u8, the converted symbols of the last iteration
  *          (sign << (E+M) | exponent << M | mantissa).

@@ -20,8 +20,11 @@ EXPORTS = [
     "co3_plan_create", "co3_plan_destroy", "co3_sizes", "co3_encode", "co3_decode_aggregate",
     "co3_iteration_host", "co3_status", "co3_get_fit", "co3_state_export", "co3_state_import",
     "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
-    "co3_strerror",
+    "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
 ]
+
+KERNEL_NAMES = ["stats", "fit", "convert", "code_enc", "enc_len", "enc_scan", "enc_pack", "code_dec",
+                "decode"]
 
 
 class Format(C.Structure):
@@ -84,6 +87,12 @@ def lib():
     L.co3_model_weights.argtypes = [Format, C.c_int32, C.c_int32, vp]
     L.co3_partition.restype = C.c_int64
     L.co3_partition.argtypes = [C.c_int64, C.c_int32, vp, vp, vp, vp, vp, i64p]
+    L.co3_profile_enable.restype = C.c_int
+    L.co3_profile_enable.argtypes = [vp, C.c_uint32, C.c_int32]
+    L.co3_profile_collect.restype = C.c_int
+    L.co3_profile_collect.argtypes = [vp, vp, vp]
+    L.co3_launch_count.restype = C.c_int64
+    L.co3_launch_count.argtypes = [vp]
     L.co3_strerror.restype = C.c_char_p
     L.co3_strerror.argtypes = [C.c_int]
     _lib = L
@@ -226,6 +235,28 @@ class Plan:
         rc = lib().co3_state_import(self.handle, int(iteration), nb.ctypes.data)
         if rc != OK:
             raise Co3Error(rc, "co3_state_import")
+
+    def profile_enable(self, kernel_names=None, max_records=4096):
+        """Trace the named kernel classes (all if None; [] switches tracing off)."""
+        names = KERNEL_NAMES if kernel_names is None else kernel_names
+        mask = 0
+        for n in names:
+            mask |= 1 << KERNEL_NAMES.index(n)
+        rc = lib().co3_profile_enable(self.handle, mask, max_records)
+        if rc != OK:
+            raise Co3Error(rc, "co3_profile_enable")
+
+    def profile_collect(self):
+        """{kernel class: (total ms, launches)} since the last collect (synchronises)."""
+        ms = np.zeros(len(KERNEL_NAMES), np.float64)
+        n = np.zeros(len(KERNEL_NAMES), np.int64)
+        rc = lib().co3_profile_collect(self.handle, ms.ctypes.data, n.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_profile_collect")
+        return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_NAMES)}
+
+    def launch_count(self):
+        return int(lib().co3_launch_count(self.handle))
 
     def debug_symbols(self, stream=None):
         t = self.torch

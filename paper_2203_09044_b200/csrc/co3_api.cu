@@ -47,6 +47,8 @@ bool g_kernels_ready = false;
 
 }  // namespace
 
+#define CO3_SYNC_OR_FAIL(pl) do { if (cudaStreamSynchronize((pl)->last_stream) != cudaSuccess) { (void)cudaGetLastError(); return CO3_ECUDA; } } while (0)
+
 extern "C" const char* co3_strerror(int code) {
     switch (code) {
         case CO3_OK: return "ok";
@@ -60,8 +62,53 @@ extern "C" const char* co3_strerror(int code) {
     }
 }
 
+static void free_events(co3_plan* pl) {
+    if (pl->prof_ev) {
+        for (size_t i = 0; i < (size_t)CO3_NUM_KERNELS * pl->prof_cap * 2; ++i) cudaEventDestroy(pl->prof_ev[i]);
+        free(pl->prof_ev);
+    }
+    pl->prof_ev = nullptr; pl->prof_cap = 0; pl->prof_mask = 0;
+    memset(pl->prof_n, 0, sizeof(pl->prof_n));
+}
+
+extern "C" int co3_profile_enable(co3_plan* pl, uint32_t kernel_mask, int32_t max_records) {
+    if (!pl || max_records < 0 || max_records > (1 << 20)) return CO3_EINVAL;
+    CO3_SYNC_OR_FAIL(pl);
+    free_events(pl);
+    if (!kernel_mask || !max_records) return CO3_OK;
+    const size_t n = (size_t)CO3_NUM_KERNELS * max_records * 2;
+    pl->prof_ev = (cudaEvent_t*)calloc(n, sizeof(cudaEvent_t));
+    if (!pl->prof_ev) return CO3_ENOMEM;
+    pl->prof_cap = max_records;
+    for (size_t i = 0; i < n; ++i)
+        if (cudaEventCreate(&pl->prof_ev[i]) != cudaSuccess) { (void)cudaGetLastError(); free_events(pl); return CO3_ECUDA; }
+    pl->prof_mask = kernel_mask;
+    return CO3_OK;
+}
+
+extern "C" int co3_profile_collect(co3_plan* pl, double* total_ms, int64_t* launches) {
+    if (!pl || !total_ms || !launches) return CO3_EINVAL;
+    CO3_SYNC_OR_FAIL(pl);
+    for (int k = 0; k < CO3_NUM_KERNELS; ++k) {
+        double tot = 0.0;
+        for (int i = 0; i < pl->prof_n[k]; ++i) {
+            float ms = 0.0f;
+            const size_t o = ((size_t)k * pl->prof_cap + i) * 2;
+            if (cudaEventElapsedTime(&ms, pl->prof_ev[o], pl->prof_ev[o + 1]) != cudaSuccess) { (void)cudaGetLastError(); return CO3_ECUDA; }
+            tot += ms;
+        }
+        total_ms[k] = tot;
+        launches[k] = pl->prof_n[k];
+        pl->prof_n[k] = 0;
+    }
+    return CO3_OK;
+}
+
+extern "C" int64_t co3_launch_count(const co3_plan* pl) { return pl ? pl->launches : 0; }
+
 extern "C" void co3_plan_destroy(co3_plan* pl) {
     if (!pl) return;
+    free_events(pl);
     for (int i = 0; i < pl->n_allocs; ++i) cudaFree(pl->allocs[i]);
     free(pl->h_seg_off);
     delete pl;

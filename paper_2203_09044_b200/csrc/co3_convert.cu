@@ -193,14 +193,18 @@ static int ef_grid(const co3_plan* pl, int which) {
     return (int)(items < grid ? items : grid);
 }
 
-cudaError_t co3_launch_stats(const co3_plan* pl, const float* g, const float* m, cudaStream_t st) {
+cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st) {
+    co3_prof_begin(pl, CO3_K_STATS, st);
     ef_kernel<false><<<ef_grid(pl, 0), CO3_THREADS, 0, st>>>(pl->dev, g, const_cast<float*>(m));
+    co3_prof_end(pl, CO3_K_STATS, st, 1);
     return cudaGetLastError();
 }
 
-cudaError_t co3_launch_convert(const co3_plan* pl, const float* g, float* m, cudaStream_t st) {
+cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st) {
     cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * (size_t)pl->dev.S * CO3_MAXSYM, st);
     if (e != cudaSuccess) return e;
+    co3_prof_begin(pl, CO3_K_CONVERT, st);
     ef_kernel<true><<<ef_grid(pl, 1), CO3_THREADS, 0, st>>>(pl->dev, g, m);
+    co3_prof_end(pl, CO3_K_CONVERT, st, 1);
     return cudaGetLastError();
 }

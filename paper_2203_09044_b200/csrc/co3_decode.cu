@@ -305,10 +305,11 @@ cudaError_t co3_setup_decode_kernels(void) {
                                 (int)sizeof(SmemB));
 }
 
-cudaError_t co3_launch_decode(const co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
                               cudaStream_t st) {
     const Co3Dev& p = pl->dev;
+    co3_prof_begin(pl, CO3_K_DECODE, st);
     if (p.U <= NW) {
         const size_t smem = smem_a_bytes(p.U);
         int bpsm = 0;
@@ -326,5 +327,6 @@ cudaError_t co3_launch_decode(const co3_plan* pl, const uint32_t* bitstream, con
         decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), CO3_THREADS, sizeof(SmemB), st>>>(
             p, pl->cb_dec, bitstream, sub_bits, chunk_off, hdr, avg);
     }
+    co3_prof_end(pl, CO3_K_DECODE, st, 1);
     return cudaGetLastError();
 }

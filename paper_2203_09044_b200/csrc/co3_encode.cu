@@ -221,7 +221,7 @@ cudaError_t co3_setup_kernels(void) {
                                 (CO3_MAXSYM * 32 + BUF_WORDS + 4) * (int)sizeof(uint32_t));
 }
 
-cudaError_t co3_launch_encode(const co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
+cudaError_t co3_launch_encode(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
                               uint32_t* chunk_off, unsigned long long* user_bits, cudaStream_t st) {
     const Co3Dev& p = pl->dev;
     const int64_t items = p.n_chunks * (int64_t)p.U;
@@ -232,9 +232,13 @@ cudaError_t co3_launch_encode(const co3_plan* pl, uint32_t* bitstream, uint16_t*
         if (g_len_bpsm < 1) g_len_bpsm = 1;
     }
     int64_t grid = (int64_t)pl->num_sms * g_len_bpsm;
+    co3_prof_begin(pl, CO3_K_ENC_LEN, st);
     enc_len_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, 0, st>>>(p, pl->cb_enc, sub_bits, user_bits);
+    co3_prof_end(pl, CO3_K_ENC_LEN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
     enc_scan_kernel<<<p.U, 1024, 0, st>>>(p, chunk_off);
+    co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const size_t smem = ((size_t)p.nsym * 32 + BUF_WORDS + 4) * sizeof(uint32_t);
     const int fi = p.nsym == 256 ? 0 : (p.nsym == 128 ? 1 : (p.nsym == 64 ? 2 : 3));
@@ -243,6 +247,8 @@ cudaError_t co3_launch_encode(const co3_plan* pl, uint32_t* bitstream, uint16_t*
         if (g_pack_bpsm[fi] < 1) g_pack_bpsm[fi] = 1;
     }
     grid = (int64_t)pl->num_sms * g_pack_bpsm[fi];
+    co3_prof_begin(pl, CO3_K_ENC_PACK, st);
     enc_pack_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, smem, st>>>(p, pl->cb_enc, chunk_off, bitstream);
+    co3_prof_end(pl, CO3_K_ENC_PACK, st, 1);
     return cudaGetLastError();
 }

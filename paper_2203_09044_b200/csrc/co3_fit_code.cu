@@ -271,17 +271,24 @@ code_finalize_kernel(Co3Dev p, Co3CodeBook cb, int want_decode) {
 
 }  // namespace
 
-cudaError_t co3_launch_fit(const co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
+cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
+    co3_prof_begin(pl, CO3_K_FIT, st);
     fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr);
+    co3_prof_end(pl, CO3_K_FIT, st, 1);
     return cudaGetLastError();
 }
 
-cudaError_t co3_launch_codebook(const co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
+cudaError_t co3_launch_codebook(co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
                                 int want_decode_tables, cudaStream_t st) {
+    const int k = want_decode_tables ? CO3_K_CODE_DEC : CO3_K_CODE_ENC;
     dim3 grid(pl->dev.S, CO3_NCAND);
+    co3_prof_begin(pl, k, st);
     huff_cand_kernel<<<grid, CO3_MAXSYM, 0, st>>>(pl->dev, cb, hdr);
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    code_finalize_kernel<<<pl->dev.S, CO3_MAXSYM, 0, st>>>(pl->dev, cb, want_decode_tables);
-    return cudaGetLastError();
+    if (e == cudaSuccess) {
+        code_finalize_kernel<<<pl->dev.S, CO3_MAXSYM, 0, st>>>(pl->dev, cb, want_decode_tables);
+        e = cudaGetLastError();
+    }
+    co3_prof_end(pl, k, st, 2);
+    return e;
 }

@@ -89,7 +89,30 @@ struct co3_plan {
     void* allocs[64];
     int n_allocs;
     int64_t* h_seg_off;
+    // tracing
+    uint32_t prof_mask;
+    int prof_cap;
+    int prof_n[CO3_NUM_KERNELS];
+    cudaEvent_t* prof_ev;         // [CO3_NUM_KERNELS][prof_cap][2]
+    int64_t launches;
 };
+
+// Event pair around the launches of kernel class k (no-ops unless the class is being traced).
+inline void co3_prof_begin(co3_plan* pl, int k, cudaStream_t st) {
+    if ((pl->prof_mask >> k) & 1u) {
+        if (pl->prof_n[k] < pl->prof_cap)
+            cudaEventRecord(pl->prof_ev[((size_t)k * pl->prof_cap + pl->prof_n[k]) * 2], st);
+    }
+}
+inline void co3_prof_end(co3_plan* pl, int k, cudaStream_t st, int n_launches) {
+    pl->launches += n_launches;
+    if ((pl->prof_mask >> k) & 1u) {
+        if (pl->prof_n[k] < pl->prof_cap) {
+            cudaEventRecord(pl->prof_ev[((size_t)k * pl->prof_cap + pl->prof_n[k]) * 2 + 1], st);
+            pl->prof_n[k]++;
+        }
+    }
+}
 
 // host-side helpers (co3_model.cu)
 int co3_host_fmt_ok(co3_format f);
@@ -98,14 +121,14 @@ int64_t co3_host_K(int M, int j);
 const uint32_t* co3_host_weight_table(int E, int M);   // [NIBETA][NIR][J], cached per format
 
 // kernel launchers (each returns a cudaError_t from the launch)
-cudaError_t co3_launch_stats(const co3_plan* pl, const float* g, const float* m, cudaStream_t st);
-cudaError_t co3_launch_convert(const co3_plan* pl, const float* g, float* m, cudaStream_t st);
-cudaError_t co3_launch_fit(const co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
-cudaError_t co3_launch_codebook(const co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
+cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st);
+cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st);
+cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
+cudaError_t co3_launch_codebook(co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
                                 int want_decode_tables, cudaStream_t st);
-cudaError_t co3_launch_encode(const co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
+cudaError_t co3_launch_encode(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
                               uint32_t* chunk_off, unsigned long long* user_bits, cudaStream_t st);
-cudaError_t co3_launch_decode(const co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
                               cudaStream_t st);
 cudaError_t co3_setup_kernels(void);
