@@ -88,7 +88,9 @@ typedef struct {
 
 /* Algorithm 1 line 2 and Table I: fixes d, U, the format, the layers, gamma.  Validates the
  * configuration, computes the static chunk partition, builds the GenNorm model-weight table on
- * the host and allocates all device scratch on the current device.  The iteration counter
+ * the host, allocates all device scratch on the current device and builds there, once, the
+ * Huffman code (Sec. III (ii)) of every (shape, scale) pair a header can name, so that an
+ * iteration only selects codes.  The iteration counter
  * starts at 0 (memory m_0 = 0 is the caller's zero-filled `residual`). */
 int co3_plan_create(co3_plan** out, const co3_config* cfg);
 void co3_plan_destroy(co3_plan* plan);
@@ -154,11 +156,11 @@ int co3_state_import(co3_plan* plan, int64_t iteration, const int32_t* next_bias
 #define CO3_K_STATS 0        /* moments of g + gamma m (t = 0, or every t in CURRENT mode) */
 #define CO3_K_FIT 1          /* GenNorm fit, bias, header                                   */
 #define CO3_K_CONVERT 2      /* fused EF-add / convert / residual / histogram / moments      */
-#define CO3_K_CODE_ENC 3     /* Huffman code build, user side                                */
+#define CO3_K_CODE_ENC 3     /* (unused: codes are built once at plan creation)              */
 #define CO3_K_ENC_LEN 4      /* code lengths -> sub-chunk bits, chunk words                  */
 #define CO3_K_ENC_SCAN 5     /* chunk offsets                                                */
 #define CO3_K_ENC_PACK 6     /* bit packing                                                  */
-#define CO3_K_CODE_DEC 7     /* Huffman code + decode tables, server side                    */
+#define CO3_K_CODE_DEC 7     /* (unused: codes are built once at plan creation)              */
 #define CO3_K_DECODE 8       /* decode + aggregate                                           */
 #define CO3_NUM_KERNELS 9
 int co3_profile_enable(co3_plan* plan, uint32_t kernel_mask, int32_t max_records);
@@ -170,10 +172,11 @@ int64_t co3_launch_count(const co3_plan* plan);
  *          (sign << (E+M) | exponent << M | mantissa).
  * hist:    host out [n_segments][2^(1+E+M)] u64, symbol counts pooled over users.
  * code:    host out, lengths [n_segments][2^B] u8 and codewords [n_segments][2^B] u32 (root bit
- *          = most significant of `length` bits) of the last encode. */
+ *          = most significant of `length` bits) of the codes that the headers `hdr` (device,
+ *          [n_segments]) select. */
 int co3_debug_symbols(co3_plan* plan, uint8_t* symbols, void* cuda_stream);
 int co3_debug_hist(co3_plan* plan, uint64_t* hist);
-int co3_debug_code(co3_plan* plan, uint8_t* lengths, uint32_t* codewords);
+int co3_debug_code(co3_plan* plan, const co3_seg_header* hdr, uint8_t* lengths, uint32_t* codewords);
 
 /* Host only, no GPU needed: integer model weights of the quantised GenNorm source for header
  * indices (ibeta in [-14, 8], ir in [-96, 31]), one per symbol byte, 2^(1+E+M) entries.  The

@@ -82,7 +82,7 @@ def lib():
     L.co3_debug_hist.restype = C.c_int
     L.co3_debug_hist.argtypes = [vp, vp]
     L.co3_debug_code.restype = C.c_int
-    L.co3_debug_code.argtypes = [vp, vp, vp]
+    L.co3_debug_code.argtypes = [vp, vp, vp, vp]
     L.co3_model_weights.restype = C.c_int
     L.co3_model_weights.argtypes = [Format, C.c_int32, C.c_int32, vp]
     L.co3_partition.restype = C.c_int64
@@ -273,10 +273,10 @@ class Plan:
             raise Co3Error(rc, "co3_debug_hist")
         return h
 
-    def debug_code(self):
+    def debug_code(self, hdr):
         ln = np.zeros((self.S, self.nsym), np.uint8)
         cw = np.zeros((self.S, self.nsym), np.uint32)
-        rc = lib().co3_debug_code(self.handle, ln.ctypes.data, cw.ctypes.data)
+        rc = lib().co3_debug_code(self.handle, _ptr(hdr), ln.ctypes.data, cw.ctypes.data)
         if rc != OK:
             raise Co3Error(rc, "co3_debug_code")
         return ln, cw

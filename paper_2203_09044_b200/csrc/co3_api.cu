@@ -25,19 +25,20 @@ int dev_alloc(co3_plan* pl, T** out, size_t count) {
     return CO3_OK;
 }
 
-int alloc_codebook(co3_plan* pl, Co3CodeBook& cb, int S) {
+int alloc_codebook(co3_plan* pl, Co3CodeBook& cb) {
+    const size_t R = CO3_NROWS;
     int rc = 0;
-    rc |= dev_alloc(pl, &cb.cand_len, (size_t)S * CO3_NCAND * CO3_MAXSYM);
-    rc |= dev_alloc(pl, &cb.cand_max, (size_t)S * CO3_NCAND);
-    rc |= dev_alloc(pl, &cb.len8, (size_t)S * CO3_MAXSYM);
-    rc |= dev_alloc(pl, &cb.enc, (size_t)S * CO3_MAXSYM);
-    rc |= dev_alloc(pl, &cb.code_msb, (size_t)S * CO3_MAXSYM);
-    rc |= dev_alloc(pl, &cb.lut, (size_t)S * CO3_LUT_SIZE);
-    rc |= dev_alloc(pl, &cb.first, (size_t)S * (CO3_MAXLEN + 1));
-    rc |= dev_alloc(pl, &cb.count, (size_t)S * (CO3_MAXLEN + 1));
-    rc |= dev_alloc(pl, &cb.offs, (size_t)S * (CO3_MAXLEN + 1));
-    rc |= dev_alloc(pl, &cb.perm, (size_t)S * CO3_MAXSYM);
-    rc |= dev_alloc(pl, &cb.ksign, (size_t)S * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.cand_len, R * CO3_NCAND * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.cand_max, R * CO3_NCAND);
+    rc |= dev_alloc(pl, &cb.len8, R * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.enc, R * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.code_msb, R * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.lut, R * CO3_LUT_SIZE);
+    rc |= dev_alloc(pl, &cb.first, R * (CO3_MAXLEN + 1));
+    rc |= dev_alloc(pl, &cb.count, R * (CO3_MAXLEN + 1));
+    rc |= dev_alloc(pl, &cb.offs, R * (CO3_MAXLEN + 1));
+    rc |= dev_alloc(pl, &cb.perm, R * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.ksign, (size_t)CO3_MAXSYM);
     return rc ? CO3_ENOMEM : CO3_OK;
 }
 
@@ -154,7 +155,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
     int32_t* h_seg_chunk0 = (int32_t*)malloc(sizeof(int32_t) * (size_t)(S + 1));
     Co3Group* h_groups = (Co3Group*)calloc((size_t)nc, sizeof(Co3Group));
     const uint32_t* wtab = co3_host_weight_table(E, M);
-    if (!h_chunks || !h_seg || !h_start || !h_end || !h_sub || !h_seg_chunk0 || !h_groups || !wtab) rc = CO3_ENOMEM;
+    const double* logr = co3_host_logr_table();
+    if (!h_chunks || !h_seg || !h_start || !h_end || !h_sub || !h_seg_chunk0 || !h_groups || !wtab || !logr) rc = CO3_ENOMEM;
 
     int64_t n_groups = 0, worst = 0;
     if (rc == CO3_OK) {
@@ -201,7 +203,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         pl->worst_case_words = worst;
 
         Co3Chunk* d_chunks = nullptr; Co3Group* d_groups = nullptr; int64_t* d_seg_off = nullptr;
-        int32_t* d_seg_chunk0 = nullptr; uint32_t* d_wtab = nullptr;
+        int32_t* d_seg_chunk0 = nullptr; uint32_t* d_wtab = nullptr; double* d_logr = nullptr;
         const size_t items = (size_t)nc * (size_t)dv.U;
         int a = 0;
         a |= dev_alloc(pl, &d_chunks, (size_t)nc);
@@ -209,6 +211,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &d_seg_off, (size_t)S + 1);
         a |= dev_alloc(pl, &d_seg_chunk0, (size_t)S + 1);
         a |= dev_alloc(pl, &d_wtab, (size_t)CO3_NIBETA * CO3_NIR * J);
+        a |= dev_alloc(pl, &d_logr, (size_t)CO3_FIT_GRID + 1);
         a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
         a |= dev_alloc(pl, &dv.hist, (size_t)S * CO3_MAXSYM);
         a |= dev_alloc(pl, &dv.part_s1, items);
@@ -220,8 +223,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);
-        a |= alloc_codebook(pl, pl->cb_enc, S);
-        a |= alloc_codebook(pl, pl->cb_dec, S);
+        a |= alloc_codebook(pl, dv.cb);
         if (a) rc = CO3_ENOMEM;
         if (rc == CO3_OK) {
             cudaError_t e = cudaSuccess;
@@ -233,6 +235,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             up(d_seg_off, pl->h_seg_off, sizeof(int64_t) * (size_t)(S + 1));
             up(d_seg_chunk0, h_seg_chunk0, sizeof(int32_t) * (size_t)(S + 1));
             up(d_wtab, wtab, sizeof(uint32_t) * (size_t)CO3_NIBETA * CO3_NIR * J);
+            up(d_logr, logr, sizeof(double) * ((size_t)CO3_FIT_GRID + 1));
             if (e == cudaSuccess) e = cudaMemset(dv.flags, 0, sizeof(uint32_t));
             if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
             if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);
@@ -246,7 +249,13 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             }
             if (e != cudaSuccess) { (void)cudaGetLastError(); rc = CO3_ECUDA; }
             dv.chunks = d_chunks; dv.groups = d_groups; dv.seg_off = d_seg_off;
-            dv.seg_chunk0 = d_seg_chunk0; dv.wtab = d_wtab;
+            dv.seg_chunk0 = d_seg_chunk0; dv.wtab = d_wtab; dv.logr_tab = d_logr;
+            if (rc == CO3_OK) {                      // Huffman codes of all model rows, once
+                if (co3_build_codebook(pl, 0) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    rc = CO3_ECUDA;
+                }
+            }
         }
     }
     free(h_chunks); free(h_seg); free(h_start); free(h_end); free(h_sub); free(h_seg_chunk0); free(h_groups);
@@ -278,8 +287,7 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
     }
     CO3_TRY(co3_launch_convert(pl, grad, residual, st));
     CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
-    CO3_TRY(co3_launch_codebook(pl, pl->cb_enc, hdr, 0, st));
-    CO3_TRY(co3_launch_encode(pl, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
+    CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;
     return CO3_OK;
 }
@@ -291,7 +299,6 @@ extern "C" int co3_decode_aggregate(co3_plan* pl, const uint32_t* bitstream, con
     if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
-    CO3_TRY(co3_launch_codebook(pl, pl->cb_dec, hdr, 1, st));
     CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, st));
     return CO3_OK;
 }
@@ -378,13 +385,25 @@ extern "C" int co3_debug_hist(co3_plan* pl, uint64_t* hist) {
     return CO3_OK;
 }
 
-extern "C" int co3_debug_code(co3_plan* pl, uint8_t* lengths, uint32_t* codewords) {
-    if (!pl || !lengths || !codewords) return CO3_EINVAL;
+extern "C" int co3_debug_code(co3_plan* pl, const co3_seg_header* hdr, uint8_t* lengths, uint32_t* codewords) {
+    if (!pl || !hdr || !lengths || !codewords) return CO3_EINVAL;
     CO3_TRY(cudaStreamSynchronize(pl->last_stream));
-    CO3_TRY(cudaMemcpy2D(lengths, (size_t)pl->dev.nsym, pl->cb_enc.len8, CO3_MAXSYM, (size_t)pl->dev.nsym,
-                         (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
-    CO3_TRY(cudaMemcpy2D(codewords, sizeof(uint32_t) * (size_t)pl->dev.nsym, pl->cb_enc.code_msb,
-                         sizeof(uint32_t) * CO3_MAXSYM, sizeof(uint32_t) * (size_t)pl->dev.nsym,
-                         (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
-    return CO3_OK;
+    const int S = pl->dev.S, nsym = pl->dev.nsym;
+    co3_seg_header* h = (co3_seg_header*)malloc(sizeof(co3_seg_header) * (size_t)S);
+    if (!h) return CO3_ENOMEM;
+    int rc = CO3_OK;
+    if (cudaMemcpy(h, hdr, sizeof(co3_seg_header) * (size_t)S, cudaMemcpyDeviceToHost) != cudaSuccess) rc = CO3_ECUDA;
+    for (int l = 0; l < S && rc == CO3_OK; ++l) {
+        bool bad = false;
+        const size_t row = (size_t)co3_row_of(h[l], &bad);
+        if (bad) { rc = CO3_ECORRUPT; break; }
+        if (cudaMemcpy(lengths + (size_t)l * nsym, pl->dev.cb.len8 + row * CO3_MAXSYM, (size_t)nsym,
+                       cudaMemcpyDeviceToHost) != cudaSuccess ||
+            cudaMemcpy(codewords + (size_t)l * nsym, pl->dev.cb.code_msb + row * CO3_MAXSYM,
+                       sizeof(uint32_t) * (size_t)nsym, cudaMemcpyDeviceToHost) != cudaSuccess)
+            rc = CO3_ECUDA;
+    }
+    free(h);
+    if (rc == CO3_ECUDA) (void)cudaGetLastError();
+    return rc;
 }

@@ -10,8 +10,8 @@
 // traffic is fully coalesced.
 //
 // Two variants: U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
-// per sub-chunk (small accumulator, several chunks per block when U < 8); U > 8 keeps a whole
-// chunk accumulator and loops over user groups.
+// per sub-chunk (small double-buffered accumulator, several chunks per block when U < 8); U > 8
+// keeps a whole chunk accumulator and loops over user groups.
 //
 // Bound: HBM for U = 1 (4 B written per element); for U >= 4 the serial decode (issue slots and
 // shared-memory look-ups per symbol) dominates.
@@ -21,24 +21,30 @@ namespace {
 
 constexpr int NW = CO3_THREADS / 32;              // warps = concurrent streams per block
 constexpr int PADW = 33;                          // row stride of the transposed accumulator
+// A lane never reads more than 128 * 16 bits past the start of its sub-chunk, so with this much
+// slack after the staged words the staged reader needs no bounds checks.
+constexpr int STAGE_PAD = 72;
+constexpr int STAGE_ROW = CO3_STAGE_WORDS + STAGE_PAD;
+static_assert(STAGE_ROW % 4 == 0, "stage rows must keep 16-byte alignment");
 
 struct Tables {                                   // per-segment decoder tables in shared memory
-    uint32_t lut[CO3_LUT_SIZE];
+    alignas(16) uint32_t lut[CO3_LUT_SIZE];
     uint32_t first[CO3_MAXLEN + 1], count[CO3_MAXLEN + 1], offs[CO3_MAXLEN + 1];
     int32_t ksign[CO3_MAXSYM];
     uint8_t perm[CO3_MAXSYM];
 };
 
-__device__ void load_tables(Tables& t, const Co3CodeBook& cb, int seg, int nsym, int tid) {
-    const uint32_t* lut = cb.lut + (size_t)seg * CO3_LUT_SIZE;
-    for (int i = tid; i < CO3_LUT_SIZE; i += CO3_THREADS) t.lut[i] = lut[i];
+__device__ void load_tables(Tables& t, const Co3CodeBook& cb, int row, int nsym, int tid) {
+    const uint4* lut = reinterpret_cast<const uint4*>(cb.lut + (size_t)row * CO3_LUT_SIZE);
+    uint4* dst = reinterpret_cast<uint4*>(t.lut);
+    for (int i = tid; i < CO3_LUT_SIZE / 4; i += CO3_THREADS) dst[i] = __ldg(lut + i);
     if (tid <= CO3_MAXLEN) {
-        const size_t o = (size_t)seg * (CO3_MAXLEN + 1) + tid;
+        const size_t o = (size_t)row * (CO3_MAXLEN + 1) + tid;
         t.first[tid] = cb.first[o]; t.count[tid] = cb.count[o]; t.offs[tid] = cb.offs[o];
     }
     if (tid < nsym) {
-        t.ksign[tid] = cb.ksign[(size_t)seg * CO3_MAXSYM + tid];
-        t.perm[tid] = cb.perm[(size_t)seg * CO3_MAXSYM + tid];
+        t.ksign[tid] = cb.ksign[tid];
+        t.perm[tid] = cb.perm[(size_t)row * CO3_MAXSYM + tid];
     }
 }
 
@@ -47,74 +53,84 @@ __device__ __forceinline__ float pow2_clamped(int e) {   // 2^e; a corrupt heade
     return __uint_as_float((uint32_t)(e + 127) << 23);
 }
 
-struct Reader {                                   // LSB-first bit reader over a bounded word array
+struct Reader {                                   // LSB-first bit reader
     unsigned long long buf;
     int nb;                                       // valid bits in buf
     uint32_t wp;                                  // next word to fetch
 };
 
+template <bool CHECKED>
 __device__ __forceinline__ uint32_t fetch(const uint32_t* src, uint32_t nwords, uint32_t i) {
-    return i < nwords ? src[i] : 0u;
+    if (CHECKED) return i < nwords ? src[i] : 0u;
+    return src[i];
 }
 
+template <bool CHECKED>
 __device__ __forceinline__ void reader_init(Reader& r, const uint32_t* src, uint32_t nwords, uint32_t bitpos) {
     r.wp = bitpos >> 5;
     const uint32_t sh = bitpos & 31u;
-    r.buf = (unsigned long long)(fetch(src, nwords, r.wp) >> sh);
+    r.buf = (unsigned long long)(fetch<CHECKED>(src, nwords, r.wp) >> sh);
     r.nb = 32 - (int)sh;
     r.wp++;
-    r.buf |= (unsigned long long)fetch(src, nwords, r.wp) << r.nb;
+    r.buf |= (unsigned long long)fetch<CHECKED>(src, nwords, r.wp) << r.nb;
     r.nb += 32;
     r.wp++;
 }
 
-// Decode one codeword; returns its signed integer magnitude.  bad is set if no codeword matches
-// (cannot happen for a complete code; kept so that corrupt tables cannot loop or read outside).
-__device__ __forceinline__ int32_t decode_one(Reader& r, const Tables& t, const uint32_t* src,
-                                              uint32_t nwords, bool& bad) {
-    const uint32_t window = (uint32_t)r.buf;
-    uint32_t e = t.lut[window & (CO3_LUT_SIZE - 1)];
-    int32_t k;
-    uint32_t len = e & 0xFFu;
-    if (len != 0) {
-        k = (int32_t)e >> 8;
-    } else {                                      // codeword longer than 11 bits: canonical search
-        const uint32_t v = __brev(window) >> 16;  // 16 stream bits, root bit on top
-        k = 0;
-        len = CO3_MAXLEN;
-        bool found = false;
-        for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
-            const uint32_t dd = (v >> (CO3_MAXLEN - L)) - t.first[L];
-            if (dd < t.count[L]) {
-                k = t.ksign[t.perm[(t.offs[L] + dd) & (CO3_MAXSYM - 1)]];
-                len = (uint32_t)L;
-                found = true;
-                break;
-            }
+// Codeword longer than the primary table: canonical search over lengths 12..16.
+__device__ __noinline__ uint32_t decode_long(uint32_t window, const Tables& t, int32_t& k, bool& bad) {
+    const uint32_t v = __brev(window) >> 16;      // 16 stream bits, root bit on top
+    for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
+        const uint32_t dd = (v >> (CO3_MAXLEN - L)) - t.first[L];
+        if (dd < t.count[L]) {
+            k = t.ksign[t.perm[(t.offs[L] + dd) & (CO3_MAXSYM - 1)]];
+            return (uint32_t)L;
         }
-        bad |= !found;
     }
-    r.buf >>= len;
-    r.nb -= (int)len;
-    if (r.nb < 32) {
-        r.buf |= (unsigned long long)fetch(src, nwords, r.wp) << r.nb;
-        r.nb += 32;
-        r.wp++;
+    bad = true;                                   // cannot happen for a complete code
+    k = 0;
+    return CO3_MAXLEN;
+}
+
+// Decode n symbols of this lane's sub-chunk, adding their signed magnitudes to acc[0],
+// acc[PADW], ... (one accumulator row per symbol position).
+template <bool CHECKED>
+__device__ __forceinline__ void decode_run(Reader& r, const Tables& t, const uint32_t* src, uint32_t nwords,
+                                           int32_t* acc, int n, bool& bad) {
+    unsigned long long buf = r.buf;
+    int nb = r.nb;
+    uint32_t wp = r.wp;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t window = (uint32_t)buf;
+        const uint32_t e = t.lut[window & (CO3_LUT_SIZE - 1)];
+        int32_t k = (int32_t)e >> 8;
+        uint32_t len = e & 0xFFu;
+        if (len == 0) len = decode_long(window, t, k, bad);
+        buf >>= len;
+        nb -= (int)len;
+        atomicAdd(acc, k);
+        acc += PADW;
+        if (nb < 32) {
+            buf |= (unsigned long long)fetch<CHECKED>(src, nwords, wp) << nb;
+            nb += 32;
+            wp++;
+        }
     }
-    return k;
+    r.buf = buf; r.nb = nb; r.wp = wp;
 }
 
 struct Stream {                                   // one (chunk, user) stream as seen by a lane
-    const uint32_t* src;                          // staged or global words of the chunk
     uint32_t nwords;
     uint32_t bitpos;                              // start of this lane's sub-chunk
     uint32_t sub_len_bits;                        // recorded length of this lane's sub-chunk
     int i_lo, i_hi;                               // this lane's symbols within its 128-window
     bool active;
+    bool staged;                                  // words are in shared memory (else read from global)
+    const uint32_t* gsrc;
 };
 
-// Stage the words of (chunk c, user u) into `stage` (or point at global memory if they do not
-// fit) and give every lane the start of its sub-chunk.  Called by one whole warp.
+// Stage the words of (chunk c, user u) into `stage` (if they fit) and give every lane the start
+// of its sub-chunk.  Called by one whole warp.
 __device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co3Chunk& cd, int64_t c, int u,
                                             const uint32_t* __restrict__ bitstream,
                                             const uint16_t* __restrict__ sub_bits,
@@ -125,15 +141,13 @@ __device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co
     uint32_t nwords = 0;
     if ((w0 & 3u) || w1 < w0 || (int64_t)w1 > p.cap_words) bad = true;   // offsets must be sane
     else nwords = w1 - w0;
-    const uint32_t* g = bitstream + (size_t)u * p.cap_words + w0;
-    if (nwords <= CO3_STAGE_WORDS) {
+    const uint32_t* g = bitstream + (size_t)u * p.cap_words + (nwords ? w0 : 0u);
+    s.gsrc = g;
+    s.staged = nwords <= CO3_STAGE_WORDS;
+    if (s.staged) {
         const uint4* gv = reinterpret_cast<const uint4*>(g);
         uint4* sv = reinterpret_cast<uint4*>(stage);
         for (uint32_t i = lane; i < nwords / 4; i += 32) sv[i] = __ldg(gv + i);
-        for (uint32_t i = (nwords & ~3u) + lane; i < nwords; i += 32) stage[i] = __ldg(g + i);
-        s.src = stage;
-    } else {
-        s.src = g;
     }
     s.nwords = nwords;
     const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
@@ -151,39 +165,35 @@ __device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co
     }
     s.bitpos = x - sb;
     s.sub_len_bits = sb;
+    if (s.bitpos > nwords * 32u) {                // a start outside the chunk: corrupt side info
+        bad = true;
+        s.bitpos = nwords * 32u;
+    }
     __syncwarp();
 }
 
-__device__ __forceinline__ void write_out(const Co3Dev& p, float* __restrict__ avg, const int32_t* acc,
-                                          const Co3Chunk& cd, int i0, int ni, float scale, float fu,
-                                          int t, int nt) {
-    // acc holds symbols i0 .. i0+ni-1 of every sub-chunk: acc[(i - i0) * PADW + kk]
-    const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-    const int lo = (int)(cd.start - tb), hi = lo + cd.len;
-    for (int x = t; x < 32 * ni; x += nt) {
-        const int kk = x / ni, il = x - kk * ni;
-        const int e = kk * CO3_SUB + i0 + il;
-        if (e >= lo && e < hi)
-            avg[tb + e] = __fdiv_rn(__fmul_rn((float)acc[il * PADW + kk], scale), fu);
-    }
+__device__ __forceinline__ float finish(int32_t ksum, float scale, float fu, float inv_u) {
+    const float v = __fmul_rn((float)ksum, scale);                  // exact
+    return inv_u != 0.0f ? __fmul_rn(v, inv_u) : __fdiv_rn(v, fu);  // U a power of two: exact either way
 }
 
 // ---- U <= 8: one stream per warp, quarter batches ------------------------------------------
-static_assert(CO3_STAGE_WORDS % 4 == 0, "stage rows must keep 16-byte alignment");
 constexpr int QB = 32;                            // symbols per lane per batch
+constexpr int ACC_Q = QB * PADW;                  // accumulator words per chunk per batch
 
 struct SmemA {
     Tables t;
-    alignas(16) uint32_t stage[NW][CO3_STAGE_WORDS];   // filled with 128-bit stores
-    int32_t acc[1][QB * PADW];                    // one accumulator per chunk of the group:
-};                                                // really [chunks per group], sized at launch
+    alignas(16) uint32_t stage[NW][STAGE_ROW];    // filled with 128-bit stores
+    alignas(16) int32_t acc[2][ACC_Q];            // really [2][chunks per group][ACC_Q], sized at launch
+};
 
+__host__ __device__ inline int acc_words_a(int U) { return ((NW / U) * ACC_Q + 3) & ~3; }
 __host__ __device__ inline size_t smem_a_bytes(int U) {
-    return sizeof(SmemA) + (size_t)(NW / U - 1) * QB * PADW * sizeof(int32_t);
+    return sizeof(SmemA) - sizeof(int32_t) * 2 * ACC_Q + sizeof(int32_t) * 2 * (size_t)acc_words_a(U);
 }
 
 __global__ void __launch_bounds__(CO3_THREADS)
-decode_small_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bitstream,
+decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                       const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
                       const co3_seg_header* __restrict__ hdr, float* __restrict__ avg) {
     extern __shared__ __align__(16) unsigned char s_raw[];
@@ -191,47 +201,69 @@ decode_small_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bit
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int U = p.U;
     const int cpg = NW / U;                        // chunks per group (>= 1)
+    const int accw = acc_words_a(U);               // words per accumulator buffer
+    int32_t* acc0 = &sm.acc[0][0];
     const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
     const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
     const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
     const float fu = (float)U;
+    const float inv_u = (U & (U - 1)) == 0 ? 1.0f / fu : 0.0f;
     int cur_seg = -1;
     bool bad = false;
     for (int64_t gi = g0; gi < g1; ++gi) {
         const Co3Group grp = p.groups[gi];
+        __syncthreads();                           // previous group's read-out is finished
         if (grp.seg != cur_seg) {
-            __syncthreads();
-            load_tables(sm.t, cb, grp.seg, p.nsym, tid);
+            load_tables(sm.t, p.cb, co3_row_of(hdr[grp.seg], &bad), p.nsym, tid);
             cur_seg = grp.seg;
-            __syncthreads();
         }
+        for (int i = tid; i < accw / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
         const bool mine = ci < cpg && ci < grp.count;
         Stream s;
-        s.active = false;
-        Co3Chunk cd;
-        cd.start = 0; cd.len = 0; cd.seg = 0; cd.sub0 = 0;
+        s.active = false; s.staged = true; s.nwords = 0; s.bitpos = 0; s.sub_len_bits = 0;
+        s.i_lo = 0; s.i_hi = 0; s.gsrc = nullptr;
         Reader r;
         r.buf = 0; r.nb = 0; r.wp = 0;
         if (mine) {
-            cd = p.chunks[grp.chunk0 + ci];
+            const Co3Chunk cd = p.chunks[grp.chunk0 + ci];
             open_stream(s, p, cd, grp.chunk0 + ci, us, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
-            if (s.active) reader_init(r, s.src, s.nwords, s.bitpos);
+            if (s.active) {
+                if (s.staged) reader_init<false>(r, sm.stage[warp], s.nwords, s.bitpos);
+                else reader_init<true>(r, s.gsrc, s.nwords, s.bitpos);
+            }
         }
         const float scale = pow2_clamped((int)hdr[grp.seg].bias + p.cF);
+        __syncthreads();                           // tables, zeroed accumulator 0
+#pragma unroll 1
         for (int q = 0; q < CO3_SUB / QB; ++q) {
-            for (int i = tid; i < grp.count * QB * PADW; i += CO3_THREADS) (&sm.acc[0][0])[i] = 0;
-            __syncthreads();
+            int32_t* accq = acc0 + (q & 1) * accw;
             if (mine && s.active) {
                 const int a = max(s.i_lo, q * QB), b = min(s.i_hi, (q + 1) * QB);
-                int32_t* acc = sm.acc[ci];
-                for (int i = a; i < b; ++i) {
-                    const int32_t k = decode_one(r, sm.t, s.src, s.nwords, bad);
-                    atomicAdd(&acc[(i - q * QB) * PADW + lane], k);
+                if (b > a) {
+                    int32_t* dst = accq + ci * ACC_Q + (a - q * QB) * PADW + lane;
+                    if (s.staged) decode_run<false>(r, sm.t, sm.stage[warp], s.nwords, dst, b - a, bad);
+                    else decode_run<true>(r, sm.t, s.gsrc, s.nwords, dst, b - a, bad);
                 }
             }
             __syncthreads();
-            for (int cc = 0; cc < grp.count; ++cc)
-                write_out(p, avg, sm.acc[cc], p.chunks[grp.chunk0 + cc], q * QB, QB, scale, fu, tid, CO3_THREADS);
+            // clear the other buffer for the next quarter while this one is written out
+            if (q + 1 < CO3_SUB / QB) {
+                uint4* z = reinterpret_cast<uint4*>(acc0 + ((q + 1) & 1) * accw);
+                for (int i = tid; i < accw / 4; i += CO3_THREADS) z[i] = make_uint4(0, 0, 0, 0);
+            }
+            for (int cc = 0; cc < grp.count; ++cc) {
+                const Co3Chunk cd = p.chunks[grp.chunk0 + cc];
+                const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+                const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+                const int32_t* a = accq + cc * ACC_Q;
+#pragma unroll
+                for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+                    const int x = tid + rr * CO3_THREADS;
+                    const int kk = x >> 5, il = x & 31;
+                    const int e = kk * CO3_SUB + q * QB + il;
+                    if (e >= lo && e < hi) avg[tb + e] = finish(a[il * PADW + kk], scale, fu, inv_u);
+                }
+            }
             __syncthreads();
         }
         if (mine && s.active) {
@@ -245,12 +277,12 @@ decode_small_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bit
 // ---- U > 8: whole-chunk accumulator, user groups of 8 --------------------------------------
 struct SmemB {
     Tables t;
-    int32_t acc[CO3_SUB * PADW];
-    alignas(16) uint32_t stage[NW][CO3_STAGE_WORDS];   // filled with 128-bit stores
+    alignas(16) int32_t acc[CO3_SUB * PADW];
+    alignas(16) uint32_t stage[NW][STAGE_ROW];    // filled with 128-bit stores
 };
 
 __global__ void __launch_bounds__(CO3_THREADS)
-decode_large_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bitstream,
+decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                       const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
                       const co3_seg_header* __restrict__ hdr, float* __restrict__ avg) {
     extern __shared__ __align__(16) unsigned char s_raw[];
@@ -259,26 +291,29 @@ decode_large_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bit
     const int64_t per = (p.n_chunks + gridDim.x - 1) / gridDim.x;
     const int64_t c0 = (int64_t)blockIdx.x * per, c1 = min(p.n_chunks, c0 + per);
     const float fu = (float)p.U;
+    const float inv_u = (p.U & (p.U - 1)) == 0 ? 1.0f / fu : 0.0f;
     int cur_seg = -1;
     bool bad = false;
     for (int64_t c = c0; c < c1; ++c) {
         const Co3Chunk cd = p.chunks[c];
         if (cd.seg != cur_seg) {
-            __syncthreads();
-            load_tables(sm.t, cb, cd.seg, p.nsym, tid);
+            load_tables(sm.t, p.cb, co3_row_of(hdr[cd.seg], &bad), p.nsym, tid);
             cur_seg = cd.seg;
         }
-        for (int i = tid; i < CO3_SUB * PADW; i += CO3_THREADS) sm.acc[i] = 0;
+        for (int i = tid; i < CO3_SUB * PADW / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(sm.acc)[i] = make_uint4(0, 0, 0, 0);
         __syncthreads();
         for (int u = warp; u < p.U; u += NW) {
             Stream s;
             open_stream(s, p, cd, c, u, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
             if (s.active) {
                 Reader r;
-                reader_init(r, s.src, s.nwords, s.bitpos);
-                for (int i = s.i_lo; i < s.i_hi; ++i) {
-                    const int32_t k = decode_one(r, sm.t, s.src, s.nwords, bad);
-                    atomicAdd(&sm.acc[i * PADW + lane], k);
+                int32_t* dst = sm.acc + s.i_lo * PADW + lane;
+                if (s.staged) {
+                    reader_init<false>(r, sm.stage[warp], s.nwords, s.bitpos);
+                    decode_run<false>(r, sm.t, sm.stage[warp], s.nwords, dst, s.i_hi - s.i_lo, bad);
+                } else {
+                    reader_init<true>(r, s.gsrc, s.nwords, s.bitpos);
+                    decode_run<true>(r, sm.t, s.gsrc, s.nwords, dst, s.i_hi - s.i_lo, bad);
                 }
                 const uint32_t endpos = r.wp * 32u - (uint32_t)r.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
@@ -287,7 +322,14 @@ decode_large_u_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ bit
         }
         __syncthreads();
         const float scale = pow2_clamped((int)hdr[cd.seg].bias + p.cF);
-        write_out(p, avg, sm.acc, cd, 0, CO3_SUB, scale, fu, tid, CO3_THREADS);
+        const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+        const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+#pragma unroll 4
+        for (int rr = 0; rr < CO3_TILE / CO3_THREADS; ++rr) {
+            const int e = tid + rr * CO3_THREADS;
+            const int kk = e >> 7, il = e & (CO3_SUB - 1);
+            if (e >= lo && e < hi) avg[tb + e] = finish(sm.acc[il * PADW + kk], scale, fu, inv_u);
+        }
         __syncthreads();
     }
     if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
@@ -317,7 +359,7 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
         if (bpsm < 1) bpsm = 1;
         const int64_t grid = (int64_t)pl->num_sms * bpsm;
         decode_small_u_kernel<<<(int)(p.n_groups < grid ? p.n_groups : grid), CO3_THREADS, smem, st>>>(
-            p, pl->cb_dec, bitstream, sub_bits, chunk_off, hdr, avg);
+            p, bitstream, sub_bits, chunk_off, hdr, avg);
     } else {
         if (!g_bpsm_b) {
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_bpsm_b, decode_large_u_kernel, CO3_THREADS, sizeof(SmemB));
@@ -325,7 +367,7 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
         }
         const int64_t grid = (int64_t)pl->num_sms * g_bpsm_b;
         decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), CO3_THREADS, sizeof(SmemB), st>>>(
-            p, pl->cb_dec, bitstream, sub_bits, chunk_off, hdr, avg);
+            p, bitstream, sub_bits, chunk_off, hdr, avg);
     }
     co3_prof_end(pl, CO3_K_DECODE, st, 1);
     return cudaGetLastError();

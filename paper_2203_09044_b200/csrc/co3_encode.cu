@@ -6,87 +6,131 @@
 //   3. enc_pack_kernel -- per chunk: per-thread bit offsets by a block scan, codewords merged
 //                         into a shared-memory image of the chunk, 128-bit coalesced stores
 // Work item = (user, chunk); a thread owns 16 consecutive symbols (one 128-bit load), 8 threads
-// own a sub-chunk, a block owns a chunk.  Blocks are persistent over contiguous item ranges and
-// keep the segment's code table in shared memory, replicated once per lane so that the table
-// look-ups are free of bank conflicts.  Bound: HBM for the symbol reads (1 B/element, twice) and
-// payload writes (~0.85 B/element), with integer issue slots close behind.
+// own a sub-chunk, a block owns a chunk.  Blocks are persistent over contiguous item ranges, keep
+// the segment's table in shared memory (replicated once per lane, so the look-ups are free of
+// bank conflicts) and always have the next item's symbols in flight.  In the pack kernel a thread
+// first merges its 16 codewords pairwise in registers (16 -> 8 -> 4 pieces of at most 64 bits),
+// then ORs the four pieces into the chunk image at its scanned bit offset.
+// Bound: HBM for the symbol reads (1 B/element, twice) and payload writes (~0.85 B/element), with
+// integer issue slots and shared-memory look-ups (one per symbol per pass) close behind.
 #include "co3_internal.h"
 
 namespace {
 
 constexpr int BUF_WORDS = CO3_TILE * CO3_MAXLEN / 32;   // 2048: a chunk at 16 bits per symbol
 
-__device__ __forceinline__ void load_symbols(const Co3Dev& p, int u, const Co3Chunk& cd, int tid,
-                                             uint32_t w[4], uint32_t& mask) {
-    const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-    const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+struct Item {                    // one (user, chunk) work item as a thread sees it
+    uint32_t u;
+    Co3Chunk cd;
+    uint32_t w[4];               // this thread's 16 symbols
+    uint32_t mask;               // which of them belong to the chunk
+};
+
+__device__ __forceinline__ void fetch_item(Item& it, const Co3Dev& p, uint32_t u, uint32_t c, int tid) {
+    it.u = u;
+    it.cd = p.chunks[c];
+    const int64_t tb = it.cd.start & ~(int64_t)(CO3_TILE - 1);
+    const int lo = (int)(it.cd.start - tb), hi = lo + it.cd.len;
     const int e0 = 16 * tid;
-    mask = 0;
-    w[0] = w[1] = w[2] = w[3] = 0;
+    it.mask = 0;
+    it.w[0] = it.w[1] = it.w[2] = it.w[3] = 0;
     if (e0 < hi && e0 + 16 > lo) {
         const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.sym + (size_t)u * p.sld + tb + e0));
-        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        it.w[0] = v.x; it.w[1] = v.y; it.w[2] = v.z; it.w[3] = v.w;
         const int a = max(lo - e0, 0), b = min(hi - e0, 16);     // valid bytes [a, b)
-        mask = (b >= 16 ? 0xFFFFu : ((1u << b) - 1u)) & ~((1u << a) - 1u);
+        it.mask = (b >= 16 ? 0xFFFFu : ((1u << b) - 1u)) & ~((1u << a) - 1u);
     }
 }
 
-__global__ void __launch_bounds__(CO3_THREADS)
-enc_len_kernel(Co3Dev p, Co3CodeBook cb, uint16_t* __restrict__ sub_bits, unsigned long long* user_bits) {
-    __shared__ uint32_t s_len[(CO3_MAXSYM / 4) * 32];   // [word of 4 lengths][lane]
-    __shared__ uint32_t s_warp[CO3_THREADS / 32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t n_items = p.n_chunks * (int64_t)p.U;
-    const int64_t per = (n_items + gridDim.x - 1) / gridDim.x;
-    const int64_t it0 = (int64_t)blockIdx.x * per, it1 = min(n_items, it0 + per);
-    int cur_seg = -1;
-    for (int64_t item = it0; item < it1; ++item) {
-        const int u = (int)(item / p.n_chunks);
-        const int64_t c = item - (int64_t)u * p.n_chunks;
-        const Co3Chunk cd = p.chunks[c];
-        if (cd.seg != cur_seg) {
-            __syncthreads();
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(cb.len8 + (size_t)cd.seg * CO3_MAXSYM);
-            for (int i = tid; i < (p.nsym / 4) * 32; i += CO3_THREADS) s_len[i] = src[i >> 5];
-            cur_seg = cd.seg;
-            __syncthreads();
-        }
-        uint32_t w[4], mask;
-        load_symbols(p, u, cd, tid, w, mask);
-        uint32_t bits = 0;
+// Look up the 16 table entries of a thread's symbols; entries of masked-out symbols are 0.
+__device__ __forceinline__ void lookup16(const uint32_t* s_tab, int lane, const uint32_t w[4],
+                                         uint32_t mask, uint32_t ent[16]) {
+    if (mask == 0xFFFFu) {
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-            const uint32_t s = (w[i >> 2] >> (8 * (i & 3))) & 0xFFu;
-            const uint32_t l4 = s_len[(s >> 2) * 32 + lane];
-            const uint32_t l = (l4 >> (8 * (s & 3))) & 0xFFu;
-            bits += ((mask >> i) & 1u) ? l : 0u;
+            const uint32_t s = __byte_perm(w[i >> 2], 0, 0x4440 + (i & 3));
+            ent[i] = s_tab[s * 32 + lane];
         }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t s = __byte_perm(w[i >> 2], 0, 0x4440 + (i & 3));
+            ent[i] = ((mask >> i) & 1u) ? s_tab[s * 32 + lane] : 0u;
+        }
+    }
+}
+
+// Contiguous item range of this block and the (user, chunk) of its first item.
+__device__ __forceinline__ void block_range(const Co3Dev& p, uint32_t& it0, uint32_t& it1, uint32_t& u, uint32_t& c) {
+    const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.U;
+    const uint32_t per = (n_items + gridDim.x - 1) / gridDim.x;
+    it0 = blockIdx.x * per;
+    it1 = min(n_items, it0 + per);
+    u = it0 / (uint32_t)p.n_chunks;
+    c = it0 - u * (uint32_t)p.n_chunks;
+}
+
+__global__ void __launch_bounds__(CO3_THREADS)
+enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits,
+               unsigned long long* user_bits) {
+    extern __shared__ __align__(16) uint32_t s_dyn[];
+    uint32_t* s_len = s_dyn;                          // [nsym][32 lanes] code lengths
+    __shared__ uint32_t s_warp[2][CO3_THREADS / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t it0, it1, u, c;
+    block_range(p, it0, it1, u, c);
+    if (it0 >= it1) return;
+    const uint32_t n_chunks = (uint32_t)p.n_chunks;
+    int cur_seg = -1;
+    bool bad = false;
+    Item cur;
+    fetch_item(cur, p, u, c, tid);
+    for (uint32_t item = it0; item < it1; ++item) {
+        Item nxt = cur;
+        if (item + 1 < it1) {                         // next item's symbols in flight
+            uint32_t un = u, cn = c + 1;
+            if (cn == n_chunks) { cn = 0; ++un; }
+            fetch_item(nxt, p, un, cn, tid);
+            u = un; c = cn;
+        }
+        if (cur.cd.seg != cur_seg) {
+            __syncthreads();
+            const uint8_t* src = p.cb.len8 + (size_t)co3_row_of(hdr[cur.cd.seg], &bad) * CO3_MAXSYM;
+            for (int i = tid; i < p.nsym * 32; i += CO3_THREADS) s_len[i] = src[i >> 5];
+            cur_seg = cur.cd.seg;
+            __syncthreads();
+        }
+        uint32_t ent[16];
+        lookup16(s_len, lane, cur.w, cur.mask, ent);
+        uint32_t bits = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) bits += ent[i];
         // 8 threads = one sub-chunk
         uint32_t sb = bits;
         sb += __shfl_xor_sync(0xffffffffu, sb, 1);
         sb += __shfl_xor_sync(0xffffffffu, sb, 2);
         sb += __shfl_xor_sync(0xffffffffu, sb, 4);
-        const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-        const int sub_first = (int)((cd.start - tb) / CO3_SUB);
-        const int sub_last = (int)((cd.start - tb + cd.len - 1) / CO3_SUB);
+        const int tlo = (int)(cur.cd.start & (CO3_TILE - 1));
+        const int sub_first = tlo / CO3_SUB, sub_last = (tlo + cur.cd.len - 1) / CO3_SUB;
         const int kk = tid >> 3;
         if ((tid & 7) == 0 && kk >= sub_first && kk <= sub_last)
-            sub_bits[(size_t)u * p.n_sub + cd.sub0 + (kk - sub_first)] = (uint16_t)sb;
-        uint32_t wb = sb;                       // every lane of a sub-chunk holds sb: count it once
-        wb = ((lane & 7) == 0) ? wb : 0u;
+            sub_bits[(size_t)cur.u * p.n_sub + cur.cd.sub0 + (kk - sub_first)] = (uint16_t)sb;
+        uint32_t wb = ((lane & 7) == 0) ? sb : 0u;     // every lane of a sub-chunk holds sb: count it once
         wb += __shfl_xor_sync(0xffffffffu, wb, 8);
         wb += __shfl_xor_sync(0xffffffffu, wb, 16);
-        if (lane == 0) s_warp[warp] = wb;
+        const int par = (int)(item & 1);
+        if (lane == 0) s_warp[par][warp] = wb;
         __syncthreads();
         if (tid == 0) {
             uint32_t tot = 0;
 #pragma unroll
-            for (int k = 0; k < CO3_THREADS / 32; ++k) tot += s_warp[k];
+            for (int k = 0; k < CO3_THREADS / 32; ++k) tot += s_warp[par][k];
             p.chunk_words[item] = 4u * ((tot + 127u) / 128u);
-            atomicAdd(&user_bits[u], (unsigned long long)tot);
+            atomicAdd(&user_bits[cur.u], (unsigned long long)tot);
         }
-        __syncthreads();
+        cur = nxt;
     }
+    if (bad && tid == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
 
 // chunk_off[u][c] = exclusive prefix of the chunk word counts of user u; one block per user.
@@ -135,105 +179,140 @@ __global__ void __launch_bounds__(1024) enc_scan_kernel(Co3Dev p, uint32_t* __re
     }
 }
 
-__global__ void __launch_bounds__(CO3_THREADS)
-enc_pack_kernel(Co3Dev p, Co3CodeBook cb, const uint32_t* __restrict__ chunk_off, uint32_t* __restrict__ bitstream) {
-    extern __shared__ __align__(16) uint32_t s_dyn[];
-    uint32_t* s_enc = s_dyn;                          // [nsym][32 lanes]
-    uint32_t* s_buf = s_dyn + p.nsym * 32;            // BUF_WORDS + 4
-    __shared__ uint32_t s_warp[CO3_THREADS / 32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t n_items = p.n_chunks * (int64_t)p.U;
-    const int64_t per = (n_items + gridDim.x - 1) / gridDim.x;
-    const int64_t it0 = (int64_t)blockIdx.x * per, it1 = min(n_items, it0 + per);
-    int cur_seg = -1;
-    for (int64_t item = it0; item < it1; ++item) {
-        const int u = (int)(item / p.n_chunks);
-        const int64_t c = item - (int64_t)u * p.n_chunks;
-        if (p.user_ovf[u]) continue;                  // block-uniform
-        const Co3Chunk cd = p.chunks[c];
-        if (cd.seg != cur_seg) {
-            __syncthreads();
-            const uint32_t* src = cb.enc + (size_t)cd.seg * CO3_MAXSYM;
-            for (int i = tid; i < p.nsym * 32; i += CO3_THREADS) s_enc[i] = src[i >> 5];
-            cur_seg = cd.seg;
-            __syncthreads();
-        }
-        uint32_t w[4], mask;
-        load_symbols(p, u, cd, tid, w, mask);
-        uint32_t ent[16];
-        uint32_t bits = 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const uint32_t s = (w[i >> 2] >> (8 * (i & 3))) & 0xFFu;
-            const uint32_t e = s_enc[s * 32 + lane];
-            ent[i] = ((mask >> i) & 1u) ? e : 0u;
-            bits += ent[i] >> 16;
-        }
-        // exclusive scan of the per-thread bit counts over the block
-        uint32_t x = bits;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
-            if (lane >= o) x += y;
-        }
-        if (lane == 31) s_warp[warp] = x;
-        __syncthreads();
-        uint32_t pre = 0, total = 0;
-#pragma unroll
-        for (int k = 0; k < CO3_THREADS / 32; ++k) {
-            const uint32_t t = s_warp[k];
-            pre += (k < warp) ? t : 0u;
-            total += t;
-        }
-        const uint32_t nwords = 4u * ((total + 127u) / 128u);
-        for (uint32_t i = tid; i < nwords; i += CO3_THREADS) s_buf[i] = 0;
-        __syncthreads();
-        uint32_t pos = pre + x - bits;
-        uint32_t wi = pos >> 5, nb = pos & 31u;
-        unsigned long long acc = 0;
-        bool first = true;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            acc |= (unsigned long long)(ent[i] & 0xFFFFu) << nb;
-            nb += ent[i] >> 16;
-            if (nb >= 32u) {
-                if (first) { atomicOr(&s_buf[wi], (uint32_t)acc); first = false; }
-                else s_buf[wi] = (uint32_t)acc;        // a word wholly inside this thread's span
-                acc >>= 32; nb -= 32u; ++wi;
-            }
-        }
-        if (acc) atomicOr(&s_buf[wi], (uint32_t)acc);
-        __syncthreads();
-        uint4* dst = reinterpret_cast<uint4*>(bitstream + (size_t)u * p.cap_words +
-                                              chunk_off[(size_t)u * (p.n_chunks + 1) + c]);
-        const uint4* srcv = reinterpret_cast<const uint4*>(s_buf);
-        for (uint32_t i = tid; i < nwords / 4; i += CO3_THREADS) dst[i] = srcv[i];
-        __syncthreads();
-    }
+// OR a piece of at most 64 bits into the chunk image at bit position pos.
+__device__ __forceinline__ void put_piece(uint32_t* s_buf, uint32_t pos, unsigned long long v) {
+    const uint32_t wi = pos >> 5, bs = pos & 31u;
+    const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+    const uint32_t w0 = lo << bs;
+    const uint32_t w1 = __funnelshift_l(lo, hi, bs);
+    const uint32_t w2 = __funnelshift_l(hi, 0u, bs);
+    if (w0) atomicOr(&s_buf[wi], w0);
+    if (w1) atomicOr(&s_buf[wi + 1], w1);
+    if (w2) atomicOr(&s_buf[wi + 2], w2);
 }
 
-int g_len_bpsm = 0, g_pack_bpsm[4] = {0, 0, 0, 0};
+__global__ void __launch_bounds__(CO3_THREADS)
+enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t* __restrict__ chunk_off,
+                uint32_t* __restrict__ bitstream) {
+    extern __shared__ __align__(16) uint32_t s_dyn[];
+    uint32_t* s_enc = s_dyn;                          // [nsym][32 lanes] codeword | length << 16
+    uint32_t* s_buf = s_dyn + p.nsym * 32;            // BUF_WORDS + 4
+    __shared__ uint32_t s_warp[2][CO3_THREADS / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t it0, it1, u, c;
+    block_range(p, it0, it1, u, c);
+    if (it0 >= it1) return;
+    const uint32_t n_chunks = (uint32_t)p.n_chunks;
+    int cur_seg = -1;
+    bool bad = false;
+    uint32_t prev_words = BUF_WORDS + 4;              // words of the image that may be non-zero
+    Item cur;
+    fetch_item(cur, p, u, c, tid);
+    uint32_t cur_c = c;
+    for (uint32_t item = it0; item < it1; ++item) {
+        Item nxt = cur;
+        uint32_t nxt_c = cur_c;
+        if (item + 1 < it1) {                         // next item's symbols in flight
+            uint32_t un = u, cn = c + 1;
+            if (cn == n_chunks) { cn = 0; ++un; }
+            fetch_item(nxt, p, un, cn, tid);
+            u = un; c = cn; nxt_c = cn;
+        }
+        if (!p.user_ovf[cur.u]) {                     // block-uniform
+            if (cur.cd.seg != cur_seg) {
+                const uint32_t* src = p.cb.enc + (size_t)co3_row_of(hdr[cur.cd.seg], &bad) * CO3_MAXSYM;
+                for (int i = tid; i < p.nsym * 32; i += CO3_THREADS) s_enc[i] = src[i >> 5];
+                cur_seg = cur.cd.seg;
+            }
+            {   // clear what the previous chunk left in the image (all of it the first time)
+                uint4* z = reinterpret_cast<uint4*>(s_buf);
+                for (uint32_t i = tid; i < (prev_words + 3) / 4; i += CO3_THREADS) z[i] = make_uint4(0, 0, 0, 0);
+            }
+            const uint32_t dst_word = chunk_off[(size_t)cur.u * (n_chunks + 1) + cur_c];
+            __syncthreads();                          // table and cleared image visible
+            uint32_t ent[16];
+            lookup16(s_enc, lane, cur.w, cur.mask, ent);
+            // merge 16 codewords -> 8 pieces (<= 32 bits) -> 4 pieces (<= 64 bits)
+            uint32_t c1[8], l1[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t a = ent[2 * k], b = ent[2 * k + 1];
+                c1[k] = (a & 0xFFFFu) | ((b & 0xFFFFu) << (a >> 16));
+                l1[k] = (a >> 16) + (b >> 16);
+            }
+            unsigned long long c2[4];
+            uint32_t l2[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                c2[k] = (unsigned long long)c1[2 * k] | ((unsigned long long)c1[2 * k + 1] << l1[2 * k]);
+                l2[k] = l1[2 * k] + l1[2 * k + 1];
+            }
+            const uint32_t bits = l2[0] + l2[1] + l2[2] + l2[3];
+            // exclusive scan of the per-thread bit counts over the block
+            uint32_t x = bits;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += y;
+            }
+            const int par = (int)(item & 1);
+            if (lane == 31) s_warp[par][warp] = x;
+            __syncthreads();
+            uint32_t pre = 0, total = 0;
+#pragma unroll
+            for (int k = 0; k < CO3_THREADS / 32; ++k) {
+                const uint32_t t = s_warp[par][k];
+                pre += (k < warp) ? t : 0u;
+                total += t;
+            }
+            const uint32_t nwords = 4u * ((total + 127u) / 128u);
+            uint32_t pos = pre + x - bits;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                put_piece(s_buf, pos, c2[k]);
+                pos += l2[k];
+            }
+            __syncthreads();
+            uint4* dst = reinterpret_cast<uint4*>(bitstream + (size_t)cur.u * p.cap_words + dst_word);
+            const uint4* srcv = reinterpret_cast<const uint4*>(s_buf);
+            for (uint32_t i = tid; i < nwords / 4; i += CO3_THREADS) dst[i] = srcv[i];
+            prev_words = nwords;
+            __syncthreads();
+        }
+        cur = nxt;
+        cur_c = nxt_c;
+    }
+    if (bad && tid == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);
+}
+
+int g_len_bpsm[4] = {0, 0, 0, 0}, g_pack_bpsm[4] = {0, 0, 0, 0};
 
 }  // namespace
 
 cudaError_t co3_setup_kernels(void) {
-    return cudaFuncSetAttribute(enc_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (CO3_MAXSYM * 32 + BUF_WORDS + 4) * (int)sizeof(uint32_t));
+    cudaError_t e = cudaFuncSetAttribute(enc_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (CO3_MAXSYM * 32 + BUF_WORDS + 4) * (int)sizeof(uint32_t));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(enc_len_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                CO3_MAXSYM * 32 * (int)sizeof(uint32_t));
 }
 
-cudaError_t co3_launch_encode(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
-                              uint32_t* chunk_off, unsigned long long* user_bits, cudaStream_t st) {
+cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
+                              uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
+                              cudaStream_t st) {
     const Co3Dev& p = pl->dev;
     const int64_t items = p.n_chunks * (int64_t)p.U;
     cudaError_t e = cudaMemsetAsync(user_bits, 0, sizeof(unsigned long long) * (size_t)p.U, st);
     if (e != cudaSuccess) return e;
-    if (!g_len_bpsm) {
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_len_bpsm, enc_len_kernel, CO3_THREADS, 0);
-        if (g_len_bpsm < 1) g_len_bpsm = 1;
+    const int fi = p.nsym == 256 ? 0 : (p.nsym == 128 ? 1 : (p.nsym == 64 ? 2 : 3));
+    const size_t smem_len = (size_t)p.nsym * 32 * sizeof(uint32_t);
+    if (!g_len_bpsm[fi]) {
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_len_bpsm[fi], enc_len_kernel, CO3_THREADS, smem_len);
+        if (g_len_bpsm[fi] < 1) g_len_bpsm[fi] = 1;
     }
-    int64_t grid = (int64_t)pl->num_sms * g_len_bpsm;
+    int64_t grid = (int64_t)pl->num_sms * g_len_bpsm[fi];
     co3_prof_begin(pl, CO3_K_ENC_LEN, st);
-    enc_len_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, 0, st>>>(p, pl->cb_enc, sub_bits, user_bits);
+    enc_len_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, smem_len, st>>>(p, hdr, sub_bits, user_bits);
     co3_prof_end(pl, CO3_K_ENC_LEN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
@@ -241,14 +320,13 @@ cudaError_t co3_launch_encode(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_b
     co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const size_t smem = ((size_t)p.nsym * 32 + BUF_WORDS + 4) * sizeof(uint32_t);
-    const int fi = p.nsym == 256 ? 0 : (p.nsym == 128 ? 1 : (p.nsym == 64 ? 2 : 3));
     if (!g_pack_bpsm[fi]) {
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_pack_bpsm[fi], enc_pack_kernel, CO3_THREADS, smem);
         if (g_pack_bpsm[fi] < 1) g_pack_bpsm[fi] = 1;
     }
     grid = (int64_t)pl->num_sms * g_pack_bpsm[fi];
     co3_prof_begin(pl, CO3_K_ENC_PACK, st);
-    enc_pack_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, smem, st>>>(p, pl->cb_enc, chunk_off, bitstream);
+    enc_pack_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, smem, st>>>(p, hdr, chunk_off, bitstream);
     co3_prof_end(pl, CO3_K_ENC_PACK, st, 1);
     return cudaGetLastError();
 }

@@ -1,30 +1,26 @@
-// Small per-segment kernels between the streaming passes (sm_100a):
+// Small per-segment / per-model-row kernels (sm_100a):
 //  * fit_kernel      -- pooled moments -> GenNorm shape/scale by moment matching -> exponent bias
 //                       (Eq. "approximate") and the header indices that name the code model.
+//                       Runs once per iteration (twice when the bias is taken from the current
+//                       iteration's own moments).
 //  * huff_cand_kernel / code_finalize_kernel -- element-wise Huffman code of the quantised GenNorm
-//                       model (Sec. III (ii)), canonical codewords, encoder and decoder tables.
-// All are latency-bound (O(segments * alphabet) work); they are organised so that the serial part
-// of each (one two-queue merge of <= 255 steps) runs once, with every weight-floor candidate of
-// the depth limit in its own block.
+//                       model (Sec. III (ii)), canonical codewords, encoder and decoder tables,
+//                       for EVERY model row.  A code depends only on the format and on the two
+//                       header indices, so these run once, when the plan is created; an iteration
+//                       only selects rows.
+// All are latency-bound.  The moment ratio is inverted through a table of log R(beta) (uniform in
+// log2 beta) by a two-level parallel search and inverse cubic interpolation, so the solve costs no
+// lgamma evaluation; the depth limit of the code is resolved by building every weight-floor
+// candidate in its own block.
 #include "co3_internal.h"
 
 namespace {
 
-constexpr int FIT_THREADS = 128;
-constexpr int FIT_POINTS = 42;   // interior points per search round (3 lgamma each = 126 threads)
-constexpr int FIT_ROUNDS = 9;    // (hi - lo) shrinks by 43 per round: 1.7 / 43^9 < 4e-15
+constexpr int FIT_THREADS = 128;   // = FIT_GRID / 64: one coarse table interval per thread
 
 __device__ __forceinline__ double poly_bias(double b) {
     const double b2 = b * b;
     return 0.46 - 2.85 * b + 5.37 * b2 - 2.85 * b2 * b + 0.52 * b2 * b2;
-}
-
-// log R(beta) = lgamma(1/b) + lgamma(3/b) - 2 lgamma(2/b) at K points, three threads per point.
-__device__ void eval_logR(const double* pts, int K, double* out, double* s_lg, int tid) {
-    if (tid < 3 * K) s_lg[tid] = lgamma((double)(tid % 3 + 1) / pts[tid / 3]);
-    __syncthreads();
-    if (tid < K) out[tid] = s_lg[3 * tid] + s_lg[3 * tid + 2] - 2.0 * s_lg[3 * tid + 1];
-    __syncthreads();
 }
 
 // mode 0: after the stats pass -- write the bias for the coming convert pass.
@@ -33,21 +29,22 @@ __device__ void eval_logR(const double* pts, int K, double* out, double* s_lg, i
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr) {
     __shared__ double s_a[FIT_THREADS], s_b[FIT_THREADS];
     __shared__ unsigned long long s_n[FIT_THREADS];
-    __shared__ double s_pts[FIT_POINTS + 2], s_val[FIT_POINTS + 2], s_lg[3 * (FIT_POINTS + 2)];
-    __shared__ double s_lo, s_hi, s_target;
-    __shared__ int s_state;   // 0 search, 1 beta fixed in s_lo
+    __shared__ double s_lg[2];
+    __shared__ double s_target, s_t;        // log rho; log2(beta)
+    __shared__ int s_state, s_coarse, s_fine;
 
     const int seg = blockIdx.x, tid = threadIdx.x;
     const int c0 = p.seg_chunk0[seg], c1 = p.seg_chunk0[seg + 1];
-    const int64_t nci = c1 - c0, total = nci * p.U;
     double a1 = 0.0, a2 = 0.0;
     unsigned long long an = 0;
-    for (int64_t k = tid; k < total; k += FIT_THREADS) {
-        const int64_t u = k / nci, c = c0 + (k - u * nci);
-        const int64_t idx = u * p.n_chunks + c;
-        a1 += p.part_s1[idx];
-        a2 += p.part_s2[idx];
-        an += p.part_nf[idx];
+    for (int u = 0; u < p.U; ++u) {                       // fixed order: users, then chunks
+        const size_t base = (size_t)u * (size_t)p.n_chunks;
+#pragma unroll 4
+        for (int c = c0 + tid; c < c1; c += FIT_THREADS) {
+            a1 += p.part_s1[base + c];
+            a2 += p.part_s2[base + c];
+            an += p.part_nf[base + c];
+        }
     }
     s_a[tid] = a1; s_b[tid] = a2; s_n[tid] = an;
     __syncthreads();
@@ -58,44 +55,51 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     const double S1 = s_a[0], S2 = s_b[0];
     const unsigned long long nf = s_n[0];
     const double N = (double)((unsigned long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * (unsigned long long)p.U - nf);
-    __syncthreads();
 
-    // beta = clamp(R^-1(rho), 0.3, 2.0), rho = N S2 / S1^2, R strictly decreasing
+    // beta = clamp(R^-1(rho), 0.3, 2.0), rho = N S2 / S1^2; R is strictly decreasing in beta, and
+    // the table holds log R at log2(beta) = T0 + i * H.
+    const double T0 = log2(0.3), H = (1.0 - T0) / (double)CO3_FIT_GRID;
+    const double* tab = p.logr_tab;
     if (tid == 0) {
-        s_state = 0;
-        if (!(N > 0.0) || !(S1 > 0.0)) { s_state = 2; s_lo = 1.0; }
-        else s_target = log(N) + log(S2) - 2.0 * log(S1);
-        s_pts[0] = 0.3; s_pts[1] = 2.0;
+        s_state = 0; s_coarse = 0; s_fine = 0;
+        if (!(N > 0.0) || !(S1 > 0.0)) { s_state = 2; s_t = 0.0; }          // beta = 1, alpha = 0
+        else {
+            s_target = log(N) + log(S2) - 2.0 * log(S1);
+            if (s_target >= tab[0]) { s_state = 1; s_t = T0; }
+            else if (s_target <= tab[CO3_FIT_GRID]) { s_state = 1; s_t = 1.0; }
+        }
     }
     __syncthreads();
     if (s_state == 0) {
-        eval_logR(s_pts, 2, s_val, s_lg, tid);
+        // interval i with tab[i] > target >= tab[i+1]: coarse then fine, 64 entries each
+        constexpr int STEP = CO3_FIT_GRID / FIT_THREADS;       // 64
+        const double target = s_target;
+        if (tab[tid * STEP] > target && target >= tab[(tid + 1) * STEP]) s_coarse = tid;
+        __syncthreads();
+        if (tid < STEP) {
+            const int i = s_coarse * STEP + tid;
+            if (tab[i] > target && target >= tab[i + 1]) s_fine = i;
+        }
+        __syncthreads();
         if (tid == 0) {
-            if (s_target >= s_val[0]) { s_state = 1; s_lo = 0.3; }
-            else if (s_target <= s_val[1]) { s_state = 1; s_lo = 2.0; }
-            else { s_lo = 0.3; s_hi = 2.0; }
-        }
-        __syncthreads();
-    }
-    if (s_state == 0) {
-        for (int round = 0; round < FIT_ROUNDS; ++round) {
-            if (tid < FIT_POINTS) s_pts[tid] = s_lo + (s_hi - s_lo) * ((double)(tid + 1) / (double)(FIT_POINTS + 1));
-            __syncthreads();
-            eval_logR(s_pts, FIT_POINTS, s_val, s_lg, tid);
-            if (tid == 0) {
-                double lo = s_lo, hi = s_hi;
-                for (int k = 0; k < FIT_POINTS; ++k) {
-                    if (s_val[k] > s_target) lo = s_pts[k];
-                    else { hi = s_pts[k]; break; }
-                }
-                s_lo = lo; s_hi = hi;
+            // inverse cubic (Lagrange) interpolation of log2(beta) as a function of log R through
+            // the four grid points around the bracket
+            int i = s_fine;
+            i = i < 1 ? 1 : (i > CO3_FIT_GRID - 2 ? CO3_FIT_GRID - 2 : i);
+            double xs[4], acc = 0.0;
+            for (int k = 0; k < 4; ++k) xs[k] = tab[i - 1 + k];
+            for (int a = 0; a < 4; ++a) {
+                double term = T0 + H * (double)(i - 1 + a);
+                for (int c = 0; c < 4; ++c)
+                    if (c != a) term *= (target - xs[c]) / (xs[a] - xs[c]);
+                acc += term;
             }
-            __syncthreads();
+            s_t = acc;
         }
-        if (tid == 0) s_lo = 0.5 * (s_lo + s_hi);
         __syncthreads();
     }
-    const double beta = s_lo;
+    const double t = s_t;
+    const double beta = (s_state == 1) ? (t == T0 ? 0.3 : 2.0) : exp2(t);
     if (tid < 2) s_lg[tid] = lgamma((double)(tid + 1) / beta);
     __syncthreads();
     if (tid != 0) return;
@@ -130,26 +134,18 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     }
 }
 
-// One (segment, weight floor 2^cand) pair per block: Huffman code lengths of the floored model
+// One (model row, weight floor 2^cand) pair per block: Huffman code lengths of the floored model
 // weights.  Leaves sorted by (weight, symbol); two queues; on equal weights the leaf goes first.
-__global__ void __launch_bounds__(CO3_MAXSYM)
-huff_cand_kernel(Co3Dev p, Co3CodeBook cb, const co3_seg_header* __restrict__ hdr) {
+__global__ void __launch_bounds__(CO3_MAXSYM) huff_cand_kernel(Co3Dev p) {
     __shared__ uint32_t s_w[CO3_MAXSYM], s_sw[CO3_MAXSYM], s_iw[CO3_MAXSYM];
     __shared__ uint16_t s_ssym[CO3_MAXSYM], s_parent[2 * CO3_MAXSYM];
     __shared__ int s_max;
-    const int seg = blockIdx.x, cand = blockIdx.y, tid = threadIdx.x, n = p.nsym;
-    const co3_seg_header h = hdr[seg];
-    int ib = (int)h.ibeta, ir = (int)h.ir;
-    if (ib < CO3_IBETA_MIN || ib > CO3_IBETA_MAX || ir < CO3_IR_MIN || ir > CO3_IR_MAX) {
-        if (tid == 0 && cand == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);   // header out of range
-        ib = min(max(ib, CO3_IBETA_MIN), CO3_IBETA_MAX);
-        ir = min(max(ir, CO3_IR_MIN), CO3_IR_MAX);
-    }
-    const uint32_t* row = p.wtab + ((size_t)(ib - CO3_IBETA_MIN) * CO3_NIR + (ir - CO3_IR_MIN)) * p.J;
+    const int rowi = blockIdx.x, cand = blockIdx.y, tid = threadIdx.x, n = p.nsym;
+    const uint32_t* row = p.wtab + (size_t)rowi * p.J;
     if (tid == 0) s_max = 0;
     if (tid < n) {
         const int j = tid & (p.J - 1);
-        const uint32_t w = ((tid >> p.nm) && j == 0) ? 1u : row[j];
+        const uint32_t w = ((tid >> p.nm) && j == 0) ? 1u : row[j];     // "-0" is never emitted
         s_w[tid] = max(w, 1u << cand);
     }
     __syncthreads();
@@ -172,7 +168,7 @@ huff_cand_kernel(Co3Dev p, Co3CodeBook cb, const co3_seg_header* __restrict__ hd
             uint32_t sum = 0;
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
-                if (lw <= iw) {                      // leaf first on ties; lw = UINT_MAX when exhausted
+                if (lw <= iw) {                      // leaf first on ties; UINT_MAX when exhausted
                     sum += lw;
                     s_parent[i] = (uint16_t)(n + k);
                     ++i;
@@ -194,31 +190,31 @@ huff_cand_kernel(Co3Dev p, Co3CodeBook cb, const co3_seg_header* __restrict__ hd
         int node = tid, depth = 0;
         while (node != root && depth <= CO3_MAXLEN) { node = s_parent[node]; ++depth; }
         atomicMax(&s_max, depth);
-        cb.cand_len[((size_t)seg * CO3_NCAND + cand) * CO3_MAXSYM + s_ssym[tid]] = (uint8_t)depth;
+        p.cb.cand_len[((size_t)rowi * CO3_NCAND + cand) * CO3_MAXSYM + s_ssym[tid]] = (uint8_t)depth;
     }
     __syncthreads();
-    if (tid == 0) cb.cand_max[seg * CO3_NCAND + cand] = s_max;
+    if (tid == 0) p.cb.cand_max[rowi * CO3_NCAND + cand] = s_max;
 }
 
-// Per segment: take the smallest floor whose code is at most 16 deep, assign canonical
-// codewords (symbols ordered by (length, symbol)), and write the encoder table and, if asked,
-// the decoder tables (11-bit primary table + canonical arrays for the rare longer codewords).
-__global__ void __launch_bounds__(CO3_MAXSYM)
-code_finalize_kernel(Co3Dev p, Co3CodeBook cb, int want_decode) {
+// Per model row: take the smallest floor whose code is at most 16 deep, assign canonical
+// codewords (symbols ordered by (length, symbol)), and write the encoder table and the decoder
+// tables (11-bit primary table + canonical arrays for the rare longer codewords).
+__global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p) {
     __shared__ uint8_t s_len[CO3_MAXSYM], s_perm[CO3_MAXSYM];
     __shared__ uint32_t s_count[CO3_MAXLEN + 2], s_first[CO3_MAXLEN + 2], s_offs[CO3_MAXLEN + 2];
     __shared__ int s_sel;
-    const int seg = blockIdx.x, tid = threadIdx.x, n = p.nsym;
+    const Co3CodeBook& cb = p.cb;
+    const int rowi = blockIdx.x, tid = threadIdx.x, n = p.nsym;
     if (tid == 0) {
         int sel = CO3_NCAND - 1;
         for (int c = 0; c < CO3_NCAND; ++c)
-            if (cb.cand_max[seg * CO3_NCAND + c] <= CO3_MAXLEN) { sel = c; break; }
+            if (cb.cand_max[rowi * CO3_NCAND + c] <= CO3_MAXLEN) { sel = c; break; }
         s_sel = sel;
     }
     if (tid < CO3_MAXLEN + 2) s_count[tid] = 0;
     __syncthreads();
     if (tid < n) {
-        const uint8_t L = cb.cand_len[((size_t)seg * CO3_NCAND + s_sel) * CO3_MAXSYM + tid];
+        const uint8_t L = cb.cand_len[((size_t)rowi * CO3_NCAND + s_sel) * CO3_MAXSYM + tid];
         s_len[tid] = L;
         atomicAdd(&s_count[L], 1u);
     }
@@ -238,18 +234,17 @@ code_finalize_kernel(Co3Dev p, Co3CodeBook cb, int want_decode) {
         for (int s = 0; s < tid; ++s) r += (s_len[s] == L);
         const uint32_t code = s_first[L] + r;
         const uint32_t rev = __brev(code) >> (32 - L);
-        const size_t o = (size_t)seg * CO3_MAXSYM + tid;
+        const size_t o = (size_t)rowi * CO3_MAXSYM + tid;
         cb.len8[o] = (uint8_t)L;
         cb.enc[o] = rev | ((uint32_t)L << 16);
         cb.code_msb[o] = code;
         s_perm[s_offs[L] + r] = (uint8_t)tid;
-        if (want_decode) cb.ksign[o] = co3_ksigned(tid, p.M, p.nm);
+        if (rowi == 0) cb.ksign[tid] = co3_ksigned(tid, p.M, p.nm);
     }
     __syncthreads();
-    if (!want_decode) return;
-    if (tid < n) cb.perm[(size_t)seg * CO3_MAXSYM + tid] = s_perm[tid];
+    if (tid < n) cb.perm[(size_t)rowi * CO3_MAXSYM + tid] = s_perm[tid];
     if (tid <= CO3_MAXLEN) {
-        const size_t o = (size_t)seg * (CO3_MAXLEN + 1) + tid;
+        const size_t o = (size_t)rowi * (CO3_MAXLEN + 1) + tid;
         cb.first[o] = tid ? s_first[tid] : 0;
         cb.count[o] = tid ? s_count[tid] : 0;
         cb.offs[o] = tid ? s_offs[tid] : 0;
@@ -265,7 +260,7 @@ code_finalize_kernel(Co3Dev p, Co3CodeBook cb, int want_decode) {
                 break;
             }
         }
-        cb.lut[(size_t)seg * CO3_LUT_SIZE + i] = entry;
+        cb.lut[(size_t)rowi * CO3_LUT_SIZE + i] = entry;
     }
 }
 
@@ -278,17 +273,12 @@ cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStre
     return cudaGetLastError();
 }
 
-cudaError_t co3_launch_codebook(co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
-                                int want_decode_tables, cudaStream_t st) {
-    const int k = want_decode_tables ? CO3_K_CODE_DEC : CO3_K_CODE_ENC;
-    dim3 grid(pl->dev.S, CO3_NCAND);
-    co3_prof_begin(pl, k, st);
-    huff_cand_kernel<<<grid, CO3_MAXSYM, 0, st>>>(pl->dev, cb, hdr);
+// Builds the code tables of all model rows (plan creation).
+cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st) {
+    dim3 grid(CO3_NROWS, CO3_NCAND);
+    huff_cand_kernel<<<grid, CO3_MAXSYM, 0, st>>>(pl->dev);
     cudaError_t e = cudaGetLastError();
-    if (e == cudaSuccess) {
-        code_finalize_kernel<<<pl->dev.S, CO3_MAXSYM, 0, st>>>(pl->dev, cb, want_decode_tables);
-        e = cudaGetLastError();
-    }
-    co3_prof_end(pl, k, st, 2);
-    return e;
+    if (e != cudaSuccess) return e;
+    code_finalize_kernel<<<CO3_NROWS, CO3_MAXSYM, 0, st>>>(pl->dev);
+    return cudaGetLastError();
 }

@@ -14,6 +14,8 @@ constexpr int CO3_NCAND = 10;       // weight floors 2^0 .. 2^9 tried in paralle
 constexpr int CO3_NIBETA = 23;      // ibeta in [-14, 8]
 constexpr int CO3_NIR = 128;        // ir in [-96, 31]
 constexpr int CO3_IBETA_MIN = -14, CO3_IBETA_MAX = 8, CO3_IR_MIN = -96, CO3_IR_MAX = 31;
+constexpr int CO3_NROWS = CO3_NIBETA * CO3_NIR;   // model rows (codes) per format
+constexpr int CO3_FIT_GRID = 8192;  // log R(beta) is tabulated at FIT_GRID + 1 points, uniform in log2 beta
 constexpr int CO3_MAXSYM = 256;     // alphabet rows are padded to 256 entries
 constexpr int CO3_STAGE_WORDS = 1024;  // shared-memory staging per (chunk, user) stream in decode
 constexpr int CO3_THREADS = 256;
@@ -36,20 +38,22 @@ struct Co3Group {
     int32_t pad_;
 };
 
-// Per-segment code tables built on the device from the header (one instance for the encoder,
-// one for the decoder; rows are CO3_MAXSYM / CO3_LUT_SIZE wide).
+// Code tables for every model row r = (ibeta - IBETA_MIN) * NIR + (ir - IR_MIN).  The Huffman
+// code of a segment is a pure function of the format and of the two header indices, so all
+// CO3_NROWS codes are built on the device once, when the plan is created; an iteration only
+// selects rows.  Rows are CO3_MAXSYM / CO3_LUT_SIZE wide.
 struct Co3CodeBook {
-    uint8_t* cand_len;   // [S][NCAND][256] code lengths per weight-floor candidate
-    int32_t* cand_max;   // [S][NCAND]      longest codeword per candidate
-    uint8_t* len8;       // [S][256]        chosen lengths
-    uint32_t* enc;       // [S][256]        bit-reversed codeword | length << 16
-    uint32_t* code_msb;  // [S][256]        canonical codeword, root bit most significant
-    uint32_t* lut;       // [S][2048]       (signed magnitude << 8) | length, 0 = longer than 11 bits
-    uint32_t* first;     // [S][17]         first canonical code of each length
-    uint32_t* count;     // [S][17]
-    uint32_t* offs;      // [S][17]         start of each length in perm
-    uint8_t* perm;       // [S][256]        symbols ordered by (length, symbol)
-    int32_t* ksign;      // [S][256]        signed integer magnitude of each symbol
+    uint8_t* cand_len;   // [R][NCAND][256] code lengths per weight-floor candidate (build scratch)
+    int32_t* cand_max;   // [R][NCAND]      longest codeword per candidate (build scratch)
+    uint8_t* len8;       // [R][256]        chosen lengths
+    uint32_t* enc;       // [R][256]        bit-reversed codeword | length << 16
+    uint32_t* code_msb;  // [R][256]        canonical codeword, root bit most significant
+    uint32_t* lut;       // [R][2048]       (signed magnitude << 8) | length, 0 = longer than 11 bits
+    uint32_t* first;     // [R][17]         first canonical code of each length
+    uint32_t* count;     // [R][17]
+    uint32_t* offs;      // [R][17]         start of each length in perm
+    uint8_t* perm;       // [R][256]        symbols ordered by (length, symbol)
+    int32_t* ksign;      // [256]           signed integer magnitude of each symbol
 };
 
 // Everything the kernels need, passed by value.
@@ -71,6 +75,8 @@ struct Co3Dev {
     double* fit;                  // [S][5] beta, alpha, N, S1, S2
     int32_t* bias_cur;            // [S] bias used by the next convert pass
     const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
+    const double* logr_tab;       // [FIT_GRID + 1] log R(beta) at log2(beta) uniform in [log2 0.3, 1]
+    Co3CodeBook cb;               // code tables of all model rows
     uint32_t* chunk_words;        // [U][n_chunks]
     uint32_t* user_ovf;           // [U] 1 if the user's payload exceeds cap_words
     uint32_t* flags;              // sticky status flags
@@ -80,11 +86,11 @@ struct Co3Dev {
 struct co3_plan {
     co3_config cfg;
     Co3Dev dev;
-    Co3CodeBook cb_enc, cb_dec;
     int64_t iteration;
     int64_t worst_case_words;
     int device;
     int num_sms;
+    int grid_stats, grid_convert;   // launch grids (fixed per plan: they define the reduction order)
     cudaStream_t last_stream;
     void* allocs[64];
     int n_allocs;
@@ -119,19 +125,31 @@ int co3_host_fmt_ok(co3_format f);
 int co3_host_cF(int E, int M);
 int64_t co3_host_K(int M, int j);
 const uint32_t* co3_host_weight_table(int E, int M);   // [NIBETA][NIR][J], cached per format
+const double* co3_host_logr_table(void);               // [FIT_GRID + 1], cached
 
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st);
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st);
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
-cudaError_t co3_launch_codebook(co3_plan* pl, const Co3CodeBook& cb, const co3_seg_header* hdr,
-                                int want_decode_tables, cudaStream_t st);
-cudaError_t co3_launch_encode(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits,
-                              uint32_t* chunk_off, unsigned long long* user_bits, cudaStream_t st);
+cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st);
+cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
+                              uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
+                              cudaStream_t st);
 cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
                               cudaStream_t st);
 cudaError_t co3_setup_kernels(void);
+
+// Model row of a segment header; out-of-range indices (a corrupt header) are clamped and reported.
+__host__ __device__ inline int co3_row_of(const co3_seg_header h, bool* bad) {
+    int ib = (int)h.ibeta, ir = (int)h.ir;
+    if (ib < CO3_IBETA_MIN || ib > CO3_IBETA_MAX || ir < CO3_IR_MIN || ir > CO3_IR_MAX) {
+        *bad = true;
+        ib = ib < CO3_IBETA_MIN ? CO3_IBETA_MIN : (ib > CO3_IBETA_MAX ? CO3_IBETA_MAX : ib);
+        ir = ir < CO3_IR_MIN ? CO3_IR_MIN : (ir > CO3_IR_MAX ? CO3_IR_MAX : ir);
+    }
+    return (ib - CO3_IBETA_MIN) * CO3_NIR + (ir - CO3_IR_MIN);
+}
 
 // Signed integer magnitude of a symbol byte: K(j) = f (e = 0) or (2^M + f) << (e - 1).
 __host__ __device__ inline int32_t co3_ksigned(int sym, int M, int nm) {

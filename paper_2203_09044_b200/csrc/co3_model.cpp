@@ -123,6 +123,24 @@ const uint32_t* co3_host_weight_table(int E, int M) {
     return t;
 }
 
+// log R(beta) = lgamma(1/b) + lgamma(3/b) - 2 lgamma(2/b) on a grid uniform in log2(beta) over
+// [log2 0.3, log2 2]; the device inverts it by inverse cubic interpolation (the moment ratio of a
+// GenNorm sample determines its shape).
+const double* co3_host_logr_table(void) {
+    static double* tab = nullptr;
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (tab) return tab;
+    double* t = (double*)malloc(sizeof(double) * (CO3_FIT_GRID + 1));
+    if (!t) return nullptr;
+    const double t0 = log2(0.3), t1 = 1.0;
+    for (int i = 0; i <= CO3_FIT_GRID; ++i) {
+        double b = (i == 0) ? 0.3 : (i == CO3_FIT_GRID ? 2.0 : exp2(t0 + (t1 - t0) * ((double)i / CO3_FIT_GRID)));
+        t[i] = lgamma(1.0 / b) + lgamma(3.0 / b) - 2.0 * lgamma(2.0 / b);
+    }
+    tab = t;
+    return tab;
+}
+
 extern "C" int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint32_t* weights) {
     if (!co3_host_fmt_ok(fmt) || !weights || ibeta < CO3_IBETA_MIN || ibeta > CO3_IBETA_MAX ||
         ir < CO3_IR_MIN || ir > CO3_IR_MAX)

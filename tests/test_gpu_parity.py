@@ -37,7 +37,7 @@ def compare_iteration(b, plan, out, r, m_gpu, m_cpu, tag=""):
         np.testing.assert_allclose([beta, alpha], r.fit[l], rtol=1e-5, err_msg=f"{tag} fit")
     hdr = b.hdr_to_numpy(out["hdr"])
     assert np.array_equal(hdr, r.hdr), f"{tag} header {hdr[hdr != r.hdr]} vs {r.hdr[hdr != r.hdr]}"
-    lens, codes = plan.debug_code()
+    lens, codes = plan.debug_code(out["hdr"])
     assert np.array_equal(lens, r.lens), f"{tag} code lengths"
     assert np.array_equal(codes, r.codes), f"{tag} codewords"
     co = out["chunk_off"].cpu().numpy().view(np.uint32)
