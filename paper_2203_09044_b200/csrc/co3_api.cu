@@ -220,6 +220,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.fit, (size_t)S * 5);
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
         a |= dev_alloc(pl, &dv.chunk_words, items);
+        a |= dev_alloc(pl, &dv.chunk_bits, items);
         a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);

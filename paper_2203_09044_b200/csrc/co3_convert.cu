@@ -8,212 +8,271 @@
 // in the row, so segment boundaries never misalign the vectors; the vectors that straddle a
 // chunk edge are handled element by element.
 //
-// Work item = (user, chunk).  Blocks are persistent and take contiguous item ranges, so a block
-// stays inside one segment for long stretches: the histogram lives in shared memory (one copy
-// per warp) and is flushed with 64-bit global atomics only when the segment changes.  Moments
-// are reduced in a fixed order per item and stored per item, so the fit does not depend on the
-// launch geometry or on scheduling.  A thread handles one 4-element vector per step (4 steps per
-// item) and always has the next step's two 128-bit loads in flight (register double buffer that
-// runs across item boundaries), so with four resident blocks per SM the memory system stays full
-// while the conversion arithmetic runs.
+// Work item = (user, chunk).  Blocks are persistent and take every gridDim-th item, so a block
+// meets its segments in order and stays inside one for long stretches, while the grid as a whole
+// sweeps one window of memory: the histogram lives in shared memory (one copy
+// per warp) and is flushed with 64-bit global atomics only when the segment changes; the moments
+// are kept per thread over such a run of items and reduced in a fixed order once per run (the
+// sum lands in the per-item array at the run's last item, zeros elsewhere), so there is no
+// barrier inside a run and the fit does not depend on scheduling.
+//
+// Memory pipeline: a thread handles one 4-element vector of g and of m per step (4 steps per
+// item).  The loads are asynchronous copies (cp.async, 16 B, L2-only) into thread-private slots of
+// a 4-stage shared-memory ring that runs across item boundaries, so three steps (24 KB per block)
+// are always in flight without holding registers, and no barrier is needed: a thread only ever
+// reads the slots it filled itself, after cp.async.wait_group.
 #include "co3_internal.h"
 
 namespace {
 
 constexpr int STEPS = CO3_TILE / (4 * CO3_THREADS);   // vectors per thread per item (4)
+constexpr int STAGES = 4;                             // ring depth of the asynchronous copies
 
-struct QParams {
-    int lambda;        // grid value = K * 2^lambda
-    float inv_scale;   // 2^-lambda
-    float top;         // K_max * 2^lambda
+struct QParams {                 // per segment
+    float top;                   // K_max * 2^lambda: largest grid value (grid value = K * 2^lambda)
+    uint32_t low_bits;           // bits of 2^(lambda + M): below it the quantum stays 2^lambda
+    uint32_t e0;                 // exponent field of 1.5 * 2^(lambda + 23): lambda + 150
 };
 
 __device__ __forceinline__ float pow2f(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
 
-// Q_fp on one element.  Round-to-nearest-even at the quantum of a's binade (or the subnormal
-// quantum 2^lambda, whichever is larger) by adding and subtracting 1.5 * 2^(qe+23); saturate;
-// then read the magnitude code off the bits of the integer magnitude.  M = mantissa bits,
-// NM = exponent + mantissa bits (position of the sign in the symbol byte).
-template <int M, bool CONVERT>
-__device__ __forceinline__ void ef_element(float g, float m, float gamma, const QParams& q, int nm,
-                                           uint32_t& sym, float& m_new, double& s1, double& s2,
-                                           uint32_t& nf) {
-    const float a = __fadd_rn(g, __fmul_rn(gamma, m));
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+// Q_fp on one finite element, branch-free.  |a| (clamped to the top grid value) is rounded to
+// nearest even at the quantum 2^qe of its binade -- or the subnormal quantum 2^lambda, whichever
+// is larger -- by adding 1.5 * 2^(qe+23): the sum t holds n = |a| / 2^qe rounded, as an integer, in
+// its low mantissa bits, and subtracting the constant again gives the rounded value r.  The
+// magnitude code is j = ((qe - lambda) << M) + n for every binade (n < 2^(M+1) below the second
+// binade, where it is the code itself; 2^M <= n <= 2^(M+1) above, where it carries the mantissa
+// and, on a carry, the next exponent).
+template <int M>
+__device__ __forceinline__ void quantize(float a, const QParams& q, int sign_shift, uint32_t& sym, float& m_new) {
     const uint32_t ab = __float_as_uint(a);
-    if ((ab & 0x7F800000u) == 0x7F800000u) {  // NaN / Inf: counted, coded as +0, memory reset
-        nf += 1;
-        sym = 0;
-        m_new = 0.0f;
-        return;
+    const float axc = fminf(fabsf(a), q.top);
+    // exponent field of max(|a|, 2^(lambda+M)), moved up by 23 - M binades, plus the 1.5
+    const uint32_t mb = (max(__float_as_uint(axc), q.low_bits) & 0x7F800000u) + (((23u - M) << 23) | 0x400000u);
+    const float magic = __uint_as_float(mb);
+    const float t = __fadd_rn(axc, magic);
+    const float r = __fsub_rn(t, magic);      // multiple of 2^qe, <= top
+    const uint32_t tb = __float_as_uint(t);
+    const uint32_t j = (((tb >> 23) - q.e0) << M) + (tb & 0x3FFFFFu);
+    const uint32_t sb = (r != 0.0f) ? (ab & 0x80000000u) : 0u;  // "-0" is never emitted
+    sym = j | (sb >> sign_shift);
+    m_new = __fsub_rn(a, __uint_as_float(__float_as_uint(r) | sb));
+}
+
+// a = g + gamma m for the four elements of a vector; moments of the finite ones; NaN/Inf are
+// counted and replaced by 0 (so they are coded as +0 and their memory is reset to 0).
+__device__ __forceinline__ void ef_add4(const float4& gv, const float4& mv, float gamma, float a[4],
+                                        double& s1, double& s2, uint32_t& nf) {
+    a[0] = __fadd_rn(gv.x, __fmul_rn(gamma, mv.x));
+    a[1] = __fadd_rn(gv.y, __fmul_rn(gamma, mv.y));
+    a[2] = __fadd_rn(gv.z, __fmul_rn(gamma, mv.z));
+    a[3] = __fadd_rn(gv.w, __fmul_rn(gamma, mv.w));
+    const uint32_t big = max(max(__float_as_uint(a[0]) & 0x7FFFFFFFu, __float_as_uint(a[1]) & 0x7FFFFFFFu),
+                             max(__float_as_uint(a[2]) & 0x7FFFFFFFu, __float_as_uint(a[3]) & 0x7FFFFFFFu));
+    if (big >= 0x7F800000u) {                 // rare: some element is NaN or Inf
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if ((__float_as_uint(a[e]) & 0x7FFFFFFFu) >= 0x7F800000u) { a[e] = 0.0f; ++nf; }
     }
-    const float ax = fabsf(a);
-    const double ad = (double)ax;
-    s1 += ad;
-    s2 = __fma_rn(ad, ad, s2);                // ad*ad is exact in double, so this rounds once
-    if (!CONVERT) return;
-    const float axc = fminf(ax, q.top);
-    const int qe = max((int)(__float_as_uint(axc) >> 23) - (127 + M), q.lambda);
-    const float magic = __uint_as_float((uint32_t)(qe << 23) + ((150u << 23) | 0x400000u));
-    const float r = __fsub_rn(__fadd_rn(axc, magic), magic);   // multiple of 2^qe, <= top
-    const float kf = __fmul_rn(r, q.inv_scale);                 // integer magnitude, exact
-    const uint32_t k = (uint32_t)kf;
-    const uint32_t j = (k < (2u << M)) ? k : ((__float_as_uint(kf) >> (23 - M)) - ((uint32_t)(127 + M - 1) << M));
-    const uint32_t s = (k != 0) ? (ab >> 31) : 0u;
-    sym = (s << nm) | j;
-    m_new = __fsub_rn(a, __uint_as_float(__float_as_uint(r) | (s << 31)));
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const double ad = (double)fabsf(a[e]);
+        s1 += ad;
+        s2 = __fma_rn(ad, ad, s2);            // ad*ad is exact in double, so this rounds once
+    }
 }
 
 struct ItemCtx {                  // what a step needs to know about its item
-    const float* gr;              // row pointers at the start of the item's tile
-    float* mr;
-    uint8_t* sr;
-    int lo, hi;                   // the item's elements within the tile
+    const float* gp;              // this thread's first vector of the item's tile (g, m, symbols)
+    float* mp;
+    uint8_t* sp;
+    int lo, hi, seg;              // the item's elements within the tile; its segment
+    bool whole;                   // the item covers its whole tile: no edge handling
 };
 
 template <int M, bool CONVERT>
-__global__ void __launch_bounds__(CO3_THREADS, CONVERT ? 4 : 4)
+__global__ void __launch_bounds__(CO3_THREADS, 4)
 ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
+    extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS]
     __shared__ uint32_t s_hist[CONVERT ? CO3_THREADS / 32 : 1][CO3_MAXSYM];
-    __shared__ double s_red[2][2][CO3_THREADS / 32];
-    __shared__ uint32_t s_rednf[2][CO3_THREADS / 32];
+    __shared__ double s_red[2][CO3_THREADS / 32];
+    __shared__ uint32_t s_rednf[CO3_THREADS / 32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // items blockIdx.x, blockIdx.x + gridDim.x, ...: at any time the blocks of the grid work on
+    // neighbouring chunks, so the whole GPU sweeps one window of each array (DRAM page and L2
+    // locality of a streaming copy) while a block still meets its segments in order
     const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.U;
-    const uint32_t per = (n_items + gridDim.x - 1) / gridDim.x;
-    const uint32_t it0 = blockIdx.x * per;
-    const uint32_t it1 = min(n_items, it0 + per);
+    const uint32_t it0 = blockIdx.x, it1 = n_items, stride = gridDim.x;
     if (it0 >= it1) return;
 
     if (CONVERT) {
         for (int i = tid; i < (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
         __syncthreads();
     }
-    const int nm = p.nm;
+    const int sign_shift = 31 - p.nm;
     const uint32_t n_chunks = (uint32_t)p.n_chunks;
-    uint32_t u = it0 / n_chunks, c = it0 - u * n_chunks;
+    constexpr int VSTRIDE = 4 * CO3_THREADS;          // elements between a thread's vectors
 
-    auto make_ctx = [&](uint32_t uu, const Co3Chunk& cd) {
+    auto make_ctx = [&](uint32_t uu, uint32_t cc) {
+        const Co3Chunk cd = p.chunks[cc];
         ItemCtx x;
         const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-        x.gr = g + (size_t)uu * p.ld + tb;
-        x.mr = m + (size_t)uu * p.ld + tb;
-        x.sr = p.sym + (size_t)uu * p.sld + tb;
+        x.gp = g + (size_t)uu * p.ld + tb + 4 * tid;
+        x.mp = m + (size_t)uu * p.ld + tb + 4 * tid;
+        x.sp = p.sym + (size_t)uu * p.sld + tb + 4 * tid;
         x.lo = (int)(cd.start - tb);
         x.hi = x.lo + cd.len;
+        x.seg = cd.seg;
+        x.whole = cd.len == CO3_TILE;
         return x;
     };
-    auto load_step = [&](const ItemCtx& x, int r, float4& gv, float4& mv) {
-        const int e0 = 4 * (tid + CO3_THREADS * r);
-        if (e0 < x.hi && e0 + 4 > x.lo) {
-            gv = __ldg(reinterpret_cast<const float4*>(x.gr + e0));
-            mv = *reinterpret_cast<const float4*>(x.mr + e0);
+    const uint32_t ring_g = (uint32_t)__cvta_generic_to_shared(s_ring + tid);
+    const uint32_t ring_m = (uint32_t)__cvta_generic_to_shared(s_ring + CO3_THREADS + tid);
+    constexpr uint32_t SLOT_BYTES = 2 * CO3_THREADS * sizeof(float4);
+
+    // producer cursor (runs STAGES-1 steps ahead of the consumer)
+    uint32_t pu = it0 / n_chunks, pc = it0 - pu * n_chunks, pitem = it0;
+    int pr = 0;
+    uint32_t pslot = 0;
+    ItemCtx pctx = make_ctx(pu, pc);
+    auto produce = [&]() {
+        if (pitem < it1) {
+            const int e0 = 4 * tid + VSTRIDE * pr;
+            if (pctx.whole || (e0 < pctx.hi && e0 + 4 > pctx.lo)) {
+                cp_async16(ring_g + pslot, pctx.gp + VSTRIDE * pr);
+                cp_async16(ring_m + pslot, pctx.mp + VSTRIDE * pr);
+            }
+            if (++pr == STEPS) {
+                pr = 0;
+                pitem += stride;
+                pc += stride;
+                while (pc >= n_chunks) { pc -= n_chunks; ++pu; }
+                if (pitem < it1) pctx = make_ctx(pu, pc);
+            }
         }
+        cp_async_commit();                            // one group per step, even if empty
+        pslot = (pslot + SLOT_BYTES == STAGES * SLOT_BYTES) ? 0 : pslot + SLOT_BYTES;
     };
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) produce();
 
-    Co3Chunk cd = p.chunks[c];
-    ItemCtx cur = make_ctx(u, cd);
-    float4 gbuf[2], mbuf[2];
-    load_step(cur, 0, gbuf[0], mbuf[0]);
-
+    // consumer cursor
+    uint32_t cu = it0 / n_chunks, cc = it0 - cu * n_chunks;
+    ItemCtx cur = make_ctx(cu, cc);
+    uint32_t cslot = 0;
     int cur_seg = -1;
     QParams q;
-    q.lambda = 0; q.inv_scale = 1.0f; q.top = 0.0f;
+    q.top = 0.0f; q.low_bits = 0; q.e0 = 0;
 
-    for (uint32_t item = it0; item < it1; ++item) {
-        if (CONVERT && cd.seg != cur_seg) {
-            if (cur_seg >= 0) {               // flush the histogram of the segment just left
-                __syncthreads();
-                if (tid < p.nsym) {
-                    unsigned long long tot = 0;
-#pragma unroll
-                    for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[w][tid]; s_hist[w][tid] = 0; }
-                    if (tot) atomicAdd(&p.hist[(size_t)cur_seg * CO3_MAXSYM + tid], tot);
-                }
-                __syncthreads();
-            }
-            cur_seg = cd.seg;
-            q.lambda = p.bias_cur[cd.seg] + p.cF;
-            q.inv_scale = pow2f(-q.lambda);
-            q.top = __fmul_rn((float)p.Kmax, pow2f(q.lambda));
-        }
-        // the next item (for the prefetch that crosses the item boundary)
-        uint32_t un = u, cn = c + 1;
-        if (cn == n_chunks) { cn = 0; ++un; }
-        const bool has_next = item + 1 < it1;
-        Co3Chunk cdn = cd;
-        ItemCtx nxt = cur;
-        if (has_next) { cdn = p.chunks[cn]; nxt = make_ctx(un, cdn); }
-
-        double s1 = 0.0, s2 = 0.0;
-        uint32_t nf = 0;
-#pragma unroll
-        for (int r = 0; r < STEPS; ++r) {
-            // keep the next step's loads in flight while this one is converted
-            if (r + 1 < STEPS) load_step(cur, r + 1, gbuf[(r + 1) & 1], mbuf[(r + 1) & 1]);
-            else if (has_next) load_step(nxt, 0, gbuf[0], mbuf[0]);
-            const int e0 = 4 * (tid + CO3_THREADS * r);
-            if (!(e0 < cur.hi && e0 + 4 > cur.lo)) continue;
-            const float4 gv = gbuf[r & 1], mv = mbuf[r & 1];
-            const float ge[4] = {gv.x, gv.y, gv.z, gv.w};
-            const float me[4] = {mv.x, mv.y, mv.z, mv.w};
-            float mo[4];
-            uint32_t so[4];
-            const bool full = (e0 >= cur.lo) && (e0 + 4 <= cur.hi);
-            if (full) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    ef_element<M, CONVERT>(ge[e], me[e], p.gamma, q, nm, so[e], mo[e], s1, s2, nf);
-                    if (CONVERT) atomicAdd(&s_hist[warp][so[e]], 1u);
-                }
-                if (CONVERT) {
-                    *reinterpret_cast<float4*>(cur.mr + e0) = make_float4(mo[0], mo[1], mo[2], mo[3]);
-                    *reinterpret_cast<uint32_t*>(cur.sr + e0) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (e0 + e >= cur.lo && e0 + e < cur.hi) {
-                        ef_element<M, CONVERT>(ge[e], me[e], p.gamma, q, nm, so[e], mo[e], s1, s2, nf);
-                        if (CONVERT) {
-                            atomicAdd(&s_hist[warp][so[e]], 1u);
-                            cur.mr[e0 + e] = mo[e];
-                            cur.sr[e0 + e] = (uint8_t)so[e];
-                        }
-                    }
-                }
-            }
-        }
-        // fixed-order reduction of this item's moments: lanes, then warps
+    // reduce the moments of the run of items that ends with `last_item` and start a new run
+    double s1 = 0.0, s2 = 0.0;
+    uint32_t nf = 0;
+    auto close_run = [&](uint32_t last_item, int seg) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             s1 += __shfl_down_sync(0xffffffffu, s1, o);
             s2 += __shfl_down_sync(0xffffffffu, s2, o);
             nf += __shfl_down_sync(0xffffffffu, nf, o);
         }
-        const int par = (int)(item & 1);
-        if (lane == 0) { s_red[par][0][warp] = s1; s_red[par][1][warp] = s2; s_rednf[par][warp] = nf; }
+        if (lane == 0) { s_red[0][warp] = s1; s_red[1][warp] = s2; s_rednf[warp] = nf; }
         __syncthreads();
         if (tid == 0) {
             double t1 = 0.0, t2 = 0.0;
             uint32_t tn = 0;
 #pragma unroll
-            for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
-            p.part_s1[item] = t1; p.part_s2[item] = t2; p.part_nf[item] = tn;
+            for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[0][w]; t2 += s_red[1][w]; tn += s_rednf[w]; }
+            p.part_s1[last_item] = t1; p.part_s2[last_item] = t2; p.part_nf[last_item] = tn;
         }
-        u = un; c = cn; cd = cdn; cur = nxt;
-    }
-    if (CONVERT && cur_seg >= 0) {
-        __syncthreads();
-        if (tid < p.nsym) {
+        if (CONVERT && tid < p.nsym) {                // flush the histogram of the run's segment
             unsigned long long tot = 0;
 #pragma unroll
-            for (int w = 0; w < CO3_THREADS / 32; ++w) tot += s_hist[w][tid];
-            if (tot) atomicAdd(&p.hist[(size_t)cur_seg * CO3_MAXSYM + tid], tot);
+            for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[w][tid]; s_hist[w][tid] = 0; }
+            if (tot) atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + tid], tot);
+        }
+        __syncthreads();
+        s1 = 0.0; s2 = 0.0; nf = 0;
+    };
+
+    uint32_t last = it0;
+    for (uint32_t item = it0; item < it1; item += stride) {
+        if (cur.seg != cur_seg) {
+            if (cur_seg >= 0) close_run(item - stride, cur_seg);
+            cur_seg = cur.seg;
+            if (CONVERT) {
+                const int lambda = p.bias_cur[cur.seg] + p.cF;
+                q.top = __fmul_rn((float)p.Kmax, pow2f(lambda));
+                q.low_bits = __float_as_uint(pow2f(lambda + M));
+                q.e0 = (uint32_t)(lambda + 150);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < STEPS; ++r) {
+            produce();                                // step (this + STAGES - 1) goes in flight
+            cp_async_wait<STAGES - 1>();              // this step's copies have landed
+            const uint32_t slot = cslot;
+            cslot = (cslot + SLOT_BYTES == STAGES * SLOT_BYTES) ? 0 : cslot + SLOT_BYTES;
+            const int e0 = 4 * tid + VSTRIDE * r;
+            const bool full = cur.whole || ((e0 >= cur.lo) && (e0 + 4 <= cur.hi));
+            if (!full && !(e0 < cur.hi && e0 + 4 > cur.lo)) continue;
+            float4 gv = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_ring + tid) + slot);
+            float4 mv = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_ring + CO3_THREADS + tid) + slot);
+            float a[4], mo[4];
+            uint32_t so[4];
+            if (full) {
+                ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
+                if (CONVERT) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        quantize<M>(a[e], q, sign_shift, so[e], mo[e]);
+                        atomicAdd(&s_hist[warp][so[e]], 1u);
+                    }
+                    *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+                    *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
+                }
+            } else {                                  // a vector on the chunk's edge: element by element
+                const bool in0 = e0 >= cur.lo && e0 < cur.hi, in1 = e0 + 1 >= cur.lo && e0 + 1 < cur.hi;
+                const bool in2 = e0 + 2 >= cur.lo && e0 + 2 < cur.hi, in3 = e0 + 3 >= cur.lo && e0 + 3 < cur.hi;
+                const bool in[4] = {in0, in1, in2, in3};
+                if (!in0) { gv.x = 0.0f; mv.x = 0.0f; }   // elements of the neighbouring chunk count as 0
+                if (!in1) { gv.y = 0.0f; mv.y = 0.0f; }
+                if (!in2) { gv.z = 0.0f; mv.z = 0.0f; }
+                if (!in3) { gv.w = 0.0f; mv.w = 0.0f; }
+                ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
+                if (CONVERT) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (in[e]) {
+                            quantize<M>(a[e], q, sign_shift, so[e], mo[e]);
+                            atomicAdd(&s_hist[warp][so[e]], 1u);
+                            cur.mp[VSTRIDE * r + e] = mo[e];
+                            cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
+                        }
+                    }
+                }
+            }
+        }
+        last = item;
+        if (item + stride < it1) {
+            if (tid == 0) { p.part_s1[item] = 0.0; p.part_s2[item] = 0.0; p.part_nf[item] = 0; }
+            cc += stride;
+            while (cc >= n_chunks) { cc -= n_chunks; ++cu; }
+            cur = make_ctx(cu, cc);
         }
     }
+    cp_async_wait<0>();
+    close_run(last, cur_seg);
 }
 
 typedef void (*ef_fn)(Co3Dev, const float*, float*);
+constexpr size_t RING_BYTES = (size_t)STAGES * 2 * CO3_THREADS * sizeof(float4);
 
 template <bool CONVERT>
 ef_fn pick_kernel(int M) {
@@ -229,7 +288,7 @@ ef_fn pick_kernel(int M) {
 
 int ef_grid(const co3_plan* pl, ef_fn fn) {
     int n = 0;
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, CO3_THREADS, 0);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, CO3_THREADS, RING_BYTES);
     if (n < 1) n = 1;
     const int64_t items = pl->dev.n_chunks * (int64_t)pl->dev.U;
     const int64_t grid = (int64_t)pl->num_sms * n;
@@ -242,7 +301,7 @@ cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaS
     ef_fn fn = pick_kernel<false>(pl->dev.M);
     if (!pl->grid_stats) pl->grid_stats = ef_grid(pl, fn);
     co3_prof_begin(pl, CO3_K_STATS, st);
-    fn<<<pl->grid_stats, CO3_THREADS, 0, st>>>(pl->dev, g, const_cast<float*>(m));
+    fn<<<pl->grid_stats, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, const_cast<float*>(m));
     co3_prof_end(pl, CO3_K_STATS, st, 1);
     return cudaGetLastError();
 }
@@ -253,7 +312,7 @@ cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStrea
     ef_fn fn = pick_kernel<true>(pl->dev.M);
     if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn);
     co3_prof_begin(pl, CO3_K_CONVERT, st);
-    fn<<<pl->grid_convert, CO3_THREADS, 0, st>>>(pl->dev, g, m);
+    fn<<<pl->grid_convert, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, m);
     co3_prof_end(pl, CO3_K_CONVERT, st, 1);
     return cudaGetLastError();
 }

@@ -20,17 +20,30 @@ namespace {
 constexpr int BUF_WORDS = CO3_TILE * CO3_MAXLEN / 32;   // 2048: a chunk at 16 bits per symbol
 
 struct Item {                    // one (user, chunk) work item as a thread sees it
-    uint32_t u;
-    Co3Chunk cd;
+    uint32_t u, c;
     uint32_t w[4];               // this thread's 16 symbols
     uint32_t mask;               // which of them belong to the chunk
+    uint32_t dst_word, skip;     // pack pass: the chunk's word offset; user's payload does not fit
+};
+
+// Cursor over a block's contiguous item range in (user, chunk) order.  (Contiguous, not
+// interleaved across blocks: a block then changes segment -- and reloads its replicated table --
+// only a few times.)
+struct Cursor {
+    uint32_t next, end, u, c, n_chunks;
+    __device__ __forceinline__ bool more() const { return next < end; }
+    __device__ __forceinline__ void advance() {
+        ++next;
+        if (++c == n_chunks) { c = 0; ++u; }
+    }
 };
 
 __device__ __forceinline__ void fetch_item(Item& it, const Co3Dev& p, uint32_t u, uint32_t c, int tid) {
     it.u = u;
-    it.cd = p.chunks[c];
-    const int64_t tb = it.cd.start & ~(int64_t)(CO3_TILE - 1);
-    const int lo = (int)(it.cd.start - tb), hi = lo + it.cd.len;
+    it.c = c;
+    const Co3Chunk cd = p.chunks[c];
+    const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+    const int lo = (int)(cd.start - tb), hi = lo + cd.len;
     const int e0 = 16 * tid;
     it.mask = 0;
     it.w[0] = it.w[1] = it.w[2] = it.w[3] = 0;
@@ -60,44 +73,35 @@ __device__ __forceinline__ void lookup16(const uint32_t* s_tab, int lane, const 
     }
 }
 
-// Contiguous item range of this block and the (user, chunk) of its first item.
-__device__ __forceinline__ void block_range(const Co3Dev& p, uint32_t& it0, uint32_t& it1, uint32_t& u, uint32_t& c) {
-    const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.U;
+__device__ __forceinline__ void cursor_init(Cursor& cu, const Co3Dev& p) {
+    cu.n_chunks = (uint32_t)p.n_chunks;
+    const uint32_t n_items = cu.n_chunks * (uint32_t)p.U;
     const uint32_t per = (n_items + gridDim.x - 1) / gridDim.x;
-    it0 = blockIdx.x * per;
-    it1 = min(n_items, it0 + per);
-    u = it0 / (uint32_t)p.n_chunks;
-    c = it0 - u * (uint32_t)p.n_chunks;
+    cu.next = blockIdx.x * per;
+    cu.end = min(n_items, cu.next + per);
+    cu.u = cu.next / cu.n_chunks;
+    cu.c = cu.next - cu.u * cu.n_chunks;
 }
 
 __global__ void __launch_bounds__(CO3_THREADS)
-enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits,
-               unsigned long long* user_bits) {
+enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits) {
     extern __shared__ __align__(16) uint32_t s_dyn[];
     uint32_t* s_len = s_dyn;                          // [nsym][32 lanes] code lengths
     __shared__ uint32_t s_warp[2][CO3_THREADS / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t it0, it1, u, c;
-    block_range(p, it0, it1, u, c);
-    if (it0 >= it1) return;
-    const uint32_t n_chunks = (uint32_t)p.n_chunks;
-    int cur_seg = -1;
+    Cursor cu;
+    cursor_init(cu, p);
+    if (!cu.more()) return;
+    int cur_seg = -1, par = 0;
     bool bad = false;
-    Item cur;
-    fetch_item(cur, p, u, c, tid);
-    for (uint32_t item = it0; item < it1; ++item) {
-        Item nxt = cur;
-        if (item + 1 < it1) {                         // next item's symbols in flight
-            uint32_t un = u, cn = c + 1;
-            if (cn == n_chunks) { cn = 0; ++un; }
-            fetch_item(nxt, p, un, cn, tid);
-            u = un; c = cn;
-        }
-        if (cur.cd.seg != cur_seg) {
+
+    auto process = [&](const Item& cur, uint32_t item) {
+        const Co3Chunk cd = p.chunks[cur.c];
+        if (cd.seg != cur_seg) {
             __syncthreads();
-            const uint8_t* src = p.cb.len8 + (size_t)co3_row_of(hdr[cur.cd.seg], &bad) * CO3_MAXSYM;
+            const uint8_t* src = p.cb.len8 + (size_t)co3_row_of(hdr[cd.seg], &bad) * CO3_MAXSYM;
             for (int i = tid; i < p.nsym * 32; i += CO3_THREADS) s_len[i] = src[i >> 5];
-            cur_seg = cur.cd.seg;
+            cur_seg = cd.seg;
             __syncthreads();
         }
         uint32_t ent[16];
@@ -110,15 +114,15 @@ enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __res
         sb += __shfl_xor_sync(0xffffffffu, sb, 1);
         sb += __shfl_xor_sync(0xffffffffu, sb, 2);
         sb += __shfl_xor_sync(0xffffffffu, sb, 4);
-        const int tlo = (int)(cur.cd.start & (CO3_TILE - 1));
-        const int sub_first = tlo / CO3_SUB, sub_last = (tlo + cur.cd.len - 1) / CO3_SUB;
+        const int tlo = (int)(cd.start & (CO3_TILE - 1));
+        const int sub_first = tlo / CO3_SUB, sub_last = (tlo + cd.len - 1) / CO3_SUB;
         const int kk = tid >> 3;
         if ((tid & 7) == 0 && kk >= sub_first && kk <= sub_last)
-            sub_bits[(size_t)cur.u * p.n_sub + cur.cd.sub0 + (kk - sub_first)] = (uint16_t)sb;
+            sub_bits[(size_t)cur.u * p.n_sub + cd.sub0 + (kk - sub_first)] = (uint16_t)sb;
         uint32_t wb = ((lane & 7) == 0) ? sb : 0u;     // every lane of a sub-chunk holds sb: count it once
         wb += __shfl_xor_sync(0xffffffffu, wb, 8);
         wb += __shfl_xor_sync(0xffffffffu, wb, 16);
-        const int par = (int)(item & 1);
+        par ^= 1;
         if (lane == 0) s_warp[par][warp] = wb;
         __syncthreads();
         if (tid == 0) {
@@ -126,25 +130,46 @@ enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __res
 #pragma unroll
             for (int k = 0; k < CO3_THREADS / 32; ++k) tot += s_warp[par][k];
             p.chunk_words[item] = 4u * ((tot + 127u) / 128u);
-            atomicAdd(&user_bits[cur.u], (unsigned long long)tot);
+            p.chunk_bits[item] = tot;
         }
-        cur = nxt;
+    };
+
+    // two item buffers used alternately, so that the next item's loads stay in flight while the
+    // current one is processed (no register copies that would wait for them)
+    Item a, b;
+    fetch_item(a, p, cu.u, cu.c, tid);
+    while (true) {
+        const uint32_t ia = cu.next;
+        cu.advance();
+        if (cu.more()) fetch_item(b, p, cu.u, cu.c, tid);
+        process(a, ia);
+        if (!cu.more()) break;
+        const uint32_t ib = cu.next;
+        cu.advance();
+        if (cu.more()) fetch_item(a, p, cu.u, cu.c, tid);
+        process(b, ib);
+        if (!cu.more()) break;
     }
     if (bad && tid == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
 
 // chunk_off[u][c] = exclusive prefix of the chunk word counts of user u; one block per user.
-__global__ void __launch_bounds__(1024) enc_scan_kernel(Co3Dev p, uint32_t* __restrict__ chunk_off) {
+__global__ void __launch_bounds__(1024)
+enc_scan_kernel(Co3Dev p, uint32_t* __restrict__ chunk_off, unsigned long long* __restrict__ user_bits) {
     __shared__ uint32_t s_warp[32];
     __shared__ uint32_t s_carry;
+    __shared__ unsigned long long s_bits[32];
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t* in = p.chunk_words + (size_t)u * p.n_chunks;
+    const uint32_t* inb = p.chunk_bits + (size_t)u * p.n_chunks;
     uint32_t* out = chunk_off + (size_t)u * (p.n_chunks + 1);
+    unsigned long long my_bits = 0;                   // r_t^(u): code bits of this user
     if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int64_t base = 0; base < p.n_chunks; base += 1024) {
         const int64_t i = base + tid;
         const uint32_t v = (i < p.n_chunks) ? in[i] : 0u;
+        my_bits += (i < p.n_chunks) ? inb[i] : 0u;
         uint32_t x = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -170,7 +195,14 @@ __global__ void __launch_bounds__(1024) enc_scan_kernel(Co3Dev p, uint32_t* __re
         if (tid == 1023) s_carry = carry + s_warp[31];
         __syncthreads();
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) my_bits += __shfl_xor_sync(0xffffffffu, my_bits, o);
+    if (lane == 0) s_bits[warp] = my_bits;
+    __syncthreads();
     if (tid == 0) {
+        unsigned long long tb = 0;
+        for (int k = 0; k < 32; ++k) tb += s_bits[k];
+        user_bits[u] = tb;
         const uint32_t total = s_carry;
         out[p.n_chunks] = total;
         const uint32_t ovf = (int64_t)total > p.cap_words;
@@ -199,88 +231,94 @@ enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t
     uint32_t* s_buf = s_dyn + p.nsym * 32;            // BUF_WORDS + 4
     __shared__ uint32_t s_warp[2][CO3_THREADS / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t it0, it1, u, c;
-    block_range(p, it0, it1, u, c);
-    if (it0 >= it1) return;
-    const uint32_t n_chunks = (uint32_t)p.n_chunks;
-    int cur_seg = -1;
+    Cursor cu;
+    cursor_init(cu, p);
+    if (!cu.more()) return;
+    int cur_seg = -1, par = 0;
     bool bad = false;
     uint32_t prev_words = BUF_WORDS + 4;              // words of the image that may be non-zero
-    Item cur;
-    fetch_item(cur, p, u, c, tid);
-    uint32_t cur_c = c;
-    for (uint32_t item = it0; item < it1; ++item) {
-        Item nxt = cur;
-        uint32_t nxt_c = cur_c;
-        if (item + 1 < it1) {                         // next item's symbols in flight
-            uint32_t un = u, cn = c + 1;
-            if (cn == n_chunks) { cn = 0; ++un; }
-            fetch_item(nxt, p, un, cn, tid);
-            u = un; c = cn; nxt_c = cn;
+
+    auto fetch = [&](Item& it) {
+        fetch_item(it, p, cu.u, cu.c, tid);
+        it.skip = p.user_ovf[cu.u];
+        it.dst_word = chunk_off[(size_t)cu.u * (cu.n_chunks + 1) + cu.c];
+    };
+    auto process = [&](const Item& cur, uint32_t item) {
+        if (cur.skip) return;                         // block-uniform: this user's payload does not fit
+        const int seg = p.chunks[cur.c].seg;
+        if (seg != cur_seg) {
+            const uint32_t* src = p.cb.enc + (size_t)co3_row_of(hdr[seg], &bad) * CO3_MAXSYM;
+            for (int i = tid; i < p.nsym * 32; i += CO3_THREADS) s_enc[i] = src[i >> 5];
+            cur_seg = seg;
         }
-        if (!p.user_ovf[cur.u]) {                     // block-uniform
-            if (cur.cd.seg != cur_seg) {
-                const uint32_t* src = p.cb.enc + (size_t)co3_row_of(hdr[cur.cd.seg], &bad) * CO3_MAXSYM;
-                for (int i = tid; i < p.nsym * 32; i += CO3_THREADS) s_enc[i] = src[i >> 5];
-                cur_seg = cur.cd.seg;
-            }
-            {   // clear what the previous chunk left in the image (all of it the first time)
-                uint4* z = reinterpret_cast<uint4*>(s_buf);
-                for (uint32_t i = tid; i < (prev_words + 3) / 4; i += CO3_THREADS) z[i] = make_uint4(0, 0, 0, 0);
-            }
-            const uint32_t dst_word = chunk_off[(size_t)cur.u * (n_chunks + 1) + cur_c];
-            __syncthreads();                          // table and cleared image visible
-            uint32_t ent[16];
-            lookup16(s_enc, lane, cur.w, cur.mask, ent);
-            // merge 16 codewords -> 8 pieces (<= 32 bits) -> 4 pieces (<= 64 bits)
-            uint32_t c1[8], l1[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t a = ent[2 * k], b = ent[2 * k + 1];
-                c1[k] = (a & 0xFFFFu) | ((b & 0xFFFFu) << (a >> 16));
-                l1[k] = (a >> 16) + (b >> 16);
-            }
-            unsigned long long c2[4];
-            uint32_t l2[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                c2[k] = (unsigned long long)c1[2 * k] | ((unsigned long long)c1[2 * k + 1] << l1[2 * k]);
-                l2[k] = l1[2 * k] + l1[2 * k + 1];
-            }
-            const uint32_t bits = l2[0] + l2[1] + l2[2] + l2[3];
-            // exclusive scan of the per-thread bit counts over the block
-            uint32_t x = bits;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
-                if (lane >= o) x += y;
-            }
-            const int par = (int)(item & 1);
-            if (lane == 31) s_warp[par][warp] = x;
-            __syncthreads();
-            uint32_t pre = 0, total = 0;
-#pragma unroll
-            for (int k = 0; k < CO3_THREADS / 32; ++k) {
-                const uint32_t t = s_warp[par][k];
-                pre += (k < warp) ? t : 0u;
-                total += t;
-            }
-            const uint32_t nwords = 4u * ((total + 127u) / 128u);
-            uint32_t pos = pre + x - bits;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                put_piece(s_buf, pos, c2[k]);
-                pos += l2[k];
-            }
-            __syncthreads();
-            uint4* dst = reinterpret_cast<uint4*>(bitstream + (size_t)cur.u * p.cap_words + dst_word);
-            const uint4* srcv = reinterpret_cast<const uint4*>(s_buf);
-            for (uint32_t i = tid; i < nwords / 4; i += CO3_THREADS) dst[i] = srcv[i];
-            prev_words = nwords;
-            __syncthreads();
+        {   // clear what the previous chunk left in the image (all of it the first time)
+            uint4* z = reinterpret_cast<uint4*>(s_buf);
+            for (uint32_t i = tid; i < (prev_words + 3) / 4; i += CO3_THREADS) z[i] = make_uint4(0, 0, 0, 0);
         }
-        cur = nxt;
-        cur_c = nxt_c;
+        __syncthreads();                              // table and cleared image visible
+        uint32_t ent[16];
+        lookup16(s_enc, lane, cur.w, cur.mask, ent);
+        // merge 16 codewords -> 8 pieces (<= 32 bits) -> 4 pieces (<= 64 bits)
+        uint32_t c1[8], l1[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t x0 = ent[2 * k], x1 = ent[2 * k + 1];
+            c1[k] = (x0 & 0xFFFFu) | ((x1 & 0xFFFFu) << (x0 >> 16));
+            l1[k] = (x0 >> 16) + (x1 >> 16);
+        }
+        unsigned long long c2[4];
+        uint32_t l2[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            c2[k] = (unsigned long long)c1[2 * k] | ((unsigned long long)c1[2 * k + 1] << l1[2 * k]);
+            l2[k] = l1[2 * k] + l1[2 * k + 1];
+        }
+        const uint32_t bits = l2[0] + l2[1] + l2[2] + l2[3];
+        // exclusive scan of the per-thread bit counts over the block
+        uint32_t x = bits;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        par ^= 1;
+        if (lane == 31) s_warp[par][warp] = x;
+        __syncthreads();
+        uint32_t pre = 0, total = 0;
+#pragma unroll
+        for (int k = 0; k < CO3_THREADS / 32; ++k) {
+            const uint32_t t = s_warp[par][k];
+            pre += (k < warp) ? t : 0u;
+            total += t;
+        }
+        const uint32_t nwords = 4u * ((total + 127u) / 128u);
+        uint32_t pos = pre + x - bits;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            put_piece(s_buf, pos, c2[k]);
+            pos += l2[k];
+        }
+        __syncthreads();
+        uint4* dst = reinterpret_cast<uint4*>(bitstream + (size_t)cur.u * p.cap_words + cur.dst_word);
+        const uint4* srcv = reinterpret_cast<const uint4*>(s_buf);
+        for (uint32_t i = tid; i < nwords / 4; i += CO3_THREADS) dst[i] = srcv[i];
+        prev_words = nwords;
+        __syncthreads();
+    };
+
+    Item a, b;
+    fetch(a);
+    while (true) {
+        const uint32_t ia = cu.next;
+        cu.advance();
+        if (cu.more()) fetch(b);
+        process(a, ia);
+        if (!cu.more()) break;
+        const uint32_t ib = cu.next;
+        cu.advance();
+        if (cu.more()) fetch(a);
+        process(b, ib);
+        if (!cu.more()) break;
     }
     if (bad && tid == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
@@ -302,8 +340,7 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
                               cudaStream_t st) {
     const Co3Dev& p = pl->dev;
     const int64_t items = p.n_chunks * (int64_t)p.U;
-    cudaError_t e = cudaMemsetAsync(user_bits, 0, sizeof(unsigned long long) * (size_t)p.U, st);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
     const int fi = p.nsym == 256 ? 0 : (p.nsym == 128 ? 1 : (p.nsym == 64 ? 2 : 3));
     const size_t smem_len = (size_t)p.nsym * 32 * sizeof(uint32_t);
     if (!g_len_bpsm[fi]) {
@@ -312,11 +349,11 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
     }
     int64_t grid = (int64_t)pl->num_sms * g_len_bpsm[fi];
     co3_prof_begin(pl, CO3_K_ENC_LEN, st);
-    enc_len_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, smem_len, st>>>(p, hdr, sub_bits, user_bits);
+    enc_len_kernel<<<(int)(items < grid ? items : grid), CO3_THREADS, smem_len, st>>>(p, hdr, sub_bits);
     co3_prof_end(pl, CO3_K_ENC_LEN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
-    enc_scan_kernel<<<p.U, 1024, 0, st>>>(p, chunk_off);
+    enc_scan_kernel<<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
     co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const size_t smem = ((size_t)p.nsym * 32 + BUF_WORDS + 4) * sizeof(uint32_t);

@@ -77,7 +77,8 @@ struct Co3Dev {
     const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
     const double* logr_tab;       // [FIT_GRID + 1] log R(beta) at log2(beta) uniform in [log2 0.3, 1]
     Co3CodeBook cb;               // code tables of all model rows
-    uint32_t* chunk_words;        // [U][n_chunks]
+    uint32_t* chunk_words;        // [U][n_chunks] payload words of each chunk (multiple of 4)
+    uint32_t* chunk_bits;         // [U][n_chunks] code bits of each chunk
     uint32_t* user_ovf;           // [U] 1 if the user's payload exceeds cap_words
     uint32_t* flags;              // sticky status flags
     unsigned long long* nonfinite_total;
