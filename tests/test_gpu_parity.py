@@ -275,3 +275,48 @@ def test_config1_full_two_iterations(binding, oracle):
     from paper_2203_09044_b200 import inputs
     wl = inputs.workload(1)
     run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+def test_config2_full_one_iteration(binding, oracle):
+    """16 users x d = 14,728,266 in 16 segments with odd offsets, E3M2 (the U > 8 decode path)."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(2)
+    run_case(binding, oracle, wl.d, wl.n_users, 3, 2, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+def test_config3_full_one_iteration(binding, oracle):
+    """4 users x d = 124,439,808 heavy-tailed with outliers, E4M3: the shape estimate clamps at 0.3."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(3)
+    plan, orc, out, res = run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 1),
+                                   gamma=wl.gamma)
+    assert res[0][0].fit[0, 0] == 0.3
+
+
+# ---- the size / users / shape / format sweep (a subset the oracle can follow) ----------------
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("beta", [0.5, 1.0, 2.0])
+@pytest.mark.parametrize("U", [1, 8, 64])
+def test_sweep_d_2p16(binding, oracle, U, beta, E, M):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 16, U, beta, E, M)
+    run_case(binding, oracle, wl.d, U, E, M, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("beta", [0.5, 2.0])
+def test_sweep_d_2p20_8_users(binding, oracle, beta, E, M):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 20, 8, beta, E, M)
+    run_case(binding, oracle, wl.d, 8, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+def test_sweep_d_2p24_and_2p28_single_user(binding, oracle):
+    from paper_2203_09044_b200 import inputs
+    for d, E, M in ((1 << 24, 3, 2), (1 << 28, 1, 2)):
+        wl = inputs.sweep_cell(d, 1, 1.0, E, M)
+        run_case(binding, oracle, wl.d, 1, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
