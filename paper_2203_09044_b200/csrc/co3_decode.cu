@@ -2,19 +2,27 @@
 // decode every user's stream and write the average of the reconstructed gradients.
 //
 // A lane decodes one sub-chunk (<= 128 codewords) serially with an 11-bit primary table whose
-// entries already hold the signed integer magnitude; the 32 sub-chunks of a chunk are the 32
-// lanes of a warp, so a warp is one (chunk, user) stream.  The integer magnitudes of all users
-// are accumulated with shared-memory atomics into a transposed, padded tile (conflict-free both
-// for the per-lane scattered adds and for the coalesced read-out), scaled once by 2^lambda and
-// divided by U.  The stream words are staged in shared memory with 128-bit loads, so global
-// traffic is fully coalesced.
+// entries already hold the signed integer magnitude ((K << 8) | length); the 32 sub-chunks of a
+// chunk are the 32 lanes of a warp, so a warp is one (chunk, user) stream.  The magnitudes of all
+// users are accumulated with shared-memory reductions into a transposed, padded tile
+// (conflict-free both for the per-lane scattered adds and for the coalesced read-out), scaled
+// once by 2^lambda and divided by U.  The stream words are staged in shared memory with 128-bit
+// loads, so global traffic is fully coalesced.
+//
+// The inner loop is written for issue slots: shared memory is addressed with 32-bit
+// shared-space addresses (ld.shared / red.shared), the bit buffer is kept shifted left by two so
+// that one AND gives the table's byte offset, the funnel shifts take the table entry itself as
+// shift amount (only its low five bits count), and four symbols are decoded per loop trip with
+// immediate accumulator offsets.
 //
 // Two variants: U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
-// per sub-chunk (small double-buffered accumulator, several chunks per block when U < 8); U > 8
-// keeps a whole chunk accumulator and loops over user groups.
+// per sub-chunk (small double-buffered accumulator, several chunks per block when U < 8); the
+// whole table entries are accumulated (the length bytes of at most 8 users cannot carry into
+// the magnitude) and the magnitude sum is taken out with one shift at the end.  U > 8 keeps a
+// whole chunk accumulator and loops over user groups.
 //
 // Bound: HBM for U = 1 (4 B written per element); for U >= 4 the serial decode (issue slots and
-// shared-memory look-ups per symbol) dominates.
+// shared-memory wavefronts: the table look-up of 32 lanes hits random banks) dominates.
 #include "co3_internal.h"
 
 namespace {
@@ -53,70 +61,127 @@ __device__ __forceinline__ float pow2_clamped(int e) {   // 2^e; a corrupt heade
     return __uint_as_float((uint32_t)(e + 127) << 23);
 }
 
-struct Reader {                                   // LSB-first bit reader
-    unsigned long long buf;
-    int nb;                                       // valid bits in buf
-    uint32_t wp;                                  // next word to fetch
-};
-
-template <bool CHECKED>
-__device__ __forceinline__ uint32_t fetch(const uint32_t* src, uint32_t nwords, uint32_t i) {
-    if (CHECKED) return i < nwords ? src[i] : 0u;
-    return src[i];
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ void red_add(uint32_t addr, uint32_t v) {
+    asm volatile("red.shared.add.u32 [%0+%2], %1;" ::"r"(addr), "r"(v), "n"(OFF) : "memory");
 }
 
-template <bool CHECKED>
-__device__ __forceinline__ void reader_init(Reader& r, const uint32_t* src, uint32_t nwords, uint32_t bitpos) {
-    r.wp = bitpos >> 5;
-    const uint32_t sh = bitpos & 31u;
-    r.buf = (unsigned long long)(fetch<CHECKED>(src, nwords, r.wp) >> sh);
-    r.nb = 32 - (int)sh;
-    r.wp++;
-    r.buf |= (unsigned long long)fetch<CHECKED>(src, nwords, r.wp) << r.nb;
-    r.nb += 32;
-    r.wp++;
-}
-
-// Codeword longer than the primary table: canonical search over lengths 12..16.
-__device__ __noinline__ uint32_t decode_long(uint32_t window, const Tables& t, int32_t& k, bool& bad) {
+// Codeword longer than the primary table: canonical search over lengths 12..16.  Returns the
+// entry (K << 8) | length.
+__device__ __noinline__ uint32_t decode_long(uint32_t window, const Tables& t, bool& bad) {
     const uint32_t v = __brev(window) >> 16;      // 16 stream bits, root bit on top
     for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
         const uint32_t dd = (v >> (CO3_MAXLEN - L)) - t.first[L];
-        if (dd < t.count[L]) {
-            k = t.ksign[t.perm[(t.offs[L] + dd) & (CO3_MAXSYM - 1)]];
-            return (uint32_t)L;
-        }
+        if (dd < t.count[L])
+            return ((uint32_t)t.ksign[t.perm[(t.offs[L] + dd) & (CO3_MAXSYM - 1)]] << 8) | (uint32_t)L;
     }
     bad = true;                                   // cannot happen for a complete code
-    k = 0;
     return CO3_MAXLEN;
 }
 
-// Decode n symbols of this lane's sub-chunk, adding their signed magnitudes to acc[0],
-// acc[PADW], ... (one accumulator row per symbol position).
-template <bool CHECKED>
-__device__ __forceinline__ void decode_run(Reader& r, const Tables& t, const uint32_t* src, uint32_t nwords,
-                                           int32_t* acc, int n, bool& bad) {
-    unsigned long long buf = r.buf;
-    int nb = r.nb;
-    uint32_t wp = r.wp;
+// LSB-first bit reader over staged words.  The stream sits at bits [2, 2 + nb) of hi:lo, so
+// (lo & 0x1FFC) is the byte offset of the 11-bit table entry; rp is the shared-space byte
+// address of the next word.  Before every symbol nb >= 31.
+struct Reader {
+    uint32_t lo, hi;
+    int nb;
+    uint32_t rp;
+};
+
+__device__ __forceinline__ void refill(Reader& r) {
+    if (r.nb <= 30) {
+        const unsigned long long w = (unsigned long long)lds32(r.rp) << (r.nb + 2);
+        r.lo |= (uint32_t)w;
+        r.hi |= (uint32_t)(w >> 32);
+        r.nb += 32;
+        r.rp += 4;
+    }
+}
+
+__device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint32_t bitpos) {
+    r.rp = stage_addr + ((bitpos >> 5) << 2);
+    const uint32_t sh = bitpos & 31u;
+    const unsigned long long v = (unsigned long long)(lds32(r.rp) >> sh) << 2;
+    r.lo = (uint32_t)v;
+    r.hi = (uint32_t)(v >> 32);
+    r.nb = 32 - (int)sh;
+    r.rp += 4;
+    refill(r);
+}
+
+// One symbol: look up, consume, add to the accumulator row at byte offset OFF.
+// PACKED: add the whole entry (length byte included); else add the signed magnitude.
+template <int OFF, bool PACKED>
+__device__ __forceinline__ void decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr, const Tables& t, bool& bad) {
+    uint32_t e = lds32(lut_addr + (r.lo & ((CO3_LUT_SIZE - 1) << 2)));
+    if ((e & 0xFFu) == 0u) e = decode_long(__funnelshift_r(r.lo, r.hi, 2), t, bad);
+    r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
+    r.hi = __funnelshift_r(r.hi, 0u, e);
+    r.nb -= (int)(e & 0xFFu);
+    red_add<OFF>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
+    refill(r);
+}
+
+template <bool PACKED>
+__device__ __forceinline__ void decode_run(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int n,
+                                           const Tables& t, bool& bad) {
+    int i = 0;
+    for (; i + 4 <= n; i += 4) {
+        decode_step<0, PACKED>(r, lut_addr, acc_addr, t, bad);
+        decode_step<PADW * 4, PACKED>(r, lut_addr, acc_addr, t, bad);
+        decode_step<PADW * 8, PACKED>(r, lut_addr, acc_addr, t, bad);
+        decode_step<PADW * 12, PACKED>(r, lut_addr, acc_addr, t, bad);
+        acc_addr += PADW * 16;
+    }
+    for (; i < n; ++i) {
+        decode_step<0, PACKED>(r, lut_addr, acc_addr, t, bad);
+        acc_addr += PADW * 4;
+    }
+}
+
+// The same for a stream that did not fit the staging row: words come from global memory with
+// bounds checks.  Rare (a chunk above 8 bits per symbol), so written plainly.
+struct SlowReader {
+    unsigned long long buf;
+    int nb;
+    uint32_t wp;
+};
+__device__ __forceinline__ uint32_t fetch_checked(const uint32_t* src, uint32_t nwords, uint32_t i) {
+    return i < nwords ? src[i] : 0u;
+}
+__device__ void slow_init(SlowReader& r, const uint32_t* src, uint32_t nwords, uint32_t bitpos) {
+    r.wp = bitpos >> 5;
+    const uint32_t sh = bitpos & 31u;
+    r.buf = (unsigned long long)(fetch_checked(src, nwords, r.wp) >> sh);
+    r.nb = 32 - (int)sh;
+    r.wp++;
+    r.buf |= (unsigned long long)fetch_checked(src, nwords, r.wp) << r.nb;
+    r.nb += 32;
+    r.wp++;
+}
+template <bool PACKED>
+__device__ void slow_run(SlowReader& r, const Tables& t, const uint32_t* src, uint32_t nwords, int32_t* acc,
+                         int n, bool& bad) {
     for (int i = 0; i < n; ++i) {
-        const uint32_t window = (uint32_t)buf;
-        const uint32_t e = t.lut[window & (CO3_LUT_SIZE - 1)];
-        int32_t k = (int32_t)e >> 8;
-        uint32_t len = e & 0xFFu;
-        if (len == 0) len = decode_long(window, t, k, bad);
-        buf >>= len;
-        nb -= (int)len;
-        atomicAdd(acc, k);
+        const uint32_t window = (uint32_t)r.buf;
+        uint32_t e = t.lut[window & (CO3_LUT_SIZE - 1)];
+        if ((e & 0xFFu) == 0u) e = decode_long(window, t, bad);
+        const uint32_t len = e & 0xFFu;
+        r.buf >>= len;
+        r.nb -= (int)len;
+        atomicAdd(acc, PACKED ? (int32_t)e : ((int32_t)e >> 8));
         acc += PADW;
-        if (nb < 32) {
-            buf |= (unsigned long long)fetch<CHECKED>(src, nwords, wp) << nb;
-            nb += 32;
-            wp++;
+        if (r.nb < 32) {
+            r.buf |= (unsigned long long)fetch_checked(src, nwords, r.wp) << r.nb;
+            r.nb += 32;
+            r.wp++;
         }
     }
-    r.buf = buf; r.nb = nb; r.wp = wp;
 }
 
 struct Stream {                                   // one (chunk, user) stream as seen by a lane
@@ -203,6 +268,9 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     const int cpg = NW / U;                        // chunks per group (>= 1)
     const int accw = acc_words_a(U);               // words per accumulator buffer
     int32_t* acc0 = &sm.acc[0][0];
+    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(acc0);
+    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(sm.stage[warp]);
     const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
     const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
     const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
@@ -223,26 +291,28 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
         s.active = false; s.staged = true; s.nwords = 0; s.bitpos = 0; s.sub_len_bits = 0;
         s.i_lo = 0; s.i_hi = 0; s.gsrc = nullptr;
         Reader r;
-        r.buf = 0; r.nb = 0; r.wp = 0;
+        r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr;
+        SlowReader sr;
+        sr.buf = 0; sr.nb = 0; sr.wp = 0;
         if (mine) {
             const Co3Chunk cd = p.chunks[grp.chunk0 + ci];
             open_stream(s, p, cd, grp.chunk0 + ci, us, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
             if (s.active) {
-                if (s.staged) reader_init<false>(r, sm.stage[warp], s.nwords, s.bitpos);
-                else reader_init<true>(r, s.gsrc, s.nwords, s.bitpos);
+                if (s.staged) reader_init(r, stage_addr, s.bitpos);
+                else slow_init(sr, s.gsrc, s.nwords, s.bitpos);
             }
         }
         const float scale = pow2_clamped((int)hdr[grp.seg].bias + p.cF);
         __syncthreads();                           // tables, zeroed accumulator 0
 #pragma unroll 1
         for (int q = 0; q < CO3_SUB / QB; ++q) {
-            int32_t* accq = acc0 + (q & 1) * accw;
+            const int qoff = (q & 1) * accw;
             if (mine && s.active) {
                 const int a = max(s.i_lo, q * QB), b = min(s.i_hi, (q + 1) * QB);
                 if (b > a) {
-                    int32_t* dst = accq + ci * ACC_Q + (a - q * QB) * PADW + lane;
-                    if (s.staged) decode_run<false>(r, sm.t, sm.stage[warp], s.nwords, dst, b - a, bad);
-                    else decode_run<true>(r, sm.t, s.gsrc, s.nwords, dst, b - a, bad);
+                    const int row0 = qoff + ci * ACC_Q + (a - q * QB) * PADW + lane;
+                    if (s.staged) decode_run<true>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, b - a, sm.t, bad);
+                    else slow_run<true>(sr, sm.t, s.gsrc, s.nwords, acc0 + row0, b - a, bad);
                 }
             }
             __syncthreads();
@@ -255,19 +325,21 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                 const Co3Chunk cd = p.chunks[grp.chunk0 + cc];
                 const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
                 const int lo = (int)(cd.start - tb), hi = lo + cd.len;
-                const int32_t* a = accq + cc * ACC_Q;
+                const int32_t* a = acc0 + qoff + cc * ACC_Q;
 #pragma unroll
                 for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
                     const int x = tid + rr * CO3_THREADS;
                     const int kk = x >> 5, il = x & 31;
                     const int e = kk * CO3_SUB + q * QB + il;
-                    if (e >= lo && e < hi) avg[tb + e] = finish(a[il * PADW + kk], scale, fu, inv_u);
+                    // the accumulator holds sum((K << 8) | length): the lengths of <= 8 users stay below 256
+                    if (e >= lo && e < hi) avg[tb + e] = finish(a[il * PADW + kk] >> 8, scale, fu, inv_u);
                 }
             }
             __syncthreads();
         }
         if (mine && s.active) {
-            const uint32_t endpos = r.wp * 32u - (uint32_t)r.nb;
+            const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - (uint32_t)r.nb
+                                             : sr.wp * 32u - (uint32_t)sr.nb;
             if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
         }
     }
@@ -288,6 +360,9 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     extern __shared__ __align__(16) unsigned char s_raw[];
     SmemB& sm = *reinterpret_cast<SmemB*>(s_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(sm.acc);
+    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(sm.stage[warp]);
     const int64_t per = (p.n_chunks + gridDim.x - 1) / gridDim.x;
     const int64_t c0 = (int64_t)blockIdx.x * per, c1 = min(p.n_chunks, c0 + per);
     const float fu = (float)p.U;
@@ -306,16 +381,19 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
             Stream s;
             open_stream(s, p, cd, c, u, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
             if (s.active) {
-                Reader r;
-                int32_t* dst = sm.acc + s.i_lo * PADW + lane;
+                const int row0 = s.i_lo * PADW + lane;
+                uint32_t endpos;
                 if (s.staged) {
-                    reader_init<false>(r, sm.stage[warp], s.nwords, s.bitpos);
-                    decode_run<false>(r, sm.t, sm.stage[warp], s.nwords, dst, s.i_hi - s.i_lo, bad);
+                    Reader r;
+                    reader_init(r, stage_addr, s.bitpos);
+                    decode_run<false>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, s.i_hi - s.i_lo, sm.t, bad);
+                    endpos = ((r.rp - stage_addr) << 3) - (uint32_t)r.nb;
                 } else {
-                    reader_init<true>(r, s.gsrc, s.nwords, s.bitpos);
-                    decode_run<true>(r, sm.t, s.gsrc, s.nwords, dst, s.i_hi - s.i_lo, bad);
+                    SlowReader sr;
+                    slow_init(sr, s.gsrc, s.nwords, s.bitpos);
+                    slow_run<false>(sr, sm.t, s.gsrc, s.nwords, sm.acc + row0, s.i_hi - s.i_lo, bad);
+                    endpos = sr.wp * 32u - (uint32_t)sr.nb;
                 }
-                const uint32_t endpos = r.wp * 32u - (uint32_t)r.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
             }
             __syncwarp();                          // the stage is reused by this warp's next user
