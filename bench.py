@@ -30,9 +30,10 @@ UNIT = "GB/s"
 POOL = 4                      # distinct gradient batches cycled through (each > L2)
 # algorithmic bytes per user-element of the fused convert pass: read g, m (8), write m (4), symbol (1)
 CONVERT_BYTES_PER_ELEMENT = 13.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel on this workload,
-# from the ncu capture summarised in profiles/ (None until one has been taken)
-CONVERT_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel on the full 8-user
+# workload (mean of three launches of the one-pass ncu capture summarised in
+# profiles/dram_traffic_config1_8users.md); it grows in proportion with the number of users
+CONVERT_DRAM_TRAFFIC_BYTES_8_USERS = 1112.6e6
 
 
 def measured_peaks():
@@ -227,7 +228,7 @@ def run_ours(args):
         "roofline": {"kernel": "ef_kernel<convert> (fused EF-add/convert/residual/histogram/moments)",
                      "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
-                     "traffic": CONVERT_DRAM_TRAFFIC_BYTES,
+                     "traffic": CONVERT_DRAM_TRAFFIC_BYTES_8_USERS * U / 8.0,
                      "algorithmic_bytes_per_launch": CONVERT_BYTES_PER_ELEMENT * U * d,
                      "avg_launch_ms": conv_avg_ms, "launches_timed": conv_n,
                      "timing": "cudaEvent pair around each launch on the launching stream, inside the timed region"},
