@@ -49,6 +49,7 @@ extern "C" {
 #define CO3_ECAPACITY (-4)  /* a user's payload does not fit cap_words               */
 #define CO3_ECORRUPT (-5)   /* a stream did not decode to its recorded lengths       */
 #define CO3_ENONFINITE (-6) /* NaN/Inf met in g + gamma m (coded as 0, memory reset) */
+#define CO3_ELIMIT (-7)     /* input larger than the fixed scratch of co3_moments_static */
 
 #define CO3_FLAG_CAPACITY 1u
 #define CO3_FLAG_CORRUPT 2u
@@ -188,6 +189,26 @@ int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint32_t* weigh
 int64_t co3_partition(int64_t d, int32_t n_segments, const int64_t* seg_offsets,
                       int32_t* chunk_seg, int64_t* chunk_start, int64_t* chunk_end,
                       int64_t* sub_base, int64_t* n_sub);
+
+/* (The paper has no counterpart of this call: it is a convenience of this library.)
+ * Pooled moments of a = g + gamma m over n elements, WITHOUT allocating anything: for callers
+ * that may not allocate device memory when they need these statistics -- code living inside a
+ * host application whose device memory belongs to that application's own pool, or loops that
+ * cannot take the device-wide synchronisation of cudaMalloc/cudaFree -- and that therefore cannot
+ * create a plan (co3_plan_create allocates tables and scratch).
+ *   grad, residual  device, const, n fp32 each, 16-byte aligned (for several users pass the
+ *                   rows back to back: n = U * d with ld == d)
+ *   moments         device, out, 4 doubles: N (finite elements), sum |a|, sum a^2, non-finite count
+ * The partial sums live in a 3 MiB array that is part of the library's device image (every GPU
+ * that loads the library holds it until the process exits); n may be at most
+ * CO3_STATIC_MAX_ELEMENTS, else CO3_ELIMIT is returned and nothing is launched.  The first call
+ * on each device looks the array's device address up: make it before any stream capture begins.
+ * All calls share the array, so calls whose kernels could overlap on the GPU (other streams,
+ * other host threads) must be serialised by the caller; nothing in it needs clearing between
+ * calls.  Work is enqueued on cuda_stream; the caller synchronises before reading `moments`. */
+#define CO3_STATIC_MAX_ELEMENTS ((int64_t)1 << 29)
+int co3_moments_static(const float* grad, const float* residual, int64_t n, float gamma,
+                       double* moments, void* cuda_stream);
 
 const char* co3_strerror(int code);
 

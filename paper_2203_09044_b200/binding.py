@@ -21,7 +21,10 @@ EXPORTS = [
     "co3_iteration_host", "co3_status", "co3_get_fit", "co3_state_export", "co3_state_import",
     "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
+    "co3_moments_static",
 ]
+ELIMIT = -7
+STATIC_MAX_ELEMENTS = 1 << 29
 
 KERNEL_NAMES = ["stats", "fit", "convert", "code_enc", "enc_len", "enc_scan", "enc_pack", "code_dec",
                 "decode"]
@@ -93,6 +96,8 @@ def lib():
     L.co3_profile_collect.argtypes = [vp, vp, vp]
     L.co3_launch_count.restype = C.c_int64
     L.co3_launch_count.argtypes = [vp]
+    L.co3_moments_static.restype = C.c_int
+    L.co3_moments_static.argtypes = [vp, vp, C.c_int64, C.c_float, vp, vp]
     L.co3_strerror.restype = C.c_char_p
     L.co3_strerror.argtypes = [C.c_int]
     _lib = L
@@ -124,6 +129,16 @@ def partition(d, seg_offsets):
 
 def _ptr(t):
     return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def moments_static(grad, residual, n, gamma, moments, stream=None):
+    """co3_moments_static: N, sum|a|, sum a^2, non-finite count of a = g + gamma m over n elements
+    into `moments` (4 float64 on the device), with no allocation inside the library.  Returns the
+    C return code (0, or a negative CO3_E* value such as ELIMIT)."""
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(lib().co3_moments_static(_ptr(grad), _ptr(residual), int(n), float(gamma), _ptr(moments),
+                                        C.c_void_p(s.cuda_stream)))
 
 
 class Plan:

@@ -59,6 +59,7 @@ extern "C" const char* co3_strerror(int code) {
         case CO3_ECAPACITY: return "payload exceeds cap_words";
         case CO3_ECORRUPT: return "stream does not decode to its recorded lengths";
         case CO3_ENONFINITE: return "non-finite value in g + gamma*m";
+        case CO3_ELIMIT: return "input exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown error";
     }
 }
