@@ -126,6 +126,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
     if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED) return CO3_EINVAL;
     if (!(cfg->gamma >= 0.0f) || !(cfg->gamma <= 1.0f)) return CO3_EINVAL;
     if (cfg->d > ((int64_t)1 << 31)) return CO3_EINVAL;
+    if (((cfg->d + 4095) / 4096 + (cfg->seg_offsets ? cfg->n_segments : 1)) * (int64_t)cfg->n_users > 0x7FFFFFFFLL) return CO3_EINVAL;
     const int nm = E + M, J = 1 << nm, nsym = 2 * J;
     const int64_t Kmax = co3_host_K(M, J - 1);
     if ((int64_t)cfg->n_users * Kmax >= ((int64_t)1 << 24)) return CO3_EINVAL;   // exact integer sums
@@ -222,6 +223,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
         a |= dev_alloc(pl, &dv.chunk_words, items);
         a |= dev_alloc(pl, &dv.chunk_bits, items);
+        a |= dev_alloc(pl, &dv.gran_bits, items * 64);
         a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);

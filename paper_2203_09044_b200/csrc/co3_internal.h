@@ -79,6 +79,7 @@ struct Co3Dev {
     Co3CodeBook cb;               // code tables of all model rows
     uint32_t* chunk_words;        // [U][n_chunks] payload words of each chunk (multiple of 4)
     uint32_t* chunk_bits;         // [U][n_chunks] code bits of each chunk
+    uint16_t* gran_bits;          // [U][n_chunks][64] code bits of each 64-symbol granule
     uint32_t* user_ovf;           // [U] 1 if the user's payload exceeds cap_words
     uint32_t* flags;              // sticky status flags
     unsigned long long* nonfinite_total;
