@@ -213,7 +213,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &d_seg_off, (size_t)S + 1);
         a |= dev_alloc(pl, &d_seg_chunk0, (size_t)S + 1);
         a |= dev_alloc(pl, &d_wtab, (size_t)CO3_NIBETA * CO3_NIR * J);
-        a |= dev_alloc(pl, &d_logr, (size_t)CO3_FIT_GRID + 1);
+        a |= dev_alloc(pl, &d_logr, 2 * ((size_t)CO3_FIT_GRID + 1));
         a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
         a |= dev_alloc(pl, &dv.hist, (size_t)S * CO3_MAXSYM);
         a |= dev_alloc(pl, &dv.part_s1, items);
@@ -239,7 +239,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             up(d_seg_off, pl->h_seg_off, sizeof(int64_t) * (size_t)(S + 1));
             up(d_seg_chunk0, h_seg_chunk0, sizeof(int32_t) * (size_t)(S + 1));
             up(d_wtab, wtab, sizeof(uint32_t) * (size_t)CO3_NIBETA * CO3_NIR * J);
-            up(d_logr, logr, sizeof(double) * ((size_t)CO3_FIT_GRID + 1));
+            up(d_logr, logr, sizeof(double) * 2 * ((size_t)CO3_FIT_GRID + 1));
             if (e == cudaSuccess) e = cudaMemset(dv.flags, 0, sizeof(uint32_t));
             if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
             if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);

@@ -10,10 +10,9 @@
 // loads, so global traffic is fully coalesced.
 //
 // The inner loop is written for issue slots: shared memory is addressed with 32-bit
-// shared-space addresses (ld.shared / red.shared), the bit buffer is kept shifted left by two so
-// that one AND gives the table's byte offset, the funnel shifts take the table entry itself as
-// shift amount (only its low five bits count), and four symbols are decoded per loop trip with
-// immediate accumulator offsets.
+// shared-space addresses (ld.shared / red.shared), the funnel shifts take the table entry itself
+// as shift amount (only its low five bits count), the bit buffer is topped up once per pair of
+// symbols, and four symbols are decoded per loop trip with immediate accumulator offsets.
 //
 // Two variants: U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
 // per sub-chunk (small double-buffered accumulator, several chunks per block when U < 8); the
@@ -72,7 +71,8 @@ __device__ __forceinline__ void red_add(uint32_t addr, uint32_t v) {
 }
 
 // Codeword longer than the primary table: canonical search over lengths 12..16.  Returns the
-// entry (K << 8) | length.
+// entry (K << 8) | length.  Kept out of line: it is rare, and inlining it four times into the
+// unrolled decode loop made the loop slower.
 __device__ __noinline__ uint32_t decode_long(uint32_t window, const Tables& t, bool& bad) {
     const uint32_t v = __brev(window) >> 16;      // 16 stream bits, root bit on top
     for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
@@ -84,9 +84,11 @@ __device__ __noinline__ uint32_t decode_long(uint32_t window, const Tables& t, b
     return CO3_MAXLEN;
 }
 
-// LSB-first bit reader over staged words.  The stream sits at bits [2, 2 + nb) of hi:lo, so
-// (lo & 0x1FFC) is the byte offset of the 11-bit table entry; rp is the shared-space byte
-// address of the next word.  Before every symbol nb >= 31.
+// LSB-first bit reader over staged words: the stream sits at bits [0, nb) of hi:lo; rp is the
+// shared-space byte address of the next word.  A refill is checked once per PAIR of symbols:
+// with nb >= 32 two codewords (at most 16 bits each) can be taken without looking at nb, and one
+// more word then always fits.  (With 32 lanes a per-symbol refill branch would be taken on nearly
+// every step, so its cost is paid per step, not per refill.)
 struct Reader {
     uint32_t lo, hi;
     int nb;
@@ -94,8 +96,8 @@ struct Reader {
 };
 
 __device__ __forceinline__ void refill(Reader& r) {
-    if (r.nb <= 30) {
-        const unsigned long long w = (unsigned long long)lds32(r.rp) << (r.nb + 2);
+    if (r.nb < 32) {
+        const unsigned long long w = (unsigned long long)lds32(r.rp) << r.nb;
         r.lo |= (uint32_t)w;
         r.hi |= (uint32_t)(w >> 32);
         r.nb += 32;
@@ -106,25 +108,23 @@ __device__ __forceinline__ void refill(Reader& r) {
 __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint32_t bitpos) {
     r.rp = stage_addr + ((bitpos >> 5) << 2);
     const uint32_t sh = bitpos & 31u;
-    const unsigned long long v = (unsigned long long)(lds32(r.rp) >> sh) << 2;
+    const unsigned long long v = (((unsigned long long)lds32(r.rp + 4) << 32) | lds32(r.rp)) >> sh;
     r.lo = (uint32_t)v;
     r.hi = (uint32_t)(v >> 32);
-    r.nb = 32 - (int)sh;
-    r.rp += 4;
-    refill(r);
+    r.nb = 64 - (int)sh;
+    r.rp += 8;
 }
 
 // One symbol: look up, consume, add to the accumulator row at byte offset OFF.
 // PACKED: add the whole entry (length byte included); else add the signed magnitude.
 template <int OFF, bool PACKED>
 __device__ __forceinline__ void decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr, const Tables& t, bool& bad) {
-    uint32_t e = lds32(lut_addr + (r.lo & ((CO3_LUT_SIZE - 1) << 2)));
-    if ((e & 0xFFu) == 0u) e = decode_long(__funnelshift_r(r.lo, r.hi, 2), t, bad);
+    uint32_t e = lds32(lut_addr + ((r.lo & (CO3_LUT_SIZE - 1)) << 2));
+    if ((e & 0xFFu) == 0u) e = decode_long(r.lo, t, bad);
     r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= (int)(e & 0xFFu);
     red_add<OFF>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
-    refill(r);
 }
 
 template <bool PACKED>
@@ -132,13 +132,16 @@ __device__ __forceinline__ void decode_run(Reader& r, uint32_t lut_addr, uint32_
                                            const Tables& t, bool& bad) {
     int i = 0;
     for (; i + 4 <= n; i += 4) {
+        refill(r);
         decode_step<0, PACKED>(r, lut_addr, acc_addr, t, bad);
         decode_step<PADW * 4, PACKED>(r, lut_addr, acc_addr, t, bad);
+        refill(r);
         decode_step<PADW * 8, PACKED>(r, lut_addr, acc_addr, t, bad);
         decode_step<PADW * 12, PACKED>(r, lut_addr, acc_addr, t, bad);
         acc_addr += PADW * 16;
     }
     for (; i < n; ++i) {
+        refill(r);
         decode_step<0, PACKED>(r, lut_addr, acc_addr, t, bad);
         acc_addr += PADW * 4;
     }

@@ -203,15 +203,21 @@ enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t
     if (lane == 31) s_warp[warp] = x;
     __syncthreads();                                  // table, cleared image, warp totals
     uint32_t pos = x - bits + (warp ? s_warp[0] : 0u);
+    const bool whole = it.a == 0 && it.b == GRANULE;  // no symbol of this granule lies outside the chunk
 #pragma unroll
     for (int k = 0; k < GRANULE / 16; ++k) {
-        const uint32_t mask = round_mask(it, k);
+        const uint32_t mask = whole ? 0xFFFFu : round_mask(it, k);
         if (mask == 0) continue;
         uint32_t ent[16];
+        if (whole) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const uint32_t e = s_enc[__byte_perm(it.w[4 * k + (i >> 2)], 0, 0x4440 + (i & 3))];
-            ent[i] = (mask == 0xFFFFu || ((mask >> i) & 1u)) ? e : 0u;
+            for (int i = 0; i < 16; ++i) ent[i] = s_enc[__byte_perm(it.w[4 * k + (i >> 2)], 0, 0x4440 + (i & 3))];
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint32_t e = s_enc[__byte_perm(it.w[4 * k + (i >> 2)], 0, 0x4440 + (i & 3))];
+                ent[i] = ((mask >> i) & 1u) ? e : 0u;
+            }
         }
         // merge 16 codewords -> 8 pieces (<= 32 bits) -> 4 pieces (<= 64 bits)
         uint32_t c1[8], l1[8];

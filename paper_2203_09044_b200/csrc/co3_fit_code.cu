@@ -16,7 +16,8 @@
 
 namespace {
 
-constexpr int FIT_THREADS = 128;   // = FIT_GRID / 64: one coarse table interval per thread
+constexpr int FIT_THREADS = 512;   // reduction width
+constexpr int FIT_SEARCH = 128;    // = FIT_GRID / 64: one coarse table interval per searching thread
 
 __device__ __forceinline__ double poly_bias(double b) {
     const double b2 = b * b;
@@ -29,7 +30,7 @@ __device__ __forceinline__ double poly_bias(double b) {
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr) {
     __shared__ double s_a[FIT_THREADS], s_b[FIT_THREADS];
     __shared__ unsigned long long s_n[FIT_THREADS];
-    __shared__ double s_lg[2];
+    __shared__ double s_lg[3];
     __shared__ double s_target, s_t;        // log rho; log2(beta)
     __shared__ int s_state, s_coarse, s_fine;
 
@@ -57,57 +58,71 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     const double N = (double)((unsigned long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * (unsigned long long)p.U - nf);
 
     // beta = clamp(R^-1(rho), 0.3, 2.0), rho = N S2 / S1^2; R is strictly decreasing in beta, and
-    // the table holds log R at log2(beta) = T0 + i * H.
+    // the tables hold log R and log G at log2(beta) = T0 + i * H.
     const double T0 = log2(0.3), H = (1.0 - T0) / (double)CO3_FIT_GRID;
     const double* tab = p.logr_tab;
+    const double* tabg = p.logr_tab + CO3_FIT_GRID + 1;
+    if (tid < 3) s_lg[tid] = log(tid == 0 ? N : (tid == 1 ? S2 : S1));   // three logarithms side by side
+    __syncthreads();
     if (tid == 0) {
         s_state = 0; s_coarse = 0; s_fine = 0;
         if (!(N > 0.0) || !(S1 > 0.0)) { s_state = 2; s_t = 0.0; }          // beta = 1, alpha = 0
         else {
-            s_target = log(N) + log(S2) - 2.0 * log(S1);
-            if (s_target >= tab[0]) { s_state = 1; s_t = T0; }
-            else if (s_target <= tab[CO3_FIT_GRID]) { s_state = 1; s_t = 1.0; }
+            s_target = s_lg[0] + s_lg[1] - 2.0 * s_lg[2];
+            if (s_target >= tab[0]) { s_state = 1; s_t = T0; s_fine = 0; }
+            else if (s_target <= tab[CO3_FIT_GRID]) { s_state = 1; s_t = 1.0; s_fine = CO3_FIT_GRID; }
         }
     }
     __syncthreads();
     if (s_state == 0) {
         // interval i with tab[i] > target >= tab[i+1]: coarse then fine, 64 entries each
-        constexpr int STEP = CO3_FIT_GRID / FIT_THREADS;       // 64
+        constexpr int STEP = CO3_FIT_GRID / FIT_SEARCH;        // 64
         const double target = s_target;
-        if (tab[tid * STEP] > target && target >= tab[(tid + 1) * STEP]) s_coarse = tid;
+        if (tid < FIT_SEARCH && tab[tid * STEP] > target && target >= tab[(tid + 1) * STEP]) s_coarse = tid;
         __syncthreads();
         if (tid < STEP) {
             const int i = s_coarse * STEP + tid;
             if (tab[i] > target && target >= tab[i + 1]) s_fine = i;
         }
         __syncthreads();
-        if (tid == 0) {
-            // inverse cubic (Lagrange) interpolation of log2(beta) as a function of log R through
-            // the four grid points around the bracket
-            int i = s_fine;
-            i = i < 1 ? 1 : (i > CO3_FIT_GRID - 2 ? CO3_FIT_GRID - 2 : i);
-            double xs[4], acc = 0.0;
-            for (int k = 0; k < 4; ++k) xs[k] = tab[i - 1 + k];
-            for (int a = 0; a < 4; ++a) {
-                double term = T0 + H * (double)(i - 1 + a);
-                for (int c = 0; c < 4; ++c)
-                    if (c != a) term *= (target - xs[c]) / (xs[a] - xs[c]);
-                acc += term;
-            }
-            s_t = acc;
-        }
-        __syncthreads();
     }
-    const double t = s_t;
-    const double beta = (s_state == 1) ? (t == T0 ? 0.3 : 2.0) : exp2(t);
-    if (tid < 2) s_lg[tid] = lgamma((double)(tid + 1) / beta);
-    __syncthreads();
     if (tid != 0) return;
 
-    const double alpha = (s_state == 2) ? 0.0 : (S1 / N) * exp(s_lg[0] - s_lg[1]);
+    double t = s_t, beta, log_g;
+    if (s_state == 0) {
+        // inverse cubic (Lagrange) interpolation of log2(beta) as a function of log R through the
+        // four grid points around the bracket, then cubic interpolation of log G at that point
+        int i = s_fine;
+        i = i < 1 ? 1 : (i > CO3_FIT_GRID - 2 ? CO3_FIT_GRID - 2 : i);
+        const double target = s_target;
+        double xs[4], gs[4], acc = 0.0;
+        for (int k = 0; k < 4; ++k) { xs[k] = tab[i - 1 + k]; gs[k] = tabg[i - 1 + k]; }
+        for (int a = 0; a < 4; ++a) {
+            double term = T0 + H * (double)(i - 1 + a);
+            for (int c = 0; c < 4; ++c)
+                if (c != a) term *= (target - xs[c]) / (xs[a] - xs[c]);
+            acc += term;
+        }
+        t = acc;
+        const double x = (t - (T0 + H * (double)(i - 1))) / H;           // position among the four nodes 0..3
+        log_g = gs[0] * ((x - 1.0) * (x - 2.0) * (x - 3.0) / -6.0) + gs[1] * (x * (x - 2.0) * (x - 3.0) / 2.0) +
+                gs[2] * (x * (x - 1.0) * (x - 3.0) / -2.0) + gs[3] * (x * (x - 1.0) * (x - 2.0) / 6.0);
+        beta = exp2(t);
+    } else if (s_state == 1) {
+        beta = (t == T0) ? 0.3 : 2.0;
+        log_g = tabg[s_fine];
+    } else {
+        beta = 1.0;
+        log_g = 0.0;
+    }
+    const double log2e = 1.4426950408889634;
+    // alpha = (S1 / N) * G(beta); its base-2 logarithm without forming alpha first
+    const double log2_alpha = (s_state == 2) ? 0.0 : (s_lg[2] - s_lg[0] + log_g) * log2e;
+    const bool has_alpha = s_state != 2;
+    const double alpha = has_alpha ? exp2(log2_alpha) : 0.0;
     int b_rule = p.b_lo;
-    if (alpha > 0.0) {
-        const double bf = floor(log2(alpha) - log2(poly_bias(beta)) + 0.5);
+    if (has_alpha && alpha > 0.0) {
+        const double bf = floor(log2_alpha - log2(poly_bias(beta)) + 0.5);
         b_rule = bf < (double)p.b_lo ? p.b_lo : (bf > (double)p.b_hi ? p.b_hi : (int)bf);
     }
     if (mode == 0) {
@@ -115,11 +130,11 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         return;
     }
     const int b_used = p.bias_cur[seg];
-    double x = floor(8.0 * log2(beta) + 0.5);
+    double x = floor(8.0 * (s_state == 0 ? t : log2(beta)) + 0.5);
     x = x < (double)CO3_IBETA_MIN ? (double)CO3_IBETA_MIN : (x > (double)CO3_IBETA_MAX ? (double)CO3_IBETA_MAX : x);
     double y = (double)CO3_IR_MIN;
-    if (alpha > 0.0) {
-        y = floor(8.0 * (log2(alpha) - (double)b_used) + 0.5);
+    if (has_alpha && alpha > 0.0) {
+        y = floor(8.0 * (log2_alpha - (double)b_used) + 0.5);
         y = y < (double)CO3_IR_MIN ? (double)CO3_IR_MIN : (y > (double)CO3_IR_MAX ? (double)CO3_IR_MAX : y);
     }
     co3_seg_header h;

@@ -75,7 +75,7 @@ struct Co3Dev {
     double* fit;                  // [S][5] beta, alpha, N, S1, S2
     int32_t* bias_cur;            // [S] bias used by the next convert pass
     const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
-    const double* logr_tab;       // [FIT_GRID + 1] log R(beta) at log2(beta) uniform in [log2 0.3, 1]
+    const double* logr_tab;       // [2][FIT_GRID + 1] log R(beta), log G(beta) at log2(beta) uniform in [log2 0.3, 1]
     Co3CodeBook cb;               // code tables of all model rows
     uint32_t* chunk_words;        // [U][n_chunks] payload words of each chunk (multiple of 4)
     uint32_t* chunk_bits;         // [U][n_chunks] code bits of each chunk
@@ -127,7 +127,7 @@ int co3_host_fmt_ok(co3_format f);
 int co3_host_cF(int E, int M);
 int64_t co3_host_K(int M, int j);
 const uint32_t* co3_host_weight_table(int E, int M);   // [NIBETA][NIR][J], cached per format
-const double* co3_host_logr_table(void);               // [FIT_GRID + 1], cached
+const double* co3_host_logr_table(void);               // [2][FIT_GRID + 1], cached
 
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st);

@@ -123,19 +123,22 @@ const uint32_t* co3_host_weight_table(int E, int M) {
     return t;
 }
 
-// log R(beta) = lgamma(1/b) + lgamma(3/b) - 2 lgamma(2/b) on a grid uniform in log2(beta) over
-// [log2 0.3, log2 2]; the device inverts it by inverse cubic interpolation (the moment ratio of a
-// GenNorm sample determines its shape).
+// Two functions of the GenNorm shape on a grid uniform in log2(beta) over [log2 0.3, log2 2]:
+//   [0 .. FIT_GRID]              log R(beta) = lgamma(1/b) + lgamma(3/b) - 2 lgamma(2/b)
+//   [FIT_GRID+1 .. 2 FIT_GRID+1] log G(beta) = lgamma(1/b) - lgamma(2/b)
+// The moment ratio of a GenNorm sample is R(beta) (the device inverts the first table by inverse
+// cubic interpolation) and its scale is alpha = E|X| * G(beta) (second table, cubic interpolation).
 const double* co3_host_logr_table(void) {
     static double* tab = nullptr;
     std::lock_guard<std::mutex> lk(g_mu);
     if (tab) return tab;
-    double* t = (double*)malloc(sizeof(double) * (CO3_FIT_GRID + 1));
+    double* t = (double*)malloc(sizeof(double) * 2 * (CO3_FIT_GRID + 1));
     if (!t) return nullptr;
     const double t0 = log2(0.3), t1 = 1.0;
     for (int i = 0; i <= CO3_FIT_GRID; ++i) {
         double b = (i == 0) ? 0.3 : (i == CO3_FIT_GRID ? 2.0 : exp2(t0 + (t1 - t0) * ((double)i / CO3_FIT_GRID)));
         t[i] = lgamma(1.0 / b) + lgamma(3.0 / b) - 2.0 * lgamma(2.0 / b);
+        t[CO3_FIT_GRID + 1 + i] = lgamma(1.0 / b) - lgamma(2.0 / b);
     }
     tab = t;
     return tab;
