@@ -31,6 +31,7 @@ int alloc_codebook(co3_plan* pl, Co3CodeBook& cb) {
     rc |= dev_alloc(pl, &cb.cand_len, R * CO3_NCAND * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.cand_max, R * CO3_NCAND);
     rc |= dev_alloc(pl, &cb.len8, R * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.len_pub, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.enc, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.code_msb, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.lut, R * CO3_LUT_SIZE);
@@ -374,8 +375,7 @@ extern "C" int co3_state_import(co3_plan* pl, int64_t iteration, const int32_t* 
 extern "C" int co3_debug_symbols(co3_plan* pl, uint8_t* symbols, void* cuda_stream) {
     if (!pl || !symbols) return CO3_EINVAL;
     cudaStream_t st = as_stream(cuda_stream);
-    CO3_TRY(cudaMemcpy2DAsync(symbols, (size_t)pl->dev.d, pl->dev.sym, (size_t)pl->dev.sld, (size_t)pl->dev.d,
-                              (size_t)pl->dev.U, cudaMemcpyDeviceToDevice, st));
+    CO3_TRY(co3_launch_symbol_export(pl, symbols, st));
     CO3_TRY(cudaStreamSynchronize(st));
     return CO3_OK;
 }
@@ -383,9 +383,18 @@ extern "C" int co3_debug_symbols(co3_plan* pl, uint8_t* symbols, void* cuda_stre
 extern "C" int co3_debug_hist(co3_plan* pl, uint64_t* hist) {
     if (!pl || !hist) return CO3_EINVAL;
     CO3_TRY(cudaStreamSynchronize(pl->last_stream));
-    CO3_TRY(cudaMemcpy2D(hist, sizeof(uint64_t) * (size_t)pl->dev.nsym, pl->dev.hist,
-                         sizeof(uint64_t) * CO3_MAXSYM, sizeof(uint64_t) * (size_t)pl->dev.nsym,
-                         (size_t)pl->dev.S, cudaMemcpyDeviceToHost));
+    const int S = pl->dev.S, nsym = pl->dev.nsym, nm = pl->dev.nm;
+    uint64_t* tmp = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)S * CO3_MAXSYM);
+    if (!tmp) return CO3_ENOMEM;
+    if (cudaMemcpy(tmp, pl->dev.hist, sizeof(uint64_t) * (size_t)S * CO3_MAXSYM, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        (void)cudaGetLastError();
+        free(tmp);
+        return CO3_ECUDA;
+    }
+    for (int l = 0; l < S; ++l)                          // stored by internal symbol, reported by public symbol
+        for (int sym = 0; sym < nsym; ++sym)
+            hist[(size_t)l * nsym + sym] = tmp[(size_t)l * CO3_MAXSYM + co3_sym_internal(sym, nm)];
+    free(tmp);
     return CO3_OK;
 }
 
@@ -401,7 +410,7 @@ extern "C" int co3_debug_code(co3_plan* pl, const co3_seg_header* hdr, uint8_t* 
         bool bad = false;
         const size_t row = (size_t)co3_row_of(h[l], &bad);
         if (bad) { rc = CO3_ECORRUPT; break; }
-        if (cudaMemcpy(lengths + (size_t)l * nsym, pl->dev.cb.len8 + row * CO3_MAXSYM, (size_t)nsym,
+        if (cudaMemcpy(lengths + (size_t)l * nsym, pl->dev.cb.len_pub + row * CO3_MAXSYM, (size_t)nsym,
                        cudaMemcpyDeviceToHost) != cudaSuccess ||
             cudaMemcpy(codewords + (size_t)l * nsym, pl->dev.cb.code_msb + row * CO3_MAXSYM,
                        sizeof(uint32_t) * (size_t)nsym, cudaMemcpyDeviceToHost) != cudaSuccess)

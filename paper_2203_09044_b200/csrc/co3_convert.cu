@@ -51,7 +51,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // binade, where it is the code itself; 2^M <= n <= 2^(M+1) above, where it carries the mantissa
 // and, on a carry, the next exponent).
 template <int M>
-__device__ __forceinline__ void quantize(float a, const QParams& q, int sign_shift, uint32_t& sym, float& m_new) {
+__device__ __forceinline__ void quantize(float a, const QParams& q, uint32_t& sym, float& m_new) {
     const uint32_t ab = __float_as_uint(a);
     const float axc = fminf(fabsf(a), q.top);
     // exponent field of max(|a|, 2^(lambda+M)), moved up by 23 - M binades, plus the 1.5
@@ -62,7 +62,7 @@ __device__ __forceinline__ void quantize(float a, const QParams& q, int sign_shi
     const uint32_t tb = __float_as_uint(t);
     const uint32_t j = (((tb >> 23) - q.e0) << M) + (tb & 0x3FFFFFu);
     const uint32_t sb = (r != 0.0f) ? (ab & 0x80000000u) : 0u;  // "-0" is never emitted
-    sym = j | (sb >> sign_shift);
+    sym = (j << 1) | (sb >> 31);                                 // internal form: code << 1 | sign
     m_new = __fsub_rn(a, __uint_as_float(__float_as_uint(r) | sb));
 }
 
@@ -117,7 +117,6 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
         for (int i = tid; i < (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
         __syncthreads();
     }
-    const int sign_shift = 31 - p.nm;
     const uint32_t n_chunks = (uint32_t)p.n_chunks;
     constexpr int VSTRIDE = 4 * CO3_THREADS;          // elements between a thread's vectors
 
@@ -137,37 +136,29 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
     const uint32_t ring_g = (uint32_t)__cvta_generic_to_shared(s_ring + tid);
     const uint32_t ring_m = (uint32_t)__cvta_generic_to_shared(s_ring + CO3_THREADS + tid);
     constexpr uint32_t SLOT_BYTES = 2 * CO3_THREADS * sizeof(float4);
+    static_assert(STAGES == STEPS, "step r of every item lives in ring slot r");
 
-    // producer cursor (runs STAGES-1 steps ahead of the consumer)
-    uint32_t pu = it0 / n_chunks, pc = it0 - pu * n_chunks, pitem = it0;
-    int pr = 0;
-    uint32_t pslot = 0;
-    ItemCtx pctx = make_ctx(pu, pc);
-    auto produce = [&]() {
-        if (pitem < it1) {
-            const int e0 = 4 * tid + VSTRIDE * pr;
-            if (pctx.whole || (e0 < pctx.hi && e0 + 4 > pctx.lo)) {
-                cp_async16(ring_g + pslot, pctx.gp + VSTRIDE * pr);
-                cp_async16(ring_m + pslot, pctx.mp + VSTRIDE * pr);
-            }
-            if (++pr == STEPS) {
-                pr = 0;
-                pitem += stride;
-                pc += stride;
-                while (pc >= n_chunks) { pc -= n_chunks; ++pu; }
-                if (pitem < it1) pctx = make_ctx(pu, pc);
-            }
+    // one asynchronous step: vector r of item x into ring slot r (one commit group per step)
+    auto issue = [&](const ItemCtx& x, bool valid, int r) {
+        const int e0 = 4 * tid + VSTRIDE * r;
+        if (valid && (x.whole || (e0 < x.hi && e0 + 4 > x.lo))) {
+            cp_async16(ring_g + r * SLOT_BYTES, x.gp + VSTRIDE * r);
+            cp_async16(ring_m + r * SLOT_BYTES, x.mp + VSTRIDE * r);
         }
-        cp_async_commit();                            // one group per step, even if empty
-        pslot = (pslot + SLOT_BYTES == STAGES * SLOT_BYTES) ? 0 : pslot + SLOT_BYTES;
+        cp_async_commit();
     };
-#pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) produce();
 
-    // consumer cursor
-    uint32_t cu = it0 / n_chunks, cc = it0 - cu * n_chunks;
+    uint32_t cu = it0 / n_chunks, cc = it0 - cu * n_chunks;        // (user, chunk) of the current item
     ItemCtx cur = make_ctx(cu, cc);
-    uint32_t cslot = 0;
+    issue(cur, true, 0);
+    issue(cur, true, 1);
+    issue(cur, true, 2);
+    uint32_t nu = cu, nc = cc + stride;                             // ... and of the next one
+    while (nc >= n_chunks) { nc -= n_chunks; ++nu; }
+    bool has_nxt = it0 + stride < it1;
+    ItemCtx nxt = cur;
+    if (has_nxt) nxt = make_ctx(nu, nc);
+
     int cur_seg = -1;
     QParams q;
     q.top = 0.0f; q.low_bits = 0; q.e0 = 0;
@@ -215,10 +206,12 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
         }
 #pragma unroll
         for (int r = 0; r < STEPS; ++r) {
-            produce();                                // step (this + STAGES - 1) goes in flight
+            // the producer is always STAGES - 1 = 3 steps ahead: step 3 of this item, then steps
+            // 0..2 of the next one, each into the slot the consumer has just left
+            if (r == 0) issue(cur, true, 3);
+            else issue(nxt, has_nxt, r - 1);
             cp_async_wait<STAGES - 1>();              // this step's copies have landed
-            const uint32_t slot = cslot;
-            cslot = (cslot + SLOT_BYTES == STAGES * SLOT_BYTES) ? 0 : cslot + SLOT_BYTES;
+            const uint32_t slot = r * SLOT_BYTES;
             const int e0 = 4 * tid + VSTRIDE * r;
             const bool full = cur.whole || ((e0 >= cur.lo) && (e0 + 4 <= cur.hi));
             if (!full && !(e0 < cur.hi && e0 + 4 > cur.lo)) continue;
@@ -231,7 +224,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
                 if (CONVERT) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        quantize<M>(a[e], q, sign_shift, so[e], mo[e]);
+                        quantize<M>(a[e], q, so[e], mo[e]);
                         atomicAdd(&s_hist[warp][so[e]], 1u);
                     }
                     *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
@@ -250,7 +243,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if (in[e]) {
-                            quantize<M>(a[e], q, sign_shift, so[e], mo[e]);
+                            quantize<M>(a[e], q, so[e], mo[e]);
                             atomicAdd(&s_hist[warp][so[e]], 1u);
                             cur.mp[VSTRIDE * r + e] = mo[e];
                             cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
@@ -260,15 +253,28 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             }
         }
         last = item;
-        if (item + stride < it1) {
+        if (has_nxt) {
             if (tid == 0) { p.part_s1[item] = 0.0; p.part_s2[item] = 0.0; p.part_nf[item] = 0; }
-            cc += stride;
-            while (cc >= n_chunks) { cc -= n_chunks; ++cu; }
-            cur = make_ctx(cu, cc);
+            cur = nxt;
+            has_nxt = item + 2 * stride < it1;
+            if (has_nxt) {
+                nc += stride;
+                while (nc >= n_chunks) { nc -= n_chunks; ++nu; }
+                nxt = make_ctx(nu, nc);
+            }
         }
     }
     cp_async_wait<0>();
     close_run(last, cur_seg);
+}
+
+// Inspection: copy the stored symbols to a caller buffer [U][d] in the public form.
+__global__ void symbol_export_kernel(Co3Dev p, uint8_t* __restrict__ out) {
+    const int64_t n = (int64_t)p.U * p.d;
+    for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t u = k / p.d, i = k - u * p.d;
+        out[k] = (uint8_t)co3_sym_public(p.sym[(size_t)u * p.sld + i], p.nm);
+    }
 }
 
 typedef void (*ef_fn)(Co3Dev, const float*, float*);
@@ -296,6 +302,11 @@ int ef_grid(const co3_plan* pl, ef_fn fn) {
 }
 
 }  // namespace
+
+cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_t st) {
+    symbol_export_kernel<<<pl->num_sms * 8, 256, 0, st>>>(pl->dev, symbols);
+    return cudaGetLastError();
+}
 
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st) {
     ef_fn fn = pick_kernel<false>(pl->dev.M);

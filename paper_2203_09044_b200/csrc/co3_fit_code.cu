@@ -250,8 +250,10 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p) {
         const uint32_t code = s_first[L] + r;
         const uint32_t rev = __brev(code) >> (32 - L);
         const size_t o = (size_t)rowi * CO3_MAXSYM + tid;
-        cb.len8[o] = (uint8_t)L;
-        cb.enc[o] = rev | ((uint32_t)L << 16);
+        const size_t oi = (size_t)rowi * CO3_MAXSYM + co3_sym_internal(tid, p.nm);
+        cb.len8[oi] = (uint8_t)L;                   // the encoder looks up stored (internal) symbols
+        cb.enc[oi] = rev | ((uint32_t)L << 16);
+        cb.len_pub[o] = (uint8_t)L;
         cb.code_msb[o] = code;
         s_perm[s_offs[L] + r] = (uint8_t)tid;
         if (rowi == 0) cb.ksign[tid] = co3_ksigned(tid, p.M, p.nm);

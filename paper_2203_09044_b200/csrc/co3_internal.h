@@ -45,9 +45,10 @@ struct Co3Group {
 struct Co3CodeBook {
     uint8_t* cand_len;   // [R][NCAND][256] code lengths per weight-floor candidate (build scratch)
     int32_t* cand_max;   // [R][NCAND]      longest codeword per candidate (build scratch)
-    uint8_t* len8;       // [R][256]        chosen lengths
-    uint32_t* enc;       // [R][256]        bit-reversed codeword | length << 16
-    uint32_t* code_msb;  // [R][256]        canonical codeword, root bit most significant
+    uint8_t* len8;       // [R][256]        chosen lengths, by internal symbol
+    uint8_t* len_pub;    // [R][256]        the same by public symbol (inspection only)
+    uint32_t* enc;       // [R][256]        bit-reversed codeword | length << 16, by internal symbol
+    uint32_t* code_msb;  // [R][256]        canonical codeword, root bit most significant, by public symbol
     uint32_t* lut;       // [R][2048]       (signed magnitude << 8) | length, 0 = longer than 11 bits
     uint32_t* first;     // [R][17]         first canonical code of each length
     uint32_t* count;     // [R][17]
@@ -67,8 +68,8 @@ struct Co3Dev {
     const Co3Group* groups;       // [n_groups]
     const int64_t* seg_off;       // [S+1]
     const int32_t* seg_chunk0;    // [S+1] first chunk of each segment
-    uint8_t* sym;                 // [U][sld]
-    unsigned long long* hist;     // [S][256]
+    uint8_t* sym;                 // [U][sld] internal symbols (co3_sym_internal)
+    unsigned long long* hist;     // [S][256] by internal symbol
     double* part_s1;              // [U*n_chunks] per-(user,chunk) partial sums of |a|
     double* part_s2;              //              ... of a^2
     uint32_t* part_nf;            //              ... count of non-finite a
@@ -141,6 +142,7 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
                               cudaStream_t st);
 cudaError_t co3_setup_kernels(void);
+cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_t st);
 
 // Model row of a segment header; out-of-range indices (a corrupt header) are clamped and reported.
 __host__ __device__ inline int co3_row_of(const co3_seg_header h, bool* bad) {
@@ -152,6 +154,12 @@ __host__ __device__ inline int co3_row_of(const co3_seg_header h, bool* bad) {
     }
     return (ib - CO3_IBETA_MIN) * CO3_NIR + (ir - CO3_IR_MIN);
 }
+
+// Inside the library a symbol is stored as (magnitude code << 1) | sign instead of the public
+// sign << (E+M) | magnitude code: the frequent symbols (small and medium magnitudes of both
+// signs) are then neighbours, so table look-ups of a warp spread over distinct shared-memory banks.
+__host__ __device__ inline int co3_sym_internal(int sym, int nm) { return ((sym & ((1 << nm) - 1)) << 1) | (sym >> nm); }
+__host__ __device__ inline int co3_sym_public(int isym, int nm) { return ((isym & 1) << nm) | (isym >> 1); }
 
 // Signed integer magnitude of a symbol byte: K(j) = f (e = 0) or (2^M + f) << (e - 1).
 __host__ __device__ inline int32_t co3_ksigned(int sym, int M, int nm) {
