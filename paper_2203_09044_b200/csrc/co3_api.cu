@@ -216,7 +216,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &d_wtab, (size_t)CO3_NIBETA * CO3_NIR * J);
         a |= dev_alloc(pl, &d_logr, 2 * ((size_t)CO3_FIT_GRID + 1));
         a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
-        a |= dev_alloc(pl, &dv.hist, (size_t)S * CO3_MAXSYM);
+        a |= dev_alloc(pl, &dv.hist, (size_t)S * CO3_MAXSYM + 1);
         a |= dev_alloc(pl, &dv.part_s1, items);
         a |= dev_alloc(pl, &dv.part_s2, items);
         a |= dev_alloc(pl, &dv.part_nf, items);
@@ -245,7 +245,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
             if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);
             if (e == cudaSuccess) e = cudaMemset(dv.fit, 0, sizeof(double) * (size_t)S * 5);
-            if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * (size_t)S * CO3_MAXSYM);
+            if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * ((size_t)S * CO3_MAXSYM + 1));
+            dv.ticket = reinterpret_cast<unsigned int*>(dv.hist + (size_t)S * CO3_MAXSYM);
             if (e == cudaSuccess) e = cudaMemset(dv.sym, 0, (size_t)dv.U * (size_t)dv.sld);
             if (e == cudaSuccess && !g_kernels_ready) {
                 e = co3_setup_kernels();

@@ -8,13 +8,12 @@
 // in the row, so segment boundaries never misalign the vectors; the vectors that straddle a
 // chunk edge are handled element by element.
 //
-// Work item = (user, chunk).  Blocks are persistent and take every gridDim-th item, so a block
-// meets its segments in order and stays inside one for long stretches, while the grid as a whole
-// sweeps one window of memory: the histogram lives in shared memory (one copy
-// per warp) and is flushed with 64-bit global atomics only when the segment changes; the moments
-// are kept per thread over such a run of items and reduced in a fixed order once per run (the
-// sum lands in the per-item array at the run's last item, zeros elsewhere), so there is no
-// barrier inside a run and the fit does not depend on scheduling.
+// Work item = (user, chunk).  Blocks are persistent and claim items in order through an atomic
+// ticket, so the grid as a whole sweeps one window of memory (with a fixed assignment of items to
+// blocks the blocks drift apart and a plain streaming kernel loses ~10 % of the bandwidth).  The
+// histogram lives in shared memory (one copy per warp) and is flushed with 64-bit global atomics
+// when the block leaves a segment; the moments are reduced in a fixed order per item and stored
+// per item, so the fit does not depend on which block converted which item.
 //
 // Memory pipeline: a thread handles one 4-element vector of g and of m per step (4 steps per
 // item).  The loads are asynchronous copies (cp.async, 16 B, L2-only) into thread-private slots of
@@ -102,25 +101,32 @@ __global__ void __launch_bounds__(CO3_THREADS, 4)
 ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
     extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS]
     __shared__ uint32_t s_hist[CONVERT ? CO3_THREADS / 32 : 1][CO3_MAXSYM];
-    __shared__ double s_red[2][CO3_THREADS / 32];
-    __shared__ uint32_t s_rednf[CO3_THREADS / 32];
+    __shared__ double s_red[2][2][CO3_THREADS / 32];
+    __shared__ uint32_t s_rednf[2][CO3_THREADS / 32];
+    __shared__ uint32_t s_ticket[2];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // items blockIdx.x, blockIdx.x + gridDim.x, ...: at any time the blocks of the grid work on
-    // neighbouring chunks, so the whole GPU sweeps one window of each array (DRAM page and L2
-    // locality of a streaming copy) while a block still meets its segments in order
     const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.U;
-    const uint32_t it0 = blockIdx.x, it1 = n_items, stride = gridDim.x;
-    if (it0 >= it1) return;
-
-    if (CONVERT) {
-        for (int i = tid; i < (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
-        __syncthreads();
-    }
     const uint32_t n_chunks = (uint32_t)p.n_chunks;
     constexpr int VSTRIDE = 4 * CO3_THREADS;          // elements between a thread's vectors
 
-    auto make_ctx = [&](uint32_t uu, uint32_t cc) {
+    // Items are claimed through an atomic ticket, two ahead of the one being converted (the copy
+    // ring needs the next item's addresses).  Tickets are handed out in item order, so at any time
+    // the blocks of the grid work on neighbouring chunks -- the whole GPU sweeps one window of each
+    // array like a streaming copy -- and no block falls behind as it does with a fixed assignment.
+    if (tid == 0) {
+        s_ticket[0] = atomicAdd(p.ticket, 1u);
+        s_ticket[1] = atomicAdd(p.ticket, 1u);
+    }
+    if (CONVERT)
+        for (int i = tid; i < (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
+    __syncthreads();
+    uint32_t item = s_ticket[0], nitem = s_ticket[1];
+    if (item >= n_items) return;
+    __syncthreads();                                  // both tickets read before slot 0 is reused
+
+    auto make_ctx = [&](uint32_t it) {
+        const uint32_t uu = it / n_chunks, cc = it - uu * n_chunks;
         const Co3Chunk cd = p.chunks[cc];
         ItemCtx x;
         const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
@@ -148,62 +154,29 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
         cp_async_commit();
     };
 
-    uint32_t cu = it0 / n_chunks, cc = it0 - cu * n_chunks;        // (user, chunk) of the current item
-    ItemCtx cur = make_ctx(cu, cc);
+    ItemCtx cur = make_ctx(item);
     issue(cur, true, 0);
     issue(cur, true, 1);
     issue(cur, true, 2);
-    uint32_t nu = cu, nc = cc + stride;                             // ... and of the next one
-    while (nc >= n_chunks) { nc -= n_chunks; ++nu; }
-    bool has_nxt = it0 + stride < it1;
+    bool has_nxt = nitem < n_items;
     ItemCtx nxt = cur;
-    if (has_nxt) nxt = make_ctx(nu, nc);
+    if (has_nxt) nxt = make_ctx(nitem);
 
-    int cur_seg = -1;
+    int cur_seg = -1, par = 0;
     QParams q;
     q.top = 0.0f; q.low_bits = 0; q.e0 = 0;
 
-    // reduce the moments of the run of items that ends with `last_item` and start a new run
-    double s1 = 0.0, s2 = 0.0;
-    uint32_t nf = 0;
-    auto close_run = [&](uint32_t last_item, int seg) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            s1 += __shfl_down_sync(0xffffffffu, s1, o);
-            s2 += __shfl_down_sync(0xffffffffu, s2, o);
-            nf += __shfl_down_sync(0xffffffffu, nf, o);
-        }
-        if (lane == 0) { s_red[0][warp] = s1; s_red[1][warp] = s2; s_rednf[warp] = nf; }
-        __syncthreads();
-        if (tid == 0) {
-            double t1 = 0.0, t2 = 0.0;
-            uint32_t tn = 0;
-#pragma unroll
-            for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[0][w]; t2 += s_red[1][w]; tn += s_rednf[w]; }
-            p.part_s1[last_item] = t1; p.part_s2[last_item] = t2; p.part_nf[last_item] = tn;
-        }
-        if (CONVERT && tid < p.nsym) {                // flush the histogram of the run's segment
-            unsigned long long tot = 0;
-#pragma unroll
-            for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[w][tid]; s_hist[w][tid] = 0; }
-            if (tot) atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + tid], tot);
-        }
-        __syncthreads();
-        s1 = 0.0; s2 = 0.0; nf = 0;
-    };
-
-    uint32_t last = it0;
-    for (uint32_t item = it0; item < it1; item += stride) {
-        if (cur.seg != cur_seg) {
-            if (cur_seg >= 0) close_run(item - stride, cur_seg);
+    while (true) {
+        if (tid == 0 && has_nxt) s_ticket[par] = atomicAdd(p.ticket, 1u);   // the item after next
+        if (CONVERT && cur.seg != cur_seg) {
             cur_seg = cur.seg;
-            if (CONVERT) {
-                const int lambda = p.bias_cur[cur.seg] + p.cF;
-                q.top = __fmul_rn((float)p.Kmax, pow2f(lambda));
-                q.low_bits = __float_as_uint(pow2f(lambda + M));
-                q.e0 = (uint32_t)(lambda + 150);
-            }
+            const int lambda = p.bias_cur[cur.seg] + p.cF;
+            q.top = __fmul_rn((float)p.Kmax, pow2f(lambda));
+            q.low_bits = __float_as_uint(pow2f(lambda + M));
+            q.e0 = (uint32_t)(lambda + 150);
         }
+        double s1 = 0.0, s2 = 0.0;
+        uint32_t nf = 0;
 #pragma unroll
         for (int r = 0; r < STEPS; ++r) {
             // the producer is always STAGES - 1 = 3 steps ahead: step 3 of this item, then steps
@@ -252,20 +225,43 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
                 }
             }
         }
-        last = item;
-        if (has_nxt) {
-            if (tid == 0) { p.part_s1[item] = 0.0; p.part_s2[item] = 0.0; p.part_nf[item] = 0; }
-            cur = nxt;
-            has_nxt = item + 2 * stride < it1;
-            if (has_nxt) {
-                nc += stride;
-                while (nc >= n_chunks) { nc -= n_chunks; ++nu; }
-                nxt = make_ctx(nu, nc);
-            }
+        // this item's moments, reduced in a fixed order (lanes, then warps) and stored per item:
+        // the fit does not depend on which block converted which item
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s1 += __shfl_down_sync(0xffffffffu, s1, o);
+            s2 += __shfl_down_sync(0xffffffffu, s2, o);
+            nf += __shfl_down_sync(0xffffffffu, nf, o);
         }
+        if (lane == 0) { s_red[par][0][warp] = s1; s_red[par][1][warp] = s2; s_rednf[par][warp] = nf; }
+        __syncthreads();                              // partial sums, histogram adds, next ticket
+        if (tid == 0) {
+            double t1 = 0.0, t2 = 0.0;
+            uint32_t tn = 0;
+#pragma unroll
+            for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
+            p.part_s1[item] = t1; p.part_s2[item] = t2; p.part_nf[item] = tn;
+        }
+        const uint32_t after = has_nxt ? s_ticket[par] : n_items;
+        // flush the histogram when the block leaves the segment (or ends)
+        if (CONVERT && (!has_nxt || nxt.seg != cur.seg)) {
+            if (tid < p.nsym) {
+                unsigned long long tot = 0;
+#pragma unroll
+                for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[w][tid]; s_hist[w][tid] = 0; }
+                if (tot) atomicAdd(&p.hist[(size_t)cur.seg * CO3_MAXSYM + tid], tot);
+            }
+            __syncthreads();
+        }
+        if (!has_nxt) break;
+        item = nitem;
+        cur = nxt;
+        nitem = after;
+        has_nxt = nitem < n_items;
+        if (has_nxt) nxt = make_ctx(nitem);
+        par ^= 1;
     }
     cp_async_wait<0>();
-    close_run(last, cur_seg);
 }
 
 // Inspection: copy the stored symbols to a caller buffer [U][d] in the public form.
@@ -311,6 +307,8 @@ cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st) {
     ef_fn fn = pick_kernel<false>(pl->dev.M);
     if (!pl->grid_stats) pl->grid_stats = ef_grid(pl, fn);
+    cudaError_t e = cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
+    if (e != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_STATS, st);
     fn<<<pl->grid_stats, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, const_cast<float*>(m));
     co3_prof_end(pl, CO3_K_STATS, st, 1);
@@ -318,7 +316,8 @@ cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaS
 }
 
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st) {
-    cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * (size_t)pl->dev.S * CO3_MAXSYM, st);
+    // one memset clears the histogram and the item ticket that follows it in the same allocation
+    cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.S * CO3_MAXSYM + 1), st);
     if (e != cudaSuccess) return e;
     ef_fn fn = pick_kernel<true>(pl->dev.M);
     if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn);
