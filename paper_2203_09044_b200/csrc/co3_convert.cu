@@ -100,10 +100,11 @@ template <int M, bool CONVERT>
 __global__ void __launch_bounds__(CO3_THREADS, 4)
 ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
     extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS]
-    __shared__ uint32_t s_hist[CONVERT ? CO3_THREADS / 32 : 1][CO3_MAXSYM];
+    __shared__ uint32_t s_hist[2][CONVERT ? CO3_THREADS / 32 : 1][CO3_MAXSYM];   // [item parity][warp][symbol]
     __shared__ double s_red[2][2][CO3_THREADS / 32];
     __shared__ uint32_t s_rednf[2][CO3_THREADS / 32];
     __shared__ uint32_t s_ticket[2];
+    __shared__ Co3Chunk s_chunk[2];                   // descriptor of the chunk of s_ticket[.]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.U;
@@ -119,15 +120,14 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
         s_ticket[1] = atomicAdd(p.ticket, 1u);
     }
     if (CONVERT)
-        for (int i = tid; i < (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
+        for (int i = tid; i < 2 * (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0][0])[i] = 0;
     __syncthreads();
     uint32_t item = s_ticket[0], nitem = s_ticket[1];
     if (item >= n_items) return;
     __syncthreads();                                  // both tickets read before slot 0 is reused
 
-    auto make_ctx = [&](uint32_t it) {
-        const uint32_t uu = it / n_chunks, cc = it - uu * n_chunks;
-        const Co3Chunk cd = p.chunks[cc];
+    auto make_ctx = [&](uint32_t it, const Co3Chunk& cd) {
+        const uint32_t uu = it / n_chunks;
         ItemCtx x;
         const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
         x.gp = g + (size_t)uu * p.ld + tb + 4 * tid;
@@ -154,20 +154,24 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
         cp_async_commit();
     };
 
-    ItemCtx cur = make_ctx(item);
+    ItemCtx cur = make_ctx(item, p.chunks[item % n_chunks]);
     issue(cur, true, 0);
     issue(cur, true, 1);
     issue(cur, true, 2);
     bool has_nxt = nitem < n_items;
     ItemCtx nxt = cur;
-    if (has_nxt) nxt = make_ctx(nitem);
+    if (has_nxt) nxt = make_ctx(nitem, p.chunks[nitem % n_chunks]);
 
     int cur_seg = -1, par = 0;
     QParams q;
     q.top = 0.0f; q.low_bits = 0; q.e0 = 0;
 
     while (true) {
-        if (tid == 0 && has_nxt) s_ticket[par] = atomicAdd(p.ticket, 1u);   // the item after next
+        // thread 0 claims the item after next now, fetches its chunk descriptor half-way through the
+        // item and publishes both before the item's barrier: no thread ever waits for either
+        uint32_t claim = n_items;
+        Co3Chunk claim_cd;
+        if (tid == 0 && has_nxt) claim = atomicAdd(p.ticket, 1u);
         if (CONVERT && cur.seg != cur_seg) {
             cur_seg = cur.seg;
             const int lambda = p.bias_cur[cur.seg] + p.cF;
@@ -183,6 +187,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             // 0..2 of the next one, each into the slot the consumer has just left
             if (r == 0) issue(cur, true, 3);
             else issue(nxt, has_nxt, r - 1);
+            if (r == 2 && tid == 0 && claim < n_items) claim_cd = p.chunks[claim % n_chunks];
             cp_async_wait<STAGES - 1>();              // this step's copies have landed
             const uint32_t slot = r * SLOT_BYTES;
             const int e0 = 4 * tid + VSTRIDE * r;
@@ -198,7 +203,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         quantize<M>(a[e], q, so[e], mo[e]);
-                        atomicAdd(&s_hist[warp][so[e]], 1u);
+                        atomicAdd(&s_hist[par][warp][so[e]], 1u);
                     }
                     *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
                     *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
@@ -217,7 +222,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
                     for (int e = 0; e < 4; ++e) {
                         if (in[e]) {
                             quantize<M>(a[e], q, so[e], mo[e]);
-                            atomicAdd(&s_hist[warp][so[e]], 1u);
+                            atomicAdd(&s_hist[par][warp][so[e]], 1u);
                             cur.mp[VSTRIDE * r + e] = mo[e];
                             cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
                         }
@@ -234,7 +239,11 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             nf += __shfl_down_sync(0xffffffffu, nf, o);
         }
         if (lane == 0) { s_red[par][0][warp] = s1; s_red[par][1][warp] = s2; s_rednf[par][warp] = nf; }
-        __syncthreads();                              // partial sums, histogram adds, next ticket
+        if (tid == 0) {
+            s_ticket[par] = claim;
+            if (claim < n_items) s_chunk[par] = claim_cd;
+        }
+        __syncthreads();                              // the item's only barrier: sums, histogram, claim
         if (tid == 0) {
             double t1 = 0.0, t2 = 0.0;
             uint32_t tn = 0;
@@ -242,23 +251,20 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
             p.part_s1[item] = t1; p.part_s2[item] = t2; p.part_nf[item] = tn;
         }
-        const uint32_t after = has_nxt ? s_ticket[par] : n_items;
-        // flush the histogram when the block leaves the segment (or ends)
-        if (CONVERT && (!has_nxt || nxt.seg != cur.seg)) {
-            if (tid < p.nsym) {
-                unsigned long long tot = 0;
+        // The item's histogram goes to global memory now; the next item counts in the other copy,
+        // and this copy is not touched again before the next item's barrier.
+        if (CONVERT && tid < p.nsym) {
+            unsigned long long tot = 0;
 #pragma unroll
-                for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[w][tid]; s_hist[w][tid] = 0; }
-                if (tot) atomicAdd(&p.hist[(size_t)cur.seg * CO3_MAXSYM + tid], tot);
-            }
-            __syncthreads();
+            for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[par][w][tid]; s_hist[par][w][tid] = 0; }
+            if (tot) atomicAdd(&p.hist[(size_t)cur.seg * CO3_MAXSYM + tid], tot);
         }
         if (!has_nxt) break;
         item = nitem;
         cur = nxt;
-        nitem = after;
+        nitem = s_ticket[par];
         has_nxt = nitem < n_items;
-        if (has_nxt) nxt = make_ctx(nitem);
+        if (has_nxt) nxt = make_ctx(nitem, s_chunk[par]);
         par ^= 1;
     }
     cp_async_wait<0>();
@@ -290,6 +296,9 @@ ef_fn pick_kernel(int M) {
 
 int ef_grid(const co3_plan* pl, ef_fn fn) {
     int n = 0;
+    // static + dynamic shared memory exceed the 48 KiB default, so the kernel has to opt in
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RING_BYTES) != cudaSuccess)
+        (void)cudaGetLastError();
     cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, CO3_THREADS, RING_BYTES);
     if (n < 1) n = 1;
     const int64_t items = pl->dev.n_chunks * (int64_t)pl->dev.U;
