@@ -119,10 +119,10 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    wl = inputs.workload(1, n_users=args.users)
+    wl = inputs.workload(1, n_users=args.users).align_rows()
     U, d = wl.n_users, wl.d
     plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
-                        bias_mode=binding.BIAS_LAGGED)
+                        bias_mode=binding.BIAS_LAGGED, ld=wl.ld)
     out = plan.alloc_outputs()
     residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
     # every rank draws its own users' gradients (seed offset by rank): a weak-scaling replica
@@ -217,7 +217,7 @@ def run_ours(args):
         "config": {"workload": "configs[1]: %d users x ResNet-18 (10-class head) gradient, d=11173962, "
                                "62 layers, iid GenNorm(beta=0.8) per layer, E4M3, gamma=0.9, lagged bias" % U,
                    "d": d, "n_users": U, "n_segments": plan.S, "format": "E4M3", "gamma": wl.gamma,
-                   "bias_mode": "lagged", "replicas": world,
+                   "bias_mode": "lagged", "replicas": world, "row_stride": plan.ld,
                    "l2": "inputs larger than L2: %d MB of gradient+memory read per step, %d gradient "
                          "batches cycled" % (8 * U * d // 1000000, POOL)},
         "clocks": clocks,

@@ -216,7 +216,11 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &d_wtab, (size_t)CO3_NIBETA * CO3_NIR * J);
         a |= dev_alloc(pl, &d_logr, 2 * ((size_t)CO3_FIT_GRID + 1));
         a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
-        a |= dev_alloc(pl, &dv.hist, (size_t)S * CO3_MAXSYM + 1);
+        // Blocks add their shared-memory histograms to global memory with atomics; one counter takes
+        // ~1e8 atomics/s, which a large layer converted at full HBM rate exceeds, so the blocks are
+        // spread over several copies of the histogram (summed at read-out).
+        dv.hist_copies = S <= 1024 ? 8 : 1;
+        a |= dev_alloc(pl, &dv.hist, (size_t)dv.hist_copies * S * CO3_MAXSYM + 1);
         a |= dev_alloc(pl, &dv.part_s1, items);
         a |= dev_alloc(pl, &dv.part_s2, items);
         a |= dev_alloc(pl, &dv.part_nf, items);
@@ -245,8 +249,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
             if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);
             if (e == cudaSuccess) e = cudaMemset(dv.fit, 0, sizeof(double) * (size_t)S * 5);
-            if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * ((size_t)S * CO3_MAXSYM + 1));
-            dv.ticket = reinterpret_cast<unsigned int*>(dv.hist + (size_t)S * CO3_MAXSYM);
+            if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * ((size_t)dv.hist_copies * S * CO3_MAXSYM + 1));
+            dv.ticket = reinterpret_cast<unsigned int*>(dv.hist + (size_t)dv.hist_copies * S * CO3_MAXSYM);
             if (e == cudaSuccess) e = cudaMemset(dv.sym, 0, (size_t)dv.U * (size_t)dv.sld);
             if (e == cudaSuccess && !g_kernels_ready) {
                 e = co3_setup_kernels();
@@ -385,16 +389,22 @@ extern "C" int co3_debug_hist(co3_plan* pl, uint64_t* hist) {
     if (!pl || !hist) return CO3_EINVAL;
     CO3_TRY(cudaStreamSynchronize(pl->last_stream));
     const int S = pl->dev.S, nsym = pl->dev.nsym, nm = pl->dev.nm;
-    uint64_t* tmp = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)S * CO3_MAXSYM);
+    const int copies = pl->dev.hist_copies;
+    const size_t per_copy = (size_t)S * CO3_MAXSYM;
+    uint64_t* tmp = (uint64_t*)malloc(sizeof(uint64_t) * per_copy * copies);
     if (!tmp) return CO3_ENOMEM;
-    if (cudaMemcpy(tmp, pl->dev.hist, sizeof(uint64_t) * (size_t)S * CO3_MAXSYM, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    if (cudaMemcpy(tmp, pl->dev.hist, sizeof(uint64_t) * per_copy * copies, cudaMemcpyDeviceToHost) != cudaSuccess) {
         (void)cudaGetLastError();
         free(tmp);
         return CO3_ECUDA;
     }
     for (int l = 0; l < S; ++l)                          // stored by internal symbol, reported by public symbol
         for (int sym = 0; sym < nsym; ++sym)
-            hist[(size_t)l * nsym + sym] = tmp[(size_t)l * CO3_MAXSYM + co3_sym_internal(sym, nm)];
+        {
+            uint64_t tot = 0;
+            for (int k = 0; k < copies; ++k) tot += tmp[k * per_copy + (size_t)l * CO3_MAXSYM + co3_sym_internal(sym, nm)];
+            hist[(size_t)l * nsym + sym] = tot;
+        }
     free(tmp);
     return CO3_OK;
 }

@@ -11,8 +11,8 @@
 // Work item = (user, chunk).  Blocks are persistent and claim items in order through an atomic
 // ticket, so the grid as a whole sweeps one window of memory (with a fixed assignment of items to
 // blocks the blocks drift apart and a plain streaming kernel loses ~10 % of the bandwidth).  The
-// histogram lives in shared memory (one copy per warp) and is flushed with 64-bit global atomics
-// when the block leaves a segment; the moments are reduced in a fixed order per item and stored
+// histogram lives in shared memory (one copy per warp, two sets used alternately) and is flushed
+// with 64-bit global atomics when the block leaves a segment; the moments are reduced in a fixed order per item and stored
 // per item, so the fit does not depend on which block converted which item.
 //
 // Memory pipeline: a thread handles one 4-element vector of g and of m per step (4 steps per
@@ -162,7 +162,8 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
     ItemCtx nxt = cur;
     if (has_nxt) nxt = make_ctx(nitem, p.chunks[nitem % n_chunks]);
 
-    int cur_seg = -1, par = 0;
+    int cur_seg = -1, par = 0, hpar = 0;
+    unsigned long long* hist_copy = p.hist + (size_t)(blockIdx.x % (unsigned)p.hist_copies) * p.S * CO3_MAXSYM;
     QParams q;
     q.top = 0.0f; q.low_bits = 0; q.e0 = 0;
 
@@ -203,7 +204,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         quantize<M>(a[e], q, so[e], mo[e]);
-                        atomicAdd(&s_hist[par][warp][so[e]], 1u);
+                        atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
                     }
                     *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
                     *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
@@ -222,7 +223,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
                     for (int e = 0; e < 4; ++e) {
                         if (in[e]) {
                             quantize<M>(a[e], q, so[e], mo[e]);
-                            atomicAdd(&s_hist[par][warp][so[e]], 1u);
+                            atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
                             cur.mp[VSTRIDE * r + e] = mo[e];
                             cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
                         }
@@ -251,13 +252,18 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
             p.part_s1[item] = t1; p.part_s2[item] = t2; p.part_nf[item] = tn;
         }
-        // The item's histogram goes to global memory now; the next item counts in the other copy,
-        // and this copy is not touched again before the next item's barrier.
-        if (CONVERT && tid < p.nsym) {
-            unsigned long long tot = 0;
+        // When the block leaves the segment (or ends) its histogram goes to global memory; the next
+        // item counts in the other copy, and this copy is not touched again before a later barrier.
+        // (Flushing after every item instead costs a single-segment E4M3 gradient 30 % of the pass:
+        // all blocks then hammer the same 256 counters.)
+        if (CONVERT && (!has_nxt || nxt.seg != cur.seg)) {
+            if (tid < p.nsym) {
+                unsigned long long tot = 0;
 #pragma unroll
-            for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[par][w][tid]; s_hist[par][w][tid] = 0; }
-            if (tot) atomicAdd(&p.hist[(size_t)cur.seg * CO3_MAXSYM + tid], tot);
+                for (int w = 0; w < CO3_THREADS / 32; ++w) { tot += s_hist[hpar][w][tid]; s_hist[hpar][w][tid] = 0; }
+                if (tot) atomicAdd(&hist_copy[(size_t)cur.seg * CO3_MAXSYM + tid], tot);
+            }
+            hpar ^= 1;
         }
         if (!has_nxt) break;
         item = nitem;
@@ -326,7 +332,7 @@ cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaS
 
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st) {
     // one memset clears the histogram and the item ticket that follows it in the same allocation
-    cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.S * CO3_MAXSYM + 1), st);
+    cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st);
     if (e != cudaSuccess) return e;
     ef_fn fn = pick_kernel<true>(pl->dev.M);
     if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn);

@@ -69,7 +69,8 @@ struct Co3Dev {
     const int64_t* seg_off;       // [S+1]
     const int32_t* seg_chunk0;    // [S+1] first chunk of each segment
     uint8_t* sym;                 // [U][sld] internal symbols (co3_sym_internal)
-    unsigned long long* hist;     // [S][256] by internal symbol (+ one word: the item ticket)
+    unsigned long long* hist;     // [hist_copies][S][256] by internal symbol (+ one word: the item ticket)
+    int hist_copies;              // the copies are summed when the histogram is read out
     unsigned int* ticket;         // item ticket of the convert / stats pass (last word of hist)
     double* part_s1;              // [U*n_chunks] per-(user,chunk) partial sums of |a|
     double* part_s2;              //              ... of a^2

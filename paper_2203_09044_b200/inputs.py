@@ -25,6 +25,11 @@ def gennorm(n: int, beta: float, alpha, gen: torch.Generator, device="cpu") -> t
     return (x * alpha).to(torch.float32)
 
 
+def aligned_ld(d: int) -> int:
+    """Row stride in elements that puts every row on a 16 KiB boundary."""
+    return (d + 4095) // 4096 * 4096
+
+
 def resnet18_cifar_tensor_sizes(num_classes: int = 10) -> List[int]:
     """Element counts of the parameter tensors of a CIFAR-style ResNet-18, in definition order."""
     sizes = [64 * 3 * 3 * 3, 64, 64]                       # stem conv + BN weight/bias
@@ -54,11 +59,18 @@ class Workload:
     seg_alpha: Optional[List[float]] = None     # per-segment GenNorm scale
     outlier_prob: float = 0.0
     outlier_gain: float = 1.0
+    row_stride: Optional[int] = None            # elements between user rows; None = d rounded up to 4
     _alpha_vec: dict = field(default_factory=dict, repr=False)
 
     @property
     def ld(self) -> int:
-        return (self.d + 3) // 4 * 4
+        return self.row_stride if self.row_stride is not None else (self.d + 3) // 4 * 4
+
+    def align_rows(self) -> "Workload":
+        """Start every user's row on a 16 KiB boundary (what the benchmark uses: with rows that start
+        in the middle of a 128-byte line every 512-byte warp access touches five lines, not four)."""
+        self.row_stride = aligned_ld(self.d)
+        return self
 
     @property
     def n_segments(self) -> int:

@@ -1,0 +1,161 @@
+"""Throughput report over the benchmark configurations and the size / users / shape / format sweep.
+
+    python -m paper_2203_09044_b200.sweep --configs 0,1,2,3 --sweep --out report.md
+
+For every workload it runs CO3 iterations (co3_encode + co3_decode_aggregate) on seeded synthetic
+GenNorm gradients and prints one markdown table row: milliseconds per steady-state iteration, GB/s
+of fp32 gradient, the fused convert pass against its 13 B per user-element, the encode passes, the
+decode-aggregate pass, and the code / container bits per element.  All times are CUDA-event times;
+per-kernel times come from the library's own event pairs around each launch.  Nothing here touches
+the CPU oracle: this is a measurement script, parity lives in tests/.
+
+Cells whose gradients and memories alone would need more than --max-bytes of device memory are
+listed as skipped (the largest sweep cell, 2^28 elements x 64 users, needs about 160 GiB).
+"""
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+from . import binding, inputs
+
+L2_BYTES = 126e6
+NOMINAL_HBM_GBS = 8000.0
+FORMATS = ((1, 2), (3, 2), (4, 3))                      # E1M2 (fp4), E3M2 (fp6), E4M3 (fp8)
+
+
+def measured_hbm_gbs():
+    """Measured copy bandwidth of this machine's GPUs if the file is there, else the fallback figure."""
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def device_bytes_needed(wl, pool):
+    """Gradients (pool copies), memory, symbols, worst-case payload and the average."""
+    ud = wl.n_users * wl.d
+    return 4 * ud * pool + 4 * ud + ud + 2 * ud + 4 * wl.d
+
+
+def measure(wl, iters, warm, pool):
+    """Run warm + iters iterations of one workload; returns a dict of figures."""
+    wl.align_rows()
+    U, d = wl.n_users, wl.d
+    plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
+                        bias_mode=binding.BIAS_LAGGED, ld=wl.ld)
+    out = plan.alloc_outputs()
+    residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+    grads = [wl.gradient(t, device="cuda") for t in range(pool)]
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def step(t):
+        plan.encode(grads[t % pool], residual, out)
+        plan.decode_aggregate(out)
+
+    e0.record()
+    step(0)                                             # t = 0: includes the bootstrap statistics pass
+    e1.record()
+    torch.cuda.synchronize()
+    first_ms = e0.elapsed_time(e1)
+    for t in range(1, warm):
+        step(t)
+    torch.cuda.synchronize()
+    plan.profile_enable(None, max_records=2 * iters + 8)
+    e0.record()
+    for t in range(iters):
+        step(warm + t)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    prof = {k: v[0] / iters for k, v in plan.profile_collect().items() if v[1]}
+    plan.profile_enable([], 0)
+    flags, nonfinite = plan.status(clear=True)
+    code_bits = float(out["user_bits"].sum().item()) / (U * d)
+    container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
+                      + 32.0 * U * (plan.n_chunks + 1) + 32.0 * plan.S) / (U * d)
+    res = dict(name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
+               ms=ms, first_ms=first_ms, gbs=4.0 * U * d / (ms * 1e-3) / 1e9,
+               convert_ms=prof.get("convert", 0.0),
+               encode_ms=prof.get("enc_len", 0.0) + prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0),
+               fit_ms=prof.get("fit", 0.0), decode_ms=prof.get("decode", 0.0),
+               code_bits=code_bits, container_bits=container_bits, flags=flags,
+               l2_resident=8.0 * U * d * pool < L2_BYTES)
+    plan.close()
+    del out, residual, grads
+    torch.cuda.empty_cache()
+    return res
+
+
+HEADER = ("| workload | d | U | format | beta | ms/iter | GB/s fp32 in | convert us | convert GB/s (13 B) | % of {peak:.0f} "
+          "| % of 8000 | encode us | decode us | decode+encode GB/s (payload+symbols+avg) | code b/el | container b/el | t=0 ms | note |\n"
+          "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+
+
+def row(r, peak):
+    ud = r["U"] * r["d"]
+    conv_gbs = 13.0 * ud / (r["convert_ms"] * 1e-3) / 1e9 if r["convert_ms"] else 0.0
+    # encode + decode algorithmic bytes: symbols read twice, payload written and read, average written
+    ed_bytes = 2.0 * ud + 2.0 * r["code_bits"] / 8.0 * ud + 4.0 * r["d"]
+    ed_ms = r["encode_ms"] + r["decode_ms"]
+    ed_gbs = ed_bytes / (ed_ms * 1e-3) / 1e9 if ed_ms else 0.0
+    note = []
+    if r["l2_resident"]:
+        note.append("inputs fit L2, launch-bound")
+    if r["flags"]:
+        note.append("flags=%d" % r["flags"])
+    return ("| %s | %d | %d | %s | %.1f | %.4f | %.1f | %.1f | %.0f | %.1f | %.1f | %.1f | %.1f | %.0f | %.3f | %.3f | %.3f | %s |"
+            % (r["name"], r["d"], r["U"], r["fmt"], r["beta"], r["ms"], r["gbs"], r["convert_ms"] * 1e3, conv_gbs,
+               100.0 * conv_gbs / peak, 100.0 * conv_gbs / NOMINAL_HBM_GBS, r["encode_ms"] * 1e3,
+               r["decode_ms"] * 1e3, ed_gbs, r["code_bits"], r["container_bits"], r["first_ms"], "; ".join(note)))
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
+    ap.add_argument("--configs", default="0,1,2,3", help="comma list of benchmark configurations (empty: none)")
+    ap.add_argument("--sweep", action="store_true", help="also run the 108-cell sweep")
+    ap.add_argument("--iters", type=int, default=5, help="timed steady-state iterations per workload")
+    ap.add_argument("--warm", type=int, default=3, help="untimed iterations before them (>= 1)")
+    ap.add_argument("--max-bytes", type=float, default=60e9, help="skip workloads needing more device memory")
+    ap.add_argument("--filter", default=None, help="run only workloads whose name contains this text")
+    ap.add_argument("--out", default=None, help="also write the table to this file")
+    args = ap.parse_args(argv)
+    binding.lib()                                       # no CUDA library: raise, never fall back
+    peak, src = measured_hbm_gbs()
+    lines = ["Peak used for the convert column: %.1f GB/s (%s copy bandwidth); nominal 8000 GB/s beside it." % (peak, src),
+             "", HEADER.format(peak=peak)]
+    todo = [inputs.workload(int(i)) for i in args.configs.split(",") if i != ""]
+    if args.sweep:
+        for d_log in (16, 20, 24, 28):
+            for users in (1, 8, 64):
+                for beta in (0.5, 1.0, 2.0):
+                    for e, m in FORMATS:
+                        todo.append(inputs.sweep_cell(1 << d_log, users, beta, e, m))
+    if args.filter:
+        todo = [wl for wl in todo if args.filter in wl.name]
+    for wl in todo:
+        pool = 2 if device_bytes_needed(wl, 2) <= args.max_bytes else 1
+        if device_bytes_needed(wl, pool) > args.max_bytes:
+            lines.append("| %s | %d | %d | E%dM%d | %.1f | skipped: needs %.0f GB of device memory | | | | | | | | | | | |"
+                         % (wl.name, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.beta,
+                            device_bytes_needed(wl, 1) / 1e9))
+            continue
+        r = measure(wl, args.iters, max(args.warm, 1), pool)
+        lines.append(row(r, peak))
+        print(lines[-1], flush=True)
+    text = "\n".join(lines) + "\n"
+    if args.out:
+        with open(args.out, "w") as f:
+            f.write(text)
+    else:
+        sys.stdout.write(text)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -53,8 +53,8 @@ def compare_iteration(b, plan, out, r, m_gpu, m_cpu, tag=""):
 
 
 def run_case(b, oracle, d, U, E, M, off, grads, gamma=0.9, mode=1, cap=None, decode_plan=None):
-    """grads: list of [U][ld] float32 cuda tensors, one per iteration."""
-    plan = b.Plan(d, U, E, M, off, gamma=gamma, bias_mode=mode, cap_words=cap)
+    """grads: list of [U][ld] float32 cuda tensors, one per iteration (ld is taken from them)."""
+    plan = b.Plan(d, U, E, M, off, gamma=gamma, bias_mode=mode, cap_words=cap, ld=int(grads[0].shape[1]))
     orc = oracle.OracleCO3(d, U, E, M, off, gamma=gamma, mode=mode, cap_words=plan.cap_words)
     assert plan.worst_case_words == orc.worst_case_words
     assert (plan.n_chunks, plan.n_sub) == (orc.part.n_chunks, orc.part.n_sub)
@@ -93,6 +93,18 @@ def test_configs_scaled_down(binding, oracle, idx):
     wl = inputs.workload(idx, d={0: 70_001, 1: 200_000, 2: 150_010, 3: 300_007}[idx])
     run_case(binding, oracle, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.seg_offsets,
              _grads(wl, 4), gamma=wl.gamma)
+
+
+def test_padded_rows_as_the_benchmark_lays_them_out(binding, oracle):
+    """Rows that start on 16 KiB boundaries (row stride > d): the padding between users is never
+    read as data nor written."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=90_000, n_users=3).align_rows()
+    assert wl.ld % 4096 == 0 and wl.ld > wl.d
+    grads = _grads(wl, 3)
+    for g in grads:
+        g[:, wl.d:] = 7.0                         # poison: must not leak into moments, symbols or residual
+    plan, orc, out, res = run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, grads, gamma=wl.gamma)
 
 
 @pytest.mark.parametrize("E,M", FORMATS)
@@ -273,7 +285,7 @@ def test_config0_full(binding, oracle):
 @pytest.mark.slow
 def test_config1_full_two_iterations(binding, oracle):
     from paper_2203_09044_b200 import inputs
-    wl = inputs.workload(1)
+    wl = inputs.workload(1).align_rows()           # rows on 16 KiB boundaries, as the benchmark lays them out
     run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma)
 
 
