@@ -35,6 +35,8 @@ int alloc_codebook(co3_plan* pl, Co3CodeBook& cb) {
     rc |= dev_alloc(pl, &cb.enc, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.code_msb, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.lut, R * CO3_LUT_SIZE);
+    cb.long_stride = 16 * pl->dev.nsym < CO3_LONG_CACHE ? CO3_LONG_CACHE : 16 * pl->dev.nsym;
+    rc |= dev_alloc(pl, &cb.lut_long, R * (size_t)cb.long_stride);
     rc |= dev_alloc(pl, &cb.first, R * (CO3_MAXLEN + 1));
     rc |= dev_alloc(pl, &cb.count, R * (CO3_MAXLEN + 1));
     rc |= dev_alloc(pl, &cb.offs, R * (CO3_MAXLEN + 1));

@@ -2,7 +2,8 @@
 // decode every user's stream and write the average of the reconstructed gradients.
 //
 // A lane decodes one sub-chunk (<= 128 codewords) serially with an 11-bit primary table whose
-// entries already hold the signed integer magnitude ((K << 8) | length); the 32 sub-chunks of a
+// entries already hold the signed integer magnitude ((K << 8) | length) -- codewords longer than 11
+// bits go through a second table in global memory; the 32 sub-chunks of a
 // chunk are the 32 lanes of a warp, so a warp is one (chunk, user) stream.  The magnitudes of all
 // users are accumulated with shared-memory reductions into a transposed, padded tile
 // (conflict-free both for the per-lane scattered adds and for the coalesced read-out), scaled
@@ -34,24 +35,29 @@ constexpr int STAGE_PAD = 72;
 constexpr int STAGE_ROW = CO3_STAGE_WORDS + STAGE_PAD;
 static_assert(STAGE_ROW % 4 == 0, "stage rows must keep 16-byte alignment");
 
+// The long codewords of a good code carry about as much Kraft mass as probability (~1e-3 of 65536
+// windows), so the head of the second table that fits here nearly always holds all of them.
+constexpr int LONG_CACHE = CO3_LONG_CACHE;
+
 struct Tables {                                   // per-segment decoder tables in shared memory
     alignas(16) uint32_t lut[CO3_LUT_SIZE];
-    uint32_t first[CO3_MAXLEN + 1], count[CO3_MAXLEN + 1], offs[CO3_MAXLEN + 1];
-    int32_t ksign[CO3_MAXSYM];
-    uint8_t perm[CO3_MAXSYM];
+    alignas(16) uint32_t long_cache[LONG_CACHE];  // head of the row's table of 12..16-bit codewords
+    const uint32_t* lut_long;                     // the whole of it (global memory)
+    uint32_t long_first;                          // first 16-bit window it covers
+    uint32_t long_n;                              // number of windows it covers
 };
 
-__device__ void load_tables(Tables& t, const Co3CodeBook& cb, int row, int nsym, int tid) {
+__device__ void load_tables(Tables& t, const Co3CodeBook& cb, int row, int tid) {
     const uint4* lut = reinterpret_cast<const uint4*>(cb.lut + (size_t)row * CO3_LUT_SIZE);
     uint4* dst = reinterpret_cast<uint4*>(t.lut);
     for (int i = tid; i < CO3_LUT_SIZE / 4; i += CO3_THREADS) dst[i] = __ldg(lut + i);
-    if (tid <= CO3_MAXLEN) {
-        const size_t o = (size_t)row * (CO3_MAXLEN + 1) + tid;
-        t.first[tid] = cb.first[o]; t.count[tid] = cb.count[o]; t.offs[tid] = cb.offs[o];
-    }
-    if (tid < nsym) {
-        t.ksign[tid] = cb.ksign[tid];
-        t.perm[tid] = cb.perm[(size_t)row * CO3_MAXSYM + tid];
+    if (tid < LONG_CACHE / 4)
+        reinterpret_cast<uint4*>(t.long_cache)[tid] =
+            __ldg(reinterpret_cast<const uint4*>(cb.lut_long + (size_t)row * cb.long_stride) + tid);
+    if (tid == 0) {
+        t.lut_long = cb.lut_long + (size_t)row * cb.long_stride;
+        t.long_first = cb.first[(size_t)row * (CO3_MAXLEN + 1) + CO3_LUT_BITS + 1] << (CO3_MAXLEN - CO3_LUT_BITS - 1);
+        t.long_n = (uint32_t)cb.long_stride;
     }
 }
 
@@ -70,18 +76,17 @@ __device__ __forceinline__ void red_add(uint32_t addr, uint32_t v) {
     asm volatile("red.shared.add.u32 [%0+%2], %1;" ::"r"(addr), "r"(v), "n"(OFF) : "memory");
 }
 
-// Codeword longer than the primary table: canonical search over lengths 12..16.  Returns the
-// entry (K << 8) | length.  Kept out of line: it is rare, and inlining it four times into the
-// unrolled decode loop made the loop slower.
-__device__ __noinline__ uint32_t decode_long(uint32_t window, const Tables& t, bool& bad) {
+// Codeword longer than the primary table: one look-up in the row's second table (its head is in
+// shared memory, the rest in global memory; about one symbol in a thousand comes here).  Returns the entry (K << 8) | length.
+__device__ __forceinline__ uint32_t decode_long(uint32_t window, const Tables& t, bool& bad) {
     const uint32_t v = __brev(window) >> 16;      // 16 stream bits, root bit on top
-    for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
-        const uint32_t dd = (v >> (CO3_MAXLEN - L)) - t.first[L];
-        if (dd < t.count[L])
-            return ((uint32_t)t.ksign[t.perm[(t.offs[L] + dd) & (CO3_MAXSYM - 1)]] << 8) | (uint32_t)L;
+    const uint32_t i = v - t.long_first;
+    uint32_t e = i < LONG_CACHE ? t.long_cache[i] : (i < t.long_n ? __ldg(t.lut_long + i) : 0u);
+    if ((e & 0xFFu) == 0u) {                      // no codeword starts like this: corrupt stream
+        bad = true;
+        e = CO3_MAXLEN;
     }
-    bad = true;                                   // cannot happen for a complete code
-    return CO3_MAXLEN;
+    return e;
 }
 
 // LSB-first bit reader over staged words: the stream sits at bits [0, nb) of hi:lo; rp is the
@@ -115,16 +120,45 @@ __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint
     r.rp += 8;
 }
 
-// One symbol: look up, consume, add to the accumulator row at byte offset OFF.
+// One symbol, fast form: look up, consume, add to the accumulator row at byte offset OFF, return
+// the table entry.  No test for a codeword longer than the table: such an entry is 0 (nothing is
+// consumed, nothing is added), so every later look-up of the group sees the same window and returns 0
+// too, and the caller tests only the group's LAST entry.
 // PACKED: add the whole entry (length byte included); else add the signed magnitude.
 template <int OFF, bool PACKED>
-__device__ __forceinline__ void decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr, const Tables& t, bool& bad) {
-    uint32_t e = lds32(lut_addr + ((r.lo & (CO3_LUT_SIZE - 1)) << 2));
-    if ((e & 0xFFu) == 0u) e = decode_long(r.lo, t, bad);
+__device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr) {
+    const uint32_t e = lds32(lut_addr + ((r.lo & (CO3_LUT_SIZE - 1)) << 2));
     r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= (int)(e & 0xFFu);
     red_add<OFF>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
+    return e;
+}
+
+// One symbol with the test for a long codeword (group tails, and groups that met a long codeword).
+template <bool PACKED>
+__device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr, uint32_t acc_addr,
+                                                    const Tables& t, bool& bad) {
+    uint32_t e = lds32(lut_addr + ((r.lo & (CO3_LUT_SIZE - 1)) << 2));
+    if ((e & 0xFFu) == 0u) e = decode_long(r.lo, t, bad);
+    r.lo = __funnelshift_r(r.lo, r.hi, e);
+    r.hi = __funnelshift_r(r.hi, 0u, e);
+    r.nb -= (int)(e & 0xFFu);
+    red_add<0>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
+}
+
+// A group of four whose fast pass stopped at a long codeword after `done` good symbols: the reader
+// stands exactly at that codeword, so the rest of the group is decoded with the checked step.
+// Rare (about one symbol in a thousand is longer than the table).  Inlined, so that the reader stays
+// in registers (its address is never taken); the long-codeword search itself is out of line.
+template <bool PACKED>
+__device__ __forceinline__ void finish_group(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int done,
+                                          const Tables& t, bool& bad) {
+#pragma unroll 1
+    for (int k = done; k < 4; ++k) {
+        refill(r);
+        decode_step_checked<PACKED>(r, lut_addr, acc_addr + (uint32_t)k * (PADW * 4), t, bad);
+    }
 }
 
 template <bool PACKED>
@@ -133,16 +167,20 @@ __device__ __forceinline__ void decode_run(Reader& r, uint32_t lut_addr, uint32_
     int i = 0;
     for (; i + 4 <= n; i += 4) {
         refill(r);
-        decode_step<0, PACKED>(r, lut_addr, acc_addr, t, bad);
-        decode_step<PADW * 4, PACKED>(r, lut_addr, acc_addr, t, bad);
+        const uint32_t e0 = decode_step<0, PACKED>(r, lut_addr, acc_addr);
+        const uint32_t e1 = decode_step<PADW * 4, PACKED>(r, lut_addr, acc_addr);
         refill(r);
-        decode_step<PADW * 8, PACKED>(r, lut_addr, acc_addr, t, bad);
-        decode_step<PADW * 12, PACKED>(r, lut_addr, acc_addr, t, bad);
+        const uint32_t e2 = decode_step<PADW * 8, PACKED>(r, lut_addr, acc_addr);
+        const uint32_t e3 = decode_step<PADW * 12, PACKED>(r, lut_addr, acc_addr);
+        if ((e3 & 0xFFu) == 0u) {
+            const int done = ((e0 & 0xFFu) != 0u) + ((e1 & 0xFFu) != 0u) + ((e2 & 0xFFu) != 0u);
+            finish_group<PACKED>(r, lut_addr, acc_addr, done, t, bad);
+        }
         acc_addr += PADW * 16;
     }
     for (; i < n; ++i) {
         refill(r);
-        decode_step<0, PACKED>(r, lut_addr, acc_addr, t, bad);
+        decode_step_checked<PACKED>(r, lut_addr, acc_addr, t, bad);
         acc_addr += PADW * 4;
     }
 }
@@ -251,6 +289,8 @@ constexpr int ACC_Q = QB * PADW;                  // accumulator words per chunk
 
 struct SmemA {
     Tables t;
+    long long c_tb[2][NW];                        // per chunk of the group: tile base, bounds in the tile
+    int c_lo[2][NW], c_hi[2][NW];                 // (two sets: a group is read out while the next one opens)
     alignas(16) uint32_t stage[NW][STAGE_ROW];    // filled with 128-bit stores
     alignas(16) int32_t acc[2][ACC_Q];            // really [2][chunks per group][ACC_Q], sized at launch
 };
@@ -281,14 +321,17 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     const float inv_u = (U & (U - 1)) == 0 ? 1.0f / fu : 0.0f;
     int cur_seg = -1;
     bool bad = false;
+    // Both accumulator buffers start at zero and every read-out zeroes what it has read, so one
+    // barrier per quarter is enough: decode(q) -> barrier -> read-out(q), and the buffer of quarter q
+    // is next written after the barrier of quarter q + 1.
+    for (int i = tid; i < 2 * accw / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
     for (int64_t gi = g0; gi < g1; ++gi) {
         const Co3Group grp = p.groups[gi];
-        __syncthreads();                           // previous group's read-out is finished
-        if (grp.seg != cur_seg) {
-            load_tables(sm.t, p.cb, co3_row_of(hdr[grp.seg], &bad), p.nsym, tid);
+        const int gp = (int)(gi & 1);
+        if (grp.seg != cur_seg) {                  // every warp is past the last decode with the old tables
+            load_tables(sm.t, p.cb, co3_row_of(hdr[grp.seg], &bad), tid);
             cur_seg = grp.seg;
         }
-        for (int i = tid; i < accw / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
         const bool mine = ci < cpg && ci < grp.count;
         Stream s;
         s.active = false; s.staged = true; s.nwords = 0; s.bitpos = 0; s.sub_len_bits = 0;
@@ -306,7 +349,14 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
             }
         }
         const float scale = pow2_clamped((int)hdr[grp.seg].bias + p.cF);
-        __syncthreads();                           // tables, zeroed accumulator 0
+        if (tid < grp.count) {
+            const Co3Chunk cd = p.chunks[grp.chunk0 + tid];
+            const long long tb = cd.start & ~(long long)(CO3_TILE - 1);
+            sm.c_tb[gp][tid] = tb;
+            sm.c_lo[gp][tid] = (int)(cd.start - tb);
+            sm.c_hi[gp][tid] = (int)(cd.start - tb) + cd.len;
+        }
+        __syncthreads();                           // tables, chunk bounds (and the first zeroing)
 #pragma unroll 1
         for (int q = 0; q < CO3_SUB / QB; ++q) {
             const int qoff = (q & 1) * accw;
@@ -319,26 +369,28 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                 }
             }
             __syncthreads();
-            // clear the other buffer for the next quarter while this one is written out
-            if (q + 1 < CO3_SUB / QB) {
-                uint4* z = reinterpret_cast<uint4*>(acc0 + ((q + 1) & 1) * accw);
-                for (int i = tid; i < accw / 4; i += CO3_THREADS) z[i] = make_uint4(0, 0, 0, 0);
-            }
+            // read-out: warp w, round rr takes sub-chunk w + 8 rr, lane l its symbol q*QB + l
+            const int e0 = warp * CO3_SUB + q * QB + lane;
             for (int cc = 0; cc < grp.count; ++cc) {
-                const Co3Chunk cd = p.chunks[grp.chunk0 + cc];
-                const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-                const int lo = (int)(cd.start - tb), hi = lo + cd.len;
-                const int32_t* a = acc0 + qoff + cc * ACC_Q;
+                const int lo = sm.c_lo[gp][cc], hi = sm.c_hi[gp][cc];
+                // the accumulator holds sum((K << 8) | length): the lengths of <= 8 users stay below 256
+                int32_t* a = acc0 + qoff + cc * ACC_Q + lane * PADW + warp;
+                float* o = avg + sm.c_tb[gp][cc] + e0;
+                if (lo == 0 && hi == CO3_TILE) {
 #pragma unroll
-                for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
-                    const int x = tid + rr * CO3_THREADS;
-                    const int kk = x >> 5, il = x & 31;
-                    const int e = kk * CO3_SUB + q * QB + il;
-                    // the accumulator holds sum((K << 8) | length): the lengths of <= 8 users stay below 256
-                    if (e >= lo && e < hi) avg[tb + e] = finish(a[il * PADW + kk] >> 8, scale, fu, inv_u);
+                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+                        o[rr * NW * CO3_SUB] = finish(a[rr * NW] >> 8, scale, fu, inv_u);
+                        a[rr * NW] = 0;
+                    }
+                } else {
+#pragma unroll
+                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+                        const int e = e0 + rr * NW * CO3_SUB;
+                        if (e >= lo && e < hi) o[rr * NW * CO3_SUB] = finish(a[rr * NW] >> 8, scale, fu, inv_u);
+                        a[rr * NW] = 0;
+                    }
                 }
             }
-            __syncthreads();
         }
         if (mine && s.active) {
             const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - (uint32_t)r.nb
@@ -375,7 +427,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     for (int64_t c = c0; c < c1; ++c) {
         const Co3Chunk cd = p.chunks[c];
         if (cd.seg != cur_seg) {
-            load_tables(sm.t, p.cb, co3_row_of(hdr[cd.seg], &bad), p.nsym, tid);
+            load_tables(sm.t, p.cb, co3_row_of(hdr[cd.seg], &bad), tid);
             cur_seg = cd.seg;
         }
         for (int i = tid; i < CO3_SUB * PADW / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(sm.acc)[i] = make_uint4(0, 0, 0, 0);

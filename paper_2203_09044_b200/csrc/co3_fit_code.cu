@@ -279,6 +279,25 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p) {
         }
         cb.lut[(size_t)rowi * CO3_LUT_SIZE + i] = entry;
     }
+    // Second table for the codewords the first one cannot hold.  Canonical codes grow with the length,
+    // so every 16-bit window that starts with a codeword of 12..16 bits is >= first[12] << 4, and
+    // there are at most 16 per symbol of them.
+    const uint32_t long_first = s_first[CO3_LUT_BITS + 1] << (CO3_MAXLEN - CO3_LUT_BITS - 1);
+    for (int i = tid; i < cb.long_stride; i += CO3_MAXSYM) {
+        const uint32_t v = long_first + (uint32_t)i;          // 16 stream bits, root bit on top
+        uint32_t entry = 0;                                    // 0: no codeword starts like this
+        if (v < (1u << CO3_MAXLEN)) {
+            for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
+                const uint32_t dd = (v >> (CO3_MAXLEN - L)) - s_first[L];
+                if (dd < s_count[L]) {
+                    const int sym = s_perm[s_offs[L] + dd];
+                    entry = ((uint32_t)co3_ksigned(sym, p.M, p.nm) << 8) | (uint32_t)L;
+                    break;
+                }
+            }
+        }
+        cb.lut_long[(size_t)rowi * cb.long_stride + i] = entry;
+    }
 }
 
 }  // namespace

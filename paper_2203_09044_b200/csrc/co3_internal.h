@@ -42,6 +42,9 @@ struct Co3Group {
 // code of a segment is a pure function of the format and of the two header indices, so all
 // CO3_NROWS codes are built on the device once, when the plan is created; an iteration only
 // selects rows.  Rows are CO3_MAXSYM / CO3_LUT_SIZE wide.
+// entries of lut_long that the decoder keeps in shared memory
+constexpr int CO3_LONG_CACHE = 512;
+
 struct Co3CodeBook {
     uint8_t* cand_len;   // [R][NCAND][256] code lengths per weight-floor candidate (build scratch)
     int32_t* cand_max;   // [R][NCAND]      longest codeword per candidate (build scratch)
@@ -50,6 +53,10 @@ struct Co3CodeBook {
     uint32_t* enc;       // [R][256]        bit-reversed codeword | length << 16, by internal symbol
     uint32_t* code_msb;  // [R][256]        canonical codeword, root bit most significant, by public symbol
     uint32_t* lut;       // [R][2048]       (signed magnitude << 8) | length, 0 = longer than 11 bits
+    uint32_t* lut_long;  // [R][long_stride] the same for the codewords of 12..16 bits, indexed by
+                         //                 (16 stream bits, root bit on top) - (first[12] << 4)
+    int long_stride;     //                 16 * alphabet size (more 16-bit windows cannot lie under long
+                         //                 codewords), at least CO3_LONG_CACHE
     uint32_t* first;     // [R][17]         first canonical code of each length
     uint32_t* count;     // [R][17]
     uint32_t* offs;      // [R][17]         start of each length in perm
