@@ -57,6 +57,13 @@ extern "C" {
 
 #define CO3_BIAS_CURRENT 0 /* b_t from the moments of g_t + gamma m_{t-1} itself: one extra read pass */
 #define CO3_BIAS_LAGGED 1  /* that pass at t = 0 only; b_t (t >= 1) from the fit of iteration t-1      */
+/* Not in the paper's Algorithm 1, which fits "at each time t": bias AND code model of iteration
+ * t >= 1 come from the fit of iteration t-1, so the whole header of an iteration is known before its
+ * gradient is seen and conversion and packing are one pass over the data (the symbols never go to
+ * memory).  Symbols, residuals and averages are exactly those of CO3_BIAS_LAGGED; only the code
+ * differs (by one iteration), at a rate that is higher by the drift of the model per iteration.
+ * co3_debug_symbols is not available in this mode. */
+#define CO3_CODE_LAGGED 2
 
 typedef struct co3_plan co3_plan; /* opaque, library-owned */
 
@@ -83,7 +90,7 @@ typedef struct {
     int32_t n_segments;         /* S >= 1                                                          */
     const int64_t* seg_offsets; /* host, S+1 non-decreasing entries, [0] = 0, [S] = d; NULL: S = 1 */
     float gamma;                /* memory decay of Algorithm 1 line 8; 0: no feedback, 1: plain EF */
-    int32_t bias_mode;          /* CO3_BIAS_CURRENT or CO3_BIAS_LAGGED                             */
+    int32_t bias_mode;          /* CO3_BIAS_CURRENT, CO3_BIAS_LAGGED or CO3_CODE_LAGGED            */
     int64_t cap_words;          /* row pitch of `bitstream` in 32-bit words, multiple of 4         */
 } co3_config;
 
@@ -144,9 +151,12 @@ int co3_get_fit(co3_plan* plan, int32_t seg, double* beta, double* alpha, double
                 double* S2);
 
 /* Checkpoint/resume of what the method carries between iterations besides the caller's
- * residual: the iteration counter and the next bias per segment (host int32 [n_segments]). */
+ * residual: the iteration counter and the next bias per segment (host int32 [n_segments]).
+ * With CO3_CODE_LAGGED the next header is carried too: co3_state_header copies it out of
+ * (import == 0) or into (import != 0) the plan, host [n_segments]. */
 int co3_state_export(co3_plan* plan, int64_t* iteration, int32_t* next_bias);
 int co3_state_import(co3_plan* plan, int64_t iteration, const int32_t* next_bias);
+int co3_state_header(co3_plan* plan, int32_t import, co3_seg_header* next_header);
 
 /* Tracing: per-kernel device time measured with CUDA events recorded on the caller's stream
  * around the launches of the selected kernel classes.  co3_profile_enable creates the events

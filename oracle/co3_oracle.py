@@ -14,6 +14,8 @@ _lib = None
 
 MODE_CURRENT = 0   # bias b_t from the moments of a_t itself (a stats pass every iteration)
 MODE_LAGGED = 1    # stats pass at t = 0 only; b_t (t >= 1) from the fit of iteration t-1
+MODE_LAGGED_CODE = 2  # as MODE_LAGGED, and the code model of iteration t (t >= 1) is the fit of iteration
+                      # t-1 as well: the whole header of iteration t is known before g_t is seen
 
 OK, EINVAL, ECAPACITY, ECORRUPT = 0, -1, -4, -5
 
@@ -244,6 +246,7 @@ class OracleCO3:
         self.mode = mode
         self.t = 0
         self.bias_next = np.zeros(self.S, np.int32)
+        self.hdr_next = np.zeros((self.S, 3), np.int32)   # MODE_LAGGED_CODE: header of the coming iteration
         # worst case: 16 bits per symbol, every chunk padded to 128 bits
         worst = sum(4 * ((16 * int(e - s) + 127) // 128)
                     for s, e in zip(self.part.chunk_start[:self.part.n_chunks],
@@ -273,9 +276,15 @@ class OracleCO3:
             N, S1, S2, nf = convert(g, m, sym, int(off[l]), int(off[l + 1]), self.gamma, E, M,
                                     int(bias_t[l]), hist[l])
             be, al = fit(N, S1, S2)
-            ib, ir = header(be, al, int(bias_t[l]))
-            hdr[l] = (bias_t[l], ib, ir)
             self.bias_next[l] = bias(be, al, E, M)
+            if self.mode == MODE_LAGGED_CODE and self.t > 0:
+                hdr[l] = self.hdr_next[l]              # fixed by iteration t-1 (its bias is bias_t[l])
+            else:
+                ib, ir = header(be, al, int(bias_t[l]))
+                hdr[l] = (bias_t[l], ib, ir)
+            # the header the coming iteration would use: this fit, relative to the coming bias
+            ibn, irn = header(be, al, int(self.bias_next[l]))
+            self.hdr_next[l] = (self.bias_next[l], ibn, irn)
             r.fit[l] = (be, al)
             r.moments[l] = (N, S1, S2)
             r.nonfinite += nf

@@ -14,14 +14,14 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libco3.so")
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ECORRUPT, ENONFINITE = 0, -1, -2, -3, -4, -5, -6
 FLAG_CAPACITY, FLAG_CORRUPT, FLAG_NONFINITE = 1, 2, 4
-BIAS_CURRENT, BIAS_LAGGED = 0, 1
+BIAS_CURRENT, BIAS_LAGGED, CODE_LAGGED = 0, 1, 2
 
 EXPORTS = [
     "co3_plan_create", "co3_plan_destroy", "co3_sizes", "co3_encode", "co3_decode_aggregate",
     "co3_iteration_host", "co3_status", "co3_get_fit", "co3_state_export", "co3_state_import",
     "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
-    "co3_moments_static",
+    "co3_moments_static", "co3_state_header",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -98,6 +98,8 @@ def lib():
     L.co3_launch_count.argtypes = [vp]
     L.co3_moments_static.restype = C.c_int
     L.co3_moments_static.argtypes = [vp, vp, C.c_int64, C.c_float, vp, vp]
+    L.co3_state_header.restype = C.c_int
+    L.co3_state_header.argtypes = [vp, C.c_int32, vp]
     L.co3_strerror.restype = C.c_char_p
     L.co3_strerror.argtypes = [C.c_int]
     _lib = L
@@ -152,6 +154,7 @@ class Plan:
         self.d, self.U, self.E, self.M = int(d), int(n_users), int(exp_bits), int(mant_bits)
         self.ld = int(ld) if ld is not None else (self.d + 3) // 4 * 4
         self.nsym = 1 << (1 + self.E + self.M)
+        self.bias_mode = int(bias_mode)
         off = np.ascontiguousarray([0, d] if seg_offsets is None else seg_offsets, np.int64)
         self.S = len(off) - 1
         self._off = off
@@ -250,6 +253,24 @@ class Plan:
         rc = lib().co3_state_import(self.handle, int(iteration), nb.ctypes.data)
         if rc != OK:
             raise Co3Error(rc, "co3_state_import")
+
+    def state_header(self, next_header=None):
+        """CODE_LAGGED only: the header of the coming iteration, as an [S][3] int32 array
+        (bias, ibeta, ir).  With an argument it is imported instead."""
+        raw = np.zeros(self.S, np.int32)
+        if next_header is not None:
+            h = np.ascontiguousarray(next_header, np.int32)
+            raw = ((h[:, 0] & 0xFF) | ((h[:, 1] & 0xFF) << 8) | ((h[:, 2] & 0xFFFF) << 16)).astype(np.uint32).view(np.int32)
+            raw = np.ascontiguousarray(raw)
+        rc = lib().co3_state_header(self.handle, 0 if next_header is None else 1, raw.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_state_header")
+        v = raw.view(np.uint32)
+        out = np.zeros((self.S, 3), np.int32)
+        out[:, 0] = (v & 0xFF).astype(np.uint8).view(np.int8)
+        out[:, 1] = ((v >> 8) & 0xFF).astype(np.uint8).view(np.int8)
+        out[:, 2] = ((v >> 16) & 0xFFFF).astype(np.uint16).view(np.int16)
+        return out
 
     def profile_enable(self, kernel_names=None, max_records=4096):
         """Trace the named kernel classes (all if None; [] switches tracing off)."""

@@ -126,7 +126,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
     if (!co3_host_fmt_ok(cfg->fmt)) return CO3_EINVAL;
     if (cfg->d < 1 || cfg->ld < cfg->d || (cfg->ld & 3) || cfg->n_users < 1) return CO3_EINVAL;
     if (cfg->cap_words < 4 || (cfg->cap_words & 3) || cfg->cap_words > 0xFFFFFFFFLL) return CO3_EINVAL;
-    if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED) return CO3_EINVAL;
+    if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED && cfg->bias_mode != CO3_CODE_LAGGED) return CO3_EINVAL;
     if (!(cfg->gamma >= 0.0f) || !(cfg->gamma <= 1.0f)) return CO3_EINVAL;
     if (cfg->d > ((int64_t)1 << 31)) return CO3_EINVAL;
     if (((cfg->d + 4095) / 4096 + (cfg->seg_offsets ? cfg->n_segments : 1)) * (int64_t)cfg->n_users > 0x7FFFFFFFLL) return CO3_EINVAL;
@@ -217,7 +217,10 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &d_seg_chunk0, (size_t)S + 1);
         a |= dev_alloc(pl, &d_wtab, (size_t)CO3_NIBETA * CO3_NIR * J);
         a |= dev_alloc(pl, &d_logr, 2 * ((size_t)CO3_FIT_GRID + 1));
-        a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
+        const bool code_lagged = cfg->bias_mode == CO3_CODE_LAGGED;   // no stored symbols, staging slots instead
+        if (!code_lagged) a |= dev_alloc(pl, &dv.sym, (size_t)dv.U * (size_t)dv.sld);
+        else a |= dev_alloc(pl, &dv.slot_buf, items * (size_t)CO3_SLOT_WORDS);
+        a |= dev_alloc(pl, &dv.hdr_cur, (size_t)S);
         // Blocks add their shared-memory histograms to global memory with atomics; one counter takes
         // ~1e8 atomics/s, which a large layer converted at full HBM rate exceeds, so the blocks are
         // spread over several copies of the histogram (summed at read-out).
@@ -230,7 +233,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
         a |= dev_alloc(pl, &dv.chunk_words, items);
         a |= dev_alloc(pl, &dv.chunk_bits, items);
-        a |= dev_alloc(pl, &dv.gran_bits, items * 64);
+        if (!code_lagged) a |= dev_alloc(pl, &dv.gran_bits, items * 64);
         a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);
@@ -253,7 +256,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             if (e == cudaSuccess) e = cudaMemset(dv.fit, 0, sizeof(double) * (size_t)S * 5);
             if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * ((size_t)dv.hist_copies * S * CO3_MAXSYM + 1));
             dv.ticket = reinterpret_cast<unsigned int*>(dv.hist + (size_t)dv.hist_copies * S * CO3_MAXSYM);
-            if (e == cudaSuccess) e = cudaMemset(dv.sym, 0, (size_t)dv.U * (size_t)dv.sld);
+            if (e == cudaSuccess && dv.sym) e = cudaMemset(dv.sym, 0, (size_t)dv.U * (size_t)dv.sld);
+            if (e == cudaSuccess) e = cudaMemset(dv.hdr_cur, 0, sizeof(co3_seg_header) * (size_t)S);
             if (e == cudaSuccess && !g_kernels_ready) {
                 e = co3_setup_kernels();
                 if (e == cudaSuccess) e = co3_setup_decode_kernels();
@@ -293,6 +297,20 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
     if (((uintptr_t)grad | (uintptr_t)residual | (uintptr_t)bitstream) & 15) return CO3_EINVAL;
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
+    if (pl->cfg.bias_mode == CO3_CODE_LAGGED) {
+        // The header of this iteration was fixed by the previous one (at t = 0: by a statistics pass),
+        // so conversion and packing are one pass; the fit that follows prepares the next iteration.
+        if (pl->iteration == 0) {
+            CO3_TRY(co3_launch_stats(pl, grad, residual, st));
+            CO3_TRY(co3_launch_fit(pl, 2, pl->dev.hdr_cur, st));
+        }
+        CO3_TRY(cudaMemcpyAsync(hdr, pl->dev.hdr_cur, sizeof(co3_seg_header) * (size_t)pl->dev.S, cudaMemcpyDeviceToDevice, st));
+        CO3_TRY(co3_launch_convert_pack(pl, grad, residual, sub_bits, st));
+        CO3_TRY(co3_launch_scan_gather(pl, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
+        CO3_TRY(co3_launch_fit(pl, 3, pl->dev.hdr_cur, st));
+        pl->iteration++;
+        return CO3_OK;
+    }
     if (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) {
         CO3_TRY(co3_launch_stats(pl, grad, residual, st));
         CO3_TRY(co3_launch_fit(pl, 0, hdr, st));
@@ -379,8 +397,25 @@ extern "C" int co3_state_import(co3_plan* pl, int64_t iteration, const int32_t* 
     return CO3_OK;
 }
 
+extern "C" int co3_state_header(co3_plan* pl, int32_t import, co3_seg_header* next_header) {
+    if (!pl || !next_header) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    const size_t bytes = sizeof(co3_seg_header) * (size_t)pl->dev.S;
+    if (import) {
+        for (int l = 0; l < pl->dev.S; ++l) {
+            bool bad = false;
+            (void)co3_row_of(next_header[l], &bad);
+            if (bad || next_header[l].bias < pl->dev.b_lo || next_header[l].bias > pl->dev.b_hi) return CO3_EINVAL;
+        }
+        CO3_TRY(cudaMemcpy(pl->dev.hdr_cur, next_header, bytes, cudaMemcpyHostToDevice));
+    } else {
+        CO3_TRY(cudaMemcpy(next_header, pl->dev.hdr_cur, bytes, cudaMemcpyDeviceToHost));
+    }
+    return CO3_OK;
+}
+
 extern "C" int co3_debug_symbols(co3_plan* pl, uint8_t* symbols, void* cuda_stream) {
-    if (!pl || !symbols) return CO3_EINVAL;
+    if (!pl || !symbols || !pl->dev.sym) return CO3_EINVAL;    // the fully lagged code keeps no symbols
     cudaStream_t st = as_stream(cuda_stream);
     CO3_TRY(co3_launch_symbol_export(pl, symbols, st));
     CO3_TRY(cudaStreamSynchronize(st));

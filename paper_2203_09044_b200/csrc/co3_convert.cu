@@ -20,6 +20,15 @@
 // a 4-stage shared-memory ring that runs across item boundaries, so three steps (24 KB per block)
 // are always in flight without holding registers, and no barrier is needed: a thread only ever
 // reads the slots it filled itself, after cp.async.wait_group.
+//
+// Third variant (fully lagged code, where the header of the iteration is known beforehand):
+// the pass also looks every symbol's codeword up and packs it, so the symbols never go to memory.
+// A warp's step covers exactly one sub-chunk (128 consecutive elements, four per lane): the lane
+// merges its four codewords into one piece, a warp scan places the pieces inside the sub-chunk,
+// the pieces are ORed into the warp's own shared-memory slot, and the slot's words go straight to
+// the sub-chunk's place in a staging buffer (64 words per sub-chunk) together with the sub-chunk's
+// bit count.  No block barrier is involved.  Where a sub-chunk lands in the user's payload depends
+// on all earlier ones, so a scan and a concatenation pass follow (co3_encode.cu).
 #include "co3_internal.h"
 
 namespace {
@@ -93,13 +102,36 @@ struct ItemCtx {                  // what a step needs to know about its item
     float* mp;
     uint8_t* sp;
     int lo, hi, seg;              // the item's elements within the tile; its segment
+    int user;
+    int sub0;                     // index of the chunk's first sub-chunk in the user's sub_bits row
     bool whole;                   // the item covers its whole tile: no edge handling
 };
 
-template <int M, bool CONVERT>
+constexpr int SLOT_W = CO3_SUB_WORDS + 2;             // words of a sub-chunk slot (+2: a piece may spill over)
+
+struct PackSmem {                                     // only the packing variant has this
+    uint32_t enc[2][CO3_MAXSYM];                      // codeword | length << 16 of this / the next item's segment
+    uint32_t slot[CO3_THREADS / 32][SLOT_W];          // one sub-chunk being packed per warp
+};
+
+// OR a piece of at most 64 bits into a zero-initialised shared bit image at bit position pos.
+__device__ __forceinline__ void or_piece(uint32_t* img, uint32_t pos, unsigned long long v) {
+    const uint32_t wi = pos >> 5, sh = pos & 31u;
+    const uint32_t lo = (uint32_t)v, hi = (uint32_t)(v >> 32);
+    const uint32_t w0 = lo << sh;
+    const uint32_t w1 = __funnelshift_l(lo, hi, sh);  // sh in [0, 31]
+    const uint32_t w2 = sh ? (hi >> (32u - sh)) : 0u;
+    if (w0) atomicOr(&img[wi], w0);
+    if (w1) atomicOr(&img[wi + 1], w1);
+    if (w2) atomicOr(&img[wi + 2], w2);
+}
+
+// MODE 0: statistics only.  MODE 1: convert, symbols to memory.  MODE 2: convert and pack.
+template <int M, int MODE>
 __global__ void __launch_bounds__(CO3_THREADS, 4)
-ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
-    extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS]
+ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t* __restrict__ sub_bits) {
+    constexpr bool CONVERT = MODE >= 1, PACK = MODE == 2;
+    extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS] (+ PackSmem)
     __shared__ uint32_t s_hist[2][CONVERT ? CO3_THREADS / 32 : 1][CO3_MAXSYM];   // [item parity][warp][symbol]
     __shared__ double s_red[2][2][CO3_THREADS / 32];
     __shared__ uint32_t s_rednf[2][CO3_THREADS / 32];
@@ -121,6 +153,9 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
     }
     if (CONVERT)
         for (int i = tid; i < 2 * (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0][0])[i] = 0;
+    PackSmem& pk = *reinterpret_cast<PackSmem*>(s_ring + STAGES * 2 * CO3_THREADS);
+    if (PACK)
+        for (int i = tid; i < (CO3_THREADS / 32) * SLOT_W; i += CO3_THREADS) (&pk.slot[0][0])[i] = 0;
     __syncthreads();
     uint32_t item = s_ticket[0], nitem = s_ticket[1];
     if (item >= n_items) return;
@@ -136,6 +171,8 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
         x.lo = (int)(cd.start - tb);
         x.hi = x.lo + cd.len;
         x.seg = cd.seg;
+        x.user = (int)uu;
+        x.sub0 = cd.sub0;
         x.whole = cd.len == CO3_TILE;
         return x;
     };
@@ -162,6 +199,16 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
     ItemCtx nxt = cur;
     if (has_nxt) nxt = make_ctx(nitem, p.chunks[nitem % n_chunks]);
 
+    // the code table of an item's segment is fetched while the previous item is converted
+    auto enc_entry = [&](int seg) {
+        bool bad = false;
+        const int row = co3_row_of(p.hdr_cur[seg], &bad);
+        return p.cb.enc[(size_t)row * CO3_MAXSYM + tid];
+    };
+    if (PACK) {
+        pk.enc[0][tid] = enc_entry(cur.seg);
+        __syncthreads();
+    }
     int cur_seg = -1, par = 0, hpar = 0;
     unsigned long long* hist_copy = p.hist + (size_t)(blockIdx.x % (unsigned)p.hist_copies) * p.S * CO3_MAXSYM;
     QParams q;
@@ -180,6 +227,16 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             q.low_bits = __float_as_uint(pow2f(lambda + M));
             q.e0 = (uint32_t)(lambda + 150);
         }
+        uint32_t enc_next = 0;                        // PACK: my entry of the next item's code table
+        if (PACK && has_nxt) enc_next = enc_entry(nxt.seg);
+        const uint32_t* enc_tab = pk.enc[par];
+        // PACK: this lane's word of the warp's slot, of the sub-chunk's staging slot (step 0), the
+        // lane-31 pointer into sub_bits, the chunk's sub-chunk range, the warp's share of its bits
+        uint32_t* slot_l = pk.slot[warp] + lane;
+        uint32_t* pk_stage = PACK ? p.slot_buf + ((size_t)item * (CO3_TILE / CO3_SUB) + warp) * CO3_SUB_WORDS + lane : nullptr;
+        const int pk_sub_first = cur.lo / CO3_SUB, pk_sub_last = (cur.hi - 1) / CO3_SUB;
+        uint16_t* pk_sb = PACK ? sub_bits + (size_t)cur.user * p.n_sub + cur.sub0 + (warp - pk_sub_first) : nullptr;
+        uint32_t chunk_bits_w = 0;
         double s1 = 0.0, s2 = 0.0;
         uint32_t nf = 0;
 #pragma unroll
@@ -193,44 +250,89 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             const uint32_t slot = r * SLOT_BYTES;
             const int e0 = 4 * tid + VSTRIDE * r;
             const bool full = cur.whole || ((e0 >= cur.lo) && (e0 + 4 <= cur.hi));
-            if (!full && !(e0 < cur.hi && e0 + 4 > cur.lo)) continue;
-            float4 gv = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_ring + tid) + slot);
-            float4 mv = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_ring + CO3_THREADS + tid) + slot);
-            float a[4], mo[4];
-            uint32_t so[4];
-            if (full) {
-                ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
-                if (CONVERT) {
+            const bool some = full || (e0 < cur.hi && e0 + 4 > cur.lo);
+            unsigned long long piece = 0;             // PACK: this lane's four codewords, merged
+            uint32_t plen = 0;
+            if (some) {
+                float4 gv = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_ring + tid) + slot);
+                float4 mv = *reinterpret_cast<const float4*>(reinterpret_cast<const char*>(s_ring + CO3_THREADS + tid) + slot);
+                float a[4], mo[4];
+                uint32_t so[4], en[4] = {0u, 0u, 0u, 0u};
+                if (full) {
+                    ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
+                    if (CONVERT) {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        quantize<M>(a[e], q, so[e], mo[e]);
-                        atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
-                    }
-                    *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
-                    *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
-                }
-            } else {                                  // a vector on the chunk's edge: element by element
-                const bool in0 = e0 >= cur.lo && e0 < cur.hi, in1 = e0 + 1 >= cur.lo && e0 + 1 < cur.hi;
-                const bool in2 = e0 + 2 >= cur.lo && e0 + 2 < cur.hi, in3 = e0 + 3 >= cur.lo && e0 + 3 < cur.hi;
-                const bool in[4] = {in0, in1, in2, in3};
-                if (!in0) { gv.x = 0.0f; mv.x = 0.0f; }   // elements of the neighbouring chunk count as 0
-                if (!in1) { gv.y = 0.0f; mv.y = 0.0f; }
-                if (!in2) { gv.z = 0.0f; mv.z = 0.0f; }
-                if (!in3) { gv.w = 0.0f; mv.w = 0.0f; }
-                ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
-                if (CONVERT) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (in[e]) {
+                        for (int e = 0; e < 4; ++e) {
                             quantize<M>(a[e], q, so[e], mo[e]);
                             atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
-                            cur.mp[VSTRIDE * r + e] = mo[e];
-                            cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
+                            if (PACK) en[e] = enc_tab[so[e]];
+                        }
+                        *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+                        if (!PACK)
+                            *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
+                    }
+                } else {                              // a vector on the chunk's edge: element by element
+                    const bool in0 = e0 >= cur.lo && e0 < cur.hi, in1 = e0 + 1 >= cur.lo && e0 + 1 < cur.hi;
+                    const bool in2 = e0 + 2 >= cur.lo && e0 + 2 < cur.hi, in3 = e0 + 3 >= cur.lo && e0 + 3 < cur.hi;
+                    const bool in[4] = {in0, in1, in2, in3};
+                    if (!in0) { gv.x = 0.0f; mv.x = 0.0f; }   // elements of the neighbouring chunk count as 0
+                    if (!in1) { gv.y = 0.0f; mv.y = 0.0f; }
+                    if (!in2) { gv.z = 0.0f; mv.z = 0.0f; }
+                    if (!in3) { gv.w = 0.0f; mv.w = 0.0f; }
+                    ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
+                    if (CONVERT) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (in[e]) {
+                                quantize<M>(a[e], q, so[e], mo[e]);
+                                atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
+                                cur.mp[VSTRIDE * r + e] = mo[e];
+                                if (PACK) en[e] = enc_tab[so[e]];
+                                else cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
+                            }
                         }
                     }
                 }
+                if (PACK) {                           // an element outside the chunk has entry 0: no bits
+                    const uint32_t l0 = en[0] >> 16, l2 = en[2] >> 16;
+                    const uint32_t c01 = (en[0] & 0xFFFFu) | ((en[1] & 0xFFFFu) << l0);
+                    const uint32_t c23 = (en[2] & 0xFFFFu) | ((en[3] & 0xFFFFu) << l2);
+                    const uint32_t l01 = l0 + (en[1] >> 16);
+                    piece = (unsigned long long)c01 | ((unsigned long long)c23 << l01);
+                    plen = l01 + l2 + (en[3] >> 16);
+                }
+            }
+            if (PACK) {
+                // this warp's step is sub-chunk 8 r + warp: place the lane's piece after those of the
+                // lanes below, OR it into the warp's slot, then move the slot's words to the staging
+                // buffer (and leave the slot zero for the next step)
+                uint32_t x = plen;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+                    if (lane >= o) x += y;
+                }
+                constexpr int SC_STEP = CO3_THREADS / 32;           // sub-chunk of this step: SC_STEP * r + warp
+                if (plen) or_piece(pk.slot[warp], x - plen, piece);
+                const uint32_t total = __shfl_sync(0xffffffffu, x, 31);
+                chunk_bits_w += total;
+                __syncwarp();
+                if (32u * lane < total) {
+                    pk_stage[SC_STEP * r * CO3_SUB_WORDS] = *slot_l;
+                    *slot_l = 0;
+                }
+                if (total > 1024u) {                                // rare: above 8 bits per symbol
+                    if (32u * (lane + 32) < total) {
+                        pk_stage[SC_STEP * r * CO3_SUB_WORDS + 32] = slot_l[32];
+                        slot_l[32] = 0;
+                    }
+                }
+                if (lane == 31 && SC_STEP * r + warp >= pk_sub_first && SC_STEP * r + warp <= pk_sub_last)
+                    pk_sb[SC_STEP * r] = (uint16_t)total;
+                __syncwarp();
             }
         }
+        if (PACK && lane == 31) atomicAdd(&p.chunk_bits[item], chunk_bits_w);   // cleared before the launch
         // this item's moments, reduced in a fixed order (lanes, then warps) and stored per item:
         // the fit does not depend on which block converted which item
 #pragma unroll
@@ -244,7 +346,8 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m) {
             s_ticket[par] = claim;
             if (claim < n_items) s_chunk[par] = claim_cd;
         }
-        __syncthreads();                              // the item's only barrier: sums, histogram, claim
+        if (PACK) pk.enc[par ^ 1][tid] = enc_next;
+        __syncthreads();                              // sums, histogram, claim (and the next code table)
         if (tid == 0) {
             double t1 = 0.0, t2 = 0.0;
             uint32_t tn = 0;
@@ -285,27 +388,27 @@ __global__ void symbol_export_kernel(Co3Dev p, uint8_t* __restrict__ out) {
     }
 }
 
-typedef void (*ef_fn)(Co3Dev, const float*, float*);
+typedef void (*ef_fn)(Co3Dev, const float*, float*, uint16_t*);
 constexpr size_t RING_BYTES = (size_t)STAGES * 2 * CO3_THREADS * sizeof(float4);
 
-template <bool CONVERT>
+template <int MODE>
 ef_fn pick_kernel(int M) {
     switch (M) {
-        case 1: return ef_kernel<1, CONVERT>;
-        case 2: return ef_kernel<2, CONVERT>;
-        case 3: return ef_kernel<3, CONVERT>;
-        case 4: return ef_kernel<4, CONVERT>;
-        case 5: return ef_kernel<5, CONVERT>;
-        default: return ef_kernel<6, CONVERT>;
+        case 1: return ef_kernel<1, MODE>;
+        case 2: return ef_kernel<2, MODE>;
+        case 3: return ef_kernel<3, MODE>;
+        case 4: return ef_kernel<4, MODE>;
+        case 5: return ef_kernel<5, MODE>;
+        default: return ef_kernel<6, MODE>;
     }
 }
 
-int ef_grid(const co3_plan* pl, ef_fn fn) {
+int ef_grid(const co3_plan* pl, ef_fn fn, size_t smem) {
     int n = 0;
     // static + dynamic shared memory exceed the 48 KiB default, so the kernel has to opt in
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RING_BYTES) != cudaSuccess)
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         (void)cudaGetLastError();
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, CO3_THREADS, RING_BYTES);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, CO3_THREADS, smem);
     if (n < 1) n = 1;
     const int64_t items = pl->dev.n_chunks * (int64_t)pl->dev.U;
     const int64_t grid = (int64_t)pl->num_sms * n;
@@ -320,12 +423,12 @@ cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_
 }
 
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st) {
-    ef_fn fn = pick_kernel<false>(pl->dev.M);
-    if (!pl->grid_stats) pl->grid_stats = ef_grid(pl, fn);
+    ef_fn fn = pick_kernel<0>(pl->dev.M);
+    if (!pl->grid_stats) pl->grid_stats = ef_grid(pl, fn, RING_BYTES);
     cudaError_t e = cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_STATS, st);
-    fn<<<pl->grid_stats, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, const_cast<float*>(m));
+    fn<<<pl->grid_stats, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, const_cast<float*>(m), nullptr);
     co3_prof_end(pl, CO3_K_STATS, st, 1);
     return cudaGetLastError();
 }
@@ -334,10 +437,25 @@ cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStrea
     // one memset clears the histogram and the item ticket that follows it in the same allocation
     cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st);
     if (e != cudaSuccess) return e;
-    ef_fn fn = pick_kernel<true>(pl->dev.M);
-    if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn);
+    ef_fn fn = pick_kernel<1>(pl->dev.M);
+    if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn, RING_BYTES);
     co3_prof_begin(pl, CO3_K_CONVERT, st);
-    fn<<<pl->grid_convert, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, m);
+    fn<<<pl->grid_convert, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, m, nullptr);
+    co3_prof_end(pl, CO3_K_CONVERT, st, 1);
+    return cudaGetLastError();
+}
+
+// Fully lagged code: convert and pack in one pass (chunk images go to the plan's staging slots).
+cudaError_t co3_launch_convert_pack(co3_plan* pl, const float* g, float* m, uint16_t* sub_bits, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(pl->dev.chunk_bits, 0, sizeof(uint32_t) * (size_t)pl->dev.n_chunks * pl->dev.U, st);
+    if (e != cudaSuccess) return e;
+    constexpr size_t smem = RING_BYTES + sizeof(PackSmem);
+    ef_fn fn = pick_kernel<2>(pl->dev.M);
+    if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn, smem);
+    co3_prof_begin(pl, CO3_K_CONVERT, st);
+    fn<<<pl->grid_convert, CO3_THREADS, smem, st>>>(pl->dev, g, m, sub_bits);
     co3_prof_end(pl, CO3_K_CONVERT, st, 1);
     return cudaGetLastError();
 }

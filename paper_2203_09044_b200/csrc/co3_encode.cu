@@ -102,22 +102,35 @@ enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __res
 }
 
 // chunk_off[u][c] = exclusive prefix of the chunk word counts of user u; one block per user.
+// FROM_SUB: the chunk word counts are not there yet (fully lagged code: the convert-and-pack pass
+// added up only the code bits of each chunk); derive them here and store them for the concatenation.
+template <bool FROM_SUB>
 __global__ void __launch_bounds__(1024)
 enc_scan_kernel(Co3Dev p, uint32_t* __restrict__ chunk_off, unsigned long long* __restrict__ user_bits) {
     __shared__ uint32_t s_warp[32];
     __shared__ uint32_t s_carry;
     __shared__ unsigned long long s_bits[32];
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t* in = p.chunk_words + (size_t)u * p.n_chunks;
-    const uint32_t* inb = p.chunk_bits + (size_t)u * p.n_chunks;
+    uint32_t* in = p.chunk_words + (size_t)u * p.n_chunks;
+    uint32_t* inb = p.chunk_bits + (size_t)u * p.n_chunks;
     uint32_t* out = chunk_off + (size_t)u * (p.n_chunks + 1);
     unsigned long long my_bits = 0;                   // r_t^(u): code bits of this user
     if (tid == 0) s_carry = 0;
     __syncthreads();
     for (int64_t base = 0; base < p.n_chunks; base += 1024) {
         const int64_t i = base + tid;
-        const uint32_t v = (i < p.n_chunks) ? in[i] : 0u;
-        my_bits += (i < p.n_chunks) ? inb[i] : 0u;
+        uint32_t v = 0u;
+        if (i < p.n_chunks) {
+            if (FROM_SUB) {                            // the pass left the chunk's code bits only
+                const uint32_t bits = inb[i];
+                v = 4u * ((bits + 127u) / 128u);
+                in[i] = v;
+                my_bits += bits;
+            } else {
+                v = in[i];
+                my_bits += inb[i];
+            }
+        }
         uint32_t x = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -242,9 +255,88 @@ enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t
     if (bad && tid == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
 
+// Fully lagged code: the convert-and-pack pass left every sub-chunk packed from bit 0 of its own
+// staging slot.  One block per chunk shifts the sub-chunks to their places in a shared image of the
+// chunk (a scan of their bit counts) and stores the image at the chunk's place in the payload.
+constexpr int CAT_THREADS = 256;
+__global__ void __launch_bounds__(CAT_THREADS)
+enc_concat_kernel(Co3Dev p, const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
+                  uint32_t* __restrict__ bitstream) {
+    __shared__ __align__(16) uint32_t s_img[BUF_WORDS + 4];
+    __shared__ uint32_t s_pos[CO3_TILE / CO3_SUB], s_nb[CO3_TILE / CO3_SUB];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t item = blockIdx.x;
+    const uint32_t n_chunks = (uint32_t)p.n_chunks;
+    const uint32_t u = item / n_chunks, c = item - u * n_chunks;
+    // every load that does not depend on another one is issued here, before any is used
+    const uint32_t* stage = p.slot_buf + (size_t)item * CO3_SLOT_WORDS;
+    constexpr int PER_WARP = (CO3_TILE / CO3_SUB) / (CAT_THREADS / 32);     // sub-chunks per warp (4)
+    uint32_t v[PER_WARP];
+#pragma unroll
+    for (int k = 0; k < PER_WARP; ++k)                // first 32 words of each slot (what 8 bits per symbol fill)
+        v[k] = __ldg(stage + (warp + (CAT_THREADS / 32) * k) * CO3_SUB_WORDS + lane);
+    const uint32_t ovf = p.user_ovf[u];
+    const uint32_t nwords = p.chunk_words[item];
+    const uint32_t dst_word = chunk_off[(size_t)u * (p.n_chunks + 1) + c];
+    const Co3Chunk cd = p.chunks[c];
+    if (ovf) return;                                  // this user's payload does not fit: row left untouched
+    const int tlo = (int)(cd.start & (CO3_TILE - 1));
+    const int sub_first = tlo / CO3_SUB, sub_last = (tlo + cd.len - 1) / CO3_SUB;
+    if (warp == 0) {                                  // lane = sub-chunk of the tile
+        const bool in = lane >= sub_first && lane <= sub_last;
+        const uint32_t nb = in ? sub_bits[(size_t)u * p.n_sub + cd.sub0 + (lane - sub_first)] : 0u;
+        uint32_t x = nb;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        s_pos[lane] = x - nb;
+        s_nb[lane] = nb;
+    }
+    for (uint32_t i = tid; i < nwords / 4 + 1; i += CAT_THREADS) reinterpret_cast<uint4*>(s_img)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < PER_WARP; ++k) {
+        const int sc = warp + (CAT_THREADS / 32) * k;
+        const uint32_t pos = s_pos[sc], nb = s_nb[sc];
+        if (32u * lane < nb) {
+            const uint32_t at = pos + 32u * lane, wi = at >> 5, sh = at & 31u;
+            atomicOr(&s_img[wi], v[k] << sh);
+            if (sh) atomicOr(&s_img[wi + 1], v[k] >> (32u - sh));
+        }
+        const uint32_t i = lane + 32;                 // second half: only above 8 bits per symbol
+        if (32u * i < nb) {
+            const uint32_t w = stage[sc * CO3_SUB_WORDS + i];
+            const uint32_t at = pos + 32u * i, wi = at >> 5, sh = at & 31u;
+            atomicOr(&s_img[wi], w << sh);
+            if (sh) atomicOr(&s_img[wi + 1], w >> (32u - sh));
+        }
+    }
+    __syncthreads();
+    uint4* dst = reinterpret_cast<uint4*>(bitstream + (size_t)u * p.cap_words + dst_word);
+    const uint4* srcv = reinterpret_cast<const uint4*>(s_img);
+    for (uint32_t i = tid; i < nwords / 4; i += CAT_THREADS) dst[i] = srcv[i];
+}
+
 }  // namespace
 
 cudaError_t co3_setup_kernels(void) { return cudaSuccess; }
+
+cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint16_t* sub_bits, uint32_t* chunk_off,
+                                   unsigned long long* user_bits, cudaStream_t st) {
+    const Co3Dev& p = pl->dev;
+    const unsigned items = (unsigned)(p.n_chunks * (int64_t)p.U);
+    cudaError_t e;
+    co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
+    enc_scan_kernel<true><<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
+    co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    co3_prof_begin(pl, CO3_K_ENC_PACK, st);
+    enc_concat_kernel<<<items, CAT_THREADS, 0, st>>>(p, sub_bits, chunk_off, bitstream);
+    co3_prof_end(pl, CO3_K_ENC_PACK, st, 1);
+    return cudaGetLastError();
+}
 
 cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
                               uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
@@ -257,7 +349,7 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
     co3_prof_end(pl, CO3_K_ENC_LEN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
-    enc_scan_kernel<<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
+    enc_scan_kernel<false><<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
     co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_ENC_PACK, st);

@@ -27,6 +27,10 @@ __device__ __forceinline__ double poly_bias(double b) {
 // mode 0: after the stats pass -- write the bias for the coming convert pass.
 // mode 1: after the convert pass -- write the header (bias used, ibeta, ir), keep the fit, and
 //         store the bias the rule gives for these moments as the next iteration's bias.
+// Fully lagged code (the whole header of an iteration is fixed before its gradient is seen):
+// mode 2: after the stats pass of t = 0 -- bias and header of the coming pass from these moments.
+// mode 3: after the fused convert-and-pack pass -- the same for the next iteration; keep the fit.
+//         In both, `hdr` is the plan's own header array.
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr) {
     __shared__ double s_a[FIT_THREADS], s_b[FIT_THREADS];
     __shared__ unsigned long long s_n[FIT_THREADS];
@@ -129,7 +133,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         p.bias_cur[seg] = b_rule;
         return;
     }
-    const int b_used = p.bias_cur[seg];
+    const int b_used = (mode == 1) ? p.bias_cur[seg] : b_rule;   // the bias this header goes with
     double x = floor(8.0 * (s_state == 0 ? t : log2(beta)) + 0.5);
     x = x < (double)CO3_IBETA_MIN ? (double)CO3_IBETA_MIN : (x > (double)CO3_IBETA_MAX ? (double)CO3_IBETA_MAX : x);
     double y = (double)CO3_IR_MIN;
@@ -140,9 +144,10 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     co3_seg_header h;
     h.bias = (int8_t)b_used; h.ibeta = (int8_t)(int)x; h.ir = (int16_t)(int)y;
     hdr[seg] = h;
+    p.bias_cur[seg] = b_rule;
+    if (mode == 2) return;
     double* f = p.fit + 5 * (size_t)seg;
     f[0] = beta; f[1] = alpha; f[2] = N; f[3] = S1; f[4] = S2;
-    p.bias_cur[seg] = b_rule;
     if (nf) {
         atomicAdd(p.nonfinite_total, nf);
         atomicOr(p.flags, CO3_FLAG_NONFINITE);

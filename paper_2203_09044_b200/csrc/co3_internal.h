@@ -19,6 +19,8 @@ constexpr int CO3_FIT_GRID = 8192;  // log R(beta) is tabulated at FIT_GRID + 1 
 constexpr int CO3_MAXSYM = 256;     // alphabet rows are padded to 256 entries
 constexpr int CO3_STAGE_WORDS = 1024;  // shared-memory staging per (chunk, user) stream in decode
 constexpr int CO3_THREADS = 256;
+constexpr int CO3_SUB_WORDS = CO3_SUB * CO3_MAXLEN / 32;     // payload words of a sub-chunk at 16 bits per symbol (64)
+constexpr int CO3_SLOT_WORDS = CO3_TILE * CO3_MAXLEN / 32;   // ... of a chunk (2048)
 
 // One chunk of the static partition: elements [start, start+len) of every user's row, all in
 // segment `seg`, inside one 4096-aligned tile.  sub0 = index of its first sub-chunk.
@@ -84,6 +86,9 @@ struct Co3Dev {
     uint32_t* part_nf;            //              ... count of non-finite a
     double* fit;                  // [S][5] beta, alpha, N, S1, S2
     int32_t* bias_cur;            // [S] bias used by the next convert pass
+    co3_seg_header* hdr_cur;      // [S] fully lagged code: header of the coming iteration (else unused)
+    uint32_t* slot_buf;           // [U*n_chunks][32][CO3_SUB_WORDS] fully lagged code: the packed sub-chunks,
+                                  //     each from bit 0 of its own slot, before their offsets are known (else null)
     const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
     const double* logr_tab;       // [2][FIT_GRID + 1] log R(beta), log G(beta) at log2(beta) uniform in [log2 0.3, 1]
     Co3CodeBook cb;               // code tables of all model rows
@@ -142,6 +147,9 @@ const double* co3_host_logr_table(void);               // [2][FIT_GRID + 1], cac
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st);
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st);
+cudaError_t co3_launch_convert_pack(co3_plan* pl, const float* g, float* m, uint16_t* sub_bits, cudaStream_t st);
+cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint16_t* sub_bits, uint32_t* chunk_off,
+                                   unsigned long long* user_bits, cudaStream_t st);
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
 cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st);
 cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,

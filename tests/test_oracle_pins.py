@@ -518,3 +518,39 @@ def test_modes_and_state_across_iterations(oracle):
             assert r.bias[l] == oracle.bias(*oracle.fit(N, S1, S2), E, M)
             assert (N, S1, S2) == tuple(r.moments[l])
     assert any(res[0][t][0].bias[0] != res[1][t][0].bias[0] for t in range(1, 4))   # drift shows
+
+
+def test_fully_lagged_code_mode(oracle):
+    """LAGGED_CODE: symbols, residuals and biases are those of LAGGED (the conversion does not depend
+    on the code); the header of iteration t >= 1 is built from the fit of iteration t-1 relative to
+    the bias of iteration t, so it is known before the gradient of iteration t; the stream still
+    decodes to the same symbols, at a rate at most slightly above the per-iteration code."""
+    d, U, E, M = 9000, 2, 4, 3
+    runs = {}
+    for mode in (oracle.MODE_LAGGED, oracle.MODE_LAGGED_CODE):
+        o = oracle.OracleCO3(d, U, E, M, [0, 4000, d], gamma=0.9, mode=mode)
+        m = np.zeros((U, d), np.float32)
+        rng = np.random.default_rng(5)
+        out = []
+        for t in range(4):
+            g = (rng.laplace(0, 1e-3 * 1.3 ** t, (U, d))).astype(np.float32)
+            r = o.encode(g, m)
+            rc, avg, sym = o.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr, want_symbols=True)
+            assert rc == oracle.OK and np.array_equal(sym, r.sym)
+            out.append((r, avg, m.copy()))
+        runs[mode] = out
+    lag, full = runs[oracle.MODE_LAGGED], runs[oracle.MODE_LAGGED_CODE]
+    for t in range(4):
+        assert np.array_equal(lag[t][0].sym, full[t][0].sym)
+        assert np.array_equal(lag[t][0].bias, full[t][0].bias)
+        assert np.array_equal(lag[t][2], full[t][2])                          # residuals
+        assert np.array_equal(lag[t][1].view(np.uint32), full[t][1].view(np.uint32))   # averages
+    assert np.array_equal(lag[0][0].hdr, full[0][0].hdr)                      # t = 0: same header
+    for t in range(1, 4):
+        prev = full[t - 1][0]
+        for l in range(2):
+            b = int(full[t][0].bias[l])
+            ib, ir = oracle.header(prev.fit[l, 0], prev.fit[l, 1], b)
+            assert tuple(full[t][0].hdr[l]) == (b, ib, ir)
+        bits_full, bits_lag = int(full[t][0].user_bits.sum()), int(lag[t][0].user_bits.sum())
+        assert bits_lag <= bits_full * 1.0 + 0.02 * bits_lag and bits_full <= 1.02 * bits_lag
