@@ -258,7 +258,7 @@ enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t
 // Fully lagged code: the convert-and-pack pass left every sub-chunk packed from bit 0 of its own
 // staging slot.  One block per chunk shifts the sub-chunks to their places in a shared image of the
 // chunk (a scan of their bit counts) and stores the image at the chunk's place in the payload.
-constexpr int CAT_THREADS = 256;
+constexpr int CAT_THREADS = 64;
 __global__ void __launch_bounds__(CAT_THREADS)
 enc_concat_kernel(Co3Dev p, const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
                   uint32_t* __restrict__ bitstream) {
