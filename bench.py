@@ -33,7 +33,7 @@ CONVERT_BYTES_PER_ELEMENT = 13.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel on the full 8-user
 # workload (mean of three launches of the one-pass ncu capture summarised in
 # profiles/dram_traffic_config1_8users.md); it grows in proportion with the number of users
-CONVERT_DRAM_TRAFFIC_BYTES_8_USERS = 1111.2e6
+CONVERT_DRAM_TRAFFIC_BYTES_8_USERS = 1109.7e6
 
 
 def measured_peaks():
@@ -121,8 +121,10 @@ def run_ours(args):
 
     wl = inputs.workload(1, n_users=args.users).align_rows()
     U, d = wl.n_users, wl.d
+    mode = {"lagged": binding.BIAS_LAGGED, "current": binding.BIAS_CURRENT,
+            "code-lagged": binding.CODE_LAGGED}[args.mode]
     plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
-                        bias_mode=binding.BIAS_LAGGED, ld=wl.ld)
+                        bias_mode=mode, ld=wl.ld)
     out = plan.alloc_outputs()
     residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
     # every rank draws its own users' gradients (seed offset by rank): a weak-scaling replica
@@ -207,17 +209,23 @@ def run_ours(args):
     e2e_value = world * in_bytes * ne / (e2e_ms * 1e-3) / 1e9
     peak, peak_src = measured_peaks()
     conv_avg_ms = conv_ms / max(conv_n, 1)
-    achieved = CONVERT_BYTES_PER_ELEMENT * U * d / (conv_avg_ms * 1e-3) / 1e9
-    step_bytes = (15.9 * U + 4.0) * d                 # all passes of one LAGGED iteration, E4M3
+    # bytes the dominant kernel must move per user-element: g, m in, m out, and the symbol (two-pass
+    # modes) or the packed codewords (single-pass mode) out
+    conv_bytes = CONVERT_BYTES_PER_ELEMENT if args.mode != "code-lagged" else 12.0 + code_bits / 8.0
+    achieved = conv_bytes * U * d / (conv_avg_ms * 1e-3) / 1e9
+    # all passes of one iteration, E4M3: 13 + 1.9 (encode) + 0.87 (decode) per user-element + the average
+    step_bytes = ((15.9 if args.mode != "code-lagged" else 12.0 + 4.0 * code_bits / 8.0) * U + 4.0) * d
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "configs[1]: %d users x ResNet-18 (10-class head) gradient, d=11173962, "
-                               "62 layers, iid GenNorm(beta=0.8) per layer, E4M3, gamma=0.9, lagged bias" % U,
+                               "62 layers, iid GenNorm(beta=0.8) per layer, E4M3, gamma=0.9, %s" % (
+                                   U, {"lagged": "lagged bias", "current": "bias from the current moments",
+                                       "code-lagged": "lagged bias and code (single-pass encode)"}[args.mode]),
                    "d": d, "n_users": U, "n_segments": plan.S, "format": "E4M3", "gamma": wl.gamma,
-                   "bias_mode": "lagged", "replicas": world, "row_stride": plan.ld,
+                   "bias_mode": args.mode, "replicas": world, "row_stride": plan.ld,
                    "l2": "inputs larger than L2: %d MB of gradient+memory read per step, %d gradient "
                          "batches cycled" % (8 * U * d // 1000000, POOL)},
         "clocks": clocks,
@@ -225,11 +233,13 @@ def run_ours(args):
                 "d2h_bytes_per_step": int(4 * d), "steps": ne, "ms_per_step": e2e_ms / ne,
                 "call": "co3_iteration_host (pinned host gradients in, host average out)"},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "ef_kernel<convert> (fused EF-add/convert/residual/histogram/moments)",
+        "roofline": {"kernel": "ef_kernel<convert> (fused EF-add/convert/residual/histogram/moments)"
+                               if args.mode != "code-lagged" else
+                               "ef_kernel<convert+pack> (EF-add/convert/residual/histogram/moments/codeword packing)",
                      "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
-                     "traffic": CONVERT_DRAM_TRAFFIC_BYTES_8_USERS * U / 8.0,
-                     "algorithmic_bytes_per_launch": CONVERT_BYTES_PER_ELEMENT * U * d,
+                     "traffic": CONVERT_DRAM_TRAFFIC_BYTES_8_USERS * U / 8.0 if args.mode != "code-lagged" else None,
+                     "algorithmic_bytes_per_launch": conv_bytes * U * d,
                      "avg_launch_ms": conv_avg_ms, "launches_timed": conv_n,
                      "timing": "cudaEvent pair around each launch on the launching stream, inside the timed region"},
         "elements_per_s": world * U * d * args.steps / (elapsed_ms * 1e-3),
@@ -325,6 +335,8 @@ def main():
     ap.add_argument("--users", type=int, default=None,
                     help="override the number of simulated users (profiling a smaller case); default 8")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--mode", default="lagged", choices=["lagged", "current", "code-lagged"],
+                    help="bias/code mode of the plan (default: lagged bias, the benchmark configuration)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
