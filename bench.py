@@ -106,6 +106,32 @@ def physical_gpu_index(local_rank):
     return local_rank
 
 
+def max_over_ranks(ms, world, device):
+    """A job of independent replicas is as slow as its slowest one: the maximum over all ranks of a
+    device-timed interval (milliseconds).  `device` is where the exchanged scalar lives ("cuda" under
+    NCCL, "cpu" under gloo)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput_gbs(world, bytes_per_replica_step, steps, ms):
+    """Whole-job GB/s: every replica processes bytes_per_replica_step per step in the same time."""
+    return world * bytes_per_replica_step * steps / (ms * 1e-3) / 1e9
+
+
+def replica_workload(rank, n_users=None):
+    """Configuration 1 for replica `rank`: same shapes, its own users' gradients (seed offset)."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, n_users=n_users).align_rows()
+    wl.index = wl.index + 100 * rank
+    return wl
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -119,7 +145,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    wl = inputs.workload(1, n_users=args.users).align_rows()
+    wl = replica_workload(rank, args.users)            # a weak-scaling replica: its own users' gradients
     U, d = wl.n_users, wl.d
     mode = {"lagged": binding.BIAS_LAGGED, "current": binding.BIAS_CURRENT,
             "code-lagged": binding.CODE_LAGGED}[args.mode]
@@ -127,8 +153,6 @@ def run_ours(args):
                         bias_mode=mode, ld=wl.ld)
     out = plan.alloc_outputs()
     residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
-    # every rank draws its own users' gradients (seed offset by rank): a weak-scaling replica
-    wl.index = wl.index + 100 * rank
     pool = [wl.gradient(t, device="cuda") for t in range(POOL)]
     torch.cuda.synchronize()
 
@@ -169,10 +193,7 @@ def run_ours(args):
     container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
                       + 32.0 * U * (plan.n_chunks + 1) + 32.0 * plan.S) / (U * d)
 
-    if world > 1:
-        tmax = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, world, "cuda")
 
     # ---- per-kernel breakdown: the same steps again with every kernel class traced -----------
     nb = min(args.steps, 50)
@@ -197,16 +218,13 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        tmax = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
     flags, _ = plan.status(clear=True)
     assert flags == 0
 
     in_bytes = 4.0 * d * U
-    value = world * in_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9
-    e2e_value = world * in_bytes * ne / (e2e_ms * 1e-3) / 1e9
+    value = job_throughput_gbs(world, in_bytes, args.steps, elapsed_ms)
+    e2e_value = job_throughput_gbs(world, in_bytes, ne, e2e_ms)
     peak, peak_src = measured_peaks()
     conv_avg_ms = conv_ms / max(conv_n, 1)
     # bytes the dominant kernel must move per user-element: g, m in, m out, and the symbol (two-pass
