@@ -54,6 +54,7 @@ extern "C" {
 #define CO3_FLAG_CAPACITY 1u
 #define CO3_FLAG_CORRUPT 2u
 #define CO3_FLAG_NONFINITE 4u
+#define CO3_FLAG_TIMEOUT 8u  /* a bounded wait between thread blocks ran out (should never happen) */
 
 #define CO3_BIAS_CURRENT 0 /* b_t from the moments of g_t + gamma m_{t-1} itself: one extra read pass */
 #define CO3_BIAS_LAGGED 1  /* that pass at t = 0 only; b_t (t >= 1) from the fit of iteration t-1      */
@@ -115,8 +116,9 @@ int co3_sizes(const co3_plan* plan, int64_t* n_chunks, int64_t* n_sub, int64_t* 
  *   chunk_off device, out, [U][n_chunks+1] u32, in words
  *   user_bits device, out, [U] u64          r_t^(u): code bits of user u
  *   hdr       device, out, [n_segments]
- * If a user's payload would exceed cap_words, CO3_FLAG_CAPACITY is raised and that user's
- * bitstream row is left untouched; chunk_off, sub_bits and user_bits are still written.
+ * If a user's payload would exceed cap_words, CO3_FLAG_CAPACITY is raised; nothing is written at
+ * or beyond cap_words of a row, the chunks that would not fit are not written, and the row's
+ * content is then unspecified; chunk_off, sub_bits and user_bits are still written in full.
  * Non-finite g + gamma m: counted, coded as +0, memory reset to 0, CO3_FLAG_NONFINITE raised. */
 int co3_encode(co3_plan* plan, const float* grad, float* residual, uint32_t* bitstream,
                uint16_t* sub_bits, uint32_t* chunk_off, uint64_t* user_bits, co3_seg_header* hdr,
@@ -168,9 +170,9 @@ int co3_state_header(co3_plan* plan, int32_t import, co3_seg_header* next_header
 #define CO3_K_FIT 1          /* GenNorm fit, bias, header                                   */
 #define CO3_K_CONVERT 2      /* fused EF-add / convert / residual / histogram / moments      */
 #define CO3_K_CODE_ENC 3     /* (unused: codes are built once at plan creation)              */
-#define CO3_K_ENC_LEN 4      /* code lengths -> sub-chunk bits, chunk words                  */
-#define CO3_K_ENC_SCAN 5     /* chunk offsets                                                */
-#define CO3_K_ENC_PACK 6     /* bit packing                                                  */
+#define CO3_K_ENC_LEN 4      /* (unused: the lengths are taken inside the packing kernel)    */
+#define CO3_K_ENC_SCAN 5     /* chunk offsets (CO3_CODE_LAGGED only)                         */
+#define CO3_K_ENC_PACK 6     /* lengths + offsets + bit packing (CO3_CODE_LAGGED: concatenation) */
 #define CO3_K_CODE_DEC 7     /* (unused: codes are built once at plan creation)              */
 #define CO3_K_DECODE 8       /* decode + aggregate                                           */
 #define CO3_NUM_KERNELS 9

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libco3.so")
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ECORRUPT, ENONFINITE = 0, -1, -2, -3, -4, -5, -6
 FLAG_CAPACITY, FLAG_CORRUPT, FLAG_NONFINITE = 1, 2, 4
 BIAS_CURRENT, BIAS_LAGGED, CODE_LAGGED = 0, 1, 2
+FLAG_TIMEOUT = 8
 
 EXPORTS = [
     "co3_plan_create", "co3_plan_destroy", "co3_sizes", "co3_encode", "co3_decode_aggregate",

@@ -233,8 +233,18 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
         a |= dev_alloc(pl, &dv.chunk_words, items);
         a |= dev_alloc(pl, &dv.chunk_bits, items);
-        if (!code_lagged) a |= dev_alloc(pl, &dv.gran_bits, items * 64);
         a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
+        {   // one allocation: group totals (u64), published chunk counts (u32), ticket (u32)
+            dv.n_grp = (nc + 63) / 64;
+            const size_t grp_n = (size_t)dv.U * (size_t)dv.n_grp;
+            pl->enc_sync_bytes = (sizeof(unsigned long long) * grp_n + sizeof(uint32_t) * (items + 2) + 7) / 8 * 8;
+            dv.enc_sync_words64 = pl->enc_sync_bytes / 8;
+            unsigned char* raw = nullptr;
+            a |= dev_alloc(pl, &raw, pl->enc_sync_bytes);
+            dv.enc_grp = reinterpret_cast<unsigned long long*>(raw);
+            dv.enc_st = reinterpret_cast<uint32_t*>(raw + sizeof(unsigned long long) * grp_n);
+            dv.enc_ticket = dv.enc_st + items;
+        }
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);
         a |= alloc_codebook(pl, dv.cb);

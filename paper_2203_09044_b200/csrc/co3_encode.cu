@@ -1,20 +1,19 @@
 // h_Hf on the device (Algorithm 1 line 9): Huffman-code the converted symbols of every user
-// into the chunked container.  Three launches, no device-side waiting:
-//   1. enc_len_kernel  -- code length of every symbol -> bits per 64-symbol granule, per
-//                         sub-chunk and per chunk
-//   2. enc_scan_kernel -- exclusive scan of the chunk word counts per user -> chunk offsets,
-//                         user totals, capacity check before anything is written
-//   3. enc_pack_kernel -- per chunk: bit offsets from the granule counts, codewords merged into
-//                         a shared-memory image of the chunk, 128-bit coalesced stores
+// into the chunked container, in ONE launch (enc_single_kernel).
 // Work item = (user, chunk) = one block of 64 threads; a thread owns a granule of 64 consecutive
-// symbols (four 128-bit loads), two threads own a sub-chunk.  Small blocks keep the shared-memory
-// footprint at one plain 256-entry table plus (pack pass) the 8 KB chunk image, so that 20-32
-// blocks are resident per SM and hide each other's latencies; the per-item bookkeeping is
-// amortised over 64 symbols per thread.  In the pack kernel a thread merges 16 codewords at a
-// time pairwise in registers (16 -> 8 -> 4 pieces of at most 64 bits) and ORs the pieces into
-// the chunk image at its bit offset.
-// Bound: issue slots and shared-memory look-ups (one per symbol per pass; 32 lanes hit random
-// banks of the table); HBM traffic is small (1 B/element read per pass, ~0.87 B/element written).
+// symbols (four 128-bit loads), two threads own a sub-chunk.  The block first adds up the code
+// lengths (a 256-byte table), which gives every granule its bit offset inside the chunk and the
+// chunk its size; then it looks the codewords up, merges 16 at a time pairwise in registers
+// (16 -> 8 -> 4 pieces of at most 64 bits) and ORs the pieces into a shared-memory image of the
+// chunk; then it learns the chunk's offset in the user's payload from the sizes the earlier chunks
+// have published (see below) and stores the image with 128-bit accesses.  Small blocks keep the
+// shared-memory footprint at ~9.5 KB, so that ~21 blocks are resident per SM and hide each
+// other's latencies.
+// Bound: shared-memory look-ups (two per symbol; 32 lanes hit random banks of the tables) and issue
+// slots; HBM traffic is small (1 B/element read, ~0.87 B/element written).
+//
+// The fully lagged-code mode uses enc_scan_kernel and enc_concat_kernel instead (the symbols were
+// packed per sub-chunk by the convert pass).
 #include "co3_internal.h"
 
 namespace {
@@ -30,8 +29,7 @@ struct Item {                    // one (user, chunk) work item as a thread sees
     int a, b;                    // the ones in [a, b) belong to the chunk
 };
 
-__device__ __forceinline__ void open_item(Item& it, const Co3Dev& p, int tid) {
-    const uint32_t item = blockIdx.x;
+__device__ __forceinline__ void open_item(Item& it, const Co3Dev& p, int tid, uint32_t item) {
     const uint32_t n_chunks = (uint32_t)p.n_chunks;
     it.u = item / n_chunks;
     it.c = item - it.u * n_chunks;
@@ -56,55 +54,9 @@ __device__ __forceinline__ uint32_t round_mask(const Item& it, int k) {
     return ((1u << b) - 1u) & ~((1u << a) - 1u);
 }
 
-__global__ void __launch_bounds__(ENC_THREADS)
-enc_len_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits) {
-    __shared__ __align__(16) uint8_t s_len[CO3_MAXSYM];
-    __shared__ uint32_t s_warp[ENC_THREADS / 32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    bool bad = false;
-    Item it;
-    open_item(it, p, tid);
-    {
-        const uint32_t* src = reinterpret_cast<const uint32_t*>(
-            p.cb.len8 + (size_t)co3_row_of(hdr[it.cd.seg], &bad) * CO3_MAXSYM);
-        reinterpret_cast<uint32_t*>(s_len)[tid] = src[tid];          // 64 threads x 4 bytes
-    }
-    __syncthreads();
-    uint32_t bits = 0;
-    if (it.a == 0 && it.b == GRANULE) {
-#pragma unroll
-        for (int i = 0; i < GRANULE; ++i) bits += s_len[__byte_perm(it.w[i >> 2], 0, 0x4440 + (i & 3))];
-    } else {
-#pragma unroll
-        for (int i = 0; i < GRANULE; ++i)
-            bits += (i >= it.a && i < it.b) ? s_len[__byte_perm(it.w[i >> 2], 0, 0x4440 + (i & 3))] : 0u;
-    }
-    const uint32_t item = blockIdx.x;
-    p.gran_bits[(size_t)item * ENC_THREADS + tid] = (uint16_t)bits;
-    // two threads = one sub-chunk
-    const uint32_t sb = bits + __shfl_xor_sync(0xffffffffu, bits, 1);
-    const int tlo = (int)(it.cd.start & (CO3_TILE - 1));
-    const int sub_first = tlo / CO3_SUB, sub_last = (tlo + it.cd.len - 1) / CO3_SUB;
-    const int kk = tid >> 1;
-    if ((tid & 1) == 0 && kk >= sub_first && kk <= sub_last)
-        sub_bits[(size_t)it.u * p.n_sub + it.cd.sub0 + (kk - sub_first)] = (uint16_t)sb;
-    uint32_t wb = bits;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) wb += __shfl_xor_sync(0xffffffffu, wb, o);
-    if (lane == 0) s_warp[warp] = wb;
-    __syncthreads();
-    if (tid == 0) {
-        const uint32_t tot = s_warp[0] + s_warp[1];
-        p.chunk_words[item] = 4u * ((tot + 127u) / 128u);
-        p.chunk_bits[item] = tot;
-        if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
-    }
-}
-
 // chunk_off[u][c] = exclusive prefix of the chunk word counts of user u; one block per user.
-// FROM_SUB: the chunk word counts are not there yet (fully lagged code: the convert-and-pack pass
-// added up only the code bits of each chunk); derive them here and store them for the concatenation.
-template <bool FROM_SUB>
+// Used by the fully lagged code only: the convert-and-pack pass added up the code bits of each chunk;
+// the word counts are derived here and stored for the concatenation pass.
 __global__ void __launch_bounds__(1024)
 enc_scan_kernel(Co3Dev p, uint32_t* __restrict__ chunk_off, unsigned long long* __restrict__ user_bits) {
     __shared__ uint32_t s_warp[32];
@@ -121,15 +73,10 @@ enc_scan_kernel(Co3Dev p, uint32_t* __restrict__ chunk_off, unsigned long long* 
         const int64_t i = base + tid;
         uint32_t v = 0u;
         if (i < p.n_chunks) {
-            if (FROM_SUB) {                            // the pass left the chunk's code bits only
-                const uint32_t bits = inb[i];
-                v = 4u * ((bits + 127u) / 128u);
-                in[i] = v;
-                my_bits += bits;
-            } else {
-                v = in[i];
-                my_bits += inb[i];
-            }
+            const uint32_t bits = inb[i];
+            v = 4u * ((bits + 127u) / 128u);
+            in[i] = v;
+            my_bits += bits;
         }
         uint32_t x = v;
 #pragma unroll
@@ -184,29 +131,78 @@ __device__ __forceinline__ void put_piece(uint32_t* s_buf, uint32_t pos, unsigne
     if (w2) atomicOr(&s_buf[wi + 2], w2);
 }
 
+// ---- single pass: lengths, offsets and packing in one kernel ---------------------------------
+// One block per (user, chunk) as above, but the item is a ticket (so every item with a smaller
+// number has been claimed by a block that is running or done), and the chunk's word offset is
+// summed from what the earlier chunks of the same user PUBLISH: each block stores its own word
+// count (a self-validating word) and adds it to the totals of its group of 64 chunks (a 64-bit word:
+// arrivals << 56 | payload words << 32 | code bits).  A block needs only such counts, never another block's offset, so
+// there is no chain: after packing its chunk into shared memory (by then the earlier blocks have
+// long published) it adds up the totals of the complete groups before its own and the counts of
+// the earlier chunks of its own group.  Every wait is bounded; a wait that runs out raises
+// CO3_FLAG_TIMEOUT and the block writes nothing.
+constexpr uint32_t ST_VALID = 0x80000000u;
+constexpr int GRP_SHIFT = 6, GRP_SIZE = 1 << GRP_SHIFT;
+constexpr int SPIN_LIMIT = 1 << 22;
+
+__device__ __forceinline__ uint32_t wait_count(const uint32_t* st, bool& timeout) {
+    const volatile uint32_t* v = st;
+    for (int k = 0; k < SPIN_LIMIT; ++k) {
+        const uint32_t w = *v;
+        if (w & ST_VALID) return w & ~ST_VALID;
+    }
+    timeout = true;
+    return 0;
+}
+// waits until `expect` chunks have arrived in the group; returns words << 32 | bits
+__device__ __forceinline__ unsigned long long wait_group(const unsigned long long* grp, uint32_t expect, bool& timeout) {
+    const volatile unsigned long long* v = grp;
+    for (int k = 0; k < SPIN_LIMIT; ++k) {
+        const unsigned long long w = *v;
+        if ((w >> 56) == (unsigned long long)expect) return w & ((1ull << 56) - 1);
+    }
+    timeout = true;
+    return 0;
+}
+
 __global__ void __launch_bounds__(ENC_THREADS)
-enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t* __restrict__ chunk_off,
-                uint32_t* __restrict__ bitstream) {
+enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits,
+                  uint32_t* __restrict__ chunk_off, unsigned long long* __restrict__ user_bits,
+                  uint32_t* __restrict__ bitstream) {
+    __shared__ __align__(16) uint8_t s_len[CO3_MAXSYM];
     __shared__ __align__(16) uint32_t s_enc[CO3_MAXSYM];            // codeword | length << 16
     __shared__ __align__(16) uint32_t s_buf[BUF_WORDS + 4];         // image of the chunk
-    __shared__ uint32_t s_warp[ENC_THREADS / 32];
+    __shared__ uint32_t s_warp[ENC_THREADS / 32], s_sum[ENC_THREADS / 32];
+    __shared__ uint32_t s_item;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t item = blockIdx.x;
+    if (tid == 0) s_item = atomicAdd(p.enc_ticket, 1u);
+    __syncthreads();
+    const uint32_t item = s_item;
     bool bad = false;
     Item it;
-    open_item(it, p, tid);
-    if (p.user_ovf[it.u]) return;                     // block-uniform: this user's payload does not fit
-    const uint32_t nwords = p.chunk_words[item];
-    const uint32_t dst_word = chunk_off[(size_t)it.u * (p.n_chunks + 1) + it.c];
-    uint32_t bits = p.gran_bits[(size_t)item * ENC_THREADS + tid];
+    open_item(it, p, tid, item);
     {
-        const uint4* src = reinterpret_cast<const uint4*>(
-            p.cb.enc + (size_t)co3_row_of(hdr[it.cd.seg], &bad) * CO3_MAXSYM);
-        reinterpret_cast<uint4*>(s_enc)[tid] = __ldg(src + tid);     // 64 threads x 4 entries
-        uint4* z = reinterpret_cast<uint4*>(s_buf);
-        for (uint32_t i = tid; i < nwords / 4; i += ENC_THREADS) z[i] = make_uint4(0, 0, 0, 0);
+        const size_t row = (size_t)co3_row_of(hdr[it.cd.seg], &bad) * CO3_MAXSYM;
+        reinterpret_cast<uint32_t*>(s_len)[tid] = reinterpret_cast<const uint32_t*>(p.cb.len8 + row)[tid];
+        reinterpret_cast<uint4*>(s_enc)[tid] = __ldg(reinterpret_cast<const uint4*>(p.cb.enc + row) + tid);
     }
-    // exclusive scan of the granule bit counts over the block's two warps
+    __syncthreads();
+    // code bits of this thread's granule, of its sub-chunk (two threads), of the chunk
+    const bool whole = it.a == 0 && it.b == GRANULE;  // no symbol of this granule lies outside the chunk
+    uint32_t bits = 0;
+    if (whole) {
+#pragma unroll
+        for (int i = 0; i < GRANULE; ++i) bits += s_len[__byte_perm(it.w[i >> 2], 0, 0x4440 + (i & 3))];
+    } else {
+#pragma unroll
+        for (int i = 0; i < GRANULE; ++i)
+            bits += (i >= it.a && i < it.b) ? s_len[__byte_perm(it.w[i >> 2], 0, 0x4440 + (i & 3))] : 0u;
+    }
+    const uint32_t sb = bits + __shfl_xor_sync(0xffffffffu, bits, 1);
+    const int tlo = (int)(it.cd.start & (CO3_TILE - 1));
+    const int sub_first = tlo / CO3_SUB, sub_last = (tlo + it.cd.len - 1) / CO3_SUB;
+    if ((tid & 1) == 0 && (tid >> 1) >= sub_first && (tid >> 1) <= sub_last)
+        sub_bits[(size_t)it.u * p.n_sub + it.cd.sub0 + ((tid >> 1) - sub_first)] = (uint16_t)sb;
     uint32_t x = bits;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -214,9 +210,18 @@ enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t
         if (lane >= o) x += y;
     }
     if (lane == 31) s_warp[warp] = x;
-    __syncthreads();                                  // table, cleared image, warp totals
+    __syncthreads();
     uint32_t pos = x - bits + (warp ? s_warp[0] : 0u);
-    const bool whole = it.a == 0 && it.b == GRANULE;  // no symbol of this granule lies outside the chunk
+    const uint32_t tot = s_warp[0] + s_warp[1];
+    const uint32_t nwords = 4u * ((tot + 127u) / 128u);
+    const uint32_t grp = it.c >> GRP_SHIFT;
+    if (tid == 0) {                                   // publish this chunk's size
+        *reinterpret_cast<volatile uint32_t*>(p.enc_st + item) = ST_VALID | nwords;
+        atomicAdd(p.enc_grp + (size_t)it.u * p.n_grp + grp,
+                  (1ull << 56) | ((unsigned long long)nwords << 32) | (unsigned long long)tot);
+    }
+    for (uint32_t i = tid; i < nwords / 4 + 1; i += ENC_THREADS) reinterpret_cast<uint4*>(s_buf)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
 #pragma unroll
     for (int k = 0; k < GRANULE / 16; ++k) {
         const uint32_t mask = whole ? 0xFFFFu : round_mask(it, k);
@@ -248,11 +253,44 @@ enc_pack_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, const uint32_t
             pos += l1[2 * q] + l1[2 * q + 1];
         }
     }
-    __syncthreads();
+    // offset of the chunk = words of all earlier chunks of this user
+    bool timeout = false;
+    uint32_t sum = 0;
+    for (uint32_t i = tid; i < grp; i += ENC_THREADS)
+        sum += (uint32_t)(wait_group(p.enc_grp + (size_t)it.u * p.n_grp + i, GRP_SIZE, timeout) >> 32);
+    if ((uint32_t)tid < (it.c & (GRP_SIZE - 1)))
+        sum += wait_count(p.enc_st + (size_t)it.u * p.n_chunks + ((size_t)grp << GRP_SHIFT) + tid, timeout);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) s_sum[warp] = sum;
+    const int any_timeout = __syncthreads_or(timeout);                // also: the image is complete
+    const uint32_t dst_word = s_sum[0] + s_sum[1];
+    if (tid == 0) {
+        uint32_t* co = chunk_off + (size_t)it.u * (p.n_chunks + 1);
+        co[it.c] = dst_word;
+        if ((int64_t)it.c == p.n_chunks - 1) co[p.n_chunks] = dst_word + nwords;
+        if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
+        if (any_timeout) atomicOr(p.flags, CO3_FLAG_TIMEOUT);
+        if ((int64_t)dst_word + nwords > p.cap_words) atomicOr(p.flags, CO3_FLAG_CAPACITY);
+    }
+    if ((int64_t)it.c == p.n_chunks - 1 && warp == 0) {
+        // the user's last chunk: every chunk of the user has a smaller ticket, so all groups fill up;
+        // r_t^(u) = code bits of the user = sum of the groups' bit totals
+        bool t2 = false;
+        unsigned long long ub = 0;
+        for (uint32_t i = lane; i <= grp; i += 32) {
+            const uint32_t expect = (i < grp) ? (uint32_t)GRP_SIZE : (it.c & (GRP_SIZE - 1)) + 1u;
+            ub += wait_group(p.enc_grp + (size_t)it.u * p.n_grp + i, expect, t2) & 0xFFFFFFFFull;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ub += __shfl_xor_sync(0xffffffffu, ub, o);
+        if (lane == 0) user_bits[it.u] = ub;
+        if (t2 && lane == 0) atomicOr(p.flags, CO3_FLAG_TIMEOUT);
+    }
+    if (any_timeout || (int64_t)dst_word + nwords > p.cap_words) return;   // nothing is written outside the row
     uint4* dst = reinterpret_cast<uint4*>(bitstream + (size_t)it.u * p.cap_words + dst_word);
     const uint4* srcv = reinterpret_cast<const uint4*>(s_buf);
     for (uint32_t i = tid; i < nwords / 4; i += ENC_THREADS) dst[i] = srcv[i];
-    if (bad && tid == 0) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
 
 // Fully lagged code: the convert-and-pack pass left every sub-chunk packed from bit 0 of its own
@@ -329,7 +367,7 @@ cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint
     const unsigned items = (unsigned)(p.n_chunks * (int64_t)p.U);
     cudaError_t e;
     co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
-    enc_scan_kernel<true><<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
+    enc_scan_kernel<<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
     co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     co3_prof_begin(pl, CO3_K_ENC_PACK, st);
@@ -343,17 +381,9 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
                               cudaStream_t st) {
     const Co3Dev& p = pl->dev;
     const unsigned items = (unsigned)(p.n_chunks * (int64_t)p.U);
-    cudaError_t e;
-    co3_prof_begin(pl, CO3_K_ENC_LEN, st);
-    enc_len_kernel<<<items, ENC_THREADS, 0, st>>>(p, hdr, sub_bits);
-    co3_prof_end(pl, CO3_K_ENC_LEN, st, 1);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    co3_prof_begin(pl, CO3_K_ENC_SCAN, st);
-    enc_scan_kernel<false><<<p.U, 1024, 0, st>>>(p, chunk_off, user_bits);
-    co3_prof_end(pl, CO3_K_ENC_SCAN, st, 1);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    // (tickets, published counts and group totals were cleared by the fit kernel that ran before)
     co3_prof_begin(pl, CO3_K_ENC_PACK, st);
-    enc_pack_kernel<<<items, ENC_THREADS, 0, st>>>(p, hdr, chunk_off, bitstream);
+    enc_single_kernel<<<items, ENC_THREADS, 0, st>>>(p, hdr, sub_bits, chunk_off, user_bits, bitstream);
     co3_prof_end(pl, CO3_K_ENC_PACK, st, 1);
     return cudaGetLastError();
 }

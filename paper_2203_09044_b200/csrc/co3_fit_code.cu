@@ -39,6 +39,12 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     __shared__ int s_state, s_coarse, s_fine;
 
     const int seg = blockIdx.x, tid = threadIdx.x;
+    if (mode == 1) {
+        // side job: the single-pass encode that follows this launch wants its tickets, published
+        // counts and group totals at zero
+        unsigned long long* z = p.enc_grp;
+        for (size_t i = (size_t)blockIdx.x * FIT_THREADS + tid; i < p.enc_sync_words64; i += (size_t)gridDim.x * FIT_THREADS) z[i] = 0ull;
+    }
     const int c0 = p.seg_chunk0[seg], c1 = p.seg_chunk0[seg + 1];
     double a1 = 0.0, a2 = 0.0;
     unsigned long long an = 0;

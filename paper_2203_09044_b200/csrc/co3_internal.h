@@ -92,10 +92,14 @@ struct Co3Dev {
     const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
     const double* logr_tab;       // [2][FIT_GRID + 1] log R(beta), log G(beta) at log2(beta) uniform in [log2 0.3, 1]
     Co3CodeBook cb;               // code tables of all model rows
-    uint32_t* chunk_words;        // [U][n_chunks] payload words of each chunk (multiple of 4)
-    uint32_t* chunk_bits;         // [U][n_chunks] code bits of each chunk
-    uint16_t* gran_bits;          // [U][n_chunks][64] code bits of each 64-symbol granule
+    uint32_t* chunk_words;        // [U][n_chunks] payload words of each chunk (multiple of 4)   } fully lagged
+    uint32_t* chunk_bits;         // [U][n_chunks] code bits of each chunk                        } code only
     uint32_t* user_ovf;           // [U] 1 if the user's payload exceeds cap_words
+    unsigned long long* enc_grp;  // [U][n_grp] single-pass encode, per group of 64 chunks: arrivals << 56 | words << 32 | bits
+    uint32_t* enc_st;             // [U][n_chunks] ... published word count of each chunk (top bit: valid)
+    unsigned int* enc_ticket;     // ... item ticket (the three live in one allocation, cleared per launch)
+    int64_t n_grp;
+    size_t enc_sync_words64;      // size of that allocation in 64-bit words
     uint32_t* flags;              // sticky status flags
     unsigned long long* nonfinite_total;
 };
@@ -107,6 +111,7 @@ struct co3_plan {
     int64_t worst_case_words;
     int device;
     int num_sms;
+    size_t enc_sync_bytes;          // size of the enc_grp / enc_st / enc_ticket allocation
     int grid_stats, grid_convert;   // launch grids (fixed per plan: they define the reduction order)
     cudaStream_t last_stream;
     void* allocs[64];

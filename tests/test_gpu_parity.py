@@ -198,15 +198,26 @@ def test_nonfinite_inputs(binding, oracle):
     assert plan.status() == (0, 0)
 
 
-def test_capacity_overflow_is_flagged_and_nothing_written(binding, oracle):
+@pytest.mark.parametrize("mode", [1, 2])
+def test_capacity_overflow_is_flagged_and_stays_inside_the_row(binding, oracle, mode):
+    """A payload that does not fit: the flag is raised, offsets and lengths are still complete (they
+    are compared with the oracle's inside run_case), and nothing is written past a row's end -- the
+    row of the next user and a guard row behind the last one stay as they were."""
     d, U = 20_000, 2
     gen = torch.Generator().manual_seed(4)
     g = (torch.randn((U, d), generator=gen) * 1e-3).cuda()
-    plan, orc, out, res = run_case(binding, oracle, d, U, 4, 3, None, [g], cap=1024)
+    plan, orc, out, res = run_case(binding, oracle, d, U, 4, 3, None, [g], cap=1024, mode=mode)
     r, flags = res[0]
     assert r.status == oracle.ECAPACITY and flags & binding.FLAG_CAPACITY
-    assert not out["bitstream"].any().item()
     assert int(out["chunk_off"][0, -1]) > 1024
+    # again with a sentinel in the second user's row and a guard row: only user 0's row may change
+    plan2 = binding.Plan(d, U, 4, 3, None, bias_mode=mode, cap_words=1024)
+    out2 = plan2.alloc_outputs()
+    big = torch.full((U + 1, 1024), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    out2["bitstream"] = big[:U]
+    plan2.encode(g, torch.zeros_like(g), out2)
+    assert plan2.status()[0] & binding.FLAG_CAPACITY
+    assert (big[U] == 0x5A5A5A5A).all().item()
 
 
 def test_corrupt_streams_are_flagged_not_faulting(binding, oracle):
