@@ -134,6 +134,14 @@ int co3_decode_aggregate(co3_plan* plan, const uint32_t* bitstream, const uint16
                          const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
                          void* cuda_stream);
 
+/* The same with the model update of Algorithm 1 line 14 fused in: besides avg_grad,
+ * weights[i] <- fl32(weights[i] + fl32(step * avg_grad[i])) (device, in/out, [d] fp32; two roundings,
+ * no fused multiply-add).  The paper writes the update with both signs (Sec. II, Algorithm 1), so
+ * the caller passes the signed step: -eta for descent. */
+int co3_decode_aggregate_update(co3_plan* plan, const uint32_t* bitstream, const uint16_t* sub_bits,
+                                const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
+                                float* weights, float step, void* cuda_stream);
+
 /* One whole iteration from host memory (what a training loop that keeps gradients on the host
  * would call): copies h_grad (host, [U][ld], pinned for full speed) to d_grad, runs co3_encode
  * and co3_decode_aggregate with the given device buffers, and copies the average back to h_avg

@@ -311,6 +311,14 @@ class OracleCO3:
         self.t += 1
         return r
 
+    def decode_aggregate_update(self, payload, sub_bits, chunk_off, hdr, weights, step):
+        """Algorithm 1 lines 13-14 with the model update: w <- fl32(w + fl32(step * avg)), in place.
+        The caller passes the signed step (the paper writes the update with both signs)."""
+        rc, avg, _ = self.decode_aggregate(payload, sub_bits, chunk_off, hdr)
+        if rc == OK:
+            weights += (np.float32(step) * avg).astype(np.float32)
+        return rc, avg
+
     def decode_aggregate(self, payload, sub_bits, chunk_off, hdr, want_symbols=False):
         return decode_aggregate(payload, sub_bits, chunk_off, self.part, hdr, self.E, self.M,
                                 want_symbols)

@@ -22,7 +22,7 @@ EXPORTS = [
     "co3_iteration_host", "co3_status", "co3_get_fit", "co3_state_export", "co3_state_import",
     "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
-    "co3_moments_static", "co3_state_header",
+    "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -71,6 +71,8 @@ def lib():
     L.co3_encode.argtypes = [vp] * 9
     L.co3_decode_aggregate.restype = C.c_int
     L.co3_decode_aggregate.argtypes = [vp] * 7
+    L.co3_decode_aggregate_update.restype = C.c_int
+    L.co3_decode_aggregate_update.argtypes = [vp] * 7 + [C.c_float, vp]
     L.co3_iteration_host.restype = C.c_int
     L.co3_iteration_host.argtypes = [vp] * 12
     L.co3_status.restype = C.c_int
@@ -217,6 +219,16 @@ class Plan:
                                         self._stream(stream))
         if rc != OK:
             raise Co3Error(rc, "co3_decode_aggregate")
+        return avg
+
+    def decode_aggregate_update(self, out, weights, step, avg=None, stream=None):
+        """decode_aggregate with w <- w + step * avg fused in (weights: [d] fp32 cuda tensor, in place)."""
+        avg = out["avg"] if avg is None else avg
+        rc = lib().co3_decode_aggregate_update(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
+                                               _ptr(out["chunk_off"]), _ptr(out["hdr"]), _ptr(avg),
+                                               _ptr(weights), C.c_float(float(step)), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_decode_aggregate_update")
         return avg
 
     def iteration_host(self, h_grad, d_grad, residual, out, h_avg, stream=None):

@@ -339,7 +339,18 @@ extern "C" int co3_decode_aggregate(co3_plan* pl, const uint32_t* bitstream, con
     if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
-    CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, st));
+    CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, nullptr, 0.0f, st));
+    return CO3_OK;
+}
+
+extern "C" int co3_decode_aggregate_update(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+                                           const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
+                                           float* weights, float step, void* cuda_stream) {
+    if (!pl || !bitstream || !sub_bits || !chunk_off || !hdr || !avg_grad || !weights) return CO3_EINVAL;
+    if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, weights, step, st));
     return CO3_OK;
 }
 

@@ -278,6 +278,12 @@ __device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co
     __syncwarp();
 }
 
+// Algorithm 1 line 14, optional: w <- w + step * avg (two roundings; the caller chooses the sign).
+__device__ __forceinline__ void put_out(float* avg, float* weights, float step, int64_t i, float v) {
+    avg[i] = v;
+    if (weights) weights[i] = __fadd_rn(weights[i], __fmul_rn(step, v));
+}
+
 __device__ __forceinline__ float finish(int32_t ksum, float scale, float fu, float inv_u) {
     const float v = __fmul_rn((float)ksum, scale);                  // exact
     return inv_u != 0.0f ? __fmul_rn(v, inv_u) : __fdiv_rn(v, fu);  // U a power of two: exact either way
@@ -303,7 +309,8 @@ __host__ __device__ inline size_t smem_a_bytes(int U) {
 __global__ void __launch_bounds__(CO3_THREADS)
 decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                       const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
-                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg) {
+                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
+                      float* __restrict__ weights, float step) {
     extern __shared__ __align__(16) unsigned char s_raw[];
     SmemA& sm = *reinterpret_cast<SmemA*>(s_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -375,18 +382,18 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                 const int lo = sm.c_lo[gp][cc], hi = sm.c_hi[gp][cc];
                 // the accumulator holds sum((K << 8) | length): the lengths of <= 8 users stay below 256
                 int32_t* a = acc0 + qoff + cc * ACC_Q + lane * PADW + warp;
-                float* o = avg + sm.c_tb[gp][cc] + e0;
+                const int64_t o = sm.c_tb[gp][cc] + e0;
                 if (lo == 0 && hi == CO3_TILE) {
 #pragma unroll
                     for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
-                        o[rr * NW * CO3_SUB] = finish(a[rr * NW] >> 8, scale, fu, inv_u);
+                        put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
                         a[rr * NW] = 0;
                     }
                 } else {
 #pragma unroll
                     for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
                         const int e = e0 + rr * NW * CO3_SUB;
-                        if (e >= lo && e < hi) o[rr * NW * CO3_SUB] = finish(a[rr * NW] >> 8, scale, fu, inv_u);
+                        if (e >= lo && e < hi) put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
                         a[rr * NW] = 0;
                     }
                 }
@@ -411,7 +418,8 @@ struct SmemB {
 __global__ void __launch_bounds__(CO3_THREADS)
 decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                       const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
-                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg) {
+                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
+                      float* __restrict__ weights, float step) {
     extern __shared__ __align__(16) unsigned char s_raw[];
     SmemB& sm = *reinterpret_cast<SmemB*>(s_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -461,7 +469,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
         for (int rr = 0; rr < CO3_TILE / CO3_THREADS; ++rr) {
             const int e = tid + rr * CO3_THREADS;
             const int kk = e >> 7, il = e & (CO3_SUB - 1);
-            if (e >= lo && e < hi) avg[tb + e] = finish(sm.acc[il * PADW + kk], scale, fu, inv_u);
+            if (e >= lo && e < hi) put_out(avg, weights, step, tb + e, finish(sm.acc[il * PADW + kk], scale, fu, inv_u));
         }
         __syncthreads();
     }
@@ -482,7 +490,7 @@ cudaError_t co3_setup_decode_kernels(void) {
 
 cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
-                              cudaStream_t st) {
+                              float* weights, float step, cudaStream_t st) {
     const Co3Dev& p = pl->dev;
     co3_prof_begin(pl, CO3_K_DECODE, st);
     if (p.U <= NW) {
@@ -492,7 +500,7 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
         if (bpsm < 1) bpsm = 1;
         const int64_t grid = (int64_t)pl->num_sms * bpsm;
         decode_small_u_kernel<<<(int)(p.n_groups < grid ? p.n_groups : grid), CO3_THREADS, smem, st>>>(
-            p, bitstream, sub_bits, chunk_off, hdr, avg);
+            p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     } else {
         if (!g_bpsm_b) {
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_bpsm_b, decode_large_u_kernel, CO3_THREADS, sizeof(SmemB));
@@ -500,7 +508,7 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
         }
         const int64_t grid = (int64_t)pl->num_sms * g_bpsm_b;
         decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), CO3_THREADS, sizeof(SmemB), st>>>(
-            p, bitstream, sub_bits, chunk_off, hdr, avg);
+            p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     }
     co3_prof_end(pl, CO3_K_DECODE, st, 1);
     return cudaGetLastError();

@@ -162,7 +162,7 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
                               cudaStream_t st);
 cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
-                              cudaStream_t st);
+                              float* weights, float step, cudaStream_t st);
 cudaError_t co3_setup_kernels(void);
 cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_t st);
 

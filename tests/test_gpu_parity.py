@@ -251,6 +251,33 @@ def test_corrupt_streams_are_flagged_not_faulting(binding, oracle):
                                                      res[0][0].chunk_off, res[0][0].hdr)[1]))
 
 
+@pytest.mark.parametrize("U,E,M", [(3, 4, 3), (12, 3, 2)])
+def test_decode_with_fused_model_update(binding, oracle, U, E, M):
+    """Algorithm 1 line 14 fused into the decode: w <- fl32(w + fl32(step * avg)), bit for bit, over
+    several iterations of a weight vector (both decode kernels: U <= 8 and U > 8)."""
+    d, off = 50_001, [0, 4097, 30_000, 50_001]
+    gen = torch.Generator().manual_seed(31)
+    plan = binding.Plan(d, U, E, M, off)
+    orc = oracle.OracleCO3(d, U, E, M, off, cap_words=plan.cap_words)
+    out = plan.alloc_outputs()
+    m_gpu = torch.zeros((U, plan.ld), device="cuda")
+    m_cpu = np.zeros((U, plan.ld), np.float32)
+    w_cpu = torch.randn(d, generator=gen).numpy()
+    w_gpu = torch.from_numpy(w_cpu.copy()).cuda()
+    step = -0.01
+    for t in range(3):
+        g = torch.zeros((U, plan.ld))
+        g[:, :d] = torch.randn((U, d), generator=gen) * 1e-2
+        plan.encode(g.cuda(), m_gpu, out)
+        r = orc.encode(g.numpy(), m_cpu)
+        avg = plan.decode_aggregate_update(out, w_gpu, step).cpu().numpy()
+        rc, avg_o = orc.decode_aggregate_update(r.payload, r.sub_bits, r.chunk_off, r.hdr, w_cpu, step)
+        assert rc == oracle.OK
+        assert np.array_equal(_bits(avg), _bits(avg_o)), f"t={t} average"
+        assert np.array_equal(_bits(w_gpu.cpu().numpy()), _bits(w_cpu)), f"t={t} weights"
+    assert plan.status()[0] == 0
+
+
 def test_decoder_depends_only_on_the_stream(binding, oracle):
     """A second plan that never encoded anything (the parameter server) decodes the outputs."""
     from paper_2203_09044_b200 import inputs

@@ -554,3 +554,25 @@ def test_fully_lagged_code_mode(oracle):
             assert tuple(full[t][0].hdr[l]) == (b, ib, ir)
         bits_full, bits_lag = int(full[t][0].user_bits.sum()), int(lag[t][0].user_bits.sum())
         assert bits_lag <= bits_full * 1.0 + 0.02 * bits_lag and bits_full <= 1.02 * bits_lag
+
+
+def test_fused_model_update_is_the_plain_update(oracle):
+    """decode_aggregate_update = decode_aggregate followed by w + step * avg in fp32 (two roundings),
+    checked against exact rational arithmetic rounded twice."""
+    from fractions import Fraction
+    d, U, E, M = 3000, 2, 4, 3
+    rng = np.random.default_rng(9)
+    o = oracle.OracleCO3(d, U, E, M)
+    g = rng.laplace(0, 1e-3, (U, d)).astype(np.float32)
+    m = np.zeros((U, d), np.float32)
+    r = o.encode(g, m)
+    w = rng.standard_normal(d).astype(np.float32)
+    w0 = w.copy()
+    step = np.float32(-0.05)
+    rc, avg = o.decode_aggregate_update(r.payload, r.sub_bits, r.chunk_off, r.hdr, w, step)
+    rc2, avg2, _ = o.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+    assert rc == oracle.OK and np.array_equal(avg.view(np.uint32), avg2.view(np.uint32))
+    for i in range(0, d, 37):
+        prod = np.float32(float(Fraction(float(step)) * Fraction(float(avg[i]))))     # exact product, rounded once
+        want = np.float32(float(Fraction(float(w0[i])) + Fraction(float(prod))))      # exact sum, rounded once
+        assert w[i] == want
