@@ -32,8 +32,8 @@ __device__ __forceinline__ double poly_bias(double b) {
 // mode 3: after the fused convert-and-pack pass -- the same for the next iteration; keep the fit.
 //         In both, `hdr` is the plan's own header array.
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr) {
-    __shared__ double s_a[FIT_THREADS], s_b[FIT_THREADS];
-    __shared__ unsigned long long s_n[FIT_THREADS];
+    __shared__ double s_a[FIT_THREADS / 32], s_b[FIT_THREADS / 32];
+    __shared__ unsigned long long s_n[FIT_THREADS / 32];
     __shared__ double s_lg[3];
     __shared__ double s_target, s_t;        // log rho; log2(beta)
     __shared__ int s_state, s_coarse, s_fine;
@@ -46,25 +46,31 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         for (size_t i = (size_t)blockIdx.x * FIT_THREADS + tid; i < p.enc_sync_words64; i += (size_t)gridDim.x * FIT_THREADS) z[i] = 0ull;
     }
     const int c0 = p.seg_chunk0[seg], c1 = p.seg_chunk0[seg + 1];
+    // fixed order: thread t takes the (user, chunk) pairs t, t + 512, ... of the segment, all loads
+    // independent; then lanes, then warps
+    const int nck = c1 - c0, npairs = nck * p.U;
     double a1 = 0.0, a2 = 0.0;
     unsigned long long an = 0;
-    for (int u = 0; u < p.U; ++u) {                       // fixed order: users, then chunks
-        const size_t base = (size_t)u * (size_t)p.n_chunks;
 #pragma unroll 4
-        for (int c = c0 + tid; c < c1; c += FIT_THREADS) {
-            a1 += p.part_s1[base + c];
-            a2 += p.part_s2[base + c];
-            an += p.part_nf[base + c];
-        }
+    for (int k = tid; k < npairs; k += FIT_THREADS) {
+        const int u = k / nck, c = c0 + (k - u * nck);
+        const size_t i = (size_t)u * (size_t)p.n_chunks + c;
+        a1 += p.part_s1[i];
+        a2 += p.part_s2[i];
+        an += p.part_nf[i];
     }
-    s_a[tid] = a1; s_b[tid] = a2; s_n[tid] = an;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a1 += __shfl_down_sync(0xffffffffu, a1, o);
+        a2 += __shfl_down_sync(0xffffffffu, a2, o);
+        an += __shfl_down_sync(0xffffffffu, an, o);
+    }
+    if ((tid & 31) == 0) { s_a[tid >> 5] = a1; s_b[tid >> 5] = a2; s_n[tid >> 5] = an; }
     __syncthreads();
-    for (int o = FIT_THREADS / 2; o > 0; o >>= 1) {
-        if (tid < o) { s_a[tid] += s_a[tid + o]; s_b[tid] += s_b[tid + o]; s_n[tid] += s_n[tid + o]; }
-        __syncthreads();
-    }
-    const double S1 = s_a[0], S2 = s_b[0];
-    const unsigned long long nf = s_n[0];
+    double S1 = 0.0, S2 = 0.0;
+    unsigned long long nf = 0;
+#pragma unroll
+    for (int w = 0; w < FIT_THREADS / 32; ++w) { S1 += s_a[w]; S2 += s_b[w]; nf += s_n[w]; }
     const double N = (double)((unsigned long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * (unsigned long long)p.U - nf);
 
     // beta = clamp(R^-1(rho), 0.3, 2.0), rho = N S2 / S1^2; R is strictly decreasing in beta, and
