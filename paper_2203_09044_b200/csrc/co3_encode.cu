@@ -143,7 +143,7 @@ __device__ __forceinline__ void put_piece(uint32_t* s_buf, uint32_t pos, unsigne
 // CO3_FLAG_TIMEOUT and the block writes nothing.
 constexpr uint32_t ST_VALID = 0x80000000u;
 constexpr int GRP_SHIFT = 6, GRP_SIZE = 1 << GRP_SHIFT;
-constexpr int SPIN_LIMIT = 1 << 22;
+constexpr int SPIN_LIMIT = 1 << 20;          // polls of a word in L2: about a second, then give up
 
 __device__ __forceinline__ uint32_t wait_count(const uint32_t* st, bool& timeout) {
     const volatile uint32_t* v = st;

@@ -91,3 +91,18 @@ def test_partition_identical_to_oracle(binding, oracle):
         n = p.n_chunks
         assert np.array_equal(seg, p.chunk_seg[:n]) and np.array_equal(st, p.chunk_start[:n])
         assert np.array_equal(en, p.chunk_end[:n]) and np.array_equal(sb, p.sub_base[:n])
+
+
+def test_sweep_report_helpers_need_no_gpu():
+    """The throughput report module: which workloads it would skip for lack of device memory, and
+    one formatted table row (no GPU is touched by these helpers)."""
+    from paper_2203_09044_b200 import inputs, sweep
+    big = inputs.sweep_cell(1 << 28, 64, 1.0, 4, 3)
+    small = inputs.sweep_cell(1 << 16, 8, 1.0, 1, 2)
+    assert sweep.device_bytes_needed(big, 1) > 150e9 > 60e9 > sweep.device_bytes_needed(small, 2)
+    r = dict(name="x", d=1 << 20, U=8, S=1, fmt="E4M3", beta=1.0, ms=0.5, first_ms=1.0, gbs=67.1, convert_ms=0.02,
+             encode_ms=0.03, fit_ms=0.01, decode_ms=0.03, code_bits=6.8, container_bits=6.95, flags=0, l2_resident=True)
+    cells = [c.strip() for c in sweep.row(r, 6550.7).split("|")]
+    assert cells[1] == "x" and cells[4] == "E4M3" and "launch-bound" in cells[-2]
+    conv_gbs = 13.0 * 8 * (1 << 20) / 0.02e-3 / 1e9
+    assert abs(float(cells[9]) - round(conv_gbs)) <= 1
