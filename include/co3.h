@@ -145,7 +145,11 @@ int co3_decode_aggregate_update(co3_plan* plan, const uint32_t* bitstream, const
 /* One whole iteration from host memory (what a training loop that keeps gradients on the host
  * would call): copies h_grad (host, [U][ld], pinned for full speed) to d_grad, runs co3_encode
  * and co3_decode_aggregate with the given device buffers, and copies the average back to h_avg
- * (host, [d]).  Everything is enqueued on cuda_stream; the caller synchronises. */
+ * (host, [d]).  The caller synchronises cuda_stream, as for the other calls: the two copies run on
+ * streams of the plan, ordered against cuda_stream with events, so that the gradient copy of the next
+ * call overlaps this call's encode, decode and copy back.  d_grad is scratch of this call sequence:
+ * nothing else may touch it between calls, and h_grad may be reused once cuda_stream has been
+ * synchronised (or the next call's work on it has completed). */
 int co3_iteration_host(co3_plan* plan, const float* h_grad, float* d_grad, float* d_residual,
                        uint32_t* d_bitstream, uint16_t* d_sub_bits, uint32_t* d_chunk_off,
                        uint64_t* d_user_bits, co3_seg_header* d_hdr, float* d_avg, float* h_avg,

@@ -114,6 +114,10 @@ extern "C" int64_t co3_launch_count(const co3_plan* pl) { return pl ? pl->launch
 extern "C" void co3_plan_destroy(co3_plan* pl) {
     if (!pl) return;
     free_events(pl);
+    if (pl->host_pipe_ready) {
+        cudaStreamDestroy(pl->s_in); cudaStreamDestroy(pl->s_out);
+        cudaEventDestroy(pl->ev_h2d); cudaEventDestroy(pl->ev_conv); cudaEventDestroy(pl->ev_dec); cudaEventDestroy(pl->ev_d2h);
+    }
     for (int i = 0; i < pl->n_allocs; ++i) cudaFree(pl->allocs[i]);
     free(pl->h_seg_off);
     delete pl;
@@ -316,6 +320,7 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
         }
         CO3_TRY(cudaMemcpyAsync(hdr, pl->dev.hdr_cur, sizeof(co3_seg_header) * (size_t)pl->dev.S, cudaMemcpyDeviceToDevice, st));
         CO3_TRY(co3_launch_convert_pack(pl, grad, residual, sub_bits, st));
+        if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));
         CO3_TRY(co3_launch_scan_gather(pl, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
         CO3_TRY(co3_launch_fit(pl, 3, pl->dev.hdr_cur, st));
         pl->iteration++;
@@ -326,6 +331,7 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
         CO3_TRY(co3_launch_fit(pl, 0, hdr, st));
     }
     CO3_TRY(co3_launch_convert(pl, grad, residual, st));
+    if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));   // the gradient buffer is free from here on
     CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
     CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;
@@ -360,13 +366,37 @@ extern "C" int co3_iteration_host(co3_plan* pl, const float* h_grad, float* d_gr
                                   void* cuda_stream) {
     if (!pl || !h_grad || !d_grad || !h_avg || !d_avg) return CO3_EINVAL;
     cudaStream_t st = as_stream(cuda_stream);
+    // The copies run on two streams of the plan so that consecutive calls overlap: the gradient of
+    // call k+1 goes to the device while call k is still encoding, decoding and copying its average
+    // back (PCIe is full duplex).  d_grad is free as soon as the convert pass of the previous call
+    // has read it; everything else is ordered through the caller's stream, which at the end of the
+    // call also waits for the copy of the average, so synchronising it is still all the caller does.
+    if (!pl->host_pipe_ready) {
+        CO3_TRY(cudaStreamCreateWithFlags(&pl->s_in, cudaStreamNonBlocking));
+        CO3_TRY(cudaStreamCreateWithFlags(&pl->s_out, cudaStreamNonBlocking));
+        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_h2d, cudaEventDisableTiming));
+        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_conv, cudaEventDisableTiming));
+        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_dec, cudaEventDisableTiming));
+        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_d2h, cudaEventDisableTiming));
+        pl->host_pipe_ready = true;
+    }
+    if (pl->ev_conv_recorded) CO3_TRY(cudaStreamWaitEvent(pl->s_in, pl->ev_conv, 0));
     CO3_TRY(cudaMemcpyAsync(d_grad, h_grad, sizeof(float) * (size_t)pl->dev.U * (size_t)pl->dev.ld,
-                            cudaMemcpyHostToDevice, st));
+                            cudaMemcpyHostToDevice, pl->s_in));
+    CO3_TRY(cudaEventRecord(pl->ev_h2d, pl->s_in));
+    CO3_TRY(cudaStreamWaitEvent(st, pl->ev_h2d, 0));
+    pl->record_conv = true;
     int rc = co3_encode(pl, d_grad, d_residual, d_bitstream, d_sub_bits, d_chunk_off, d_user_bits, d_hdr, cuda_stream);
+    pl->record_conv = false;
     if (rc != CO3_OK) return rc;
+    pl->ev_conv_recorded = true;
     rc = co3_decode_aggregate(pl, d_bitstream, d_sub_bits, d_chunk_off, d_hdr, d_avg, cuda_stream);
     if (rc != CO3_OK) return rc;
-    CO3_TRY(cudaMemcpyAsync(h_avg, d_avg, sizeof(float) * (size_t)pl->dev.d, cudaMemcpyDeviceToHost, st));
+    CO3_TRY(cudaEventRecord(pl->ev_dec, st));
+    CO3_TRY(cudaStreamWaitEvent(pl->s_out, pl->ev_dec, 0));
+    CO3_TRY(cudaMemcpyAsync(h_avg, d_avg, sizeof(float) * (size_t)pl->dev.d, cudaMemcpyDeviceToHost, pl->s_out));
+    CO3_TRY(cudaEventRecord(pl->ev_d2h, pl->s_out));
+    CO3_TRY(cudaStreamWaitEvent(st, pl->ev_d2h, 0));
     return CO3_OK;
 }
 

@@ -114,6 +114,12 @@ struct co3_plan {
     size_t enc_sync_bytes;          // size of the enc_grp / enc_st / enc_ticket allocation
     int grid_stats, grid_convert;   // launch grids (fixed per plan: they define the reduction order)
     cudaStream_t last_stream;
+    // co3_iteration_host: copy streams and the events that order them against the caller's stream
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_h2d, ev_conv, ev_dec, ev_d2h;
+    bool host_pipe_ready;           // streams and events exist
+    bool ev_conv_recorded;          // a convert pass that read d_grad has been recorded
+    bool record_conv;               // co3_encode records ev_conv after its last pass over the gradient
     void* allocs[64];
     int n_allocs;
     int64_t* h_seg_off;

@@ -337,6 +337,31 @@ def test_host_iteration_entry_point(binding, oracle):
         assert np.array_equal(_bits(h_avg.numpy()), _bits(avg_o))
 
 
+def test_host_iterations_back_to_back_overlap_their_copies(binding, oracle):
+    """Four co3_iteration_host calls enqueued without any synchronisation in between (the copies of
+    one call overlap the work of the previous one on the plan's own streams): every average and
+    the final memory must still be the oracle's."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=1_500_000, n_users=4)
+    plan = binding.Plan(wl.d, 4, 4, 3, wl.seg_offsets)
+    orc = oracle.OracleCO3(wl.d, 4, 4, 3, wl.seg_offsets, cap_words=plan.cap_words)
+    out = plan.alloc_outputs()
+    m = torch.zeros((4, plan.ld), device="cuda")
+    m_cpu = np.zeros((4, plan.ld), np.float32)
+    d_grad = torch.empty((4, plan.ld), device="cuda")
+    h_grads = [wl.gradient(t).pin_memory() for t in range(4)]
+    h_avgs = [torch.empty(wl.d).pin_memory() for _ in range(4)]
+    for t in range(4):
+        plan.iteration_host(h_grads[t], d_grad, m, out, h_avgs[t])
+    torch.cuda.synchronize()
+    for t in range(4):
+        r = orc.encode(h_grads[t].numpy().copy(), m_cpu)
+        rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+        assert rc == oracle.OK and np.array_equal(_bits(h_avgs[t].numpy()), _bits(avg_o)), f"t={t}"
+    assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_cpu))
+    assert plan.status()[0] == 0
+
+
 # ---- full sizes, in the launch configuration the benchmark times ---------------------------
 @pytest.mark.slow
 def test_config0_full(binding, oracle):
