@@ -66,6 +66,16 @@ extern "C" {
  * co3_debug_symbols is not available in this mode. */
 #define CO3_CODE_LAGGED 2
 
+/* How the exponent bias follows from the fitted GenNorm (Sec. III (i)).
+ * CO3_RULE_POLY: the paper's closed form (Eq. "approximate"): b = nearest integer to
+ *   log2(alpha) - log2(0.46 - 2.85 beta + 5.37 beta^2 - 2.85 beta^3 + 0.52 beta^4), fitted by the
+ *   paper for its 4-bit format.
+ * CO3_RULE_OPT: what that closed form approximates (Eq. "exp bias", L2 reading), for the plan's own
+ *   format: the integer b that minimises the expected squared conversion error of the fitted
+ *   GenNorm, evaluated on the header grid (shape 2^(ibeta/8), log2(alpha) - b in steps of 1/8). */
+#define CO3_RULE_POLY 0
+#define CO3_RULE_OPT 1
+
 typedef struct co3_plan co3_plan; /* opaque, library-owned */
 
 /* Sec. III (i): one sign bit is implied.  Supported: 1 <= exp_bits <= 4, 1 <= mant_bits,
@@ -93,6 +103,8 @@ typedef struct {
     float gamma;                /* memory decay of Algorithm 1 line 8; 0: no feedback, 1: plain EF */
     int32_t bias_mode;          /* CO3_BIAS_CURRENT, CO3_BIAS_LAGGED or CO3_CODE_LAGGED            */
     int64_t cap_words;          /* row pitch of `bitstream` in 32-bit words, multiple of 4         */
+    int32_t bias_rule;          /* CO3_RULE_POLY (the paper's, default 0) or CO3_RULE_OPT          */
+    int32_t reserved;           /* 0                                                               */
 } co3_config;
 
 /* Algorithm 1 line 2 and Table I: fixes d, U, the format, the layers, gamma.  Validates the
@@ -207,6 +219,13 @@ int co3_debug_code(co3_plan* plan, const co3_seg_header* hdr, uint8_t* lengths, 
  * indices (ibeta in [-14, 8], ir in [-96, 31]), one per symbol byte, 2^(1+E+M) entries.  The
  * Huffman code of a segment is built from exactly these numbers (Sec. III (ii)). */
 int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint32_t* weights);
+
+/* Host only: the table behind CO3_RULE_OPT, 23 x 8 int16: for shape index ibeta + 14 and residue
+ * rho = round(8 log2 alpha) mod 8, the ir (congruent to rho) of least expected squared conversion
+ * error; the rule's bias is (round(8 log2 alpha) - ir) / 8, clamped.  co3_grid_distortion is the
+ * objective itself, E[(Q(X) - X)^2] / alpha^2 at a header cell (negative: invalid arguments). */
+int co3_bias_opt_table(co3_format fmt, int16_t* table);
+double co3_grid_distortion(co3_format fmt, int32_t ibeta, int32_t ir);
 
 /* Host only: the static partition for (d, segments), as co3_plan_create computes it.  Arrays
  * are host, sized by a first call with NULL arrays that returns the chunk count. */

@@ -294,6 +294,69 @@ double co3o_gammainc(double a, double x) {
     return 1.0 - q;
 }
 
+/* ------------------------------------------------------------------------------------------
+ * The quantity the exponent bias is meant to minimise (Eq. "exp bias", L2 reading): the expected
+ * squared conversion error of X ~ GenNorm(alpha, beta), here divided by alpha^2 and evaluated on the
+ * header grid: beta = 2^(ibeta/8), log2(alpha) - b = ir/8.  In units of alpha the grid values are
+ * v_j = K(j) u with u = 2^(c_F - ir/8), the cells end at the midpoints t_j = (v_j + v_(j+1)) / 2 (the
+ * last one at infinity: saturation), and with z = (x/alpha)^beta
+ *   int_0^t (x/alpha)^k dF = Gamma((k+1)/beta) / Gamma(1/beta) * P((k+1)/beta, t^beta),
+ * so each cell contributes m2 - 2 v m1 + v^2 m0 from differences of three incomplete gammas.
+ * ------------------------------------------------------------------------------------------ */
+double co3o_distortion(int E, int M, int ibeta, int ir) {
+    if (!fmt_ok(E, M)) return -1.0;
+    int J = 1 << (E + M);
+    double beta = exp2((double)ibeta / 8.0);
+    double u = exp2((double)co3o_cF(E, M) - (double)ir / 8.0);
+    double a0 = 1.0 / beta, a1 = 2.0 / beta, a2 = 3.0 / beta;
+    double c1 = exp(lgamma(a1) - lgamma(a0)), c2 = exp(lgamma(a2) - lgamma(a0));
+    double p0 = 0.0, p1 = 0.0, p2 = 0.0, total = 0.0;
+    for (int j = 0; j < J; j++) {
+        double q0 = 1.0, q1 = 1.0, q2 = 1.0;
+        if (j < J - 1) {
+            double t = 0.5 * (double)(co3o_K(E, M, j) + co3o_K(E, M, j + 1)) * u;
+            double z = pow(t, beta);
+            q0 = co3o_gammainc(a0, z); q1 = co3o_gammainc(a1, z); q2 = co3o_gammainc(a2, z);
+        }
+        double v = (double)co3o_K(E, M, j) * u;
+        total += c2 * (q2 - p2) - 2.0 * v * c1 * (q1 - p1) + v * v * (q0 - p0);
+        p0 = q0; p1 = q1; p2 = q2;
+    }
+    return total;
+}
+
+/* Bias rule "optimal": the integer b that minimises that distortion.  Shifting b by one moves ir by
+ * eight, so for a shape index ibeta and a residue rho = round(8 log2 alpha) mod 8 the choice is the
+ * best ir among those congruent to rho: a table of 23 x 8 entries per format (first minimum in
+ * ascending ir, i.e. the larger bias on an exact tie). */
+void co3o_bias_opt_table(int E, int M, int16_t* tab) {
+    for (int ib = -14; ib <= 8; ib++)
+        for (int rho = 0; rho < 8; rho++) {
+            int best = 0, have = 0;
+            double dbest = 0.0;
+            for (int ir = -96; ir <= 31; ir++) {
+                if ((((ir % 8) + 8) % 8) != rho) continue;
+                double dd = co3o_distortion(E, M, ib, ir);
+                if (!have || dd < dbest) { have = 1; dbest = dd; best = ir; }
+            }
+            tab[(ib + 14) * 8 + rho] = (int16_t)best;
+        }
+}
+
+int co3o_bias_opt(double beta, double alpha, int E, int M, const int16_t* tab) {
+    int lo = co3o_b_lo(E, M), hi = co3o_b_hi(E, M);
+    if (!(alpha > 0.0)) return lo;
+    double x = floor(8.0 * log2(beta) + 0.5);
+    if (x < -14.0) x = -14.0;
+    if (x > 8.0) x = 8.0;
+    double t8 = floor(8.0 * log2(alpha) + 0.5);
+    if (t8 < -16000.0) return lo;
+    if (t8 > 16000.0) return hi;
+    int t = (int)t8, rho = ((t % 8) + 8) % 8;
+    int b = (t - (int)tab[((int)x + 14) * 8 + rho]) / 8;      /* exact: same residue */
+    return b < lo ? lo : (b > hi ? hi : b);
+}
+
 /* Integer symbol weights of the quantised GenNorm model (Sec. IV-B "Huffman coding": the
  * converted samples follow the quantised GenNorm distribution) for header indices (ibeta, ir).
  * Cell edges are the midpoints between neighbouring grid magnitudes, in units of alpha.

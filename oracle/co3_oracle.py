@@ -60,6 +60,12 @@ def lib():
     L.co3o_poly.argtypes = [C.c_double]
     L.co3o_bias.restype = C.c_int
     L.co3o_bias.argtypes = [C.c_double, C.c_double, C.c_int, C.c_int]
+    L.co3o_distortion.restype = C.c_double
+    L.co3o_distortion.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
+    L.co3o_bias_opt_table.restype = None
+    L.co3o_bias_opt_table.argtypes = [C.c_int, C.c_int, C.c_void_p]
+    L.co3o_bias_opt.restype = C.c_int
+    L.co3o_bias_opt.argtypes = [C.c_double, C.c_double, C.c_int, C.c_int, C.c_void_p]
     L.co3o_header.restype = None
     L.co3o_header.argtypes = [C.c_double, C.c_double, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     L.co3o_gammainc.restype = C.c_double
@@ -142,6 +148,34 @@ def poly(beta):
 
 def bias(beta, alpha, E, M):
     return int(lib().co3o_bias(beta, alpha, E, M))
+
+
+RULE_POLY = 0   # the paper's polynomial (Eq. "approximate"), nearest integer exponent
+RULE_OPT = 1    # the integer bias that minimises the L2 conversion error of the fitted GenNorm
+_OPT_TABLES = {}
+
+
+def distortion(E, M, ibeta, ir):
+    """E[(Q(X) - X)^2] / alpha^2 for X ~ GenNorm(alpha, 2^(ibeta/8)) with log2(alpha) - b = ir/8."""
+    return float(lib().co3o_distortion(E, M, ibeta, ir))
+
+
+def bias_opt_table(E, M):
+    """[23][8] int16: best ir for (ibeta + 14, round(8 log2 alpha) mod 8); cached per format."""
+    if (E, M) not in _OPT_TABLES:
+        tab = np.zeros((23, 8), np.int16)
+        lib().co3o_bias_opt_table(E, M, tab.ctypes.data)
+        _OPT_TABLES[(E, M)] = tab
+    return _OPT_TABLES[(E, M)]
+
+
+def bias_opt(beta, alpha, E, M):
+    tab = bias_opt_table(E, M)
+    return int(lib().co3o_bias_opt(beta, alpha, E, M, tab.ctypes.data))
+
+
+def bias_by_rule(rule, beta, alpha, E, M):
+    return bias_opt(beta, alpha, E, M) if rule == RULE_OPT else bias(beta, alpha, E, M)
 
 
 def header(beta, alpha, b):
@@ -236,7 +270,7 @@ class OracleCO3:
     """
 
     def __init__(self, d, n_users, E, M, seg_offsets=None, gamma=0.9, mode=MODE_LAGGED,
-                 cap_words=None):
+                 cap_words=None, rule=RULE_POLY):
         self.d, self.U, self.E, self.M = int(d), int(n_users), int(E), int(M)
         self.nsym = 1 << (1 + E + M)
         off = [0, d] if seg_offsets is None else list(seg_offsets)
@@ -244,6 +278,7 @@ class OracleCO3:
         self.S = self.part.S
         self.gamma = float(np.float32(gamma))
         self.mode = mode
+        self.rule = rule
         self.t = 0
         self.bias_next = np.zeros(self.S, np.int32)
         self.hdr_next = np.zeros((self.S, 3), np.int32)   # MODE_LAGGED_CODE: header of the coming iteration
@@ -263,7 +298,7 @@ class OracleCO3:
             for l in range(S):
                 N, S1, S2, _ = stats(g, m, int(off[l]), int(off[l + 1]), self.gamma)
                 be, al = fit(N, S1, S2)
-                bias_t[l] = bias(be, al, E, M)
+                bias_t[l] = bias_by_rule(self.rule, be, al, E, M)
         else:
             bias_t[:] = self.bias_next
         sym = np.zeros((U, self.d), np.uint8)
@@ -276,7 +311,7 @@ class OracleCO3:
             N, S1, S2, nf = convert(g, m, sym, int(off[l]), int(off[l + 1]), self.gamma, E, M,
                                     int(bias_t[l]), hist[l])
             be, al = fit(N, S1, S2)
-            self.bias_next[l] = bias(be, al, E, M)
+            self.bias_next[l] = bias_by_rule(self.rule, be, al, E, M)
             if self.mode == MODE_LAGGED_CODE and self.t > 0:
                 hdr[l] = self.hdr_next[l]              # fixed by iteration t-1 (its bias is bias_t[l])
             else:

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libco3.so")
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ECORRUPT, ENONFINITE = 0, -1, -2, -3, -4, -5, -6
 FLAG_CAPACITY, FLAG_CORRUPT, FLAG_NONFINITE = 1, 2, 4
 BIAS_CURRENT, BIAS_LAGGED, CODE_LAGGED = 0, 1, 2
+RULE_POLY, RULE_OPT = 0, 1
 FLAG_TIMEOUT = 8
 
 EXPORTS = [
@@ -23,6 +24,7 @@ EXPORTS = [
     "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
     "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
+    "co3_bias_opt_table", "co3_grid_distortion",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -38,7 +40,8 @@ class Format(C.Structure):
 class Config(C.Structure):
     _fields_ = [("d", C.c_int64), ("ld", C.c_int64), ("n_users", C.c_int32), ("fmt", Format),
                 ("n_segments", C.c_int32), ("seg_offsets", C.POINTER(C.c_int64)),
-                ("gamma", C.c_float), ("bias_mode", C.c_int32), ("cap_words", C.c_int64)]
+                ("gamma", C.c_float), ("bias_mode", C.c_int32), ("cap_words", C.c_int64),
+                ("bias_rule", C.c_int32), ("reserved", C.c_int32)]
 
 
 HDR_DTYPE = np.dtype([("bias", np.int8), ("ibeta", np.int8), ("ir", np.int16)])
@@ -103,6 +106,10 @@ def lib():
     L.co3_moments_static.argtypes = [vp, vp, C.c_int64, C.c_float, vp, vp]
     L.co3_state_header.restype = C.c_int
     L.co3_state_header.argtypes = [vp, C.c_int32, vp]
+    L.co3_bias_opt_table.restype = C.c_int
+    L.co3_bias_opt_table.argtypes = [Format, vp]
+    L.co3_grid_distortion.restype = C.c_double
+    L.co3_grid_distortion.argtypes = [Format, C.c_int32, C.c_int32]
     L.co3_strerror.restype = C.c_char_p
     L.co3_strerror.argtypes = [C.c_int]
     _lib = L
@@ -116,6 +123,19 @@ def model_weights(exp_bits, mant_bits, ibeta, ir):
     if rc != OK:
         raise Co3Error(rc, "co3_model_weights")
     return w
+
+
+def bias_opt_table(exp_bits, mant_bits):
+    """[23][8] int16 table behind RULE_OPT (host only)."""
+    tab = np.zeros((23, 8), np.int16)
+    rc = lib().co3_bias_opt_table(Format(exp_bits, mant_bits), tab.ctypes.data)
+    if rc != OK:
+        raise Co3Error(rc, "co3_bias_opt_table")
+    return tab
+
+
+def grid_distortion(exp_bits, mant_bits, ibeta, ir):
+    return float(lib().co3_grid_distortion(Format(exp_bits, mant_bits), int(ibeta), int(ir)))
 
 
 def partition(d, seg_offsets):
@@ -150,7 +170,7 @@ class Plan:
     """co3_plan plus the torch buffers of one pipeline instance on the current CUDA device."""
 
     def __init__(self, d, n_users, exp_bits, mant_bits, seg_offsets=None, gamma=0.9,
-                 bias_mode=BIAS_LAGGED, cap_words=None, ld=None):
+                 bias_mode=BIAS_LAGGED, cap_words=None, ld=None, bias_rule=RULE_POLY):
         import torch
         self.torch = torch
         L = lib()
@@ -167,7 +187,7 @@ class Plan:
         self.cap_words = int(cap_words) if cap_words is not None else worst
         cfg = Config(self.d, self.ld, self.U, Format(self.E, self.M), self.S,
                      off.ctypes.data_as(C.POINTER(C.c_int64)), float(gamma), int(bias_mode),
-                     self.cap_words)
+                     self.cap_words, int(bias_rule), 0)
         h = C.c_void_p()
         rc = L.co3_plan_create(C.byref(h), C.byref(cfg))
         if rc != OK:

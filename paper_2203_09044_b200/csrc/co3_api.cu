@@ -132,6 +132,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
     if (cfg->cap_words < 4 || (cfg->cap_words & 3) || cfg->cap_words > 0xFFFFFFFFLL) return CO3_EINVAL;
     if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED && cfg->bias_mode != CO3_CODE_LAGGED) return CO3_EINVAL;
     if (!(cfg->gamma >= 0.0f) || !(cfg->gamma <= 1.0f)) return CO3_EINVAL;
+    if (cfg->bias_rule != CO3_RULE_POLY && cfg->bias_rule != CO3_RULE_OPT) return CO3_EINVAL;
     if (cfg->d > ((int64_t)1 << 31)) return CO3_EINVAL;
     if (((cfg->d + 4095) / 4096 + (cfg->seg_offsets ? cfg->n_segments : 1)) * (int64_t)cfg->n_users > 0x7FFFFFFFLL) return CO3_EINVAL;
     const int nm = E + M, J = 1 << nm, nsym = 2 * J;
@@ -235,6 +236,11 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.part_nf, items);
         a |= dev_alloc(pl, &dv.fit, (size_t)S * 5);
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
+        int16_t* d_opt = nullptr;
+        const int16_t* h_opt = co3_host_bias_opt_table(E, M);
+        a |= dev_alloc(pl, &d_opt, (size_t)CO3_NIBETA * 8);
+        if (!h_opt) a = 1;
+        dv.bias_rule = cfg->bias_rule;
         a |= dev_alloc(pl, &dv.chunk_words, items);
         a |= dev_alloc(pl, &dv.chunk_bits, items);
         a |= dev_alloc(pl, &dv.user_ovf, (size_t)dv.U);
@@ -264,6 +270,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             up(d_seg_chunk0, h_seg_chunk0, sizeof(int32_t) * (size_t)(S + 1));
             up(d_wtab, wtab, sizeof(uint32_t) * (size_t)CO3_NIBETA * CO3_NIR * J);
             up(d_logr, logr, sizeof(double) * 2 * ((size_t)CO3_FIT_GRID + 1));
+            up(d_opt, h_opt, sizeof(int16_t) * (size_t)CO3_NIBETA * 8);
+            dv.bias_opt_tab = d_opt;
             if (e == cudaSuccess) e = cudaMemset(dv.flags, 0, sizeof(uint32_t));
             if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
             if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);

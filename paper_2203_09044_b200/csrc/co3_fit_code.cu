@@ -138,8 +138,22 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     const double alpha = has_alpha ? exp2(log2_alpha) : 0.0;
     int b_rule = p.b_lo;
     if (has_alpha && alpha > 0.0) {
-        const double bf = floor(log2_alpha - log2(poly_bias(beta)) + 0.5);
-        b_rule = bf < (double)p.b_lo ? p.b_lo : (bf > (double)p.b_hi ? p.b_hi : (int)bf);
+        if (p.bias_rule == CO3_RULE_OPT) {
+            // the integer bias of least expected squared error: (round(8 log2 alpha) - best ir) / 8
+            double xb = floor(8.0 * (s_state == 0 ? t : log2(beta)) + 0.5);
+            xb = xb < (double)CO3_IBETA_MIN ? (double)CO3_IBETA_MIN : (xb > (double)CO3_IBETA_MAX ? (double)CO3_IBETA_MAX : xb);
+            const double t8 = floor(8.0 * log2_alpha + 0.5);
+            if (t8 < -16000.0) b_rule = p.b_lo;
+            else if (t8 > 16000.0) b_rule = p.b_hi;
+            else {
+                const int ti = (int)t8, rho = ((ti % 8) + 8) % 8;
+                const int b = (ti - (int)p.bias_opt_tab[((int)xb - CO3_IBETA_MIN) * 8 + rho]) / 8;   // exact
+                b_rule = b < p.b_lo ? p.b_lo : (b > p.b_hi ? p.b_hi : b);
+            }
+        } else {
+            const double bf = floor(log2_alpha - log2(poly_bias(beta)) + 0.5);
+            b_rule = bf < (double)p.b_lo ? p.b_lo : (bf > (double)p.b_hi ? p.b_hi : (int)bf);
+        }
     }
     if (mode == 0) {
         p.bias_cur[seg] = b_rule;

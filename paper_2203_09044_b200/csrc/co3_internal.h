@@ -86,6 +86,8 @@ struct Co3Dev {
     uint32_t* part_nf;            //              ... count of non-finite a
     double* fit;                  // [S][5] beta, alpha, N, S1, S2
     int32_t* bias_cur;            // [S] bias used by the next convert pass
+    int bias_rule;                // CO3_RULE_POLY or CO3_RULE_OPT
+    const int16_t* bias_opt_tab;  // [NIBETA][8] best ir per (shape index, round(8 log2 alpha) mod 8)
     co3_seg_header* hdr_cur;      // [S] fully lagged code: header of the coming iteration (else unused)
     uint32_t* slot_buf;           // [U*n_chunks][32][CO3_SUB_WORDS] fully lagged code: the packed sub-chunks,
                                   //     each from bit 0 of its own slot, before their offsets are known (else null)
@@ -154,6 +156,7 @@ int co3_host_cF(int E, int M);
 int64_t co3_host_K(int M, int j);
 const uint32_t* co3_host_weight_table(int E, int M);   // [NIBETA][NIR][J], cached per format
 const double* co3_host_logr_table(void);               // [2][FIT_GRID + 1], cached
+const int16_t* co3_host_bias_opt_table(int E, int M);   // [NIBETA][8], cached per format
 
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st);

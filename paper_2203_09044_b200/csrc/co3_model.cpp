@@ -98,10 +98,45 @@ void weight_row(int E, int M, int ibeta, int ir, uint32_t* half /* J entries */)
     }
 }
 
+// Expected squared conversion error of X ~ GenNorm(alpha, beta_q), divided by alpha^2, when
+// log2(alpha) - b = ir/8 (the L2 objective of Eq. "exp bias" on the header grid).  Computed edge by
+// edge: at every cell edge t (in units of alpha) the three partial moments
+//   m_k(t) = int_0^t x^k dF = Gamma((k+1)/beta)/Gamma(1/beta) * P((k+1)/beta, t^beta),  k = 0, 1, 2
+// are evaluated once, and the cell between two edges adds (dm2 - 2 v dm1 + v^2 dm0) for its grid
+// value v; beyond the last edge (saturation) the moments are their totals.
+double grid_distortion(int E, int M, int ibeta, int ir) {
+    const int J = 1 << (E + M);
+    const double beta_q = exp2((double)ibeta / 8.0);
+    const double unit = exp2((double)co3_host_cF(E, M) - (double)ir / 8.0);   // grid quantum / alpha
+    const double s0 = 1.0 / beta_q, s1 = 2.0 / beta_q, s2 = 3.0 / beta_q;
+    const double g1 = exp(lgamma(s1) - lgamma(s0)), g2 = exp(lgamma(s2) - lgamma(s0));
+    double lo[3] = {0.0, 0.0, 0.0}, sum = 0.0;
+    for (int j = 0; j < J; ++j) {
+        double hi[3] = {1.0, g1, g2};
+        if (j + 1 < J) {
+            const double edge = 0.5 * (double)(co3_host_K(M, j) + co3_host_K(M, j + 1)) * unit;
+            const double z = pow(edge, beta_q);
+            hi[0] = reg_lower_gamma(s0, z);
+            hi[1] = g1 * reg_lower_gamma(s1, z);
+            hi[2] = g2 * reg_lower_gamma(s2, z);
+        }
+        const double v = (double)co3_host_K(M, j) * unit;
+        sum += (hi[2] - lo[2]) - 2.0 * v * (hi[1] - lo[1]) + v * v * (hi[0] - lo[0]);
+        lo[0] = hi[0]; lo[1] = hi[1]; lo[2] = hi[2];
+    }
+    return sum;
+}
+
 struct TableCache {
     int E, M;
     uint32_t* data;
 };
+struct OptCache {
+    int E, M;
+    int16_t tab[CO3_NIBETA * 8];
+};
+OptCache g_opt[16];
+int g_nopt = 0;
 TableCache g_cache[16];
 int g_ncache = 0;
 std::mutex g_mu;
@@ -121,6 +156,45 @@ const uint32_t* co3_host_weight_table(int E, int M) {
             weight_row(E, M, ib + CO3_IBETA_MIN, r + CO3_IR_MIN, t + ((size_t)ib * CO3_NIR + r) * J);
     g_cache[g_ncache++] = TableCache{E, M, t};
     return t;
+}
+
+// Bias rule "optimal": moving b by one moves ir by eight, so the L2-best integer bias for a shape
+// index and a residue rho = round(8 log2 alpha) mod 8 is the ir of least distortion among those
+// congruent to rho (the first one in ascending ir on an exact tie).  [NIBETA][8] entries, cached.
+const int16_t* co3_host_bias_opt_table(int E, int M) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (int i = 0; i < g_nopt; ++i)
+        if (g_opt[i].E == E && g_opt[i].M == M) return g_opt[i].tab;
+    if (g_nopt == 16) return nullptr;
+    OptCache& c = g_opt[g_nopt];
+    c.E = E; c.M = M;
+    for (int ib = 0; ib < CO3_NIBETA; ++ib) {
+        double best[8];
+        int arg[8];
+        for (int k = 0; k < 8; ++k) { best[k] = -1.0; arg[k] = 0; }
+        for (int ir = CO3_IR_MIN; ir <= CO3_IR_MAX; ++ir) {
+            const int rho = ((ir % 8) + 8) % 8;
+            const double dist = grid_distortion(E, M, ib + CO3_IBETA_MIN, ir);
+            if (best[rho] < 0.0 || dist < best[rho]) { best[rho] = dist; arg[rho] = ir; }
+        }
+        for (int k = 0; k < 8; ++k) c.tab[ib * 8 + k] = (int16_t)arg[k];
+    }
+    ++g_nopt;
+    return c.tab;
+}
+
+extern "C" int co3_bias_opt_table(co3_format fmt, int16_t* table) {
+    if (!co3_host_fmt_ok(fmt) || !table) return CO3_EINVAL;
+    const int16_t* t = co3_host_bias_opt_table(fmt.exp_bits, fmt.mant_bits);
+    if (!t) return CO3_ENOMEM;
+    memcpy(table, t, sizeof(int16_t) * CO3_NIBETA * 8);
+    return CO3_OK;
+}
+
+extern "C" double co3_grid_distortion(co3_format fmt, int32_t ibeta, int32_t ir) {
+    if (!co3_host_fmt_ok(fmt) || ibeta < CO3_IBETA_MIN || ibeta > CO3_IBETA_MAX || ir < CO3_IR_MIN || ir > CO3_IR_MAX)
+        return -1.0;
+    return grid_distortion(fmt.exp_bits, fmt.mant_bits, ibeta, ir);
 }
 
 // Two functions of the GenNorm shape on a grid uniform in log2(beta) over [log2 0.3, log2 2]:

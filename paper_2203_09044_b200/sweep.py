@@ -42,12 +42,12 @@ def device_bytes_needed(wl, pool):
     return 4 * ud * pool + 4 * ud + ud + 2 * ud + 4 * wl.d
 
 
-def measure(wl, iters, warm, pool):
+def measure(wl, iters, warm, pool, rule=0):
     """Run warm + iters iterations of one workload; returns a dict of figures."""
     wl.align_rows()
     U, d = wl.n_users, wl.d
     plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
-                        bias_mode=binding.BIAS_LAGGED, ld=wl.ld)
+                        bias_mode=binding.BIAS_LAGGED, ld=wl.ld, bias_rule=rule)
     out = plan.alloc_outputs()
     residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
     grads = [wl.gradient(t, device="cuda") for t in range(pool)]
@@ -79,7 +79,10 @@ def measure(wl, iters, warm, pool):
     code_bits = float(out["user_bits"].sum().item()) / (U * d)
     container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
                       + 32.0 * U * (plan.n_chunks + 1) + 32.0 * plan.S) / (U * d)
-    res = dict(name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
+    # realised relative conversion error of the last iteration: the memory is a - Q(a) exactly
+    err2 = float((residual[:, :d].double() ** 2).sum().item())
+    s2 = sum(plan.get_fit(l)[4] for l in range(plan.S))
+    res = dict(rel_mse=err2 / s2 if s2 > 0 else 0.0, name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
                ms=ms, first_ms=first_ms, gbs=4.0 * U * d / (ms * 1e-3) / 1e9,
                convert_ms=prof.get("convert", 0.0),
                encode_ms=prof.get("enc_len", 0.0) + prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0),
@@ -93,8 +96,8 @@ def measure(wl, iters, warm, pool):
 
 
 HEADER = ("| workload | d | U | format | beta | ms/iter | GB/s fp32 in | convert us | convert GB/s (13 B) | % of {peak:.0f} "
-          "| % of 8000 | encode us | decode us | decode+encode GB/s (payload+symbols+avg) | code b/el | container b/el | t=0 ms | note |\n"
-          "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+          "| % of 8000 | encode us | decode us | decode+encode GB/s (payload+symbols+avg) | code b/el | container b/el | t=0 ms | rel. sq. error | note |\n"
+          "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
 
 
 def row(r, peak):
@@ -109,10 +112,11 @@ def row(r, peak):
         note.append("inputs fit L2, launch-bound")
     if r["flags"]:
         note.append("flags=%d" % r["flags"])
-    return ("| %s | %d | %d | %s | %.1f | %.4f | %.1f | %.1f | %.0f | %.1f | %.1f | %.1f | %.1f | %.0f | %.3f | %.3f | %.3f | %s |"
+    return ("| %s | %d | %d | %s | %.1f | %.4f | %.1f | %.1f | %.0f | %.1f | %.1f | %.1f | %.1f | %.0f | %.3f | %.3f | %.3f | %.3e | %s |"
             % (r["name"], r["d"], r["U"], r["fmt"], r["beta"], r["ms"], r["gbs"], r["convert_ms"] * 1e3, conv_gbs,
                100.0 * conv_gbs / peak, 100.0 * conv_gbs / NOMINAL_HBM_GBS, r["encode_ms"] * 1e3,
-               r["decode_ms"] * 1e3, ed_gbs, r["code_bits"], r["container_bits"], r["first_ms"], "; ".join(note)))
+               r["decode_ms"] * 1e3, ed_gbs, r["code_bits"], r["container_bits"], r["first_ms"],
+               r.get("rel_mse", 0.0), "; ".join(note)))
 
 
 def main(argv=None):
@@ -122,6 +126,8 @@ def main(argv=None):
     ap.add_argument("--iters", type=int, default=5, help="timed steady-state iterations per workload")
     ap.add_argument("--warm", type=int, default=3, help="untimed iterations before them (>= 1)")
     ap.add_argument("--max-bytes", type=float, default=60e9, help="skip workloads needing more device memory")
+    ap.add_argument("--rule", default="poly", choices=["poly", "opt"],
+                    help="bias rule: the paper's polynomial (default) or the L2-optimal integer bias")
     ap.add_argument("--filter", default=None, help="run only workloads whose name contains this text")
     ap.add_argument("--out", default=None, help="also write the table to this file")
     args = ap.parse_args(argv)
@@ -141,11 +147,11 @@ def main(argv=None):
     for wl in todo:
         pool = 2 if device_bytes_needed(wl, 2) <= args.max_bytes else 1
         if device_bytes_needed(wl, pool) > args.max_bytes:
-            lines.append("| %s | %d | %d | E%dM%d | %.1f | skipped: needs %.0f GB of device memory | | | | | | | | | | | |"
+            lines.append("| %s | %d | %d | E%dM%d | %.1f | skipped: needs %.0f GB of device memory | | | | | | | | | | | | |"
                          % (wl.name, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.beta,
                             device_bytes_needed(wl, 1) / 1e9))
             continue
-        r = measure(wl, args.iters, max(args.warm, 1), pool)
+        r = measure(wl, args.iters, max(args.warm, 1), pool, binding.RULE_OPT if args.rule == "opt" else binding.RULE_POLY)
         lines.append(row(r, peak))
         print(lines[-1], flush=True)
     text = "\n".join(lines) + "\n"

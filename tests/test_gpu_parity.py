@@ -53,10 +53,11 @@ def compare_iteration(b, plan, out, r, m_gpu, m_cpu, tag=""):
             assert np.array_equal(pay[u, :n], r.payload[u, :n]), f"{tag} bitstream user {u}"
 
 
-def run_case(b, oracle, d, U, E, M, off, grads, gamma=0.9, mode=1, cap=None, decode_plan=None):
+def run_case(b, oracle, d, U, E, M, off, grads, gamma=0.9, mode=1, cap=None, decode_plan=None, rule=0):
     """grads: list of [U][ld] float32 cuda tensors, one per iteration (ld is taken from them)."""
-    plan = b.Plan(d, U, E, M, off, gamma=gamma, bias_mode=mode, cap_words=cap, ld=int(grads[0].shape[1]))
-    orc = oracle.OracleCO3(d, U, E, M, off, gamma=gamma, mode=mode, cap_words=plan.cap_words)
+    plan = b.Plan(d, U, E, M, off, gamma=gamma, bias_mode=mode, cap_words=cap, ld=int(grads[0].shape[1]),
+                  bias_rule=rule)
+    orc = oracle.OracleCO3(d, U, E, M, off, gamma=gamma, mode=mode, cap_words=plan.cap_words, rule=rule)
     assert plan.worst_case_words == orc.worst_case_words
     assert (plan.n_chunks, plan.n_sub) == (orc.part.n_chunks, orc.part.n_sub)
     out = plan.alloc_outputs()
@@ -135,6 +136,31 @@ def test_gamma_and_bias_modes(binding, oracle, gamma, mode):
         g[:, :d] = torch.randn((U, d), generator=gen) * (1e-3 * 3.0 ** t)
         grads.append(g.cuda())
     run_case(binding, oracle, d, U, 3, 2, [0, 12_345, d], grads, gamma=gamma, mode=mode)
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("E,M", FORMATS)
+def test_l2_optimal_bias_rule(binding, oracle, E, M, mode):
+    """CO3_RULE_OPT (the integer bias of least expected squared error for the plan's own format
+    instead of the paper's polynomial): bit-exact against the oracle's rule in every mode, on layers
+    of different shapes and drifting scales; for the 6- and 8-bit formats, for which the polynomial
+    was not made, it does change the bias."""
+    from paper_2203_09044_b200 import inputs
+    gen = torch.Generator().manual_seed(77 + E)
+    d, U, off = 40_000, 3, [0, 9_000, 22_222, 40_000]
+    grads = []
+    for t in range(3):
+        g = torch.zeros((U, d))
+        for l, beta in enumerate((0.5, 1.0, 2.0)):
+            n = off[l + 1] - off[l]
+            for u in range(U):
+                g[u, off[l]:off[l + 1]] = inputs.gennorm(n, beta, 1e-3 * 2.5 ** t * (l + 1), gen)
+        grads.append(g.cuda())
+    plan, orc, out, res = run_case(binding, oracle, d, U, E, M, off, grads, mode=mode, rule=1)
+    poly = oracle.OracleCO3(d, U, E, M, off, mode=mode, rule=0)
+    r0 = poly.encode(grads[0].cpu().numpy(), np.zeros((U, d), np.float32))
+    if (E, M) != (1, 2):
+        assert not np.array_equal(r0.bias, res[0][0].bias)
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])

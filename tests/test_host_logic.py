@@ -40,7 +40,7 @@ def test_bad_configurations_are_rejected_on_the_host(binding):
         cfg = binding.Config(base["d"], base["ld"], base["n_users"], binding.Format(base["E"], base["M"]),
                              0 if off is None else len(off) - 1,
                              None if off is None else off.ctypes.data_as(C.POINTER(C.c_int64)),
-                             base["gamma"], base["mode"], base["cap"])
+                             base["gamma"], base["mode"], base["cap"], base.get("rule", 0), 0)
         h = C.c_void_p()
         rc = L.co3_plan_create(C.byref(h), C.byref(cfg))
         if rc == 0:
@@ -54,6 +54,7 @@ def test_bad_configurations_are_rejected_on_the_host(binding):
     assert create(n_users=69) == binding.EINVAL          # 69 * 245760 >= 2^24: sums not exact
     assert create(cap=4001) == binding.EINVAL and create(cap=0) == binding.EINVAL
     assert create(gamma=1.5) == binding.EINVAL and create(mode=7) == binding.EINVAL
+    assert create(rule=2) == binding.EINVAL
     assert create(off=[0, 600, 500, 1000]) == binding.EINVAL
     assert create(off=[0, 500, 900]) == binding.EINVAL
     try:
@@ -104,5 +105,19 @@ def test_sweep_report_helpers_need_no_gpu():
              encode_ms=0.03, fit_ms=0.01, decode_ms=0.03, code_bits=6.8, container_bits=6.95, flags=0, l2_resident=True)
     cells = [c.strip() for c in sweep.row(r, 6550.7).split("|")]
     assert cells[1] == "x" and cells[4] == "E4M3" and "launch-bound" in cells[-2]
+    assert float(cells[-3]) == 0.0                      # no realised error given: column printed as 0
     conv_gbs = 13.0 * 8 * (1 << 20) / 0.02e-3 / 1e9
     assert abs(float(cells[9]) - round(conv_gbs)) <= 1
+
+
+@pytest.mark.parametrize("E,M", [(1, 2), (3, 2), (4, 3)])
+def test_optimal_bias_table_is_identical_in_library_and_oracle(binding, oracle, E, M):
+    """The 23 x 8 table behind the L2-optimal bias rule, and the objective it is the argmin of, from
+    the library's own incomplete-gamma code and from the oracle's: same choices everywhere, same
+    distortion to 1e-9."""
+    assert np.array_equal(binding.bias_opt_table(E, M), oracle.bias_opt_table(E, M))
+    for ib in (-14, -5, 0, 3, 8):
+        for ir in (-96, -40, -17, -3, 0, 9, 31):
+            a, b = binding.grid_distortion(E, M, ib, ir), oracle.distortion(E, M, ib, ir)
+            assert a > 0 and abs(a - b) <= 1e-9 * b
+    assert binding.grid_distortion(E, M, 9, 0) < 0 and binding.grid_distortion(E, M, 0, 32) < 0

@@ -576,3 +576,72 @@ def test_fused_model_update_is_the_plain_update(oracle):
         prod = np.float32(float(Fraction(float(step)) * Fraction(float(avg[i]))))     # exact product, rounded once
         want = np.float32(float(Fraction(float(w0[i])) + Fraction(float(prod))))      # exact sum, rounded once
         assert w[i] == want
+
+
+def _laplace_cell(lo, hi, v, a):
+    """int_lo^hi (x - v)^2 e^(-x/a)/a dx in closed form (antiderivative -e^(-x/a)((x-v)^2 + 2a(x-v) + 2a^2))."""
+    def F(x):
+        if math.isinf(x):
+            return 0.0
+        return -math.exp(-x / a) * ((x - v) ** 2 + 2 * a * (x - v) + 2 * a * a)
+    return F(hi) - F(lo)
+
+
+def test_distortion_closed_form_for_laplace_and_quadrature_for_other_shapes(oracle):
+    """The L2 objective of the bias (Eq. "exp bias"): for beta = 1 every cell has an elementary
+    antiderivative; for other shapes it is compared with numerical quadrature of the converter
+    itself (the oracle's Q_fp applied to a fine grid of inputs)."""
+    for E, M in FORMATS:
+        J = 1 << (E + M)
+        K = [oracle.K(E, M, j) for j in range(J)]
+        for ir in (-30, -8, 0, 7, 20):
+            u = 2.0 ** (oracle.cF(E, M) - ir / 8.0)          # grid quantum in units of alpha
+            edges = [0.0] + [0.5 * (K[j] + K[j + 1]) * u for j in range(J - 1)] + [math.inf]
+            want = sum(_laplace_cell(edges[j], edges[j + 1], K[j] * u, 1.0) for j in range(J))
+            got = oracle.distortion(E, M, 0, ir)
+            assert abs(got - want) <= 1e-9 * want, (E, M, ir, got, want)
+    # fp4, beta = 2^(ib/8): the paper's scalar form.  X ~ GenNorm(1, beta) is multiplied by s = 2^(ir/8)
+    # and converted at bias 0, so log2(alpha) - b = ir/8 and the error divided by alpha^2 is
+    # E[(Q(sX)/s - X)^2], taken here by quadrature through the oracle's converter
+    for ib, ir in ((-8, -33), (0, -4), (5, 5), (8, 8), (0, 12), (3, -20)):
+        beta = 2.0 ** (ib / 8.0)
+        xmax = 60.0 ** (1.0 / beta)
+        x = np.concatenate([np.linspace(0, 1, 40001)[:-1], np.geomspace(1, xmax, 120000)])
+        pdf = 2 * _gennorm_pdf(x, beta)
+        wts = np.zeros_like(x)
+        dx = np.diff(x)
+        wts[:-1] += 0.5 * dx * pdf[:-1]
+        wts[1:] += 0.5 * dx * pdf[1:]
+        quad = _fp4_mse(oracle, 2.0 ** (ir / 8.0), x, wts)
+        got = oracle.distortion(1, 2, ib, ir)
+        assert abs(got - quad) <= 2e-3 * quad, (ib, ir, got, quad)
+
+
+def test_optimal_bias_rule_minimises_the_realised_error(oracle):
+    """RULE_OPT picks, among all admissible integer biases, the one with the least model distortion,
+    and on sampled GenNorm data its realised squared error is the smallest (up to sampling noise)
+    and never above the polynomial rule's."""
+    rng = np.random.default_rng(21)
+    for (E, M), beta, alpha in (((1, 2), 1.6, 3e-3), ((1, 2), 0.6, 1e-3), ((3, 2), 1.0, 2e-2), ((4, 3), 0.8, 5e-4)):
+        g = (alpha * rng.gamma(1.0 / beta, 1.0, 200_000) ** (1.0 / beta) * rng.choice([-1.0, 1.0], 200_000))
+        g = g.astype(np.float32)[None, :]
+        N, S1, S2, _ = oracle.stats(g, np.zeros_like(g), 0, g.shape[1], 0.0)
+        be, al = oracle.fit(N, S1, S2)
+        b_opt, b_poly = oracle.bias_opt(be, al, E, M), oracle.bias(be, al, E, M)
+        ib, _ = oracle.header(be, al, b_opt)
+        t8 = math.floor(8 * math.log2(al) + 0.5)
+        lo, hi = oracle.b_range(E, M)
+        model = {b: oracle.distortion(E, M, ib, t8 - 8 * b) for b in range(lo, hi + 1) if -96 <= t8 - 8 * b <= 31}
+        assert b_opt == min(model, key=model.get)
+        mse = {}
+        for b in range(b_opt - 2, b_opt + 3):
+            m = np.zeros_like(g)
+            oracle.convert(g, m, np.zeros(g.shape, np.uint8), 0, g.shape[1], 0.0, E, M, b,
+                           np.zeros(1 << (1 + E + M), np.uint64))
+            mse[b] = float(np.sum(m.astype(np.float64) ** 2))
+        assert mse[b_opt] <= 1.02 * min(mse.values())
+        if b_poly in mse:
+            assert mse[b_opt] <= 1.001 * mse[b_poly]
+    assert oracle.bias_opt(1.0, 0.0, 4, 3) == oracle.b_range(4, 3)[0]
+    assert oracle.bias_opt(1.0, 1e300, 4, 3) == oracle.b_range(4, 3)[1]
+    assert oracle.bias_opt(1.3, 2.0 ** 5 * 1e-3, 3, 2) == oracle.bias_opt(1.3, 1e-3, 3, 2) + 5   # scale equivariance
