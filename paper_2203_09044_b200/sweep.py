@@ -42,6 +42,41 @@ def device_bytes_needed(wl, pool):
     return 4 * ud * pool + 4 * ud + ud + 2 * ud + 4 * wl.d
 
 
+def huffman_cost(counts):
+    """Total code bits of an (unrestricted-depth) Huffman code built from these symbol counts: the
+    sum of the weights of all internal nodes.  Symbols that do not occur get no codeword."""
+    import heapq
+    h = [int(c) for c in counts if c > 0]
+    if len(h) <= 1:
+        return float(sum(h))                            # one symbol still needs one bit each
+    heapq.heapify(h)
+    total = 0
+    while len(h) > 1:
+        a, b = heapq.heappop(h), heapq.heappop(h)
+        total += a + b
+        heapq.heappush(h, a + b)
+    return float(total)
+
+
+def code_mismatch(plan, out):
+    """Per element, pooled over segments and users, for the last encoded iteration: the entropy of
+    the symbol histogram, the bits of a Huffman code built from that histogram (what an
+    empirical-histogram variant would spend, its code table not counted), and the bits of the model
+    code actually used (histogram x code lengths of the rows the headers select)."""
+    import numpy as np
+    hist = plan.debug_hist().astype(np.float64)         # [S][nsym]
+    lens, _ = plan.debug_code(out["hdr"])               # [S][nsym]
+    n = hist.sum()
+    ent = 0.0
+    for row in hist:
+        t = row.sum()
+        p = row[row > 0] / t if t > 0 else row[:0]
+        ent += -float((p * np.log2(p)).sum()) * t
+    emp = sum(huffman_cost(row) for row in hist)
+    model = float((hist * lens).sum())
+    return ent / n, emp / n, model / n
+
+
 def measure(wl, iters, warm, pool, rule=0):
     """Run warm + iters iterations of one workload; returns a dict of figures."""
     wl.align_rows()
@@ -82,7 +117,9 @@ def measure(wl, iters, warm, pool, rule=0):
     # realised relative conversion error of the last iteration: the memory is a - Q(a) exactly
     err2 = float((residual[:, :d].double() ** 2).sum().item())
     s2 = sum(plan.get_fit(l)[4] for l in range(plan.S))
-    res = dict(rel_mse=err2 / s2 if s2 > 0 else 0.0, name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
+    ent_bits, emp_bits, model_bits = code_mismatch(plan, out)
+    res = dict(rel_mse=err2 / s2 if s2 > 0 else 0.0, ent_bits=ent_bits, emp_bits=emp_bits, model_bits=model_bits,
+               name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
                ms=ms, first_ms=first_ms, gbs=4.0 * U * d / (ms * 1e-3) / 1e9,
                convert_ms=prof.get("convert", 0.0),
                encode_ms=prof.get("enc_len", 0.0) + prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0),
@@ -96,8 +133,8 @@ def measure(wl, iters, warm, pool, rule=0):
 
 
 HEADER = ("| workload | d | U | format | beta | ms/iter | GB/s fp32 in | convert us | convert GB/s (13 B) | % of {peak:.0f} "
-          "| % of 8000 | encode us | decode us | decode+encode GB/s (payload+symbols+avg) | code b/el | container b/el | t=0 ms | rel. sq. error | note |\n"
-          "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+          "| % of 8000 | encode us | decode us | decode+encode GB/s (payload+symbols+avg) | code b/el | container b/el | t=0 ms | rel. sq. error | entropy b/el | Huffman(histogram) b/el | note |\n"
+          "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
 
 
 def row(r, peak):
@@ -112,11 +149,11 @@ def row(r, peak):
         note.append("inputs fit L2, launch-bound")
     if r["flags"]:
         note.append("flags=%d" % r["flags"])
-    return ("| %s | %d | %d | %s | %.1f | %.4f | %.1f | %.1f | %.0f | %.1f | %.1f | %.1f | %.1f | %.0f | %.3f | %.3f | %.3f | %.3e | %s |"
+    return ("| %s | %d | %d | %s | %.1f | %.4f | %.1f | %.1f | %.0f | %.1f | %.1f | %.1f | %.1f | %.0f | %.3f | %.3f | %.3f | %.3e | %.3f | %.3f | %s |"
             % (r["name"], r["d"], r["U"], r["fmt"], r["beta"], r["ms"], r["gbs"], r["convert_ms"] * 1e3, conv_gbs,
                100.0 * conv_gbs / peak, 100.0 * conv_gbs / NOMINAL_HBM_GBS, r["encode_ms"] * 1e3,
                r["decode_ms"] * 1e3, ed_gbs, r["code_bits"], r["container_bits"], r["first_ms"],
-               r.get("rel_mse", 0.0), "; ".join(note)))
+               r.get("rel_mse", 0.0), r.get("ent_bits", 0.0), r.get("emp_bits", 0.0), "; ".join(note)))
 
 
 def main(argv=None):
@@ -147,7 +184,7 @@ def main(argv=None):
     for wl in todo:
         pool = 2 if device_bytes_needed(wl, 2) <= args.max_bytes else 1
         if device_bytes_needed(wl, pool) > args.max_bytes:
-            lines.append("| %s | %d | %d | E%dM%d | %.1f | skipped: needs %.0f GB of device memory | | | | | | | | | | | | |"
+            lines.append("| %s | %d | %d | E%dM%d | %.1f | skipped: needs %.0f GB of device memory | | | | | | | | | | | | | | |"
                          % (wl.name, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.beta,
                             device_bytes_needed(wl, 1) / 1e9))
             continue

@@ -105,7 +105,10 @@ def test_sweep_report_helpers_need_no_gpu():
              encode_ms=0.03, fit_ms=0.01, decode_ms=0.03, code_bits=6.8, container_bits=6.95, flags=0, l2_resident=True)
     cells = [c.strip() for c in sweep.row(r, 6550.7).split("|")]
     assert cells[1] == "x" and cells[4] == "E4M3" and "launch-bound" in cells[-2]
-    assert float(cells[-3]) == 0.0                      # no realised error given: column printed as 0
+    assert float(cells[-5]) == 0.0                      # no realised error given: column printed as 0
+    # Huffman cost from counts: sum of internal node weights; dyadic counts cost exactly the entropy
+    assert sweep.huffman_cost([8, 4, 2, 1, 1]) == 8 * 1 + 4 * 2 + 2 * 3 + 1 * 4 + 1 * 4
+    assert sweep.huffman_cost([5, 0, 0]) == 5.0 and sweep.huffman_cost([3, 3, 3, 3]) == 24.0
     conv_gbs = 13.0 * 8 * (1 << 20) / 0.02e-3 / 1e9
     assert abs(float(cells[9]) - round(conv_gbs)) <= 1
 
