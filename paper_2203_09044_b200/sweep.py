@@ -132,6 +132,29 @@ def measure(wl, iters, warm, pool, rule=0):
     return res
 
 
+def gamma_sweep(wl, gammas, iters):
+    """Memory decay sweep (the quantity of the paper's Fig. 3 on synthetic streams): L1 norm of the
+    memory over L1 norm of the gradient after every iteration, per gamma, with the model update fused
+    into the decode (weights start at zero, step -0.01).  Returns {gamma: [ratio per iteration]}."""
+    U, d = wl.n_users, wl.d
+    out_rows = {}
+    for gamma in gammas:
+        plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=gamma, ld=wl.ld)
+        out = plan.alloc_outputs()
+        residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+        weights = torch.zeros(d, dtype=torch.float32, device="cuda")
+        ratios = []
+        for t in range(iters):
+            g = wl.gradient(t, device="cuda")
+            plan.encode(g, residual, out)
+            plan.decode_aggregate_update(out, weights, -0.01)
+            ratios.append(float(residual[:, :d].abs().sum().item() / g[:, :d].abs().sum().item()))
+        assert plan.status()[0] == 0
+        plan.close()
+        out_rows[gamma] = ratios
+    return out_rows
+
+
 HEADER = ("| workload | d | U | format | beta | ms/iter | GB/s fp32 in | convert us | convert GB/s (13 B) | % of {peak:.0f} "
           "| % of 8000 | encode us | decode us | decode+encode GB/s (payload+symbols+avg) | code b/el | container b/el | t=0 ms | rel. sq. error | entropy b/el | Huffman(histogram) b/el | note |\n"
           "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
@@ -165,10 +188,26 @@ def main(argv=None):
     ap.add_argument("--max-bytes", type=float, default=60e9, help="skip workloads needing more device memory")
     ap.add_argument("--rule", default="poly", choices=["poly", "opt"],
                     help="bias rule: the paper's polynomial (default) or the L2-optimal integer bias")
+    ap.add_argument("--gamma-sweep", action="store_true",
+                    help="instead: memory L1 / gradient L1 per iteration for gamma in {0, 0.1, 0.5, 0.9, 1} on "
+                         "configuration 1's layers in the 4-bit format")
     ap.add_argument("--filter", default=None, help="run only workloads whose name contains this text")
     ap.add_argument("--out", default=None, help="also write the table to this file")
     args = ap.parse_args(argv)
     binding.lib()                                       # no CUDA library: raise, never fall back
+    if args.gamma_sweep:
+        wl = inputs.workload(1).align_rows()
+        wl.exp_bits, wl.mant_bits = 1, 2                # the paper's 4-bit format, as in its gamma experiment
+        rows = gamma_sweep(wl, (0.0, 0.1, 0.5, 0.9, 1.0), 12)
+        lines = ["| gamma | " + " | ".join("t=%d" % t for t in range(12)) + " |", "|---|" + "---|" * 12]
+        for gm, r in rows.items():
+            lines.append("| %.1f | " % gm + " | ".join("%.4f" % x for x in r) + " |")
+        text = "\n".join(lines) + "\n"
+        if args.out:
+            with open(args.out, "w") as f:
+                f.write(text)
+        sys.stdout.write(text)
+        return 0
     peak, src = measured_hbm_gbs()
     lines = ["Peak used for the convert column: %.1f GB/s (%s copy bandwidth); nominal 8000 GB/s beside it." % (peak, src),
              "", HEADER.format(peak=peak)]
