@@ -65,6 +65,12 @@ extern "C" {
  * differs (by one iteration), at a rate that is higher by the drift of the model per iteration.
  * co3_debug_symbols is not available in this mode. */
 #define CO3_CODE_LAGGED 2
+/* Not the paper's code design (which builds the code from the fitted GenNorm model): the bias is
+ * handled as in CO3_BIAS_LAGGED, but the code of every layer is the Huffman code of this iteration's
+ * own symbol histogram (pooled over users, same construction as the model code: full alphabet, floor
+ * 1, depth at most 16), and the table of its code lengths is side information: 2^(1+E+M) bytes per
+ * layer per iteration.  Use co3_encode_empirical / co3_decode_aggregate_empirical with such a plan. */
+#define CO3_CODE_EMPIRICAL 3
 
 /* How the exponent bias follows from the fitted GenNorm (Sec. III (i)).
  * CO3_RULE_POLY: the paper's closed form (Eq. "approximate"): b = nearest integer to
@@ -101,7 +107,7 @@ typedef struct {
     int32_t n_segments;         /* S >= 1                                                          */
     const int64_t* seg_offsets; /* host, S+1 non-decreasing entries, [0] = 0, [S] = d; NULL: S = 1 */
     float gamma;                /* memory decay of Algorithm 1 line 8; 0: no feedback, 1: plain EF */
-    int32_t bias_mode;          /* CO3_BIAS_CURRENT, CO3_BIAS_LAGGED or CO3_CODE_LAGGED            */
+    int32_t bias_mode;          /* CO3_BIAS_CURRENT, CO3_BIAS_LAGGED, CO3_CODE_LAGGED, CO3_CODE_EMPIRICAL */
     int64_t cap_words;          /* row pitch of `bitstream` in 32-bit words, multiple of 4         */
     int32_t bias_rule;          /* CO3_RULE_POLY (the paper's, default 0) or CO3_RULE_OPT          */
     int32_t reserved;           /* 0                                                               */
@@ -145,6 +151,18 @@ int co3_encode(co3_plan* plan, const float* grad, float* residual, uint32_t* bit
 int co3_decode_aggregate(co3_plan* plan, const uint32_t* bitstream, const uint16_t* sub_bits,
                          const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
                          void* cuda_stream);
+
+/* The two calls for a CO3_CODE_EMPIRICAL plan (the others return CO3_EINVAL for it, and these for any
+ * other plan).  code_lens: device, [n_segments][2^(1+E+M)] u8, the code length of every symbol byte:
+ * written by the encoder, read by the decoder, which rebuilds the canonical codes from it and raises
+ * CO3_FLAG_CORRUPT if the lengths are not those of a complete prefix code of depth <= 16.  hdr is
+ * still written and read (the decoder needs the bias; the model indices are informational). */
+int co3_encode_empirical(co3_plan* plan, const float* grad, float* residual, uint32_t* bitstream,
+                         uint16_t* sub_bits, uint32_t* chunk_off, uint64_t* user_bits, co3_seg_header* hdr,
+                         uint8_t* code_lens, void* cuda_stream);
+int co3_decode_aggregate_empirical(co3_plan* plan, const uint32_t* bitstream, const uint16_t* sub_bits,
+                                   const uint32_t* chunk_off, const co3_seg_header* hdr,
+                                   const uint8_t* code_lens, float* avg_grad, void* cuda_stream);
 
 /* The same with the model update of Algorithm 1 line 14 fused in: besides avg_grad,
  * weights[i] <- fl32(weights[i] + fl32(step * avg_grad[i])) (device, in/out, [d] fp32; two roundings,

@@ -447,6 +447,21 @@ int co3o_huffman(const uint32_t* w, int n, uint8_t* len, uint32_t* floor_used) {
     return CO3O_OK;
 }
 
+/* Empirical-histogram variant: the code of a layer is the Huffman code of the symbol counts of
+ * this iteration (pooled over users), built exactly like the model code (full alphabet, floor 1 for
+ * symbols that did not occur, same tie-breaks and depth limit).  Counts are brought into 32 bits by
+ * dropping the k low bits that make the layer's total fit below 2^31. */
+int co3o_huffman_counts(const uint64_t* counts, int n, uint8_t* len, uint32_t* floor_used) {
+    if (n < 2 || n > 256) return CO3O_EINVAL;
+    uint64_t tot = 0;
+    for (int s = 0; s < n; s++) tot += counts[s];
+    int k = 0;
+    while ((tot >> k) >= ((uint64_t)1 << 31)) k++;
+    uint32_t w[256];
+    for (int s = 0; s < n; s++) w[s] = (uint32_t)(counts[s] >> k);
+    return co3o_huffman(w, n, len, floor_used);
+}
+
 /* Canonical codewords: symbols ordered by (length, symbol); code values as integers whose most
  * significant of `len` bits is the root branch. */
 void co3o_canonical(const uint8_t* len, int n, uint32_t* code) {
@@ -543,14 +558,16 @@ int co3o_encode_user(const uint8_t* sym, int64_t n_chunks, const int32_t* chunk_
  * alone, decode every user's stream and average,  avg = (1/U) sum_u ghat^(u)  (Eq. "aggregate").
  * The sum is taken over the integer magnitudes (exact) and scaled once:
  * avg = fl32( fl32(K_sum) * 2^lambda ) / fl32(U).
- * hdr is [S][3] int32: (b, ibeta, ir).  Returns CO3O_ECORRUPT if a sub-chunk does not decode to
- * exactly its recorded bit length or a chunk runs past its words. */
+ * hdr is [S][3] int32: (b, ibeta, ir).  With lens_in ([S][2^B] code lengths, the side information
+ * of the empirical-histogram code) the codes are the canonical codes of those lengths instead.
+ * Returns CO3O_ECORRUPT if a sub-chunk does not decode to exactly its recorded bit length, a chunk
+ * runs past its words, or given lengths are not those of a complete prefix code. */
 int co3o_decode_aggregate(const uint32_t* payload, int64_t cap_words, const uint16_t* sub_bits,
                           int64_t n_sub, const uint32_t* chunk_off, int U, int64_t n_chunks,
                           const int32_t* chunk_seg, const int64_t* chunk_start,
                           const int64_t* chunk_end, const int64_t* sub_base, int S,
                           const int32_t* hdr, int E, int M, float* avg, uint8_t* sym_out,
-                          int64_t sld) {
+                          int64_t sld, const uint8_t* lens_in) {
     int nsym = 1 << (1 + E + M), nm = E + M;
     uint8_t* len = (uint8_t*)malloc((size_t)S * (size_t)nsym);
     uint32_t* code = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)S * (size_t)nsym);
@@ -564,11 +581,22 @@ int co3o_decode_aggregate(const uint32_t* payload, int64_t cap_words, const uint
     int* sorted = (int*)malloc(sizeof(int) * (size_t)S * (size_t)nsym);
     int rc = CO3O_OK;
     for (int l = 0; l < S && rc == CO3O_OK; l++) {
-        rc = co3o_model_weights(E, M, hdr[3 * l + 1], hdr[3 * l + 2], w);
-        if (rc != CO3O_OK) break;
         uint8_t* L = len + (size_t)l * nsym;
         uint32_t* C = code + (size_t)l * nsym;
-        co3o_huffman(w, nsym, L, NULL);
+        if (lens_in) {                                  /* empirical code: the lengths are side information */
+            double kraft = 0.0;
+            for (int s = 0; s < nsym; s++) {
+                L[s] = lens_in[(size_t)l * nsym + s];
+                if (L[s] < 1 || L[s] > CO3O_MAXLEN) { rc = CO3O_ECORRUPT; break; }
+                kraft += ldexp(1.0, -(int)L[s]);
+            }
+            if (rc == CO3O_OK && kraft != 1.0) rc = CO3O_ECORRUPT;
+            if (rc != CO3O_OK) break;
+        } else {
+            rc = co3o_model_weights(E, M, hdr[3 * l + 1], hdr[3 * l + 2], w);
+            if (rc != CO3O_OK) break;
+            co3o_huffman(w, nsym, L, NULL);
+        }
         co3o_canonical(L, nsym, C);
         uint32_t *fi = first + (size_t)l * NL, *cn = count + (size_t)l * NL, *st = start + (size_t)l * NL;
         for (int s = 0; s < nsym; s++) cn[L[s]]++;

@@ -14,6 +14,8 @@ _lib = None
 
 MODE_CURRENT = 0   # bias b_t from the moments of a_t itself (a stats pass every iteration)
 MODE_LAGGED = 1    # stats pass at t = 0 only; b_t (t >= 1) from the fit of iteration t-1
+MODE_EMPIRICAL = 3    # bias as MODE_LAGGED; the code of a layer is the Huffman code of this iteration's symbol
+                      # histogram and its length table is side information (no GenNorm model in the code)
 MODE_LAGGED_CODE = 2  # as MODE_LAGGED, and the code model of iteration t (t >= 1) is the fit of iteration
                       # t-1 as well: the whole header of iteration t is known before g_t is seen
 
@@ -85,7 +87,10 @@ def lib():
     L.co3o_decode_aggregate.restype = C.c_int
     L.co3o_decode_aggregate.argtypes = [_u32p, _i64, _u16p, _i64, _u32p, C.c_int, _i64, _i32p,
                                         _i64p, _i64p, _i64p, C.c_int, _i32p, C.c_int, C.c_int,
-                                        _f32p, C.c_void_p, _i64]
+                                        _f32p, C.c_void_p, _i64, C.c_void_p]
+    L.co3o_huffman_counts.restype = C.c_int
+    L.co3o_huffman_counts.argtypes = [np.ctypeslib.ndpointer(np.uint64, flags="C_CONTIGUOUS"), C.c_int, _u8p,
+                                      C.POINTER(C.c_uint32)]
     _lib = L
     return L
 
@@ -206,6 +211,16 @@ def huffman(w):
     return ln, int(f.value)
 
 
+def huffman_counts(counts):
+    c = np.ascontiguousarray(counts, np.uint64)
+    ln = np.zeros(len(c), np.uint8)
+    f = C.c_uint32()
+    rc = lib().co3o_huffman_counts(c, len(c), ln, C.byref(f))
+    if rc != OK:
+        raise ValueError("co3o_huffman_counts: bad arguments")
+    return ln, int(f.value)
+
+
 def canonical(ln):
     ln = np.ascontiguousarray(ln, np.uint8)
     code = np.zeros(len(ln), np.uint32)
@@ -246,8 +261,9 @@ def encode_user(sym_row, part, nsym, lens, codes, cap_words):
     return rc, payload, sub_bits, chunk_off, int(ub.value)
 
 
-def decode_aggregate(payload, sub_bits, chunk_off, part, hdr, E, M, want_symbols=False):
-    """payload [U][cap], sub_bits [U][n_sub], chunk_off [U][n_chunks+1], hdr [S][3] int32."""
+def decode_aggregate(payload, sub_bits, chunk_off, part, hdr, E, M, want_symbols=False, lens=None):
+    """payload [U][cap], sub_bits [U][n_sub], chunk_off [U][n_chunks+1], hdr [S][3] int32;
+    lens [S][2^B] u8: the code lengths, when they are side information (empirical-histogram code)."""
     U, cap = payload.shape
     avg = np.zeros(part.d, np.float32)
     sym = np.zeros((U, part.d), np.uint8) if want_symbols else None
@@ -255,7 +271,8 @@ def decode_aggregate(payload, sub_bits, chunk_off, part, hdr, E, M, want_symbols
         np.ascontiguousarray(payload), cap, np.ascontiguousarray(sub_bits), sub_bits.shape[1],
         np.ascontiguousarray(chunk_off), U, part.n_chunks, part.chunk_seg, part.chunk_start,
         part.chunk_end, part.sub_base, part.S, np.ascontiguousarray(hdr, np.int32), E, M, avg,
-        sym.ctypes.data if want_symbols else None, part.d)
+        sym.ctypes.data if want_symbols else None, part.d,
+        None if lens is None else np.ascontiguousarray(lens, np.uint8).ctypes.data)
     return rc, avg, sym
 
 
@@ -327,8 +344,11 @@ class OracleCO3:
         codes = np.zeros((S, self.nsym), np.uint32)
         r.floor = np.zeros(S, np.int64)
         for l in range(S):
-            w = model_weights(E, M, int(hdr[l, 1]), int(hdr[l, 2]))
-            lens[l], r.floor[l] = huffman(w)
+            if self.mode == MODE_EMPIRICAL:
+                lens[l], r.floor[l] = huffman_counts(hist[l])
+            else:
+                w = model_weights(E, M, int(hdr[l, 1]), int(hdr[l, 2]))
+                lens[l], r.floor[l] = huffman(w)
             codes[l] = canonical(lens[l])
         cap = self.cap_words
         r.payload = np.zeros((U, max(cap, 1)), np.uint32)
@@ -354,6 +374,6 @@ class OracleCO3:
             weights += (np.float32(step) * avg).astype(np.float32)
         return rc, avg
 
-    def decode_aggregate(self, payload, sub_bits, chunk_off, hdr, want_symbols=False):
+    def decode_aggregate(self, payload, sub_bits, chunk_off, hdr, want_symbols=False, lens=None):
         return decode_aggregate(payload, sub_bits, chunk_off, self.part, hdr, self.E, self.M,
-                                want_symbols)
+                                want_symbols, lens)

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libco3.so")
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, ECORRUPT, ENONFINITE = 0, -1, -2, -3, -4, -5, -6
 FLAG_CAPACITY, FLAG_CORRUPT, FLAG_NONFINITE = 1, 2, 4
-BIAS_CURRENT, BIAS_LAGGED, CODE_LAGGED = 0, 1, 2
+BIAS_CURRENT, BIAS_LAGGED, CODE_LAGGED, CODE_EMPIRICAL = 0, 1, 2, 3
 RULE_POLY, RULE_OPT = 0, 1
 FLAG_TIMEOUT = 8
 
@@ -24,7 +24,7 @@ EXPORTS = [
     "co3_debug_symbols", "co3_debug_hist", "co3_debug_code", "co3_model_weights", "co3_partition",
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
     "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
-    "co3_bias_opt_table", "co3_grid_distortion",
+    "co3_bias_opt_table", "co3_grid_distortion", "co3_encode_empirical", "co3_decode_aggregate_empirical",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -74,6 +74,10 @@ def lib():
     L.co3_encode.argtypes = [vp] * 9
     L.co3_decode_aggregate.restype = C.c_int
     L.co3_decode_aggregate.argtypes = [vp] * 7
+    L.co3_encode_empirical.restype = C.c_int
+    L.co3_encode_empirical.argtypes = [vp] * 10
+    L.co3_decode_aggregate_empirical.restype = C.c_int
+    L.co3_decode_aggregate_empirical.argtypes = [vp] * 8
     L.co3_decode_aggregate_update.restype = C.c_int
     L.co3_decode_aggregate_update.argtypes = [vp] * 7 + [C.c_float, vp]
     L.co3_iteration_host.restype = C.c_int
@@ -218,6 +222,7 @@ class Plan:
             user_bits=t.zeros((self.U,), dtype=t.int64, device=device),
             hdr=t.zeros((self.S,), dtype=t.int32, device=device),
             avg=t.zeros((self.d,), dtype=t.float32, device=device),
+            code_lens=t.zeros((self.S, self.nsym), dtype=t.uint8, device=device),   # CODE_EMPIRICAL only
         )
 
     def _stream(self, stream):
@@ -226,17 +231,27 @@ class Plan:
 
     # ---- the C-ABI calls -------------------------------------------------------------------
     def encode(self, grad, residual, out, stream=None):
-        rc = lib().co3_encode(self.handle, _ptr(grad), _ptr(residual), _ptr(out["bitstream"]),
-                              _ptr(out["sub_bits"]), _ptr(out["chunk_off"]), _ptr(out["user_bits"]),
-                              _ptr(out["hdr"]), self._stream(stream))
+        if self.bias_mode == CODE_EMPIRICAL:
+            rc = lib().co3_encode_empirical(self.handle, _ptr(grad), _ptr(residual), _ptr(out["bitstream"]),
+                                            _ptr(out["sub_bits"]), _ptr(out["chunk_off"]), _ptr(out["user_bits"]),
+                                            _ptr(out["hdr"]), _ptr(out["code_lens"]), self._stream(stream))
+        else:
+            rc = lib().co3_encode(self.handle, _ptr(grad), _ptr(residual), _ptr(out["bitstream"]),
+                                  _ptr(out["sub_bits"]), _ptr(out["chunk_off"]), _ptr(out["user_bits"]),
+                                  _ptr(out["hdr"]), self._stream(stream))
         if rc != OK:
             raise Co3Error(rc, "co3_encode")
 
     def decode_aggregate(self, out, avg=None, stream=None):
         avg = out["avg"] if avg is None else avg
-        rc = lib().co3_decode_aggregate(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
-                                        _ptr(out["chunk_off"]), _ptr(out["hdr"]), _ptr(avg),
-                                        self._stream(stream))
+        if self.bias_mode == CODE_EMPIRICAL:
+            rc = lib().co3_decode_aggregate_empirical(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
+                                                      _ptr(out["chunk_off"]), _ptr(out["hdr"]),
+                                                      _ptr(out["code_lens"]), _ptr(avg), self._stream(stream))
+        else:
+            rc = lib().co3_decode_aggregate(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
+                                            _ptr(out["chunk_off"]), _ptr(out["hdr"]), _ptr(avg),
+                                            self._stream(stream))
         if rc != OK:
             raise Co3Error(rc, "co3_decode_aggregate")
         return avg

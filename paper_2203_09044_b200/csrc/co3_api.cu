@@ -25,11 +25,11 @@ int dev_alloc(co3_plan* pl, T** out, size_t count) {
     return CO3_OK;
 }
 
-int alloc_codebook(co3_plan* pl, Co3CodeBook& cb) {
-    const size_t R = CO3_NROWS;
+int alloc_codebook(co3_plan* pl, Co3CodeBook& cb, size_t R, int ncand) {
     int rc = 0;
-    rc |= dev_alloc(pl, &cb.cand_len, R * CO3_NCAND * CO3_MAXSYM);
-    rc |= dev_alloc(pl, &cb.cand_max, R * CO3_NCAND);
+    cb.ncand = ncand;
+    rc |= dev_alloc(pl, &cb.cand_len, R * (size_t)ncand * CO3_MAXSYM);
+    rc |= dev_alloc(pl, &cb.cand_max, R * (size_t)ncand);
     rc |= dev_alloc(pl, &cb.len8, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.len_pub, R * CO3_MAXSYM);
     rc |= dev_alloc(pl, &cb.enc, R * CO3_MAXSYM);
@@ -130,7 +130,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
     if (!co3_host_fmt_ok(cfg->fmt)) return CO3_EINVAL;
     if (cfg->d < 1 || cfg->ld < cfg->d || (cfg->ld & 3) || cfg->n_users < 1) return CO3_EINVAL;
     if (cfg->cap_words < 4 || (cfg->cap_words & 3) || cfg->cap_words > 0xFFFFFFFFLL) return CO3_EINVAL;
-    if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED && cfg->bias_mode != CO3_CODE_LAGGED) return CO3_EINVAL;
+    if (cfg->bias_mode != CO3_BIAS_CURRENT && cfg->bias_mode != CO3_BIAS_LAGGED && cfg->bias_mode != CO3_CODE_LAGGED && cfg->bias_mode != CO3_CODE_EMPIRICAL) return CO3_EINVAL;
     if (!(cfg->gamma >= 0.0f) || !(cfg->gamma <= 1.0f)) return CO3_EINVAL;
     if (cfg->bias_rule != CO3_RULE_POLY && cfg->bias_rule != CO3_RULE_OPT) return CO3_EINVAL;
     if (cfg->d > ((int64_t)1 << 31)) return CO3_EINVAL;
@@ -257,7 +257,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         }
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);
-        a |= alloc_codebook(pl, dv.cb);
+        a |= alloc_codebook(pl, dv.cb, CO3_NROWS, CO3_NCAND);
+        if (cfg->bias_mode == CO3_CODE_EMPIRICAL) a |= alloc_codebook(pl, pl->cb_emp, (size_t)S, CO3_NCAND_HIST);
         if (a) rc = CO3_ENOMEM;
         if (rc == CO3_OK) {
             cudaError_t e = cudaSuccess;
@@ -317,6 +318,7 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
                           co3_seg_header* hdr, void* cuda_stream) {
     if (!pl || !grad || !residual || !bitstream || !sub_bits || !chunk_off || !user_bits || !hdr) return CO3_EINVAL;
     if (((uintptr_t)grad | (uintptr_t)residual | (uintptr_t)bitstream) & 15) return CO3_EINVAL;
+    if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL && !pl->emp_lens) return CO3_EINVAL;   // use co3_encode_empirical
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
     if (pl->cfg.bias_mode == CO3_CODE_LAGGED) {
@@ -341,9 +343,20 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
     CO3_TRY(co3_launch_convert(pl, grad, residual, st));
     if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));   // the gradient buffer is free from here on
     CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
+    if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) CO3_TRY(co3_build_hist_codes(pl, pl->emp_lens, st));
     CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;
     return CO3_OK;
+}
+
+extern "C" int co3_encode_empirical(co3_plan* pl, const float* grad, float* residual, uint32_t* bitstream,
+                                    uint16_t* sub_bits, uint32_t* chunk_off, uint64_t* user_bits,
+                                    co3_seg_header* hdr, uint8_t* code_lens, void* cuda_stream) {
+    if (!pl || !code_lens || pl->cfg.bias_mode != CO3_CODE_EMPIRICAL) return CO3_EINVAL;
+    pl->emp_lens = code_lens;
+    const int rc = co3_encode(pl, grad, residual, bitstream, sub_bits, chunk_off, user_bits, hdr, cuda_stream);
+    pl->emp_lens = nullptr;
+    return rc;
 }
 
 extern "C" int co3_decode_aggregate(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
@@ -351,17 +364,29 @@ extern "C" int co3_decode_aggregate(co3_plan* pl, const uint32_t* bitstream, con
                                     void* cuda_stream) {
     if (!pl || !bitstream || !sub_bits || !chunk_off || !hdr || !avg_grad) return CO3_EINVAL;
     if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
+    if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL && !pl->emp_lens_in) return CO3_EINVAL;   // use ..._empirical
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
+    if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) CO3_TRY(co3_build_codes_from_lens(pl, pl->emp_lens_in, st));
     CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, nullptr, 0.0f, st));
     return CO3_OK;
+}
+
+extern "C" int co3_decode_aggregate_empirical(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
+                                              const uint32_t* chunk_off, const co3_seg_header* hdr,
+                                              const uint8_t* code_lens, float* avg_grad, void* cuda_stream) {
+    if (!pl || !code_lens || pl->cfg.bias_mode != CO3_CODE_EMPIRICAL) return CO3_EINVAL;
+    pl->emp_lens_in = code_lens;
+    const int rc = co3_decode_aggregate(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, cuda_stream);
+    pl->emp_lens_in = nullptr;
+    return rc;
 }
 
 extern "C" int co3_decode_aggregate_update(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                                            const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg_grad,
                                            float* weights, float step, void* cuda_stream) {
     if (!pl || !bitstream || !sub_bits || !chunk_off || !hdr || !avg_grad || !weights) return CO3_EINVAL;
-    if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
+    if ((uintptr_t)bitstream & 15 || pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) return CO3_EINVAL;
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
     CO3_TRY(co3_launch_decode(pl, bitstream, sub_bits, chunk_off, hdr, avg_grad, weights, step, st));

@@ -336,7 +336,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
         const Co3Group grp = p.groups[gi];
         const int gp = (int)(gi & 1);
         if (grp.seg != cur_seg) {                  // every warp is past the last decode with the old tables
-            load_tables(sm.t, p.cb, co3_row_of(hdr[grp.seg], &bad), tid);
+            load_tables(sm.t, p.cb, p.code_by_segment ? grp.seg : co3_row_of(hdr[grp.seg], &bad), tid);
             cur_seg = grp.seg;
         }
         const bool mine = ci < cpg && ci < grp.count;
@@ -435,7 +435,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     for (int64_t c = c0; c < c1; ++c) {
         const Co3Chunk cd = p.chunks[c];
         if (cd.seg != cur_seg) {
-            load_tables(sm.t, p.cb, co3_row_of(hdr[cd.seg], &bad), tid);
+            load_tables(sm.t, p.cb, p.code_by_segment ? cd.seg : co3_row_of(hdr[cd.seg], &bad), tid);
             cur_seg = cd.seg;
         }
         for (int i = tid; i < CO3_SUB * PADW / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(sm.acc)[i] = make_uint4(0, 0, 0, 0);
@@ -491,7 +491,8 @@ cudaError_t co3_setup_decode_kernels(void) {
 cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
                               float* weights, float step, cudaStream_t st) {
-    const Co3Dev& p = pl->dev;
+    Co3Dev p = pl->dev;
+    if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) { p.cb = pl->cb_emp; p.code_by_segment = 1; }
     co3_prof_begin(pl, CO3_K_DECODE, st);
     if (p.U <= NW) {
         const size_t smem = smem_a_bytes(p.U);

@@ -182,7 +182,7 @@ enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __
     Item it;
     open_item(it, p, tid, item);
     {
-        const size_t row = (size_t)co3_row_of(hdr[it.cd.seg], &bad) * CO3_MAXSYM;
+        const size_t row = (size_t)(p.code_by_segment ? it.cd.seg : co3_row_of(hdr[it.cd.seg], &bad)) * CO3_MAXSYM;
         reinterpret_cast<uint32_t*>(s_len)[tid] = reinterpret_cast<const uint32_t*>(p.cb.len8 + row)[tid];
         reinterpret_cast<uint4*>(s_enc)[tid] = __ldg(reinterpret_cast<const uint4*>(p.cb.enc + row) + tid);
     }
@@ -379,7 +379,8 @@ cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint
 cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
                               uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
                               cudaStream_t st) {
-    const Co3Dev& p = pl->dev;
+    Co3Dev p = pl->dev;
+    if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) { p.cb = pl->cb_emp; p.code_by_segment = 1; }
     const unsigned items = (unsigned)(p.n_chunks * (int64_t)p.U);
     // (tickets, published counts and group totals were cleared by the fit kernel that ran before)
     co3_prof_begin(pl, CO3_K_ENC_PACK, st);

@@ -182,24 +182,39 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
 
 // One (model row, weight floor 2^cand) pair per block: Huffman code lengths of the floored model
 // weights.  Leaves sorted by (weight, symbol); two queues; on equal weights the leaf goes first.
-__global__ void __launch_bounds__(CO3_MAXSYM) huff_cand_kernel(Co3Dev p) {
-    __shared__ uint32_t s_w[CO3_MAXSYM], s_sw[CO3_MAXSYM], s_iw[CO3_MAXSYM];
+// FROM_HIST: the row is a segment and the weights are this iteration's symbol counts (all copies of
+// the histogram added, low bits dropped until the segment's total is below 2^31).
+template <bool FROM_HIST>
+__global__ void __launch_bounds__(CO3_MAXSYM) huff_cand_kernel(Co3Dev p, Co3CodeBook cb) {
+    typedef unsigned long long W;                    // floors go up to 2^31: node weights need 64 bits
+    constexpr W NONE = ~(W)0;
+    __shared__ W s_w[CO3_MAXSYM], s_sw[CO3_MAXSYM], s_iw[CO3_MAXSYM];
     __shared__ uint16_t s_ssym[CO3_MAXSYM], s_parent[2 * CO3_MAXSYM];
     __shared__ int s_max;
     const int rowi = blockIdx.x, cand = blockIdx.y, tid = threadIdx.x, n = p.nsym;
-    const uint32_t* row = p.wtab + (size_t)rowi * p.J;
     if (tid == 0) s_max = 0;
     if (tid < n) {
-        const int j = tid & (p.J - 1);
-        const uint32_t w = ((tid >> p.nm) && j == 0) ? 1u : row[j];     // "-0" is never emitted
-        s_w[tid] = max(w, 1u << cand);
+        uint32_t w;
+        if (FROM_HIST) {
+            const unsigned long long tot = (unsigned long long)(p.seg_off[rowi + 1] - p.seg_off[rowi]) * (unsigned long long)p.U;
+            int k = 0;
+            while ((tot >> k) >= (1ull << 31)) ++k;
+            unsigned long long c = 0;
+            for (int h = 0; h < p.hist_copies; ++h)
+                c += p.hist[((size_t)h * p.S + rowi) * CO3_MAXSYM + co3_sym_internal(tid, p.nm)];
+            w = (uint32_t)(c >> k);
+        } else {
+            const int j = tid & (p.J - 1);
+            w = ((tid >> p.nm) && j == 0) ? 1u : p.wtab[(size_t)rowi * p.J + j];   // "-0" is never emitted
+        }
+        s_w[tid] = max((W)w, (W)1 << cand);
     }
     __syncthreads();
     if (tid < n) {
-        const uint32_t mine = s_w[tid];
+        const W mine = s_w[tid];
         int rank = 0;
         for (int s = 0; s < n; ++s) {
-            const uint32_t o = s_w[s];
+            const W o = s_w[s];
             rank += (o < mine) || (o == mine && s < tid);
         }
         s_sw[rank] = mine;
@@ -208,22 +223,22 @@ __global__ void __launch_bounds__(CO3_MAXSYM) huff_cand_kernel(Co3Dev p) {
     __syncthreads();
     if (tid == 0) {
         int i = 0, j = 0;
-        uint32_t lw = s_sw[0];                       // head of the leaf queue
-        uint32_t iw = 0xFFFFFFFFu;                   // head of the internal queue (none yet)
+        W lw = s_sw[0];                              // head of the leaf queue
+        W iw = NONE;                                 // head of the internal queue (none yet)
         for (int k = 0; k < n - 1; ++k) {
-            uint32_t sum = 0;
+            W sum = 0;
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
-                if (lw <= iw) {                      // leaf first on ties; UINT_MAX when exhausted
+                if (lw <= iw) {                      // leaf first on ties; NONE when exhausted
                     sum += lw;
                     s_parent[i] = (uint16_t)(n + k);
                     ++i;
-                    lw = (i < n) ? s_sw[i] : 0xFFFFFFFFu;
+                    lw = (i < n) ? s_sw[i] : NONE;
                 } else {
                     sum += iw;
                     s_parent[n + j] = (uint16_t)(n + k);
                     ++j;
-                    iw = (j < k) ? s_iw[j] : 0xFFFFFFFFu;
+                    iw = (j < k) ? s_iw[j] : NONE;
                 }
             }
             s_iw[k] = sum;
@@ -236,42 +251,57 @@ __global__ void __launch_bounds__(CO3_MAXSYM) huff_cand_kernel(Co3Dev p) {
         int node = tid, depth = 0;
         while (node != root && depth <= CO3_MAXLEN) { node = s_parent[node]; ++depth; }
         atomicMax(&s_max, depth);
-        p.cb.cand_len[((size_t)rowi * CO3_NCAND + cand) * CO3_MAXSYM + s_ssym[tid]] = (uint8_t)depth;
+        cb.cand_len[((size_t)rowi * cb.ncand + cand) * CO3_MAXSYM + s_ssym[tid]] = (uint8_t)depth;
     }
     __syncthreads();
-    if (tid == 0) p.cb.cand_max[rowi * CO3_NCAND + cand] = s_max;
+    if (tid == 0) cb.cand_max[rowi * cb.ncand + cand] = s_max;
 }
 
 // Per model row: take the smallest floor whose code is at most 16 deep, assign canonical
 // codewords (symbols ordered by (length, symbol)), and write the encoder table and the decoder
 // tables (11-bit primary table + canonical arrays for the rare longer codewords).
-__global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p) {
+// FROM_LENS: the lengths are given (lens_in, [rows][2^B] by public symbol: the side information of the
+// empirical-histogram code on the decoding side); lengths that are not those of a complete prefix
+// code raise CO3_FLAG_CORRUPT.  lens_out (may be null): the chosen lengths, same layout.
+template <bool FROM_LENS>
+__global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3CodeBook cb,
+                                                                   const uint8_t* __restrict__ lens_in,
+                                                                   uint8_t* __restrict__ lens_out) {
     __shared__ uint8_t s_len[CO3_MAXSYM], s_perm[CO3_MAXSYM];
     __shared__ uint32_t s_count[CO3_MAXLEN + 2], s_first[CO3_MAXLEN + 2], s_offs[CO3_MAXLEN + 2];
     __shared__ int s_sel;
-    const Co3CodeBook& cb = p.cb;
     const int rowi = blockIdx.x, tid = threadIdx.x, n = p.nsym;
-    if (tid == 0) {
-        int sel = CO3_NCAND - 1;
-        for (int c = 0; c < CO3_NCAND; ++c)
-            if (cb.cand_max[rowi * CO3_NCAND + c] <= CO3_MAXLEN) { sel = c; break; }
+    if (tid == 0 && !FROM_LENS) {
+        int sel = cb.ncand - 1;                          // the last floor always passes (see CO3_NCAND*)
+        for (int c = 0; c < cb.ncand; ++c)
+            if (cb.cand_max[rowi * cb.ncand + c] <= CO3_MAXLEN) { sel = c; break; }
         s_sel = sel;
     }
     if (tid < CO3_MAXLEN + 2) s_count[tid] = 0;
     __syncthreads();
     if (tid < n) {
-        const uint8_t L = cb.cand_len[((size_t)rowi * CO3_NCAND + s_sel) * CO3_MAXSYM + tid];
+        uint8_t L;
+        if (FROM_LENS) {
+            L = lens_in[(size_t)rowi * n + tid];
+            if (L < 1 || L > CO3_MAXLEN) { L = CO3_MAXLEN; atomicOr(p.flags, CO3_FLAG_CORRUPT); }
+        } else {
+            L = cb.cand_len[((size_t)rowi * cb.ncand + s_sel) * CO3_MAXSYM + tid];
+            if (L > CO3_MAXLEN) L = CO3_MAXLEN;            // cannot happen: the last floor passes
+            if (lens_out) lens_out[(size_t)rowi * n + tid] = L;
+        }
         s_len[tid] = L;
         atomicAdd(&s_count[L], 1u);
     }
     __syncthreads();
     if (tid == 0) {
-        uint32_t code = 0, off = 0;
+        uint32_t code = 0, off = 0, kraft = 0;
         for (int L = 1; L <= CO3_MAXLEN; ++L) {
             s_first[L] = code; s_offs[L] = off;
             code = (code + s_count[L]) << 1;
             off += s_count[L];
+            kraft += s_count[L] << (CO3_MAXLEN - L);
         }
+        if (FROM_LENS && kraft != (1u << CO3_MAXLEN)) atomicOr(p.flags, CO3_FLAG_CORRUPT);
     }
     __syncthreads();
     if (tid < n) {
@@ -343,9 +373,32 @@ cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStre
 // Builds the code tables of all model rows (plan creation).
 cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st) {
     dim3 grid(CO3_NROWS, CO3_NCAND);
-    huff_cand_kernel<<<grid, CO3_MAXSYM, 0, st>>>(pl->dev);
+    huff_cand_kernel<false><<<grid, CO3_MAXSYM, 0, st>>>(pl->dev, pl->dev.cb);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    code_finalize_kernel<<<CO3_NROWS, CO3_MAXSYM, 0, st>>>(pl->dev);
+    code_finalize_kernel<false><<<CO3_NROWS, CO3_MAXSYM, 0, st>>>(pl->dev, pl->dev.cb, nullptr, nullptr);
+    return cudaGetLastError();
+}
+
+// Empirical-histogram code, encoding side: one Huffman code per segment from the histogram the
+// convert pass has just filled; the lengths go to code_lens as well (the side information).
+cudaError_t co3_build_hist_codes(co3_plan* pl, uint8_t* code_lens, cudaStream_t st) {
+    dim3 grid(pl->dev.S, CO3_NCAND_HIST);
+    co3_prof_begin(pl, CO3_K_CODE_ENC, st);
+    huff_cand_kernel<true><<<grid, CO3_MAXSYM, 0, st>>>(pl->dev, pl->cb_emp);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) {
+        code_finalize_kernel<false><<<pl->dev.S, CO3_MAXSYM, 0, st>>>(pl->dev, pl->cb_emp, nullptr, code_lens);
+        e = cudaGetLastError();
+    }
+    co3_prof_end(pl, CO3_K_CODE_ENC, st, 2);
+    return e;
+}
+
+// Empirical-histogram code, decoding side: the tables of the canonical codes with the given lengths.
+cudaError_t co3_build_codes_from_lens(co3_plan* pl, const uint8_t* code_lens, cudaStream_t st) {
+    co3_prof_begin(pl, CO3_K_CODE_DEC, st);
+    code_finalize_kernel<true><<<pl->dev.S, CO3_MAXSYM, 0, st>>>(pl->dev, pl->cb_emp, code_lens, nullptr);
+    co3_prof_end(pl, CO3_K_CODE_DEC, st, 1);
     return cudaGetLastError();
 }

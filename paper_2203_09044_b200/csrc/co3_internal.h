@@ -10,7 +10,8 @@ constexpr int CO3_SUB = 128;        // sub-chunk grid (elements)
 constexpr int CO3_MAXLEN = 16;      // longest codeword
 constexpr int CO3_LUT_BITS = 11;    // primary decode table index width
 constexpr int CO3_LUT_SIZE = 1 << CO3_LUT_BITS;
-constexpr int CO3_NCAND = 10;       // weight floors 2^0 .. 2^9 tried in parallel (2^9 always passes)
+constexpr int CO3_NCAND = 10;       // model codes: weight floors 2^0 .. 2^9 tried in parallel (weights sum to ~2^20: 2^9 always passes)
+constexpr int CO3_NCAND_HIST = 32;  // codes from counts (total below 2^31): floors 2^0 .. 2^31 (2^31 makes all weights equal)
 constexpr int CO3_NIBETA = 23;      // ibeta in [-14, 8]
 constexpr int CO3_NIR = 128;        // ir in [-96, 31]
 constexpr int CO3_IBETA_MIN = -14, CO3_IBETA_MAX = 8, CO3_IR_MIN = -96, CO3_IR_MAX = 31;
@@ -48,8 +49,9 @@ struct Co3Group {
 constexpr int CO3_LONG_CACHE = 512;
 
 struct Co3CodeBook {
-    uint8_t* cand_len;   // [R][NCAND][256] code lengths per weight-floor candidate (build scratch)
-    int32_t* cand_max;   // [R][NCAND]      longest codeword per candidate (build scratch)
+    int ncand;           //                 weight-floor candidates of this book (NCAND or NCAND_HIST)
+    uint8_t* cand_len;   // [R][ncand][256] code lengths per weight-floor candidate (build scratch)
+    int32_t* cand_max;   // [R][ncand]      longest codeword per candidate (build scratch)
     uint8_t* len8;       // [R][256]        chosen lengths, by internal symbol
     uint8_t* len_pub;    // [R][256]        the same by public symbol (inspection only)
     uint32_t* enc;       // [R][256]        bit-reversed codeword | length << 16, by internal symbol
@@ -93,7 +95,9 @@ struct Co3Dev {
                                   //     each from bit 0 of its own slot, before their offsets are known (else null)
     const uint32_t* wtab;         // [NIBETA][NIR][J] model weights of the non-negative magnitudes
     const double* logr_tab;       // [2][FIT_GRID + 1] log R(beta), log G(beta) at log2(beta) uniform in [log2 0.3, 1]
-    Co3CodeBook cb;               // code tables of all model rows
+    Co3CodeBook cb;               // code tables the kernels use: of all model rows, or (empirical code,
+                                  // code_by_segment = 1) one row per segment, rebuilt every iteration
+    int code_by_segment;
     uint32_t* chunk_words;        // [U][n_chunks] payload words of each chunk (multiple of 4)   } fully lagged
     uint32_t* chunk_bits;         // [U][n_chunks] code bits of each chunk                        } code only
     uint32_t* user_ovf;           // [U] 1 if the user's payload exceeds cap_words
@@ -113,6 +117,9 @@ struct co3_plan {
     int64_t worst_case_words;
     int device;
     int num_sms;
+    Co3CodeBook cb_emp;             // empirical-histogram code: S rows (else unallocated)
+    uint8_t* emp_lens;              // ... the caller's length table during co3_encode_empirical
+    const uint8_t* emp_lens_in;     // ... and during co3_decode_aggregate_empirical
     size_t enc_sync_bytes;          // size of the enc_grp / enc_st / enc_ticket allocation
     int grid_stats, grid_convert;   // launch grids (fixed per plan: they define the reduction order)
     cudaStream_t last_stream;
@@ -122,7 +129,7 @@ struct co3_plan {
     bool host_pipe_ready;           // streams and events exist
     bool ev_conv_recorded;          // a convert pass that read d_grad has been recorded
     bool record_conv;               // co3_encode records ev_conv after its last pass over the gradient
-    void* allocs[64];
+    void* allocs[128];
     int n_allocs;
     int64_t* h_seg_off;
     // tracing
@@ -166,6 +173,10 @@ cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint
                                    unsigned long long* user_bits, cudaStream_t st);
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
 cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st);
+// empirical-histogram code: S codes from this iteration's histogram (lengths also to code_lens, device
+// [S][2^B]), or the tables of the codes whose lengths are given
+cudaError_t co3_build_hist_codes(co3_plan* pl, uint8_t* code_lens, cudaStream_t st);
+cudaError_t co3_build_codes_from_lens(co3_plan* pl, const uint8_t* code_lens, cudaStream_t st);
 cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
                               uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
                               cudaStream_t st);

@@ -65,7 +65,10 @@ def code_mismatch(plan, out):
     code actually used (histogram x code lengths of the rows the headers select)."""
     import numpy as np
     hist = plan.debug_hist().astype(np.float64)         # [S][nsym]
-    lens, _ = plan.debug_code(out["hdr"])               # [S][nsym]
+    if plan.bias_mode == binding.CODE_EMPIRICAL:
+        lens = out["code_lens"].cpu().numpy()           # the code is the length table itself
+    else:
+        lens, _ = plan.debug_code(out["hdr"])           # [S][nsym]
     n = hist.sum()
     ent = 0.0
     for row in hist:
@@ -77,12 +80,12 @@ def code_mismatch(plan, out):
     return ent / n, emp / n, model / n
 
 
-def measure(wl, iters, warm, pool, rule=0):
+def measure(wl, iters, warm, pool, rule=0, mode=None):
     """Run warm + iters iterations of one workload; returns a dict of figures."""
     wl.align_rows()
     U, d = wl.n_users, wl.d
     plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
-                        bias_mode=binding.BIAS_LAGGED, ld=wl.ld, bias_rule=rule)
+                        bias_mode=binding.BIAS_LAGGED if mode is None else mode, ld=wl.ld, bias_rule=rule)
     out = plan.alloc_outputs()
     residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
     grads = [wl.gradient(t, device="cuda") for t in range(pool)]
@@ -122,8 +125,9 @@ def measure(wl, iters, warm, pool, rule=0):
                name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
                ms=ms, first_ms=first_ms, gbs=4.0 * U * d / (ms * 1e-3) / 1e9,
                convert_ms=prof.get("convert", 0.0),
-               encode_ms=prof.get("enc_len", 0.0) + prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0),
-               fit_ms=prof.get("fit", 0.0), decode_ms=prof.get("decode", 0.0),
+               encode_ms=prof.get("enc_len", 0.0) + prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0)
+               + prof.get("code_enc", 0.0),
+               fit_ms=prof.get("fit", 0.0), decode_ms=prof.get("decode", 0.0) + prof.get("code_dec", 0.0),
                code_bits=code_bits, container_bits=container_bits, flags=flags,
                l2_resident=8.0 * U * d * pool < L2_BYTES)
     plan.close()
@@ -186,6 +190,8 @@ def main(argv=None):
     ap.add_argument("--iters", type=int, default=5, help="timed steady-state iterations per workload")
     ap.add_argument("--warm", type=int, default=3, help="untimed iterations before them (>= 1)")
     ap.add_argument("--max-bytes", type=float, default=60e9, help="skip workloads needing more device memory")
+    ap.add_argument("--mode", default="lagged", choices=["lagged", "current", "code-lagged", "empirical"],
+                    help="bias/code mode of the plans (default: lagged bias, the benchmark configuration)")
     ap.add_argument("--rule", default="poly", choices=["poly", "opt"],
                     help="bias rule: the paper's polynomial (default) or the L2-optimal integer bias")
     ap.add_argument("--gamma-sweep", action="store_true",
@@ -227,7 +233,10 @@ def main(argv=None):
                          % (wl.name, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.beta,
                             device_bytes_needed(wl, 1) / 1e9))
             continue
-        r = measure(wl, args.iters, max(args.warm, 1), pool, binding.RULE_OPT if args.rule == "opt" else binding.RULE_POLY)
+        mode = {"lagged": binding.BIAS_LAGGED, "current": binding.BIAS_CURRENT, "code-lagged": binding.CODE_LAGGED,
+                "empirical": binding.CODE_EMPIRICAL}[args.mode]
+        r = measure(wl, args.iters, max(args.warm, 1), pool,
+                    binding.RULE_OPT if args.rule == "opt" else binding.RULE_POLY, mode)
         lines.append(row(r, peak))
         print(lines[-1], flush=True)
     text = "\n".join(lines) + "\n"

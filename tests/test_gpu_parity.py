@@ -38,9 +38,12 @@ def compare_iteration(b, plan, out, r, m_gpu, m_cpu, tag=""):
         np.testing.assert_allclose([beta, alpha], r.fit[l], rtol=1e-5, err_msg=f"{tag} fit")
     hdr = b.hdr_to_numpy(out["hdr"])
     assert np.array_equal(hdr, r.hdr), f"{tag} header {hdr[hdr != r.hdr]} vs {r.hdr[hdr != r.hdr]}"
-    lens, codes = plan.debug_code(out["hdr"])
-    assert np.array_equal(lens, r.lens), f"{tag} code lengths"
-    assert np.array_equal(codes, r.codes), f"{tag} codewords"
+    if plan.bias_mode == b.CODE_EMPIRICAL:          # the code is the length table the encoder wrote
+        assert np.array_equal(out["code_lens"].cpu().numpy(), r.lens), f"{tag} code lengths (side information)"
+    else:
+        lens, codes = plan.debug_code(out["hdr"])
+        assert np.array_equal(lens, r.lens), f"{tag} code lengths"
+        assert np.array_equal(codes, r.codes), f"{tag} codewords"
     co = out["chunk_off"].cpu().numpy().view(np.uint32)
     assert np.array_equal(co, r.chunk_off), f"{tag} chunk offsets"
     assert np.array_equal(out["sub_bits"].cpu().numpy().view(np.uint16)[:, :plan.n_sub],
@@ -74,7 +77,8 @@ def run_case(b, oracle, d, U, E, M, off, grads, gamma=0.9, mode=1, cap=None, dec
         assert nf == r.nonfinite or t > 0
         if r.status == oracle.OK:
             avg = dec.decode_aggregate(out).cpu().numpy()
-            rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+            rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr,
+                                                lens=r.lens if mode == 3 else None)
             assert rc == oracle.OK
             assert np.array_equal(_bits(avg), _bits(avg_o)), f"t={t} averaged gradient"
             assert not (dec.status()[0] & b.FLAG_CORRUPT)
@@ -185,6 +189,56 @@ def test_fully_lagged_code_ragged_and_fp4(binding, oracle):
             g[:, :d] = torch.randn((U, d), generator=gen) * 1e-2
             grads.append(g.cuda())
         run_case(binding, oracle, d, U, E, M, off, grads, mode=2)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_empirical_histogram_code_configs_scaled_down(binding, oracle, idx):
+    """CO3_CODE_EMPIRICAL: per-iteration Huffman codes from the symbol histogram, built on the device,
+    length tables as side information; everything bit-exact against the oracle's mode, and the
+    decoder needs nothing but the stream, the header's bias and that table."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(idx, d={0: 70_001, 1: 200_000, 2: 150_010, 3: 300_007}[idx])
+    plan, orc, out, res = run_case(binding, oracle, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.seg_offsets,
+                                   _grads(wl, 3), gamma=wl.gamma, mode=3)
+    # a second plan that never encoded decodes the stream from its side information alone
+    dec = binding.Plan(wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.seg_offsets, bias_mode=3)
+    avg1 = plan.decode_aggregate(out).cpu().numpy()
+    avg2 = dec.decode_aggregate(out, avg=torch.zeros(wl.d, device="cuda")).cpu().numpy()
+    assert np.array_equal(_bits(avg1), _bits(avg2)) and dec.status()[0] == 0
+    # a length table that is not a complete prefix code is reported, never followed out of bounds
+    bad = dict(out)
+    bad["code_lens"] = out["code_lens"].clone()
+    bad["code_lens"][0, 1] = 0
+    dec.decode_aggregate(bad, avg=torch.zeros(wl.d, device="cuda"))
+    assert dec.status(clear=True)[0] & binding.FLAG_CORRUPT
+    bad["code_lens"] = out["code_lens"].clone()
+    bad["code_lens"][0, 2:5] = 1                    # three one-bit codewords: oversubscribed
+    dec.decode_aggregate(bad, avg=torch.zeros(wl.d, device="cuda"))
+    assert dec.status(clear=True)[0] & binding.FLAG_CORRUPT
+
+
+@pytest.mark.slow
+def test_empirical_histogram_code_needs_large_weight_floors(binding, oracle):
+    """A heavy-tailed layer of 67 million symbols: the unrestricted Huffman tree of its counts is far
+    deeper than 16, and the weight floor that limits it lies above 2^9 (the largest floor the model
+    codes ever need), so the device must try the same floors as the oracle, up to 2^31."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(3, d=1 << 24, n_users=4)
+    plan, orc, out, res = run_case(binding, oracle, wl.d, 4, 4, 3, wl.seg_offsets, _grads(wl, 1), mode=3)
+    assert int(res[0][0].floor[0]) > 512
+
+
+def test_empirical_histogram_code_ragged_fp4_many_users(binding, oracle):
+    gen = torch.Generator().manual_seed(26)
+    for d, off, U, E, M in ((1, [0, 1], 1, 4, 3), (10_000, [0, 1, 130, 4096, 4097, 9_999, 10_000], 3, 1, 2),
+                            (33_333, [0, 7, 8, 20_000, 33_333], 9, 3, 2)):
+        ld = (d + 3) // 4 * 4
+        grads = []
+        for t in range(2):
+            g = torch.zeros((U, ld))
+            g[:, :d] = torch.randn((U, d), generator=gen) * 1e-2
+            grads.append(g.cuda())
+        run_case(binding, oracle, d, U, E, M, off, grads, mode=3)
 
 
 def test_ragged_segments_and_tiny_inputs(binding, oracle):

@@ -645,3 +645,57 @@ def test_optimal_bias_rule_minimises_the_realised_error(oracle):
     assert oracle.bias_opt(1.0, 0.0, 4, 3) == oracle.b_range(4, 3)[0]
     assert oracle.bias_opt(1.0, 1e300, 4, 3) == oracle.b_range(4, 3)[1]
     assert oracle.bias_opt(1.3, 2.0 ** 5 * 1e-3, 3, 2) == oracle.bias_opt(1.3, 1e-3, 3, 2) + 5   # scale equivariance
+
+
+def test_empirical_histogram_code_mode(oracle):
+    """MODE_EMPIRICAL: symbols, residuals, biases and averages are those of MODE_LAGGED; the code of a
+    layer is the Huffman code of its symbol counts, so (while the depth limit is idle) its bits equal
+    the sum of the internal node weights of a Huffman tree of the counts and never exceed the model
+    code's; the stream decodes with the length table as side information and with nothing else."""
+    import heapq
+    d, U, E, M = 12_000, 3, 3, 2
+    runs = {}
+    for mode in (oracle.MODE_LAGGED, oracle.MODE_EMPIRICAL):
+        o = oracle.OracleCO3(d, U, E, M, [0, 5000, d], gamma=0.9, mode=mode)
+        m = np.zeros((U, d), np.float32)
+        rng = np.random.default_rng(8)
+        out = []
+        for t in range(3):
+            g = rng.laplace(0, 1e-3 * 1.5 ** t, (U, d)).astype(np.float32)
+            r = o.encode(g, m)
+            lens = r.lens if mode == oracle.MODE_EMPIRICAL else None
+            rc, avg, sym = o.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr, want_symbols=True, lens=lens)
+            assert rc == oracle.OK and np.array_equal(sym, r.sym)
+            out.append((r, avg, m.copy()))
+        runs[mode] = out
+    for t in range(3):
+        lag, emp = runs[oracle.MODE_LAGGED][t], runs[oracle.MODE_EMPIRICAL][t]
+        assert np.array_equal(lag[0].sym, emp[0].sym) and np.array_equal(lag[0].bias, emp[0].bias)
+        assert np.array_equal(lag[2], emp[2]) and np.array_equal(lag[1].view(np.uint32), emp[1].view(np.uint32))
+        r = emp[0]
+        for l in range(2):
+            counts = [int(c) for c in r.hist[l]]
+            h = [max(c, 1) for c in counts]                    # floor 1: every symbol keeps a codeword
+            heapq.heapify(h)
+            cost = 0
+            while len(h) > 1:
+                a, b = heapq.heappop(h), heapq.heappop(h)
+                cost += a + b
+                heapq.heappush(h, a + b)
+            floored_bits = int(sum(max(c, 1) * int(L) for c, L in zip(counts, r.lens[l])))
+            if r.floor[l] == 1:
+                assert floored_bits == cost                    # optimal for the floored counts
+            assert sum(2.0 ** -int(L) for L in r.lens[l]) == 1.0
+        assert int(emp[0].user_bits.sum()) <= int(lag[0].user_bits.sum())
+    # the model header alone does not decode an empirical stream
+    r = runs[oracle.MODE_EMPIRICAL][2][0]
+    o = oracle.OracleCO3(d, U, E, M, [0, 5000, d])
+    assert o.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)[0] == oracle.ECORRUPT
+    bad = r.lens.copy(); bad[0, 3] = 0
+    assert o.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr, lens=bad)[0] == oracle.ECORRUPT
+    bad = r.lens.copy(); bad[1, 5] += 1                         # no longer a complete code
+    assert o.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr, lens=bad)[0] == oracle.ECORRUPT
+    # counts above 32 bits are scaled, not wrapped
+    big = np.array([3 << 33, 1 << 33, 5, 0], np.uint64)
+    ln, f = oracle.huffman_counts(big)
+    assert list(ln) == [1, 2, 3, 3] and f == 1
