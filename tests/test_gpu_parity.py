@@ -417,6 +417,46 @@ def test_host_iteration_entry_point(binding, oracle):
         assert np.array_equal(_bits(h_avg.numpy()), _bits(avg_o))
 
 
+def test_steady_state_iteration_replays_from_a_cuda_graph(binding, oracle):
+    """After the first iteration (which has the extra statistics pass) an iteration is a fixed
+    sequence of memsets and kernels on one stream with no host decision in it, so it can be captured
+    once in a CUDA graph and replayed: the replays, fed through the captured input buffer, must be
+    the oracle's iterations bit for bit (state carried in device memory: residual, bias, tickets)."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=120_000, n_users=3)
+    plan = binding.Plan(wl.d, 3, 4, 3, wl.seg_offsets)
+    orc = oracle.OracleCO3(wl.d, 3, 4, 3, wl.seg_offsets, cap_words=plan.cap_words)
+    out = plan.alloc_outputs()
+    m = torch.zeros((3, plan.ld), device="cuda")
+    m_cpu = np.zeros((3, plan.ld), np.float32)
+    g_static = wl.gradient(0).cuda()                    # (drawn on the CPU: the same numbers as the oracle's)
+    plan.encode(g_static, m, out)                       # t = 0, eager
+    plan.decode_aggregate(out)
+    orc.encode(wl.gradient(0).numpy(), m_cpu)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):                       # t = 1 is captured (and not run)
+        plan.encode(g_static, m, out)
+        plan.decode_aggregate(out)
+    for t in range(1, 4):
+        g_static.copy_(wl.gradient(t))
+        graph.replay()
+        torch.cuda.synchronize()
+        r = orc.encode(wl.gradient(t).numpy(), m_cpu)
+        rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+        assert rc == oracle.OK
+        assert np.array_equal(b_hdr(binding, out), r.hdr), f"t={t} header"
+        n = int(out["chunk_off"][0, -1])
+        assert np.array_equal(out["bitstream"].cpu().numpy().view(np.uint32)[0, :n], r.payload[0, :n]), f"t={t}"
+        assert np.array_equal(_bits(out["avg"].cpu().numpy()), _bits(avg_o)), f"t={t} average"
+        assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_cpu)), f"t={t} memory"
+    assert plan.status()[0] == 0
+
+
+def b_hdr(binding, out):
+    return binding.hdr_to_numpy(out["hdr"])
+
+
 def test_host_iterations_back_to_back_overlap_their_copies(binding, oracle):
     """Four co3_iteration_host calls enqueued without any synchronisation in between (the copies of
     one call overlap the work of the previous one on the plan's own streams): every average and
