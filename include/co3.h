@@ -220,6 +220,10 @@ int co3_state_header(co3_plan* plan, int32_t import, co3_seg_header* next_header
 #define CO3_NUM_KERNELS 9
 int co3_profile_enable(co3_plan* plan, uint32_t kernel_mask, int32_t max_records);
 int co3_profile_collect(co3_plan* plan, double* total_ms, int64_t* launches);
+/* Time only every `every`-th launch of each traced class (default 1: all of them): two event records
+ * cost about as much device time as a small kernel, so a long timed loop may want to sample.
+ * co3_profile_collect then reports the sampled launches and their total. */
+int co3_profile_stride(co3_plan* plan, int32_t every);
 int64_t co3_launch_count(const co3_plan* plan);
 
 /* Inspection hooks (synchronise; used by the parity tests).

@@ -25,6 +25,7 @@ EXPORTS = [
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
     "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
     "co3_bias_opt_table", "co3_grid_distortion", "co3_encode_empirical", "co3_decode_aggregate_empirical",
+    "co3_profile_stride",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -102,6 +103,8 @@ def lib():
     L.co3_partition.argtypes = [C.c_int64, C.c_int32, vp, vp, vp, vp, vp, i64p]
     L.co3_profile_enable.restype = C.c_int
     L.co3_profile_enable.argtypes = [vp, C.c_uint32, C.c_int32]
+    L.co3_profile_stride.restype = C.c_int
+    L.co3_profile_stride.argtypes = [vp, C.c_int32]
     L.co3_profile_collect.restype = C.c_int
     L.co3_profile_collect.argtypes = [vp, vp, vp]
     L.co3_launch_count.restype = C.c_int64
@@ -329,6 +332,12 @@ class Plan:
         rc = lib().co3_profile_enable(self.handle, mask, max_records)
         if rc != OK:
             raise Co3Error(rc, "co3_profile_enable")
+
+    def profile_stride(self, every):
+        """Time only every `every`-th launch of each traced kernel class."""
+        rc = lib().co3_profile_stride(self.handle, int(every))
+        if rc != OK:
+            raise Co3Error(rc, "co3_profile_stride")
 
     def profile_collect(self):
         """{kernel class: (total ms, launches)} since the last collect (synchronises)."""

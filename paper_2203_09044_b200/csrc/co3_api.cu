@@ -91,6 +91,13 @@ extern "C" int co3_profile_enable(co3_plan* pl, uint32_t kernel_mask, int32_t ma
     return CO3_OK;
 }
 
+extern "C" int co3_profile_stride(co3_plan* pl, int32_t every) {
+    if (!pl || every < 1) return CO3_EINVAL;
+    pl->prof_every = every;
+    for (int k = 0; k < CO3_NUM_KERNELS; ++k) pl->prof_seen[k] = 0;
+    return CO3_OK;
+}
+
 extern "C" int co3_profile_collect(co3_plan* pl, double* total_ms, int64_t* launches) {
     if (!pl || !total_ms || !launches) return CO3_EINVAL;
     CO3_SYNC_OR_FAIL(pl);

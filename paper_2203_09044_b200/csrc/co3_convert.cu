@@ -12,8 +12,9 @@
 // ticket, so the grid as a whole sweeps one window of memory (with a fixed assignment of items to
 // blocks the blocks drift apart and a plain streaming kernel loses ~10 % of the bandwidth).  The
 // histogram lives in shared memory (one copy per warp, two sets used alternately) and is flushed
-// with 64-bit global atomics when the block leaves a segment; the moments are reduced in a fixed order per item and stored
-// per item, so the fit does not depend on which block converted which item.
+// with 64-bit global atomics (spread over several global copies) when the block leaves a segment;
+// the moments are reduced in a fixed order per item and stored per item, so the fit does not depend
+// on which block converted which item.
 //
 // Memory pipeline: a thread handles one 4-element vector of g and of m per step (4 steps per
 // item).  The loads are asynchronous copies (cp.async, 16 B, L2-only) into thread-private slots of

@@ -136,24 +136,30 @@ struct co3_plan {
     uint32_t prof_mask;
     int prof_cap;
     int prof_n[CO3_NUM_KERNELS];
+    int prof_every;               // only every prof_every-th launch of a class is timed (>= 1)
+    int64_t prof_seen[CO3_NUM_KERNELS];
+    bool prof_open[CO3_NUM_KERNELS];
     cudaEvent_t* prof_ev;         // [CO3_NUM_KERNELS][prof_cap][2]
     int64_t launches;
 };
 
 // Event pair around the launches of kernel class k (no-ops unless the class is being traced).
 inline void co3_prof_begin(co3_plan* pl, int k, cudaStream_t st) {
+    pl->prof_open[k] = false;
     if ((pl->prof_mask >> k) & 1u) {
-        if (pl->prof_n[k] < pl->prof_cap)
+        const int every = pl->prof_every > 1 ? pl->prof_every : 1;
+        if (pl->prof_seen[k]++ % every == 0 && pl->prof_n[k] < pl->prof_cap) {
             cudaEventRecord(pl->prof_ev[((size_t)k * pl->prof_cap + pl->prof_n[k]) * 2], st);
+            pl->prof_open[k] = true;
+        }
     }
 }
 inline void co3_prof_end(co3_plan* pl, int k, cudaStream_t st, int n_launches) {
     pl->launches += n_launches;
-    if ((pl->prof_mask >> k) & 1u) {
-        if (pl->prof_n[k] < pl->prof_cap) {
-            cudaEventRecord(pl->prof_ev[((size_t)k * pl->prof_cap + pl->prof_n[k]) * 2 + 1], st);
-            pl->prof_n[k]++;
-        }
+    if (pl->prof_open[k]) {
+        cudaEventRecord(pl->prof_ev[((size_t)k * pl->prof_cap + pl->prof_n[k]) * 2 + 1], st);
+        pl->prof_n[k]++;
+        pl->prof_open[k] = false;
     }
 }
 
