@@ -142,6 +142,26 @@ int co3_encode(co3_plan* plan, const float* grad, float* residual, uint32_t* bit
                uint16_t* sub_bits, uint32_t* chunk_off, uint64_t* user_bits, co3_seg_header* hdr,
                void* cuda_stream);
 
+/* The same iteration fed in tiles of users, for gradients of all users that do not fit the device
+ * at once (residual, payload and side information still cover all users and stay resident; only the
+ * gradient buffer holds a tile and is refilled by the caller between calls):
+ *   co3_tiled_begin       starts the iteration; *need_statistics = 1 if the bias has to come from a
+ *                         statistics pass first (t = 0, or CO3_BIAS_CURRENT)
+ *   co3_tiled_statistics  (only then) once for every tile: grad_tile is [n_tile_users][ld] for the
+ *                         users user0 .. user0 + n_tile_users - 1, residual the full [U][ld] array
+ *   co3_tiled_convert     once for every tile, after all statistics calls: as co3_encode's convert
+ *                         step for those users
+ *   co3_tiled_finish      fit, header, coding of all users; the iteration counter advances
+ * Every user must be covered exactly once per pass; the result is bit for bit that of co3_encode.
+ * Not available with CO3_CODE_LAGGED and CO3_CODE_EMPIRICAL plans. */
+int co3_tiled_begin(co3_plan* plan, int32_t* need_statistics);
+int co3_tiled_statistics(co3_plan* plan, const float* grad_tile, const float* residual, int32_t user0,
+                         int32_t n_tile_users, void* cuda_stream);
+int co3_tiled_convert(co3_plan* plan, const float* grad_tile, float* residual, int32_t user0,
+                      int32_t n_tile_users, void* cuda_stream);
+int co3_tiled_finish(co3_plan* plan, uint32_t* bitstream, uint16_t* sub_bits, uint32_t* chunk_off,
+                     uint64_t* user_bits, co3_seg_header* hdr, void* cuda_stream);
+
 /* Algorithm 1 lines 13-14 without the model update: decode all U streams and write
  * avg_grad[i] = (1/U) sum_u ghat^(u)[i] (Eq. "aggregate"), device [d] fp32.  Depends only on
  * its arguments and the plan's static configuration, never on encoder scratch.  The integer

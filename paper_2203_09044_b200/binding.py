@@ -25,7 +25,7 @@ EXPORTS = [
     "co3_strerror", "co3_profile_enable", "co3_profile_collect", "co3_launch_count",
     "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
     "co3_bias_opt_table", "co3_grid_distortion", "co3_encode_empirical", "co3_decode_aggregate_empirical",
-    "co3_profile_stride",
+    "co3_profile_stride", "co3_tiled_begin", "co3_tiled_statistics", "co3_tiled_convert", "co3_tiled_finish",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -103,6 +103,14 @@ def lib():
     L.co3_partition.argtypes = [C.c_int64, C.c_int32, vp, vp, vp, vp, vp, i64p]
     L.co3_profile_enable.restype = C.c_int
     L.co3_profile_enable.argtypes = [vp, C.c_uint32, C.c_int32]
+    L.co3_tiled_begin.restype = C.c_int
+    L.co3_tiled_begin.argtypes = [vp, C.POINTER(C.c_int32)]
+    L.co3_tiled_statistics.restype = C.c_int
+    L.co3_tiled_statistics.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp]
+    L.co3_tiled_convert.restype = C.c_int
+    L.co3_tiled_convert.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp]
+    L.co3_tiled_finish.restype = C.c_int
+    L.co3_tiled_finish.argtypes = [vp] * 7
     L.co3_profile_stride.restype = C.c_int
     L.co3_profile_stride.argtypes = [vp, C.c_int32]
     L.co3_profile_collect.restype = C.c_int
@@ -244,6 +252,28 @@ class Plan:
                                   _ptr(out["hdr"]), self._stream(stream))
         if rc != OK:
             raise Co3Error(rc, "co3_encode")
+
+    def encode_tiled(self, tile_users, make_tile, residual, out, stream=None):
+        """One iteration with the gradient supplied tile by tile: make_tile(user0, n) returns the
+        [n][ld] fp32 cuda gradient of users user0 .. user0 + n - 1 (it may reuse one buffer: each tile
+        is consumed by kernels enqueued on the stream before the next make_tile call returns work on
+        that same stream).  Bit for bit the result of encode() on the whole gradient."""
+        need = C.c_int32()
+        rc = lib().co3_tiled_begin(self.handle, C.byref(need))
+        if rc != OK:
+            raise Co3Error(rc, "co3_tiled_begin")
+        passes = (["co3_tiled_statistics"] if need.value else []) + ["co3_tiled_convert"]
+        for name in passes:
+            for u0 in range(0, self.U, tile_users):
+                n = min(tile_users, self.U - u0)
+                g = make_tile(u0, n)
+                rc = getattr(lib(), name)(self.handle, _ptr(g), _ptr(residual), u0, n, self._stream(stream))
+                if rc != OK:
+                    raise Co3Error(rc, name)
+        rc = lib().co3_tiled_finish(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]), _ptr(out["chunk_off"]),
+                                    _ptr(out["user_bits"]), _ptr(out["hdr"]), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_tiled_finish")
 
     def decode_aggregate(self, out, avg=None, stream=None):
         avg = out["avg"] if avg is None else avg

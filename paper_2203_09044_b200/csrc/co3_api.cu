@@ -214,6 +214,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         while ((Kmax >> bl) != 0) ++bl;
         dv.b_hi = (100 - bl) - dv.cF;
         dv.U = cfg->n_users; dv.S = S; dv.d = cfg->d; dv.ld = cfg->ld;
+        dv.u_base = 0; dv.u_count = cfg->n_users;
         dv.sld = (cfg->d + CO3_TILE - 1) / CO3_TILE * CO3_TILE;
         dv.n_chunks = nc; dv.n_sub = n_sub; dv.n_groups = n_groups; dv.cap_words = cfg->cap_words;
         dv.gamma = cfg->gamma;
@@ -332,7 +333,7 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
         // The header of this iteration was fixed by the previous one (at t = 0: by a statistics pass),
         // so conversion and packing are one pass; the fit that follows prepares the next iteration.
         if (pl->iteration == 0) {
-            CO3_TRY(co3_launch_stats(pl, grad, residual, st));
+            CO3_TRY(co3_launch_stats(pl, grad, residual, 0, pl->dev.U, st));
             CO3_TRY(co3_launch_fit(pl, 2, pl->dev.hdr_cur, st));
         }
         CO3_TRY(cudaMemcpyAsync(hdr, pl->dev.hdr_cur, sizeof(co3_seg_header) * (size_t)pl->dev.S, cudaMemcpyDeviceToDevice, st));
@@ -344,15 +345,72 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
         return CO3_OK;
     }
     if (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) {
-        CO3_TRY(co3_launch_stats(pl, grad, residual, st));
+        CO3_TRY(co3_launch_stats(pl, grad, residual, 0, pl->dev.U, st));
         CO3_TRY(co3_launch_fit(pl, 0, hdr, st));
     }
-    CO3_TRY(co3_launch_convert(pl, grad, residual, st));
+    CO3_TRY(co3_launch_convert(pl, grad, residual, 0, pl->dev.U, true, st));
     if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));   // the gradient buffer is free from here on
     CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) CO3_TRY(co3_build_hist_codes(pl, pl->emp_lens, st));
     CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;
+    return CO3_OK;
+}
+
+// ---- one iteration in tiles of users (gradients that do not fit the device at once) -------------
+extern "C" int co3_tiled_begin(co3_plan* pl, int32_t* need_statistics) {
+    if (!pl || !need_statistics) return CO3_EINVAL;
+    if (pl->cfg.bias_mode != CO3_BIAS_CURRENT && pl->cfg.bias_mode != CO3_BIAS_LAGGED) return CO3_EINVAL;
+    pl->tiled_state = 1;
+    pl->tiled_users = 0;
+    *need_statistics = (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) ? 1 : 0;
+    return CO3_OK;
+}
+
+static int tile_args_ok(const co3_plan* pl, const float* grad_tile, const float* residual, int32_t user0, int32_t n) {
+    if (!pl || !grad_tile || !residual || user0 < 0 || n < 1 || user0 + n > pl->dev.U) return 0;
+    if (((uintptr_t)grad_tile | (uintptr_t)residual) & 15) return 0;
+    return 1;
+}
+
+extern "C" int co3_tiled_statistics(co3_plan* pl, const float* grad_tile, const float* residual, int32_t user0,
+                                    int32_t n_tile_users, void* cuda_stream) {
+    if (!tile_args_ok(pl, grad_tile, residual, user0, n_tile_users)) return CO3_EINVAL;
+    if (pl->tiled_state != 1 && pl->tiled_state != 2) return CO3_EINVAL;       // before any convert tile
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    CO3_TRY(co3_launch_stats(pl, grad_tile, residual, user0, n_tile_users, st));
+    pl->tiled_state = 2;
+    return CO3_OK;
+}
+
+extern "C" int co3_tiled_convert(co3_plan* pl, const float* grad_tile, float* residual, int32_t user0,
+                                 int32_t n_tile_users, void* cuda_stream) {
+    if (!tile_args_ok(pl, grad_tile, residual, user0, n_tile_users)) return CO3_EINVAL;
+    if (pl->tiled_state < 1) return CO3_EINVAL;
+    const bool need_stats = pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT;
+    if (pl->tiled_state == 1 && need_stats) return CO3_EINVAL;                 // the statistics tiles come first
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    const bool first = pl->tiled_state != 3;
+    if (first && need_stats) CO3_TRY(co3_launch_fit(pl, 0, nullptr, st));       // bias from the pooled statistics
+    CO3_TRY(co3_launch_convert(pl, grad_tile, residual, user0, n_tile_users, first, st));
+    pl->tiled_state = 3;
+    pl->tiled_users += n_tile_users;
+    return CO3_OK;
+}
+
+extern "C" int co3_tiled_finish(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits, uint32_t* chunk_off,
+                                uint64_t* user_bits, co3_seg_header* hdr, void* cuda_stream) {
+    if (!pl || !bitstream || !sub_bits || !chunk_off || !user_bits || !hdr) return CO3_EINVAL;
+    if ((uintptr_t)bitstream & 15) return CO3_EINVAL;
+    if (pl->tiled_state != 3 || pl->tiled_users != pl->dev.U) return CO3_EINVAL;   // every user exactly once
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
+    CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
+    pl->iteration++;
+    pl->tiled_state = 0;
     return CO3_OK;
 }
 

@@ -140,7 +140,10 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
     __shared__ Co3Chunk s_chunk[2];                   // descriptor of the chunk of s_ticket[.]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.U;
+    // (a launch may cover only the users [u_base, u_base + u_count): the gradient pointer is then that
+    // tile's, everything else is indexed by the user's number in the plan)
+    const uint32_t n_items = (uint32_t)p.n_chunks * (uint32_t)p.u_count;
+    const uint32_t item_base = (uint32_t)p.n_chunks * (uint32_t)p.u_base;
     const uint32_t n_chunks = (uint32_t)p.n_chunks;
     constexpr int VSTRIDE = 4 * CO3_THREADS;          // elements between a thread's vectors
 
@@ -163,10 +166,10 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
     __syncthreads();                                  // both tickets read before slot 0 is reused
 
     auto make_ctx = [&](uint32_t it, const Co3Chunk& cd) {
-        const uint32_t uu = it / n_chunks;
+        const uint32_t ul = it / n_chunks, uu = ul + (uint32_t)p.u_base;
         ItemCtx x;
         const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-        x.gp = g + (size_t)uu * p.ld + tb + 4 * tid;
+        x.gp = g + (size_t)ul * p.ld + tb + 4 * tid;
         x.mp = m + (size_t)uu * p.ld + tb + 4 * tid;
         x.sp = p.sym + (size_t)uu * p.sld + tb + 4 * tid;
         x.lo = (int)(cd.start - tb);
@@ -354,7 +357,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
             uint32_t tn = 0;
 #pragma unroll
             for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
-            p.part_s1[item] = t1; p.part_s2[item] = t2; p.part_nf[item] = tn;
+            p.part_s1[item_base + item] = t1; p.part_s2[item_base + item] = t2; p.part_nf[item_base + item] = tn;
         }
         // When the block leaves the segment (or ends) its histogram goes to global memory; the next
         // item counts in the other copy, and this copy is not touched again before a later barrier.
@@ -423,25 +426,35 @@ cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_
     return cudaGetLastError();
 }
 
-cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st) {
+// u_base / u_count: the users this launch covers (g is then the gradient of those users only).
+cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u_base, int u_count, cudaStream_t st) {
     ef_fn fn = pick_kernel<0>(pl->dev.M);
     if (!pl->grid_stats) pl->grid_stats = ef_grid(pl, fn, RING_BYTES);
     cudaError_t e = cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
+    Co3Dev p = pl->dev;
+    p.u_base = u_base; p.u_count = u_count;
+    const int64_t items = p.n_chunks * (int64_t)u_count;
     co3_prof_begin(pl, CO3_K_STATS, st);
-    fn<<<pl->grid_stats, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, const_cast<float*>(m), nullptr);
+    fn<<<(int)(items < pl->grid_stats ? items : pl->grid_stats), CO3_THREADS, RING_BYTES, st>>>(p, g, const_cast<float*>(m), nullptr);
     co3_prof_end(pl, CO3_K_STATS, st, 1);
     return cudaGetLastError();
 }
 
-cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st) {
+// first: this launch starts the iteration's histogram (later tiles of the same iteration add to it)
+cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, int u_base, int u_count, bool first,
+                               cudaStream_t st) {
     // one memset clears the histogram and the item ticket that follows it in the same allocation
-    cudaError_t e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st);
+    cudaError_t e = first ? cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st)
+                          : cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     ef_fn fn = pick_kernel<1>(pl->dev.M);
     if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn, RING_BYTES);
+    Co3Dev p = pl->dev;
+    p.u_base = u_base; p.u_count = u_count;
+    const int64_t items = p.n_chunks * (int64_t)u_count;
     co3_prof_begin(pl, CO3_K_CONVERT, st);
-    fn<<<pl->grid_convert, CO3_THREADS, RING_BYTES, st>>>(pl->dev, g, m, nullptr);
+    fn<<<(int)(items < pl->grid_convert ? items : pl->grid_convert), CO3_THREADS, RING_BYTES, st>>>(p, g, m, nullptr);
     co3_prof_end(pl, CO3_K_CONVERT, st, 1);
     return cudaGetLastError();
 }

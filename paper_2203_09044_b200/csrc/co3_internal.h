@@ -73,6 +73,7 @@ struct Co3Dev {
     int E, M, nm, nsym, J, cF, b_lo, b_hi;
     uint32_t Kmax;
     int U, S;
+    int u_base, u_count;          // users covered by a statistics / convert launch (whole plan: 0, U)
     int64_t d, ld, sld, n_chunks, n_sub, n_groups, cap_words;
     float gamma;
     const Co3Chunk* chunks;       // [n_chunks]
@@ -128,6 +129,8 @@ struct co3_plan {
     cudaEvent_t ev_h2d, ev_conv, ev_dec, ev_d2h;
     bool host_pipe_ready;           // streams and events exist
     bool ev_conv_recorded;          // a convert pass that read d_grad has been recorded
+    int tiled_state;                // co3_tiled_*: 0 idle, 1 begun, 2 statistics tiles seen, 3 convert tiles seen
+    int tiled_users;                // users converted so far in this tiled iteration
     bool record_conv;               // co3_encode records ev_conv after its last pass over the gradient
     void* allocs[128];
     int n_allocs;
@@ -172,8 +175,9 @@ const double* co3_host_logr_table(void);               // [2][FIT_GRID + 1], cac
 const int16_t* co3_host_bias_opt_table(int E, int M);   // [NIBETA][8], cached per format
 
 // kernel launchers (each returns a cudaError_t from the launch)
-cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, cudaStream_t st);
-cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, cudaStream_t st);
+cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u_base, int u_count, cudaStream_t st);
+cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, int u_base, int u_count, bool first,
+                               cudaStream_t st);
 cudaError_t co3_launch_convert_pack(co3_plan* pl, const float* g, float* m, uint16_t* sub_bits, cudaStream_t st);
 cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint16_t* sub_bits, uint32_t* chunk_off,
                                    unsigned long long* user_bits, cudaStream_t st);

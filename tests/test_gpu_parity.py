@@ -417,6 +417,47 @@ def test_host_iteration_entry_point(binding, oracle):
         assert np.array_equal(_bits(h_avg.numpy()), _bits(avg_o))
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("tile", [1, 2, 4])
+def test_iteration_in_tiles_of_users(binding, oracle, mode, tile):
+    """The gradient supplied in tiles of users through ONE reused tile buffer (co3_tiled_*): every
+    output of every iteration is bit for bit what the oracle gets from the whole gradient."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=90_000, n_users=5)
+    plan = binding.Plan(wl.d, 5, 4, 3, wl.seg_offsets, bias_mode=mode)
+    orc = oracle.OracleCO3(wl.d, 5, 4, 3, wl.seg_offsets, mode=mode, cap_words=plan.cap_words)
+    out = plan.alloc_outputs()
+    m_gpu = torch.zeros((5, plan.ld), device="cuda")
+    m_cpu = np.zeros((5, plan.ld), np.float32)
+    buf = torch.empty((tile, plan.ld), device="cuda")
+    for t in range(3):
+        g = wl.gradient(t)
+
+        def make_tile(u0, n):
+            buf[:n].copy_(g[u0:u0 + n])
+            return buf
+
+        plan.encode_tiled(tile, make_tile, m_gpu, out)
+        r = orc.encode(g.numpy(), m_cpu)
+        compare_iteration(binding, plan, out, r, m_gpu, m_cpu, tag=f"tile={tile} t={t}")
+        avg = plan.decode_aggregate(out).cpu().numpy()
+        rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
+        assert rc == oracle.OK and np.array_equal(_bits(avg), _bits(avg_o))
+    assert plan.status()[0] == 0
+    # misuse is refused: a convert tile before the statistics tiles, a user twice, a finish too early
+    fresh = binding.Plan(wl.d, 5, 4, 3, wl.seg_offsets, bias_mode=mode)
+    L = binding.lib()
+    import ctypes as C
+    need = C.c_int32()
+    assert L.co3_tiled_begin(fresh.handle, C.byref(need)) == 0 and need.value == 1
+    p_buf, p_m = C.c_void_p(buf.data_ptr()), C.c_void_p(m_gpu.data_ptr())
+    assert L.co3_tiled_convert(fresh.handle, p_buf, p_m, 0, 1, None) == binding.EINVAL
+    assert L.co3_tiled_statistics(fresh.handle, p_buf, p_m, 4, 2, None) == binding.EINVAL   # beyond the last user
+    o = fresh.alloc_outputs()
+    ptrs = [C.c_void_p(o[k].data_ptr()) for k in ("bitstream", "sub_bits", "chunk_off", "user_bits", "hdr")]
+    assert L.co3_tiled_finish(fresh.handle, *ptrs, None) == binding.EINVAL
+
+
 def test_steady_state_iteration_replays_from_a_cuda_graph(binding, oracle):
     """After the first iteration (which has the extra statistics pass) an iteration is a fixed
     sequence of memsets and kernels on one stream with no host decision in it, so it can be captured
