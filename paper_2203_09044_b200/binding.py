@@ -253,11 +253,13 @@ class Plan:
         if rc != OK:
             raise Co3Error(rc, "co3_encode")
 
-    def encode_tiled(self, tile_users, make_tile, residual, out, stream=None):
+    def encode_tiled(self, tile_users, make_tile, residual, out, stream=None, around_call=None):
         """One iteration with the gradient supplied tile by tile: make_tile(user0, n) returns the
         [n][ld] fp32 cuda gradient of users user0 .. user0 + n - 1 (it may reuse one buffer: each tile
         is consumed by kernels enqueued on the stream before the next make_tile call returns work on
-        that same stream).  Bit for bit the result of encode() on the whole gradient."""
+        that same stream).  Bit for bit the result of encode() on the whole gradient.
+        around_call(False) / around_call(True), if given, run right before / after every library call
+        (a timing hook: whatever make_tile does stays outside)."""
         need = C.c_int32()
         rc = lib().co3_tiled_begin(self.handle, C.byref(need))
         if rc != OK:
@@ -267,11 +269,19 @@ class Plan:
             for u0 in range(0, self.U, tile_users):
                 n = min(tile_users, self.U - u0)
                 g = make_tile(u0, n)
+                if around_call:
+                    around_call(False)
                 rc = getattr(lib(), name)(self.handle, _ptr(g), _ptr(residual), u0, n, self._stream(stream))
+                if around_call:
+                    around_call(True)
                 if rc != OK:
                     raise Co3Error(rc, name)
+        if around_call:
+            around_call(False)
         rc = lib().co3_tiled_finish(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]), _ptr(out["chunk_off"]),
                                     _ptr(out["user_bits"]), _ptr(out["hdr"]), self._stream(stream))
+        if around_call:
+            around_call(True)
         if rc != OK:
             raise Co3Error(rc, "co3_tiled_finish")
 

@@ -36,10 +36,66 @@ def measured_hbm_gbs():
         return 6650.0, "fallback"
 
 
-def device_bytes_needed(wl, pool):
-    """Gradients (pool copies), memory, symbols, worst-case payload and the average."""
+def device_bytes_needed(wl, pool, tile_users=None):
+    """Gradients (pool copies, or two tiles of users), memory, symbols, worst-case payload and the average."""
     ud = wl.n_users * wl.d
-    return 4 * ud * pool + 4 * ud + ud + 2 * ud + 4 * wl.d
+    grads = 4 * ud * pool if tile_users is None else 2 * 4 * tile_users * wl.d
+    return grads + 4 * ud + ud + 2 * ud + 4 * wl.d
+
+
+def measure_tiled(wl, iters, warm, tile_users, rule=0):
+    """As measure(), for a workload whose gradients do not fit at once: every iteration is fed in
+    tiles of users, each drawn on the device right before it is consumed.  Only the library calls are
+    timed (event pairs around each); drawing the gradients is not."""
+    wl.align_rows()
+    U, d = wl.n_users, wl.d
+    plan = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma, ld=wl.ld, bias_rule=rule)
+    out = plan.alloc_outputs()
+    residual = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+    pairs = []
+
+    def around(after):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        if after:
+            pairs[-1].append(ev)
+        else:
+            pairs.append([ev])
+
+    def run(t):
+        del pairs[:]
+        plan.encode_tiled(tile_users, lambda u0, n: wl.gradient(t, device="cuda", users=range(u0, u0 + n)),
+                          residual, out, around_call=around)
+        around(False)
+        plan.decode_aggregate(out)
+        around(True)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in pairs)
+
+    first_ms = run(0)
+    for t in range(1, warm):
+        run(t)
+    plan.profile_enable(None, max_records=(2 * (U // tile_users + 2)) * iters + 8)
+    ms = sum(run(warm + t) for t in range(iters)) / iters
+    prof = {k: v[0] / iters for k, v in plan.profile_collect().items() if v[1]}
+    plan.profile_enable([], 0)
+    flags, _ = plan.status(clear=True)
+    code_bits = float(out["user_bits"].sum().item()) / (U * d)
+    container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
+                      + 32.0 * U * (plan.n_chunks + 1) + 32.0 * plan.S) / (U * d)
+    err2 = float(sum((residual[u, :d].double() ** 2).sum().item() for u in range(U)))
+    s2 = sum(plan.get_fit(l)[4] for l in range(plan.S))
+    ent_bits, emp_bits, model_bits = code_mismatch(plan, out)
+    res = dict(rel_mse=err2 / s2 if s2 > 0 else 0.0, ent_bits=ent_bits, emp_bits=emp_bits, model_bits=model_bits,
+               name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
+               ms=ms, first_ms=first_ms, gbs=4.0 * U * d / (ms * 1e-3) / 1e9, convert_ms=prof.get("convert", 0.0),
+               encode_ms=prof.get("enc_pack", 0.0), fit_ms=prof.get("fit", 0.0), decode_ms=prof.get("decode", 0.0),
+               code_bits=code_bits, container_bits=container_bits, flags=flags, l2_resident=False,
+               tiled=tile_users)
+    plan.close()
+    del out, residual
+    torch.cuda.empty_cache()
+    return res
 
 
 def huffman_cost(counts):
@@ -176,6 +232,8 @@ def row(r, peak):
         note.append("inputs fit L2, launch-bound")
     if r["flags"]:
         note.append("flags=%d" % r["flags"])
+    if r.get("tiled"):
+        note.append("gradients fed in tiles of %d users (co3_tiled_*), drawn per tile, drawing not timed" % r["tiled"])
     return ("| %s | %d | %d | %s | %.1f | %.4f | %.1f | %.1f | %.0f | %.1f | %.1f | %.1f | %.1f | %.0f | %.3f | %.3f | %.3f | %.3e | %.3f | %.3f | %s |"
             % (r["name"], r["d"], r["U"], r["fmt"], r["beta"], r["ms"], r["gbs"], r["convert_ms"] * 1e3, conv_gbs,
                100.0 * conv_gbs / peak, 100.0 * conv_gbs / NOMINAL_HBM_GBS, r["encode_ms"] * 1e3,
@@ -190,6 +248,10 @@ def main(argv=None):
     ap.add_argument("--iters", type=int, default=5, help="timed steady-state iterations per workload")
     ap.add_argument("--warm", type=int, default=3, help="untimed iterations before them (>= 1)")
     ap.add_argument("--max-bytes", type=float, default=60e9, help="skip workloads needing more device memory")
+    ap.add_argument("--tile-users", type=int, default=0,
+                    help="workloads over --max-bytes: feed the gradients in tiles of this many users if that "
+                         "fits --max-tiled-bytes (0: skip them)")
+    ap.add_argument("--max-tiled-bytes", type=float, default=150e9)
     ap.add_argument("--mode", default="lagged", choices=["lagged", "current", "code-lagged", "empirical"],
                     help="bias/code mode of the plans (default: lagged bias, the benchmark configuration)")
     ap.add_argument("--rule", default="poly", choices=["poly", "opt"],
@@ -228,6 +290,13 @@ def main(argv=None):
         todo = [wl for wl in todo if args.filter in wl.name]
     for wl in todo:
         pool = 2 if device_bytes_needed(wl, 2) <= args.max_bytes else 1
+        if device_bytes_needed(wl, pool) > args.max_bytes and args.tile_users > 0 and args.mode == "lagged" \
+                and device_bytes_needed(wl, 1, args.tile_users) <= args.max_tiled_bytes:
+            r = measure_tiled(wl, args.iters, max(args.warm, 1), args.tile_users,
+                              binding.RULE_OPT if args.rule == "opt" else binding.RULE_POLY)
+            lines.append(row(r, peak))
+            print(lines[-1], flush=True)
+            continue
         if device_bytes_needed(wl, pool) > args.max_bytes:
             lines.append("| %s | %d | %d | E%dM%d | %.1f | skipped: needs %.0f GB of device memory | | | | | | | | | | | | | | |"
                          % (wl.name, wl.d, wl.n_users, wl.exp_bits, wl.mant_bits, wl.beta,
