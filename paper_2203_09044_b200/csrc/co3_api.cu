@@ -243,6 +243,21 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         a |= dev_alloc(pl, &dv.part_s2, items);
         a |= dev_alloc(pl, &dv.part_nf, items);
         a |= dev_alloc(pl, &dv.fit, (size_t)S * 5);
+        {   // segments with more than 2^15 (user, chunk) pairs: sum their partials in slices first
+            int64_t max_pairs = 0;
+            for (int l = 0; l < S; ++l) {
+                const int64_t pairs = (int64_t)(h_seg_chunk0[l + 1] - h_seg_chunk0[l]) * dv.U;
+                if (pairs > max_pairs) max_pairs = pairs;
+            }
+            dv.red_k = 0;
+            if (max_pairs > (1 << 15)) {
+                const int64_t k = (max_pairs + 8191) / 8192;
+                dv.red_k = (int)(k > 512 ? 512 : k);
+                a |= dev_alloc(pl, &dv.red_s1, (size_t)S * dv.red_k);
+                a |= dev_alloc(pl, &dv.red_s2, (size_t)S * dv.red_k);
+                a |= dev_alloc(pl, &dv.red_nf, (size_t)S * dv.red_k);
+            }
+        }
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
         int16_t* d_opt = nullptr;
         const int16_t* h_opt = co3_host_bias_opt_table(E, M);

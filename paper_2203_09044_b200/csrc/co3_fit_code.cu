@@ -24,6 +24,50 @@ __device__ __forceinline__ double poly_bias(double b) {
     return 0.46 - 2.85 * b + 5.37 * b2 - 2.85 * b2 * b + 0.52 * b2 * b2;
 }
 
+// Plans with very long segments (millions of (user, chunk) pairs): slice blockIdx.x of segment
+// blockIdx.y adds its contiguous share of the pairs, in a fixed order, so that the fit kernel has
+// only red_k numbers per segment left to add.
+constexpr int RED_THREADS = 256;
+__global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int clear_enc_sync) {
+    __shared__ double s_a[RED_THREADS / 32], s_b[RED_THREADS / 32];
+    __shared__ unsigned long long s_n[RED_THREADS / 32];
+    const int seg = blockIdx.y, slice = blockIdx.x, tid = threadIdx.x;
+    if (clear_enc_sync) {                              // (see fit_kernel: here the many blocks share that job)
+        const size_t nb = (size_t)gridDim.x * gridDim.y, b = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+        for (size_t i = b * RED_THREADS + tid; i < p.enc_sync_words64; i += nb * RED_THREADS) p.enc_grp[i] = 0ull;
+    }
+    const int c0 = p.seg_chunk0[seg], nck = p.seg_chunk0[seg + 1] - c0;
+    const long long npairs = (long long)nck * p.U;
+    const long long per = (npairs + p.red_k - 1) / p.red_k;
+    const long long lo = per * slice, hi = min(npairs, lo + per);
+    double a1 = 0.0, a2 = 0.0;
+    unsigned long long an = 0;
+#pragma unroll 4
+    for (long long k = lo + tid; k < hi; k += RED_THREADS) {
+        const long long u = k / nck;
+        const size_t i = (size_t)u * (size_t)p.n_chunks + c0 + (size_t)(k - u * nck);
+        a1 += p.part_s1[i];
+        a2 += p.part_s2[i];
+        an += p.part_nf[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a1 += __shfl_down_sync(0xffffffffu, a1, o);
+        a2 += __shfl_down_sync(0xffffffffu, a2, o);
+        an += __shfl_down_sync(0xffffffffu, an, o);
+    }
+    if ((tid & 31) == 0) { s_a[tid >> 5] = a1; s_b[tid >> 5] = a2; s_n[tid >> 5] = an; }
+    __syncthreads();
+    if (tid == 0) {
+        double t1 = 0.0, t2 = 0.0;
+        unsigned long long tn = 0;
+#pragma unroll
+        for (int w = 0; w < RED_THREADS / 32; ++w) { t1 += s_a[w]; t2 += s_b[w]; tn += s_n[w]; }
+        const size_t o = (size_t)seg * p.red_k + slice;
+        p.red_s1[o] = t1; p.red_s2[o] = t2; p.red_nf[o] = tn;
+    }
+}
+
 // mode 0: after the stats pass -- write the bias for the coming convert pass.
 // mode 1: after the convert pass -- write the header (bias used, ibeta, ir), keep the fit, and
 //         store the bias the rule gives for these moments as the next iteration's bias.
@@ -39,7 +83,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     __shared__ int s_state, s_coarse, s_fine;
 
     const int seg = blockIdx.x, tid = threadIdx.x;
-    if (mode == 1) {
+    if (mode == 1 && p.red_k == 0) {
         // side job: the single-pass encode that follows this launch wants its tickets, published
         // counts and group totals at zero
         unsigned long long* z = p.enc_grp;
@@ -47,17 +91,27 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     }
     const int c0 = p.seg_chunk0[seg], c1 = p.seg_chunk0[seg + 1];
     // fixed order: thread t takes the (user, chunk) pairs t, t + 512, ... of the segment, all loads
-    // independent; then lanes, then warps
+    // independent; then lanes, then warps.  (Plans with very long segments: the pairs were summed in
+    // red_k slices by fit_reduce_kernel, and the slices are added here.)
     const int nck = c1 - c0, npairs = nck * p.U;
     double a1 = 0.0, a2 = 0.0;
     unsigned long long an = 0;
+    if (p.red_k > 0) {
+        for (int k = tid; k < p.red_k; k += FIT_THREADS) {
+            const size_t i = (size_t)seg * p.red_k + k;
+            a1 += p.red_s1[i];
+            a2 += p.red_s2[i];
+            an += p.red_nf[i];
+        }
+    } else {
 #pragma unroll 4
-    for (int k = tid; k < npairs; k += FIT_THREADS) {
-        const int u = k / nck, c = c0 + (k - u * nck);
-        const size_t i = (size_t)u * (size_t)p.n_chunks + c;
-        a1 += p.part_s1[i];
-        a2 += p.part_s2[i];
-        an += p.part_nf[i];
+        for (int k = tid; k < npairs; k += FIT_THREADS) {
+            const int u = k / nck, c = c0 + (k - u * nck);
+            const size_t i = (size_t)u * (size_t)p.n_chunks + c;
+            a1 += p.part_s1[i];
+            a2 += p.part_s2[i];
+            an += p.part_nf[i];
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -365,8 +419,9 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
     co3_prof_begin(pl, CO3_K_FIT, st);
+    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.red_k, pl->dev.S), RED_THREADS, 0, st>>>(pl->dev, mode == 1);
     fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr);
-    co3_prof_end(pl, CO3_K_FIT, st, 1);
+    co3_prof_end(pl, CO3_K_FIT, st, pl->dev.red_k > 0 ? 2 : 1);
     return cudaGetLastError();
 }
 

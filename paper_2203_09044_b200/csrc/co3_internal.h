@@ -88,6 +88,10 @@ struct Co3Dev {
     double* part_s2;              //              ... of a^2
     uint32_t* part_nf;            //              ... count of non-finite a
     double* fit;                  // [S][5] beta, alpha, N, S1, S2
+    int red_k;                    // > 0: the partials of a segment are first summed in red_k slices by
+    double* red_s1;               //      fit_reduce_kernel ([S][red_k] each) -- plans with very long segments
+    double* red_s2;
+    unsigned long long* red_nf;
     int32_t* bias_cur;            // [S] bias used by the next convert pass
     int bias_rule;                // CO3_RULE_POLY or CO3_RULE_OPT
     const int16_t* bias_opt_tab;  // [NIBETA][8] best ir per (shape index, round(8 log2 alpha) mod 8)
