@@ -173,21 +173,43 @@ def run_ours(args):
     assert flags == 0, f"status flags {flags} after warm-up"
 
     # ---- timed region: K steps, the dominant kernel traced with CUDA events --------------------
+    # A steady-state step is a fixed sequence of memsets and kernels with no host decision in it, so
+    # it is captured once per gradient batch in a CUDA graph.  Every CONVERT_TIMED_EVERY-th step of the
+    # timed region is launched eagerly with an event pair around its convert launch (the roofline
+    # figure); the steps between are graph replays, which save the launch gaps between the dependent
+    # kernels.  --no-graph launches every step eagerly.
+    graphs = None
+    per_step_launches = 0
+    if not args.no_graph:
+        graphs = []
+        for i in range(POOL):
+            n0 = plan.launch_count()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr):
+                step(i)
+            per_step_launches = plan.launch_count() - n0
+            graphs.append(gr)
+        barrier()
     plan.profile_enable(["convert"], max_records=args.steps)
-    plan.profile_stride(CONVERT_TIMED_EVERY)            # event pairs are not free: sample the launches
+    plan.profile_stride(1 if graphs else CONVERT_TIMED_EVERY)
     sampler = ClockSampler(physical_gpu_index(local_rank))
     launches0 = plan.launch_count()
+    replays = 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     sampler.start()
     e0.record()
     for t in range(args.steps):
-        step(args.warmup + t)
+        if graphs is None or t % CONVERT_TIMED_EVERY == 0:
+            step(args.warmup + t)
+        else:
+            graphs[(args.warmup + t) % POOL].replay()
+            replays += 1
     e1.record()
     barrier()
     clocks = sampler.stop()
     elapsed_ms = e0.elapsed_time(e1)
-    launches = plan.launch_count() - launches0
+    launches = plan.launch_count() - launches0 + replays * per_step_launches
     conv_ms, conv_n = plan.profile_collect()["convert"]
     flags, _ = plan.status(clear=True)
     assert flags == 0, f"status flags {flags} in the timed region"
@@ -208,9 +230,7 @@ def run_ours(args):
     plan.profile_enable([], 0)
 
     # ---- the same steps replayed from a CUDA graph (one graph = one pass over the gradient pool) --
-    # A steady-state step is a fixed sequence of memsets and kernels, so it can be captured once; the
-    # replay saves the launch gaps between the dependent kernels.  Reported beside `value`, which
-    # stays the eagerly launched number (its convert launches are event-timed one by one).
+    # All steps from one graph, no eager step in between: what the loop costs without any launch gap.
     graph_ms = None
     if world == 1 and not args.no_graph:
         graph = torch.cuda.CUDAGraph()
@@ -270,6 +290,9 @@ def run_ours(args):
                                        "code-lagged": "lagged bias and code (single-pass encode)"}[args.mode]),
                    "d": d, "n_users": U, "n_segments": plan.S, "format": "E4M3", "gamma": wl.gamma,
                    "bias_mode": args.mode, "replicas": world, "row_stride": plan.ld,
+                   "launch": ("every step launched eagerly" if graphs is None else
+                              "every %d-th step launched eagerly (its convert launch event-timed), the others "
+                              "replayed from one-step CUDA graphs" % CONVERT_TIMED_EVERY),
                    "l2": "inputs larger than L2: %d MB of gradient+memory read per step, %d gradient "
                          "batches cycled" % (8 * U * d // 1000000, POOL)},
         "clocks": clocks,
@@ -285,8 +308,8 @@ def run_ours(args):
                      "traffic": CONVERT_DRAM_TRAFFIC_BYTES_8_USERS * U / 8.0 if args.mode != "code-lagged" else None,
                      "algorithmic_bytes_per_launch": conv_bytes * U * d,
                      "avg_launch_ms": conv_avg_ms, "launches_timed": conv_n,
-                     "timing": "cudaEvent pair around every %d-th launch on the launching stream, inside the timed "
-                               "region" % CONVERT_TIMED_EVERY},
+                     "timing": "cudaEvent pair around the convert launch of every %d-th step, on the launching "
+                               "stream, inside the timed region" % CONVERT_TIMED_EVERY},
         "elements_per_s": world * U * d * args.steps / (elapsed_ms * 1e-3),
         "bits_per_element": {"code": code_bits, "container": container_bits},
         "whole_step_hbm": {"algorithmic_bytes_per_step": step_bytes,
