@@ -185,7 +185,8 @@ def run_ours(args):
         for i in range(POOL):
             n0 = plan.launch_count()
             gr = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gr):
+            # thread_local: only this thread launches; another thread (NCCL's watchdog) may query events
+            with torch.cuda.graph(gr, capture_error_mode="thread_local"):
                 step(i)
             per_step_launches = plan.launch_count() - n0
             graphs.append(gr)
@@ -234,7 +235,7 @@ def run_ours(args):
     graph_ms = None
     if world == 1 and not args.no_graph:
         graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
             for t in range(POOL):
                 step(t)
         n_rep = max(1, args.steps // POOL)
