@@ -1,9 +1,9 @@
 // Parameter-server side (Algorithm 1 lines 13-14 up to the model update, Eq. "aggregate"):
 // decode every user's stream and write the average of the reconstructed gradients.
 //
-// A lane decodes one sub-chunk (<= 128 codewords) serially with an 11-bit primary table whose
-// entries already hold the signed integer magnitude ((K << 8) | length) -- codewords longer than 11
-// bits go through a second table in global memory; the 32 sub-chunks of a
+// A lane decodes one sub-chunk (<= 128 codewords) serially with a primary table (13 or 11 index bits)
+// whose entries already hold the signed integer magnitude ((K << 8) | length) -- longer codewords
+// go through a second table in global memory; the 32 sub-chunks of a
 // chunk are the 32 lanes of a warp, so a warp is one (chunk, user) stream.  The magnitudes of all
 // users are accumulated with shared-memory reductions into a transposed, padded tile
 // (conflict-free both for the per-lane scattered adds and for the coalesced read-out), scaled
@@ -15,11 +15,15 @@
 // as shift amount (only its low five bits count), the bit buffer is topped up once per pair of
 // symbols, and four symbols are decoded per loop trip with immediate accumulator offsets.
 //
-// Two variants: U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
+// Three variants.  U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
 // per sub-chunk (small double-buffered accumulator, several chunks per block when U < 8); the
 // whole table entries are accumulated (the length bytes of at most 8 users cannot carry into
-// the magnitude) and the magnitude sum is taken out with one shift at the end.  U > 8 keeps a
-// whole chunk accumulator and loops over user groups.
+// the magnitude) and the magnitude sum is taken out with one shift at the end.  U = 8 runs four
+// such 8-warp teams in one block of 1024 threads: they share one 13-bit table (with 11 bits one
+// group of 128 look-ups in eight still meets a longer codeword and leaves the fast path, which also
+// makes the warps of a team wait for each other), each team has its own named barrier, and the whole
+// block synchronises only where the segment (the table) changes.  U > 8 keeps a whole chunk
+// accumulator and loops over user groups.
 //
 // Bound: HBM for U = 1 (4 B written per element); for U >= 4 the serial decode (issue slots and
 // shared-memory wavefronts: the table look-up of 32 lanes hits random banks) dominates.
@@ -39,25 +43,50 @@ static_assert(STAGE_ROW % 4 == 0, "stage rows must keep 16-byte alignment");
 // windows), so the head of the second table that fits here nearly always holds all of them.
 constexpr int LONG_CACHE = CO3_LONG_CACHE;
 
-struct Tables {                                   // per-segment decoder tables in shared memory
-    alignas(16) uint32_t lut[CO3_LUT_SIZE];
-    alignas(16) uint32_t long_cache[LONG_CACHE];  // head of the row's table of 12..16-bit codewords
-    const uint32_t* lut_long;                     // the whole of it (global memory)
+template <int BITS>
+struct TablesT {                                  // per-segment decoder tables in shared memory
+    static constexpr int bits = BITS;
+    alignas(16) uint32_t lut[1 << BITS];
+    alignas(16) uint32_t long_cache[LONG_CACHE];  // the row's second table from the first codeword longer than BITS
+    const uint32_t* lut_long;                     // the rest of it (global memory)
     uint32_t long_first;                          // first 16-bit window it covers
     uint32_t long_n;                              // number of windows it covers
 };
+using Tables = TablesT<CO3_LUT_SMALL_BITS>;
+using TablesWide = TablesT<CO3_LUT_BITS>;
 
-__device__ void load_tables(Tables& t, const Co3CodeBook& cb, int row, int tid) {
+__device__ __forceinline__ uint32_t keep_up_to(uint32_t e, uint32_t bits) { return (e & 0xFFu) > bits ? 0u : e; }
+
+// The stored table has 2^13 entries indexed by the next 13 stream bits (first bit lowest); its first
+// 2^BITS entries are the table for BITS index bits once the entries of longer codewords are blanked.
+template <int BITS>
+__device__ void load_tables(TablesT<BITS>& t, const Co3CodeBook& cb, int row, int tid, int nthreads) {
     const uint4* lut = reinterpret_cast<const uint4*>(cb.lut + (size_t)row * CO3_LUT_SIZE);
     uint4* dst = reinterpret_cast<uint4*>(t.lut);
-    for (int i = tid; i < CO3_LUT_SIZE / 4; i += CO3_THREADS) dst[i] = __ldg(lut + i);
-    if (tid < LONG_CACHE / 4)
+    for (int i = tid; i < (1 << BITS) / 4; i += nthreads) {
+        uint4 v = __ldg(lut + i);
+        if (BITS < CO3_LUT_BITS) {
+            v.x = keep_up_to(v.x, BITS); v.y = keep_up_to(v.y, BITS);
+            v.z = keep_up_to(v.z, BITS); v.w = keep_up_to(v.w, BITS);
+        }
+        dst[i] = v;
+    }
+    // the second table starts at the first window of a 12-bit codeword; this decoder enters it at the
+    // first window of a codeword longer than BITS (both multiples of 4, so are the row lengths)
+    const uint32_t* first = cb.first + (size_t)row * (CO3_MAXLEN + 1);
+    const uint32_t tab_first = __ldg(first + CO3_LONG_FROM) << (CO3_MAXLEN - CO3_LONG_FROM);
+    const uint32_t my_first = BITS + 1 == CO3_LONG_FROM ? tab_first : __ldg(first + BITS + 1) << (CO3_MAXLEN - BITS - 1);
+    const uint32_t base = my_first - tab_first, stride = (uint32_t)cb.long_stride;
+    const uint32_t* lg = cb.lut_long + (size_t)row * cb.long_stride;
+    if (tid < LONG_CACHE / 4) {
+        const uint32_t i = base + 4u * (uint32_t)tid;
         reinterpret_cast<uint4*>(t.long_cache)[tid] =
-            __ldg(reinterpret_cast<const uint4*>(cb.lut_long + (size_t)row * cb.long_stride) + tid);
+            i + 3u < stride ? __ldg(reinterpret_cast<const uint4*>(lg + i)) : make_uint4(0, 0, 0, 0);
+    }
     if (tid == 0) {
-        t.lut_long = cb.lut_long + (size_t)row * cb.long_stride;
-        t.long_first = cb.first[(size_t)row * (CO3_MAXLEN + 1) + CO3_LUT_BITS + 1] << (CO3_MAXLEN - CO3_LUT_BITS - 1);
-        t.long_n = (uint32_t)cb.long_stride;
+        t.lut_long = lg + (base < stride ? base : 0u);
+        t.long_first = my_first;
+        t.long_n = base < stride ? stride - base : 0u;
     }
 }
 
@@ -78,7 +107,8 @@ __device__ __forceinline__ void red_add(uint32_t addr, uint32_t v) {
 
 // Codeword longer than the primary table: one look-up in the row's second table (its head is in
 // shared memory, the rest in global memory; about one symbol in a thousand comes here).  Returns the entry (K << 8) | length.
-__device__ __forceinline__ uint32_t decode_long(uint32_t window, const Tables& t, bool& bad) {
+template <class T>
+__device__ __forceinline__ uint32_t decode_long(uint32_t window, const T& t, bool& bad) {
     const uint32_t v = __brev(window) >> 16;      // 16 stream bits, root bit on top
     const uint32_t i = v - t.long_first;
     uint32_t e = i < LONG_CACHE ? t.long_cache[i] : (i < t.long_n ? __ldg(t.lut_long + i) : 0u);
@@ -125,9 +155,9 @@ __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint
 // consumed, nothing is added), so every later look-up of the group sees the same window and returns 0
 // too, and the caller tests only the group's LAST entry.
 // PACKED: add the whole entry (length byte included); else add the signed magnitude.
-template <int OFF, bool PACKED>
+template <int OFF, bool PACKED, int BITS>
 __device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr) {
-    const uint32_t e = lds32(lut_addr + ((r.lo & (CO3_LUT_SIZE - 1)) << 2));
+    const uint32_t e = lds32(lut_addr + ((r.lo & ((1u << BITS) - 1u)) << 2));
     r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= (int)(e & 0xFFu);
@@ -136,10 +166,10 @@ __device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, ui
 }
 
 // One symbol with the test for a long codeword (group tails, and groups that met a long codeword).
-template <bool PACKED>
+template <bool PACKED, class T>
 __device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr, uint32_t acc_addr,
-                                                    const Tables& t, bool& bad) {
-    uint32_t e = lds32(lut_addr + ((r.lo & (CO3_LUT_SIZE - 1)) << 2));
+                                                    const T& t, bool& bad) {
+    uint32_t e = lds32(lut_addr + ((r.lo & ((1u << T::bits) - 1u)) << 2));
     if ((e & 0xFFu) == 0u) e = decode_long(r.lo, t, bad);
     r.lo = __funnelshift_r(r.lo, r.hi, e);
     r.hi = __funnelshift_r(r.hi, 0u, e);
@@ -151,9 +181,9 @@ __device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr
 // stands exactly at that codeword, so the rest of the group is decoded with the checked step.
 // Rare (about one symbol in a thousand is longer than the table).  Inlined, so that the reader stays
 // in registers (its address is never taken); the long-codeword search itself is out of line.
-template <bool PACKED>
+template <bool PACKED, class T>
 __device__ __forceinline__ void finish_group(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int done,
-                                          const Tables& t, bool& bad) {
+                                             const T& t, bool& bad) {
 #pragma unroll 1
     for (int k = done; k < 4; ++k) {
         refill(r);
@@ -161,17 +191,17 @@ __device__ __forceinline__ void finish_group(Reader& r, uint32_t lut_addr, uint3
     }
 }
 
-template <bool PACKED>
+template <bool PACKED, class T>
 __device__ __forceinline__ void decode_run(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int n,
-                                           const Tables& t, bool& bad) {
+                                           const T& t, bool& bad) {
     int i = 0;
     for (; i + 4 <= n; i += 4) {
         refill(r);
-        const uint32_t e0 = decode_step<0, PACKED>(r, lut_addr, acc_addr);
-        const uint32_t e1 = decode_step<PADW * 4, PACKED>(r, lut_addr, acc_addr);
+        const uint32_t e0 = decode_step<0, PACKED, T::bits>(r, lut_addr, acc_addr);
+        const uint32_t e1 = decode_step<PADW * 4, PACKED, T::bits>(r, lut_addr, acc_addr);
         refill(r);
-        const uint32_t e2 = decode_step<PADW * 8, PACKED>(r, lut_addr, acc_addr);
-        const uint32_t e3 = decode_step<PADW * 12, PACKED>(r, lut_addr, acc_addr);
+        const uint32_t e2 = decode_step<PADW * 8, PACKED, T::bits>(r, lut_addr, acc_addr);
+        const uint32_t e3 = decode_step<PADW * 12, PACKED, T::bits>(r, lut_addr, acc_addr);
         if ((e3 & 0xFFu) == 0u) {
             const int done = ((e0 & 0xFFu) != 0u) + ((e1 & 0xFFu) != 0u) + ((e2 & 0xFFu) != 0u);
             finish_group<PACKED>(r, lut_addr, acc_addr, done, t, bad);
@@ -205,12 +235,12 @@ __device__ void slow_init(SlowReader& r, const uint32_t* src, uint32_t nwords, u
     r.nb += 32;
     r.wp++;
 }
-template <bool PACKED>
-__device__ void slow_run(SlowReader& r, const Tables& t, const uint32_t* src, uint32_t nwords, int32_t* acc,
+template <bool PACKED, class T>
+__device__ void slow_run(SlowReader& r, const T& t, const uint32_t* src, uint32_t nwords, int32_t* acc,
                          int n, bool& bad) {
     for (int i = 0; i < n; ++i) {
         const uint32_t window = (uint32_t)r.buf;
-        uint32_t e = t.lut[window & (CO3_LUT_SIZE - 1)];
+        uint32_t e = t.lut[window & ((1u << T::bits) - 1u)];
         if ((e & 0xFFu) == 0u) e = decode_long(window, t, bad);
         const uint32_t len = e & 0xFFu;
         r.buf >>= len;
@@ -336,7 +366,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
         const Co3Group grp = p.groups[gi];
         const int gp = (int)(gi & 1);
         if (grp.seg != cur_seg) {                  // every warp is past the last decode with the old tables
-            load_tables(sm.t, p.cb, p.code_by_segment ? grp.seg : co3_row_of(hdr[grp.seg], &bad), tid);
+            load_tables(sm.t, p.cb, p.code_by_segment ? grp.seg : co3_row_of(hdr[grp.seg], &bad), tid, CO3_THREADS);
             cur_seg = grp.seg;
         }
         const bool mine = ci < cpg && ci < grp.count;
@@ -408,6 +438,112 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
 
+// ---- U = 8: four teams of 8 warps (one per user) share a 13-bit table ----------------------
+constexpr int TEAMS = 4;
+constexpr int WIDE_THREADS = TEAMS * CO3_THREADS;
+
+struct Team {
+    alignas(16) uint32_t stage[NW][STAGE_ROW];
+    alignas(16) int32_t acc[2][ACC_Q];
+};
+struct SmemW {
+    TablesWide t;
+    Team team[TEAMS];
+};
+
+__device__ __forceinline__ void team_barrier(int team) {   // barrier 0 is the block's own
+    asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(CO3_THREADS) : "memory");
+}
+
+__global__ void __launch_bounds__(WIDE_THREADS, 1)
+decode_u8_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
+                 const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
+                 const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
+                 float* __restrict__ weights, float step) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    SmemW& sm = *reinterpret_cast<SmemW*>(s_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int team = warp / NW, us = warp - team * NW;      // this warp's team and user
+    const int ttid = tid - team * CO3_THREADS;
+    Team& tm = sm.team[team];
+    int32_t* acc0 = &tm.acc[0][0];
+    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(acc0);
+    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[us]);
+    const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
+    const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
+    const float fu = (float)NW, inv_u = 1.0f / (float)NW;
+    bool bad = false;
+    // as in the kernel above: the accumulators start at zero and every read-out zeroes what it read
+    for (int i = ttid; i < 2 * ACC_Q / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
+    int64_t gi = g0;
+    while (gi < g1) {                                       // one trip per run of chunks of one segment
+        const int seg = p.groups[gi].seg;
+        int64_t ge = gi + 1;
+        while (ge < g1 && p.groups[ge].seg == seg) ++ge;
+        __syncthreads();                                    // every team is past its last look-up in the old tables
+        load_tables(sm.t, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, WIDE_THREADS);
+        __syncthreads();
+        const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
+        for (int64_t g = gi + team; g < ge; g += TEAMS) {
+            const int64_t c = p.groups[g].chunk0;           // a group is one chunk when U = 8
+            const Co3Chunk cd = p.chunks[c];
+            Stream s;
+            Reader r;
+            r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr;
+            SlowReader sr;
+            sr.buf = 0; sr.nb = 0; sr.wp = 0;
+            open_stream(s, p, cd, c, us, bitstream, sub_bits, chunk_off, tm.stage[us], lane, bad);
+            if (s.active) {
+                if (s.staged) reader_init(r, stage_addr, s.bitpos);
+                else slow_init(sr, s.gsrc, s.nwords, s.bitpos);
+            }
+            const long long tb = cd.start & ~(long long)(CO3_TILE - 1);
+            const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+            // No barrier here: a warp stages and reads its own stream, and the accumulator half of the
+            // first quarter was read out (and zeroed) before the barrier of the previous chunk's last quarter.
+#pragma unroll 1
+            for (int q = 0; q < CO3_SUB / QB; ++q) {
+                const int qoff = (q & 1) * ACC_Q;
+                if (s.active) {
+                    const int a = max(s.i_lo, q * QB), b = min(s.i_hi, (q + 1) * QB);
+                    if (b > a) {
+                        const int row0 = qoff + (a - q * QB) * PADW + lane;
+                        if (s.staged) decode_run<true>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, b - a, sm.t, bad);
+                        else slow_run<true>(sr, sm.t, s.gsrc, s.nwords, acc0 + row0, b - a, bad);
+                    }
+                }
+                team_barrier(team);
+                // read-out: warp w, round rr takes sub-chunk w + 8 rr, lane l its symbol q*QB + l
+                const int e0 = us * CO3_SUB + q * QB + lane;
+                int32_t* a = acc0 + qoff + lane * PADW + us;
+                const int64_t o = tb + e0;
+                if (lo == 0 && hi == CO3_TILE) {
+#pragma unroll
+                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+                        put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
+                        a[rr * NW] = 0;
+                    }
+                } else {
+#pragma unroll
+                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+                        const int e = e0 + rr * NW * CO3_SUB;
+                        if (e >= lo && e < hi) put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
+                        a[rr * NW] = 0;
+                    }
+                }
+            }
+            if (s.active) {
+                const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - (uint32_t)r.nb
+                                                 : sr.wp * 32u - (uint32_t)sr.nb;
+                if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
+            }
+        }
+        gi = ge;
+    }
+    if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
+}
+
 // ---- U > 8: whole-chunk accumulator, user groups of 8 --------------------------------------
 struct SmemB {
     Tables t;
@@ -435,7 +571,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     for (int64_t c = c0; c < c1; ++c) {
         const Co3Chunk cd = p.chunks[c];
         if (cd.seg != cur_seg) {
-            load_tables(sm.t, p.cb, p.code_by_segment ? cd.seg : co3_row_of(hdr[cd.seg], &bad), tid);
+            load_tables(sm.t, p.cb, p.code_by_segment ? cd.seg : co3_row_of(hdr[cd.seg], &bad), tid, CO3_THREADS);
             cur_seg = cd.seg;
         }
         for (int i = tid; i < CO3_SUB * PADW / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(sm.acc)[i] = make_uint4(0, 0, 0, 0);
@@ -484,6 +620,8 @@ cudaError_t co3_setup_decode_kernels(void) {
     cudaError_t e = cudaFuncSetAttribute(decode_small_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem_a_bytes(1));
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_u8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmemW));
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(decode_large_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)sizeof(SmemB));
 }
@@ -494,7 +632,11 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
     Co3Dev p = pl->dev;
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) { p.cb = pl->cb_emp; p.code_by_segment = 1; }
     co3_prof_begin(pl, CO3_K_DECODE, st);
-    if (p.U <= NW) {
+    if (p.U == NW) {
+        const int64_t grid = pl->num_sms;                    // one block of four teams per SM
+        decode_u8_kernel<<<(int)(p.n_groups < grid ? p.n_groups : grid), WIDE_THREADS, sizeof(SmemW), st>>>(
+            p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
+    } else if (p.U < NW) {
         const size_t smem = smem_a_bytes(p.U);
         int bpsm = 0;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bpsm, decode_small_u_kernel, CO3_THREADS, smem);

@@ -313,7 +313,7 @@ __global__ void __launch_bounds__(CO3_MAXSYM) huff_cand_kernel(Co3Dev p, Co3Code
 
 // Per model row: take the smallest floor whose code is at most 16 deep, assign canonical
 // codewords (symbols ordered by (length, symbol)), and write the encoder table and the decoder
-// tables (11-bit primary table + canonical arrays for the rare longer codewords).
+// tables (13-bit primary table, second table for the codewords of 12 bits and more, canonical arrays).
 // FROM_LENS: the lengths are given (lens_in, [rows][2^B] by public symbol: the side information of the
 // empirical-histogram code on the decoding side); lengths that are not those of a complete prefix
 // code raise CO3_FLAG_CORRUPT.  lens_out (may be null): the chosen lengths, same layout.
@@ -394,15 +394,15 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
         }
         cb.lut[(size_t)rowi * CO3_LUT_SIZE + i] = entry;
     }
-    // Second table for the codewords the first one cannot hold.  Canonical codes grow with the length,
+    // Second table for the codewords a primary table of 11 or 13 bits cannot hold.  Canonical codes grow with the length,
     // so every 16-bit window that starts with a codeword of 12..16 bits is >= first[12] << 4, and
     // there are at most 16 per symbol of them.
-    const uint32_t long_first = s_first[CO3_LUT_BITS + 1] << (CO3_MAXLEN - CO3_LUT_BITS - 1);
+    const uint32_t long_first = s_first[CO3_LONG_FROM] << (CO3_MAXLEN - CO3_LONG_FROM);
     for (int i = tid; i < cb.long_stride; i += CO3_MAXSYM) {
         const uint32_t v = long_first + (uint32_t)i;          // 16 stream bits, root bit on top
         uint32_t entry = 0;                                    // 0: no codeword starts like this
         if (v < (1u << CO3_MAXLEN)) {
-            for (int L = CO3_LUT_BITS + 1; L <= CO3_MAXLEN; ++L) {
+            for (int L = CO3_LONG_FROM; L <= CO3_MAXLEN; ++L) {
                 const uint32_t dd = (v >> (CO3_MAXLEN - L)) - s_first[L];
                 if (dd < s_count[L]) {
                     const int sym = s_perm[s_offs[L] + dd];

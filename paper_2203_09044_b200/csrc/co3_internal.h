@@ -8,8 +8,11 @@
 constexpr int CO3_TILE = 4096;      // chunk grid (elements)
 constexpr int CO3_SUB = 128;        // sub-chunk grid (elements)
 constexpr int CO3_MAXLEN = 16;      // longest codeword
-constexpr int CO3_LUT_BITS = 11;    // primary decode table index width
+constexpr int CO3_LUT_BITS = 13;    // index width of the stored primary decode tables
 constexpr int CO3_LUT_SIZE = 1 << CO3_LUT_BITS;
+constexpr int CO3_LUT_SMALL_BITS = 11;  // a decoder short of shared memory keeps the first 2^11 entries
+                                        // (minus those of longer codewords: the table is indexed LSB-first)
+constexpr int CO3_LONG_FROM = CO3_LUT_SMALL_BITS + 1;   // shortest codeword the second table holds
 constexpr int CO3_NCAND = 10;       // model codes: weight floors 2^0 .. 2^9 tried in parallel (weights sum to ~2^20: 2^9 always passes)
 constexpr int CO3_NCAND_HIST = 32;  // codes from counts (total below 2^31): floors 2^0 .. 2^31 (2^31 makes all weights equal)
 constexpr int CO3_NIBETA = 23;      // ibeta in [-14, 8]
@@ -56,7 +59,7 @@ struct Co3CodeBook {
     uint8_t* len_pub;    // [R][256]        the same by public symbol (inspection only)
     uint32_t* enc;       // [R][256]        bit-reversed codeword | length << 16, by internal symbol
     uint32_t* code_msb;  // [R][256]        canonical codeword, root bit most significant, by public symbol
-    uint32_t* lut;       // [R][2048]       (signed magnitude << 8) | length, 0 = longer than 11 bits
+    uint32_t* lut;       // [R][8192]       (signed magnitude << 8) | length, 0 = longer than 13 bits
     uint32_t* lut_long;  // [R][long_stride] the same for the codewords of 12..16 bits, indexed by
                          //                 (16 stream bits, root bit on top) - (first[12] << 4)
     int long_stride;     //                 16 * alphabet size (more 16-bit windows cannot lie under long
