@@ -119,23 +119,27 @@ __device__ __forceinline__ uint32_t decode_long(uint32_t window, const T& t, boo
     return e;
 }
 
-// LSB-first bit reader over staged words: the stream sits at bits [0, nb) of hi:lo; rp is the
-// shared-space byte address of the next word.  A refill is checked once per PAIR of symbols:
-// with nb >= 32 two codewords (at most 16 bits each) can be taken without looking at nb, and one
-// more word then always fits.  (With 32 lanes a per-symbol refill branch would be taken on nearly
-// every step, so its cost is paid per step, not per refill.)
+// LSB-first bit reader over staged words: the stream sits at bits [0, nb) of hi:lo and the bits above
+// are zero; rp is the shared-space byte address of the next word.  A refill is checked once per PAIR
+// of symbols: with nb >= 32 two codewords (at most 16 bits each) can be taken without looking at nb,
+// and one more word then always fits.  (With 32 lanes a per-symbol refill branch would be taken on
+// nearly every step, so its cost is paid per step, not per refill.)
+// nb is kept in the low byte of its register only: a step subtracts the whole table entry (length in
+// the low byte, which never borrows because nb >= length), and the shifts look at five bits.
 struct Reader {
     uint32_t lo, hi;
-    int nb;
+    uint32_t nb;
     uint32_t rp;
 };
 
+__device__ __forceinline__ uint32_t reader_bits(const Reader& r) { return r.nb & 0xFFu; }
+
 __device__ __forceinline__ void refill(Reader& r) {
-    if (r.nb < 32) {
-        const unsigned long long w = (unsigned long long)lds32(r.rp) << r.nb;
-        r.lo |= (uint32_t)w;
-        r.hi |= (uint32_t)(w >> 32);
-        r.nb += 32;
+    if (reader_bits(r) < 32u) {                               // then hi holds no bit
+        const uint32_t w = lds32(r.rp);
+        r.lo |= __funnelshift_l(0u, w, r.nb);                 // w << nb
+        r.hi = __funnelshift_l(w, 0u, r.nb);                  // w >> (32 - nb), 0 for nb = 0
+        r.nb += 32u;
         r.rp += 4;
     }
 }
@@ -146,7 +150,7 @@ __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint
     const unsigned long long v = (((unsigned long long)lds32(r.rp + 4) << 32) | lds32(r.rp)) >> sh;
     r.lo = (uint32_t)v;
     r.hi = (uint32_t)(v >> 32);
-    r.nb = 64 - (int)sh;
+    r.nb = 64u - sh;
     r.rp += 8;
 }
 
@@ -160,7 +164,7 @@ __device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, ui
     const uint32_t e = lds32(lut_addr + ((r.lo & ((1u << BITS) - 1u)) << 2));
     r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
     r.hi = __funnelshift_r(r.hi, 0u, e);
-    r.nb -= (int)(e & 0xFFu);
+    r.nb -= e;                                    // the low byte counts
     red_add<OFF>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
     return e;
 }
@@ -173,7 +177,7 @@ __device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr
     if ((e & 0xFFu) == 0u) e = decode_long(r.lo, t, bad);
     r.lo = __funnelshift_r(r.lo, r.hi, e);
     r.hi = __funnelshift_r(r.hi, 0u, e);
-    r.nb -= (int)(e & 0xFFu);
+    r.nb -= e;                                    // the low byte counts
     red_add<0>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
 }
 
@@ -430,7 +434,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
             }
         }
         if (mine && s.active) {
-            const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - (uint32_t)r.nb
+            const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - reader_bits(r)
                                              : sr.wp * 32u - (uint32_t)sr.nb;
             if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
         }
@@ -534,7 +538,7 @@ decode_u8_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                 }
             }
             if (s.active) {
-                const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - (uint32_t)r.nb
+                const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - reader_bits(r)
                                                  : sr.wp * 32u - (uint32_t)sr.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
             }
@@ -586,7 +590,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                     Reader r;
                     reader_init(r, stage_addr, s.bitpos);
                     decode_run<false>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, s.i_hi - s.i_lo, sm.t, bad);
-                    endpos = ((r.rp - stage_addr) << 3) - (uint32_t)r.nb;
+                    endpos = ((r.rp - stage_addr) << 3) - reader_bits(r);
                 } else {
                     SlowReader sr;
                     slow_init(sr, s.gsrc, s.nwords, s.bitpos);
