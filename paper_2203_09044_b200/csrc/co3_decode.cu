@@ -324,220 +324,145 @@ __device__ __forceinline__ float finish(int32_t ksum, float scale, float fu, flo
 }
 
 // ---- U <= 8: one stream per warp, quarter batches ------------------------------------------
+// A team = 8 warps = NW / U chunks x U users.  TEAMS teams share the block's tables (BITS index
+// bits: as wide as the shared memory left by the teams allows); a team has its own named barrier,
+// and the block synchronises as a whole only where the segment (the table) changes.
 constexpr int QB = 32;                            // symbols per lane per batch
 constexpr int ACC_Q = QB * PADW;                  // accumulator words per chunk per batch
 
-struct SmemA {
-    Tables t;
+struct TeamHead {                                 // followed by the accumulator: [2][chunks per group][ACC_Q]
     long long c_tb[2][NW];                        // per chunk of the group: tile base, bounds in the tile
     int c_lo[2][NW], c_hi[2][NW];                 // (two sets: a group is read out while the next one opens)
     alignas(16) uint32_t stage[NW][STAGE_ROW];    // filled with 128-bit stores
-    alignas(16) int32_t acc[2][ACC_Q];            // really [2][chunks per group][ACC_Q], sized at launch
 };
+static_assert(sizeof(TeamHead) % 16 == 0, "the accumulator behind it is cleared with 128-bit stores");
 
 __host__ __device__ inline int acc_words_a(int U) { return ((NW / U) * ACC_Q + 3) & ~3; }
-__host__ __device__ inline size_t smem_a_bytes(int U) {
-    return sizeof(SmemA) - sizeof(int32_t) * 2 * ACC_Q + sizeof(int32_t) * 2 * (size_t)acc_words_a(U);
-}
-
-__global__ void __launch_bounds__(CO3_THREADS)
-decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
-                      const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
-                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
-                      float* __restrict__ weights, float step) {
-    extern __shared__ __align__(16) unsigned char s_raw[];
-    SmemA& sm = *reinterpret_cast<SmemA*>(s_raw);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int U = p.U;
-    const int cpg = NW / U;                        // chunks per group (>= 1)
-    const int accw = acc_words_a(U);               // words per accumulator buffer
-    int32_t* acc0 = &sm.acc[0][0];
-    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
-    const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(acc0);
-    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(sm.stage[warp]);
-    const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
-    const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
-    const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
-    const float fu = (float)U;
-    const float inv_u = (U & (U - 1)) == 0 ? 1.0f / fu : 0.0f;
-    int cur_seg = -1;
-    bool bad = false;
-    // Both accumulator buffers start at zero and every read-out zeroes what it has read, so one
-    // barrier per quarter is enough: decode(q) -> barrier -> read-out(q), and the buffer of quarter q
-    // is next written after the barrier of quarter q + 1.
-    for (int i = tid; i < 2 * accw / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
-    for (int64_t gi = g0; gi < g1; ++gi) {
-        const Co3Group grp = p.groups[gi];
-        const int gp = (int)(gi & 1);
-        if (grp.seg != cur_seg) {                  // every warp is past the last decode with the old tables
-            load_tables(sm.t, p.cb, p.code_by_segment ? grp.seg : co3_row_of(hdr[grp.seg], &bad), tid, CO3_THREADS);
-            cur_seg = grp.seg;
-        }
-        const bool mine = ci < cpg && ci < grp.count;
-        Stream s;
-        s.active = false; s.staged = true; s.nwords = 0; s.bitpos = 0; s.sub_len_bits = 0;
-        s.i_lo = 0; s.i_hi = 0; s.gsrc = nullptr;
-        Reader r;
-        r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr;
-        SlowReader sr;
-        sr.buf = 0; sr.nb = 0; sr.wp = 0;
-        if (mine) {
-            const Co3Chunk cd = p.chunks[grp.chunk0 + ci];
-            open_stream(s, p, cd, grp.chunk0 + ci, us, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
-            if (s.active) {
-                if (s.staged) reader_init(r, stage_addr, s.bitpos);
-                else slow_init(sr, s.gsrc, s.nwords, s.bitpos);
-            }
-        }
-        const float scale = pow2_clamped((int)hdr[grp.seg].bias + p.cF);
-        if (tid < grp.count) {
-            const Co3Chunk cd = p.chunks[grp.chunk0 + tid];
-            const long long tb = cd.start & ~(long long)(CO3_TILE - 1);
-            sm.c_tb[gp][tid] = tb;
-            sm.c_lo[gp][tid] = (int)(cd.start - tb);
-            sm.c_hi[gp][tid] = (int)(cd.start - tb) + cd.len;
-        }
-        __syncthreads();                           // tables, chunk bounds (and the first zeroing)
-#pragma unroll 1
-        for (int q = 0; q < CO3_SUB / QB; ++q) {
-            const int qoff = (q & 1) * accw;
-            if (mine && s.active) {
-                const int a = max(s.i_lo, q * QB), b = min(s.i_hi, (q + 1) * QB);
-                if (b > a) {
-                    const int row0 = qoff + ci * ACC_Q + (a - q * QB) * PADW + lane;
-                    if (s.staged) decode_run<true>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, b - a, sm.t, bad);
-                    else slow_run<true>(sr, sm.t, s.gsrc, s.nwords, acc0 + row0, b - a, bad);
-                }
-            }
-            __syncthreads();
-            // read-out: warp w, round rr takes sub-chunk w + 8 rr, lane l its symbol q*QB + l
-            const int e0 = warp * CO3_SUB + q * QB + lane;
-            for (int cc = 0; cc < grp.count; ++cc) {
-                const int lo = sm.c_lo[gp][cc], hi = sm.c_hi[gp][cc];
-                // the accumulator holds sum((K << 8) | length): the lengths of <= 8 users stay below 256
-                int32_t* a = acc0 + qoff + cc * ACC_Q + lane * PADW + warp;
-                const int64_t o = sm.c_tb[gp][cc] + e0;
-                if (lo == 0 && hi == CO3_TILE) {
-#pragma unroll
-                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
-                        put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
-                        a[rr * NW] = 0;
-                    }
-                } else {
-#pragma unroll
-                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
-                        const int e = e0 + rr * NW * CO3_SUB;
-                        if (e >= lo && e < hi) put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
-                        a[rr * NW] = 0;
-                    }
-                }
-            }
-        }
-        if (mine && s.active) {
-            const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - reader_bits(r)
-                                             : sr.wp * 32u - (uint32_t)sr.nb;
-            if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
-        }
-    }
-    if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
-}
-
-// ---- U = 8: four teams of 8 warps (one per user) share a 13-bit table ----------------------
-constexpr int TEAMS = 4;
-constexpr int WIDE_THREADS = TEAMS * CO3_THREADS;
-
-struct Team {
-    alignas(16) uint32_t stage[NW][STAGE_ROW];
-    alignas(16) int32_t acc[2][ACC_Q];
-};
-struct SmemW {
-    TablesWide t;
-    Team team[TEAMS];
-};
+__host__ __device__ inline size_t team_bytes(int U) { return sizeof(TeamHead) + sizeof(int32_t) * 2 * (size_t)acc_words_a(U); }
+template <int TEAMS, int BITS>
+__host__ __device__ inline size_t smem_a_bytes(int U) { return sizeof(TablesT<BITS>) + TEAMS * team_bytes(U); }
 
 __device__ __forceinline__ void team_barrier(int team) {   // barrier 0 is the block's own
     asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(CO3_THREADS) : "memory");
 }
 
-__global__ void __launch_bounds__(WIDE_THREADS, 1)
-decode_u8_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
-                 const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
-                 const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
-                 float* __restrict__ weights, float step) {
+// One quarter of one chunk: scale the sums of warp w's sub-chunks (w, w + 8, ...) and zero them.
+__device__ __forceinline__ void read_out(int32_t* a, int64_t o, int e0, int lo, int hi, float scale, float fu,
+                                         float inv_u, float* avg, float* weights, float step) {
+    if (lo == 0 && hi == CO3_TILE) {
+#pragma unroll
+        for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+            put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
+            a[rr * NW] = 0;
+        }
+    } else {
+#pragma unroll
+        for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
+            const int e = e0 + rr * NW * CO3_SUB;
+            if (e >= lo && e < hi) put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
+            a[rr * NW] = 0;
+        }
+    }
+}
+
+// UC: the number of users when it is known at compile time (the powers of two), else 0.
+template <int TEAMS, int BITS, int UC>
+__global__ void __launch_bounds__(TEAMS * CO3_THREADS, TEAMS == 1 ? 4 : 1)
+decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
+                      const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
+                      const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
+                      float* __restrict__ weights, float step) {
     extern __shared__ __align__(16) unsigned char s_raw[];
-    SmemW& sm = *reinterpret_cast<SmemW*>(s_raw);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int team = warp / NW, us = warp - team * NW;      // this warp's team and user
-    const int ttid = tid - team * CO3_THREADS;
-    Team& tm = sm.team[team];
-    int32_t* acc0 = &tm.acc[0][0];
-    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    TablesT<BITS>& tabs = *reinterpret_cast<TablesT<BITS>*>(s_raw);
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int team = tid / CO3_THREADS, ttid = tid - team * CO3_THREADS, warp = ttid >> 5;
+    const int U = UC ? UC : p.U;
+    const bool all_mine = UC == NW;                // one chunk per group and every warp has a stream of it
+    unsigned char* team_raw = s_raw + sizeof(TablesT<BITS>) + (size_t)team * team_bytes(U);
+    TeamHead& tm = *reinterpret_cast<TeamHead*>(team_raw);
+    int32_t* acc0 = reinterpret_cast<int32_t*>(team_raw + sizeof(TeamHead));
+    const int cpg = NW / U;                        // chunks per group (>= 1)
+    const int accw = acc_words_a(U);               // words per accumulator buffer
+    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(tabs.lut);
     const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(acc0);
-    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[us]);
+    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[warp]);
+    const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
     const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
     const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
-    const float fu = (float)NW, inv_u = 1.0f / (float)NW;
+    const float fu = (float)U;
+    const float inv_u = (U & (U - 1)) == 0 ? 1.0f / fu : 0.0f;
     bool bad = false;
-    // as in the kernel above: the accumulators start at zero and every read-out zeroes what it read
-    for (int i = ttid; i < 2 * ACC_Q / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
+    int opened = 0;                                // groups this team has opened
+    // Both accumulator buffers start at zero and every read-out zeroes what it has read, so one
+    // barrier per quarter is enough: decode(q) -> barrier -> read-out(q), and the buffer of quarter q
+    // is next written after the barrier of quarter q + 1.
+    for (int i = ttid; i < 2 * accw / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(acc0)[i] = make_uint4(0, 0, 0, 0);
     int64_t gi = g0;
-    while (gi < g1) {                                       // one trip per run of chunks of one segment
+    while (gi < g1) {                              // one trip per run of groups of one segment
         const int seg = p.groups[gi].seg;
         int64_t ge = gi + 1;
         while (ge < g1 && p.groups[ge].seg == seg) ++ge;
-        __syncthreads();                                    // every team is past its last look-up in the old tables
-        load_tables(sm.t, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, WIDE_THREADS);
-        __syncthreads();
+        __syncthreads();                           // every team is past its last look-up in the old tables
+        load_tables(tabs, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, TEAMS * CO3_THREADS);
+        __syncthreads();                           // (and the first zeroing)
         const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
-        for (int64_t g = gi + team; g < ge; g += TEAMS) {
-            const int64_t c = p.groups[g].chunk0;           // a group is one chunk when U = 8
-            const Co3Chunk cd = p.chunks[c];
+        for (int64_t g = gi + team; g < ge; g += TEAMS, ++opened) {
+            const Co3Group grp = p.groups[g];
+            const int gp = opened & 1;
+            const bool mine = all_mine || (ci < cpg && ci < grp.count);
             Stream s;
+            s.active = false; s.staged = true; s.nwords = 0; s.bitpos = 0; s.sub_len_bits = 0;
+            s.i_lo = 0; s.i_hi = 0; s.gsrc = nullptr;
             Reader r;
             r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr;
             SlowReader sr;
             sr.buf = 0; sr.nb = 0; sr.wp = 0;
-            open_stream(s, p, cd, c, us, bitstream, sub_bits, chunk_off, tm.stage[us], lane, bad);
-            if (s.active) {
-                if (s.staged) reader_init(r, stage_addr, s.bitpos);
-                else slow_init(sr, s.gsrc, s.nwords, s.bitpos);
+            long long my_tb = 0;                   // bounds of this warp's own chunk (used when all_mine)
+            int my_lo = 0, my_hi = 0;
+            if (mine) {
+                const Co3Chunk cd = p.chunks[grp.chunk0 + ci];
+                open_stream(s, p, cd, grp.chunk0 + ci, us, bitstream, sub_bits, chunk_off, tm.stage[warp], lane, bad);
+                if (s.active) {
+                    if (s.staged) reader_init(r, stage_addr, s.bitpos);
+                    else slow_init(sr, s.gsrc, s.nwords, s.bitpos);
+                }
+                my_tb = cd.start & ~(long long)(CO3_TILE - 1);
+                my_lo = (int)(cd.start - my_tb);
+                my_hi = my_lo + cd.len;
             }
-            const long long tb = cd.start & ~(long long)(CO3_TILE - 1);
-            const int lo = (int)(cd.start - tb), hi = lo + cd.len;
-            // No barrier here: a warp stages and reads its own stream, and the accumulator half of the
-            // first quarter was read out (and zeroed) before the barrier of the previous chunk's last quarter.
+            if (!all_mine && ttid < grp.count) {
+                const Co3Chunk cd = p.chunks[grp.chunk0 + ttid];
+                const long long tb = cd.start & ~(long long)(CO3_TILE - 1);
+                tm.c_tb[gp][ttid] = tb;
+                tm.c_lo[gp][ttid] = (int)(cd.start - tb);
+                tm.c_hi[gp][ttid] = (int)(cd.start - tb) + cd.len;
+            }
+            // The bounds are read after the first quarter's barrier (and this set was last read two groups
+            // ago); a warp stages and reads its own stream: no barrier is needed here.
 #pragma unroll 1
             for (int q = 0; q < CO3_SUB / QB; ++q) {
-                const int qoff = (q & 1) * ACC_Q;
-                if (s.active) {
+                const int qoff = (q & 1) * accw;
+                if (mine && s.active) {
                     const int a = max(s.i_lo, q * QB), b = min(s.i_hi, (q + 1) * QB);
                     if (b > a) {
-                        const int row0 = qoff + (a - q * QB) * PADW + lane;
-                        if (s.staged) decode_run<true>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, b - a, sm.t, bad);
-                        else slow_run<true>(sr, sm.t, s.gsrc, s.nwords, acc0 + row0, b - a, bad);
+                        const int row0 = qoff + ci * ACC_Q + (a - q * QB) * PADW + lane;
+                        if (s.staged) decode_run<true>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, b - a, tabs, bad);
+                        else slow_run<true>(sr, tabs, s.gsrc, s.nwords, acc0 + row0, b - a, bad);
                     }
                 }
                 team_barrier(team);
-                // read-out: warp w, round rr takes sub-chunk w + 8 rr, lane l its symbol q*QB + l
-                const int e0 = us * CO3_SUB + q * QB + lane;
-                int32_t* a = acc0 + qoff + lane * PADW + us;
-                const int64_t o = tb + e0;
-                if (lo == 0 && hi == CO3_TILE) {
-#pragma unroll
-                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
-                        put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
-                        a[rr * NW] = 0;
-                    }
+                // read-out: warp w, round rr takes sub-chunk w + 8 rr, lane l its symbol q*QB + l; the
+                // accumulator holds sum((K << 8) | length): the lengths of <= 8 users stay below 256
+                const int e0 = warp * CO3_SUB + q * QB + lane;
+                if (all_mine) {
+                    read_out(acc0 + qoff + lane * PADW + warp, my_tb + e0, e0, my_lo, my_hi, scale, fu, inv_u, avg, weights, step);
                 } else {
-#pragma unroll
-                    for (int rr = 0; rr < 32 * QB / CO3_THREADS; ++rr) {
-                        const int e = e0 + rr * NW * CO3_SUB;
-                        if (e >= lo && e < hi) put_out(avg, weights, step, o + rr * NW * CO3_SUB, finish(a[rr * NW] >> 8, scale, fu, inv_u));
-                        a[rr * NW] = 0;
-                    }
+                    for (int cc = 0; cc < grp.count; ++cc)
+                        read_out(acc0 + qoff + cc * ACC_Q + lane * PADW + warp, tm.c_tb[gp][cc] + e0, e0,
+                                 tm.c_lo[gp][cc], tm.c_hi[gp][cc], scale, fu, inv_u, avg, weights, step);
                 }
             }
-            if (s.active) {
+            if (mine && s.active) {
                 const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - reader_bits(r)
                                                  : sr.wp * 32u - (uint32_t)sr.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
@@ -618,14 +543,39 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
 
 int g_bpsm_b = 0;
 
+typedef void (*SmallKernel)(Co3Dev, const uint32_t*, const uint16_t*, const uint32_t*, const co3_seg_header*,
+                            float*, float*, float);
+struct SmallVariant {
+    SmallKernel fn;
+    int teams;
+    size_t smem;
+};
+// The widest table and the most teams that fit the shared memory of an SM (227 KB per block); user
+// counts that do not divide 8 leave warps idle and keep the plain one-team blocks, four per SM.
+SmallVariant small_variant(int U) {
+    switch (U) {
+        case 8: return {decode_small_u_kernel<4, 13, 8>, 4, smem_a_bytes<4, 13>(U)};
+        case 4: return {decode_small_u_kernel<4, 12, 4>, 4, smem_a_bytes<4, 12>(U)};
+        case 2: return {decode_small_u_kernel<3, 12, 2>, 3, smem_a_bytes<3, 12>(U)};
+        case 1: return {decode_small_u_kernel<2, 12, 1>, 2, smem_a_bytes<2, 12>(U)};
+        default: return {decode_small_u_kernel<1, 11, 0>, 1, smem_a_bytes<1, 11>(U)};
+    }
+}
+
 }  // namespace
 
 cudaError_t co3_setup_decode_kernels(void) {
-    cudaError_t e = cudaFuncSetAttribute(decode_small_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem_a_bytes(1));
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_u8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmemW));
-    if (e != cudaSuccess) return e;
+    for (int U = 1; U <= NW; ++U) {
+        const SmallVariant v = small_variant(U);
+        size_t need = v.smem;                      // the largest of the user counts that run this variant
+        for (int U2 = 1; U2 <= NW; ++U2) {
+            const SmallVariant v2 = small_variant(U2);
+            if (v2.fn == v.fn && v2.smem > need) need = v2.smem;
+        }
+        if (need > 227u * 1024u) return cudaErrorInvalidConfiguration;
+        cudaError_t e = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+        if (e != cudaSuccess) return e;
+    }
     return cudaFuncSetAttribute(decode_large_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)sizeof(SmemB));
 }
@@ -636,17 +586,15 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
     Co3Dev p = pl->dev;
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) { p.cb = pl->cb_emp; p.code_by_segment = 1; }
     co3_prof_begin(pl, CO3_K_DECODE, st);
-    if (p.U == NW) {
-        const int64_t grid = pl->num_sms;                    // one block of four teams per SM
-        decode_u8_kernel<<<(int)(p.n_groups < grid ? p.n_groups : grid), WIDE_THREADS, sizeof(SmemW), st>>>(
-            p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
-    } else if (p.U < NW) {
-        const size_t smem = smem_a_bytes(p.U);
-        int bpsm = 0;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bpsm, decode_small_u_kernel, CO3_THREADS, smem);
-        if (bpsm < 1) bpsm = 1;
+    if (p.U <= NW) {
+        const SmallVariant v = small_variant(p.U);
+        int bpsm = 1;
+        if (v.teams == 1) {
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bpsm, v.fn, CO3_THREADS, v.smem);
+            if (bpsm < 1) bpsm = 1;
+        }
         const int64_t grid = (int64_t)pl->num_sms * bpsm;
-        decode_small_u_kernel<<<(int)(p.n_groups < grid ? p.n_groups : grid), CO3_THREADS, smem, st>>>(
+        v.fn<<<(int)(p.n_groups < grid ? p.n_groups : grid), v.teams * CO3_THREADS, v.smem, st>>>(
             p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     } else {
         if (!g_bpsm_b) {
