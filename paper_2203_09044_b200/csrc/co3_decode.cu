@@ -15,15 +15,17 @@
 // as shift amount (only its low five bits count), the bit buffer is topped up once per pair of
 // symbols, and four symbols are decoded per loop trip with immediate accumulator offsets.
 //
-// Three variants.  U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
-// per sub-chunk (small double-buffered accumulator, several chunks per block when U < 8); the
+// Two kernels.  U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
+// per sub-chunk (small double-buffered accumulator, several chunks per group when U < 8); the
 // whole table entries are accumulated (the length bytes of at most 8 users cannot carry into
-// the magnitude) and the magnitude sum is taken out with one shift at the end.  U = 8 runs four
-// such 8-warp teams in one block of 1024 threads: they share one 13-bit table (with 11 bits one
-// group of 128 look-ups in eight still meets a longer codeword and leaves the fast path, which also
-// makes the warps of a team wait for each other), each team has its own named barrier, and the whole
-// block synchronises only where the segment (the table) changes.  U > 8 keeps a whole chunk
-// accumulator and loops over user groups.
+// the magnitude) and the magnitude sum is taken out with one shift at the end.  U > 8 keeps a
+// whole-chunk accumulator and loops over the users.
+// Both run several 8-warp teams in one block per SM (1024 threads for U = 8 and U > 8): the teams
+// share one table of 13 or 12 index bits (with 11 bits one group of 128 look-ups in eight still meets
+// a longer codeword and leaves the fast path, which also makes the warps of a team wait for each
+// other), each team has its own named barrier, and the whole block synchronises only where the
+// segment (the table) changes.  User counts that do not divide 8 keep one-team blocks, four per SM,
+// with an 11-bit table.
 //
 // Bound: HBM for U = 1 (4 B written per element); for U >= 4 the serial decode (issue slots and
 // shared-memory wavefronts: the table look-up of 32 lanes hits random banks) dominates.
@@ -474,74 +476,87 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
 }
 
 // ---- U > 8: whole-chunk accumulator, user groups of 8 --------------------------------------
-struct SmemB {
-    Tables t;
+// Teams as above (four, with a 12-bit table); a team decodes all users of one chunk into a
+// whole-chunk accumulator, which the read-out leaves zeroed for the next chunk.
+struct TeamB {
     alignas(16) int32_t acc[CO3_SUB * PADW];
     alignas(16) uint32_t stage[NW][STAGE_ROW];    // filled with 128-bit stores
 };
+constexpr int TEAMS_B = 4, BITS_B = 12;
+struct SmemB {
+    TablesT<BITS_B> t;
+    TeamB team[TEAMS_B];
+};
+static_assert(sizeof(SmemB) <= 227 * 1024, "one block per SM must fit its shared memory");
 
-__global__ void __launch_bounds__(CO3_THREADS)
+__global__ void __launch_bounds__(TEAMS_B * CO3_THREADS, 1)
 decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                       const uint16_t* __restrict__ sub_bits, const uint32_t* __restrict__ chunk_off,
                       const co3_seg_header* __restrict__ hdr, float* __restrict__ avg,
                       float* __restrict__ weights, float step) {
     extern __shared__ __align__(16) unsigned char s_raw[];
     SmemB& sm = *reinterpret_cast<SmemB*>(s_raw);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int team = tid / CO3_THREADS, ttid = tid - team * CO3_THREADS, warp = ttid >> 5;
+    TeamB& tm = sm.team[team];
     const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
-    const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(sm.acc);
-    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(sm.stage[warp]);
+    const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(tm.acc);
+    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[warp]);
     const int64_t per = (p.n_chunks + gridDim.x - 1) / gridDim.x;
     const int64_t c0 = (int64_t)blockIdx.x * per, c1 = min(p.n_chunks, c0 + per);
     const float fu = (float)p.U;
     const float inv_u = (p.U & (p.U - 1)) == 0 ? 1.0f / fu : 0.0f;
-    int cur_seg = -1;
     bool bad = false;
-    for (int64_t c = c0; c < c1; ++c) {
-        const Co3Chunk cd = p.chunks[c];
-        if (cd.seg != cur_seg) {
-            load_tables(sm.t, p.cb, p.code_by_segment ? cd.seg : co3_row_of(hdr[cd.seg], &bad), tid, CO3_THREADS);
-            cur_seg = cd.seg;
-        }
-        for (int i = tid; i < CO3_SUB * PADW / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(sm.acc)[i] = make_uint4(0, 0, 0, 0);
-        __syncthreads();
-        for (int u = warp; u < p.U; u += NW) {
-            Stream s;
-            open_stream(s, p, cd, c, u, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
-            if (s.active) {
-                const int row0 = s.i_lo * PADW + lane;
-                uint32_t endpos;
-                if (s.staged) {
-                    Reader r;
-                    reader_init(r, stage_addr, s.bitpos);
-                    decode_run<false>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, s.i_hi - s.i_lo, sm.t, bad);
-                    endpos = ((r.rp - stage_addr) << 3) - reader_bits(r);
-                } else {
-                    SlowReader sr;
-                    slow_init(sr, s.gsrc, s.nwords, s.bitpos);
-                    slow_run<false>(sr, sm.t, s.gsrc, s.nwords, sm.acc + row0, s.i_hi - s.i_lo, bad);
-                    endpos = sr.wp * 32u - (uint32_t)sr.nb;
+    for (int i = ttid; i < CO3_SUB * PADW / 4; i += CO3_THREADS) reinterpret_cast<uint4*>(tm.acc)[i] = make_uint4(0, 0, 0, 0);
+    int64_t ci = c0;
+    while (ci < c1) {                              // one trip per run of chunks of one segment
+        const int seg = p.chunks[ci].seg;
+        int64_t ce = ci + 1;
+        while (ce < c1 && p.chunks[ce].seg == seg) ++ce;
+        __syncthreads();                           // every team is past its last look-up in the old tables
+        load_tables(sm.t, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, TEAMS_B * CO3_THREADS);
+        __syncthreads();                           // (and the first zeroing)
+        const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
+        for (int64_t c = ci + team; c < ce; c += TEAMS_B) {
+            const Co3Chunk cd = p.chunks[c];
+            for (int u = warp; u < p.U; u += NW) {
+                Stream s;
+                open_stream(s, p, cd, c, u, bitstream, sub_bits, chunk_off, tm.stage[warp], lane, bad);
+                if (s.active) {
+                    const int row0 = s.i_lo * PADW + lane;
+                    uint32_t endpos;
+                    if (s.staged) {
+                        Reader r;
+                        reader_init(r, stage_addr, s.bitpos);
+                        decode_run<false>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, s.i_hi - s.i_lo, sm.t, bad);
+                        endpos = ((r.rp - stage_addr) << 3) - reader_bits(r);
+                    } else {
+                        SlowReader sr;
+                        slow_init(sr, s.gsrc, s.nwords, s.bitpos);
+                        slow_run<false>(sr, sm.t, s.gsrc, s.nwords, tm.acc + row0, s.i_hi - s.i_lo, bad);
+                        endpos = sr.wp * 32u - (uint32_t)sr.nb;
+                    }
+                    if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
                 }
-                if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
+                __syncwarp();                      // the stage is reused by this warp's next user
             }
-            __syncwarp();                          // the stage is reused by this warp's next user
-        }
-        __syncthreads();
-        const float scale = pow2_clamped((int)hdr[cd.seg].bias + p.cF);
-        const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-        const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+            team_barrier(team);
+            const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+            const int lo = (int)(cd.start - tb), hi = lo + cd.len;
 #pragma unroll 4
-        for (int rr = 0; rr < CO3_TILE / CO3_THREADS; ++rr) {
-            const int e = tid + rr * CO3_THREADS;
-            const int kk = e >> 7, il = e & (CO3_SUB - 1);
-            if (e >= lo && e < hi) put_out(avg, weights, step, tb + e, finish(sm.acc[il * PADW + kk], scale, fu, inv_u));
+            for (int rr = 0; rr < CO3_TILE / CO3_THREADS; ++rr) {
+                const int e = ttid + rr * CO3_THREADS;
+                const int kk = e >> 7, il = e & (CO3_SUB - 1);
+                const int32_t k = tm.acc[il * PADW + kk];
+                tm.acc[il * PADW + kk] = 0;
+                if (e >= lo && e < hi) put_out(avg, weights, step, tb + e, finish(k, scale, fu, inv_u));
+            }
+            team_barrier(team);
         }
-        __syncthreads();
+        ci = ce;
     }
     if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
-
-int g_bpsm_b = 0;
 
 typedef void (*SmallKernel)(Co3Dev, const uint32_t*, const uint16_t*, const uint32_t*, const co3_seg_header*,
                             float*, float*, float);
@@ -597,12 +612,8 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
         v.fn<<<(int)(p.n_groups < grid ? p.n_groups : grid), v.teams * CO3_THREADS, v.smem, st>>>(
             p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     } else {
-        if (!g_bpsm_b) {
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_bpsm_b, decode_large_u_kernel, CO3_THREADS, sizeof(SmemB));
-            if (g_bpsm_b < 1) g_bpsm_b = 1;
-        }
-        const int64_t grid = (int64_t)pl->num_sms * g_bpsm_b;
-        decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), CO3_THREADS, sizeof(SmemB), st>>>(
+        const int64_t grid = pl->num_sms;                    // one block of four teams per SM
+        decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), TEAMS_B * CO3_THREADS, sizeof(SmemB), st>>>(
             p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     }
     co3_prof_end(pl, CO3_K_DECODE, st, 1);
