@@ -353,10 +353,51 @@ def cpu_baseline(wl_index, budget_s):
     t0 = time.perf_counter()
     oracle_sample_step(orc, wl, g, m)
     dt = time.perf_counter() - t0
-    return {"value": 4.0 * wl.d * users / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"1 iteration (encode + decode-aggregate) of {users} of the {full.n_users} users "
-                      f"at full d={wl.d}, {dt:.1f} s",
-            "host_cores_available": os.cpu_count()}
+    out = {"value": 4.0 * wl.d * users / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"1 iteration (encode + decode-aggregate) of {users} of the {full.n_users} users "
+                     f"at full d={wl.d}, {dt:.1f} s",
+           "host_cores_available": os.cpu_count()}
+    del g, m, orc
+    out["all_cores"] = cpu_baseline_all_cores(wl_index, full.n_users)
+    return out
+
+
+def cpu_baseline_all_cores(wl_index, n_users):
+    """The same oracle, one process per user side by side (the users' streams are independent; each
+    process fits its own user's moments, which is the same amount of work): what the host cores of
+    this box deliver together.  value = the users' bytes / the slowest process's iteration time."""
+    import subprocess
+    procs = min(n_users, os.cpu_count() or 1)
+    cmd = [sys.executable, os.path.abspath(__file__), "--oracle-worker"]
+    ps = [subprocess.Popen(cmd + [f"{wl_index}:{u}"], stdout=subprocess.PIPE, text=True) for u in range(procs)]
+    times, d = [], 0
+    for pr in ps:
+        try:
+            line = pr.communicate(timeout=300)[0].strip().splitlines()[-1]
+            rec = json.loads(line)
+            times.append(rec["seconds"])
+            d = rec["d"]
+        except Exception:                               # a worker that failed: no figure, not a wrong one
+            pr.kill()
+            return {"unavailable": "an oracle worker process failed"}
+    dt = max(times)
+    return {"value": 4.0 * d * procs / dt / 1e9, "unit": UNIT, "cores": procs,
+            "sample": f"{procs} processes, each 1 iteration of 1 user at full d={d}; slowest {dt:.1f} s"}
+
+
+def oracle_worker(spec):
+    """Child process of cpu_baseline_all_cores: one oracle iteration on one user's gradient."""
+    import numpy as np
+    from oracle import co3_oracle
+    from paper_2203_09044_b200 import inputs
+    wl_index, u = (int(x) for x in spec.split(":"))
+    wl = inputs.workload(wl_index, n_users=1)
+    g = wl.gradient(0, users=[u]).numpy()
+    m = np.zeros_like(g)
+    orc = co3_oracle.OracleCO3(wl.d, 1, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma)
+    t0 = time.perf_counter()
+    oracle_sample_step(orc, wl, g, m)
+    print(json.dumps({"seconds": time.perf_counter() - t0, "d": wl.d}), flush=True)
 
 
 def run_reference(args):
@@ -410,7 +451,11 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
     ap.add_argument("--mode", default="lagged", choices=["lagged", "current", "code-lagged"],
                     help="bias/code mode of the plan (default: lagged bias, the benchmark configuration)")
+    ap.add_argument("--oracle-worker", default=None, help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.oracle_worker:
+        oracle_worker(args.oracle_worker)
+        return
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":

@@ -165,7 +165,7 @@ __device__ __forceinline__ unsigned long long wait_group(const unsigned long lon
     return 0;
 }
 
-__global__ void __launch_bounds__(ENC_THREADS, 16)
+__global__ void __launch_bounds__(ENC_THREADS, 20)
 enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits,
                   uint32_t* __restrict__ chunk_off, unsigned long long* __restrict__ user_bits,
                   uint32_t* __restrict__ bitstream) {
