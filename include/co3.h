@@ -162,6 +162,21 @@ int co3_tiled_convert(co3_plan* plan, const float* grad_tile, float* residual, i
 int co3_tiled_finish(co3_plan* plan, uint32_t* bitstream, uint16_t* sub_bits, uint32_t* chunk_off,
                      uint64_t* user_bits, co3_seg_header* hdr, void* cuda_stream);
 
+/* Pooled moments across plans (a gradient cut into slices of d, one plan per slice, e.g. one per GPU).
+ * The shape and scale of a layer are fitted to the moments of ALL its entries (Sec. III (i), the
+ * moment-matching fit), so a layer that spans several slices needs its three sums added over the
+ * slices before the fit; everything else of an iteration is local to a slice.  Inside a tiled
+ * iteration, after the last co3_tiled_statistics call and again after the last co3_tiled_convert call:
+ *   co3_moments_export  moments: device, out, [n_segments][3] fp64 = (finite entries, sum |a|, sum a^2)
+ *                       of this plan's part of every segment, a = g + gamma m, all users pooled
+ *   co3_moments_import  moments: device, const, same layout: the sums the next fit (the bias before the
+ *                       first convert tile, or the header in co3_tiled_finish) uses INSTEAD of the
+ *                       plan's own; consumed by that fit.  The caller adds the exported sums of the
+ *                       plans that share a segment (an all-reduce of n_segments x 3 doubles) in between.
+ * Without an import the plan's own sums are used, as before.  CO3_EINVAL outside those two places. */
+int co3_moments_export(co3_plan* plan, double* moments, void* cuda_stream);
+int co3_moments_import(co3_plan* plan, const double* moments, void* cuda_stream);
+
 /* Algorithm 1 lines 13-14 without the model update: decode all U streams and write
  * avg_grad[i] = (1/U) sum_u ghat^(u)[i] (Eq. "aggregate"), device [d] fp32.  Depends only on
  * its arguments and the plan's static configuration, never on encoder scratch.  The integer

@@ -26,6 +26,7 @@ EXPORTS = [
     "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
     "co3_bias_opt_table", "co3_grid_distortion", "co3_encode_empirical", "co3_decode_aggregate_empirical",
     "co3_profile_stride", "co3_tiled_begin", "co3_tiled_statistics", "co3_tiled_convert", "co3_tiled_finish",
+    "co3_moments_export", "co3_moments_import",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -111,6 +112,10 @@ def lib():
     L.co3_tiled_convert.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp]
     L.co3_tiled_finish.restype = C.c_int
     L.co3_tiled_finish.argtypes = [vp] * 7
+    L.co3_moments_export.restype = C.c_int
+    L.co3_moments_export.argtypes = [vp, vp, vp]
+    L.co3_moments_import.restype = C.c_int
+    L.co3_moments_import.argtypes = [vp, vp, vp]
     L.co3_profile_stride.restype = C.c_int
     L.co3_profile_stride.argtypes = [vp, C.c_int32]
     L.co3_profile_collect.restype = C.c_int
@@ -284,6 +289,49 @@ class Plan:
             around_call(True)
         if rc != OK:
             raise Co3Error(rc, "co3_tiled_finish")
+
+    # The phases of a tiled iteration one by one (encode_tiled strings them together); between them a
+    # caller may pool the moments of several plans (moments_export / moments_import).
+    def tiled_begin(self):
+        """Start a tiled iteration; True if statistics tiles have to come before the convert tiles."""
+        need = C.c_int32()
+        rc = lib().co3_tiled_begin(self.handle, C.byref(need))
+        if rc != OK:
+            raise Co3Error(rc, "co3_tiled_begin")
+        return bool(need.value)
+
+    def tiled_statistics(self, grad_tile, residual, user0, n_users, stream=None):
+        rc = lib().co3_tiled_statistics(self.handle, _ptr(grad_tile), _ptr(residual), user0, n_users, self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_tiled_statistics")
+
+    def tiled_convert(self, grad_tile, residual, user0, n_users, stream=None):
+        rc = lib().co3_tiled_convert(self.handle, _ptr(grad_tile), _ptr(residual), user0, n_users, self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_tiled_convert")
+
+    def tiled_finish(self, out, stream=None):
+        rc = lib().co3_tiled_finish(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]), _ptr(out["chunk_off"]),
+                                    _ptr(out["user_bits"]), _ptr(out["hdr"]), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_tiled_finish")
+
+    def moments_export(self, moments=None, stream=None):
+        """[S][3] fp64 cuda: (finite entries, sum |a|, sum a^2) of every segment, all users pooled."""
+        import torch
+        if moments is None:
+            moments = torch.empty((self.S, 3), dtype=torch.float64, device="cuda")
+        rc = lib().co3_moments_export(self.handle, _ptr(moments), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_moments_export")
+        return moments
+
+    def moments_import(self, moments, stream=None):
+        """The sums the next fit uses instead of the plan's own ([S][3] fp64 cuda, contiguous)."""
+        assert moments.is_cuda and moments.is_contiguous() and tuple(moments.shape) == (self.S, 3)
+        rc = lib().co3_moments_import(self.handle, _ptr(moments), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_moments_import")
 
     def decode_aggregate(self, out, avg=None, stream=None):
         avg = out["avg"] if avg is None else avg

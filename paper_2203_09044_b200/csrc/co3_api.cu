@@ -259,6 +259,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             }
         }
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
+        a |= dev_alloc(pl, &pl->ext_mom, (size_t)S * 3);
         int16_t* d_opt = nullptr;
         const int16_t* h_opt = co3_host_bias_opt_table(E, M);
         a |= dev_alloc(pl, &d_opt, (size_t)CO3_NIBETA * 8);
@@ -378,6 +379,7 @@ extern "C" int co3_tiled_begin(co3_plan* pl, int32_t* need_statistics) {
     if (pl->cfg.bias_mode != CO3_BIAS_CURRENT && pl->cfg.bias_mode != CO3_BIAS_LAGGED) return CO3_EINVAL;
     pl->tiled_state = 1;
     pl->tiled_users = 0;
+    pl->use_ext_mom = false;
     *need_statistics = (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) ? 1 : 0;
     return CO3_OK;
 }
@@ -426,6 +428,29 @@ extern "C" int co3_tiled_finish(co3_plan* pl, uint32_t* bitstream, uint16_t* sub
     CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;
     pl->tiled_state = 0;
+    return CO3_OK;
+}
+
+// ---- pooled moments across plans (slices of d) ---------------------------------------------------
+extern "C" int co3_moments_export(co3_plan* pl, double* moments, void* cuda_stream) {
+    if (!pl || !moments) return CO3_EINVAL;
+    if (pl->tiled_state != 2 && pl->tiled_state != 3) return CO3_EINVAL;
+    if (pl->tiled_state == 3 && pl->tiled_users != pl->dev.U) return CO3_EINVAL;   // every user converted
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    pl->mom_out = moments;
+    CO3_TRY(co3_launch_fit(pl, 4, nullptr, st));
+    pl->mom_out = nullptr;
+    return CO3_OK;
+}
+
+extern "C" int co3_moments_import(co3_plan* pl, const double* moments, void* cuda_stream) {
+    if (!pl || !moments) return CO3_EINVAL;
+    if (pl->tiled_state != 2 && pl->tiled_state != 3) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    CO3_TRY(cudaMemcpyAsync(pl->ext_mom, moments, sizeof(double) * 3 * (size_t)pl->dev.S, cudaMemcpyDeviceToDevice, st));
+    pl->use_ext_mom = true;
     return CO3_OK;
 }
 

@@ -75,7 +75,12 @@ __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int c
 // mode 2: after the stats pass of t = 0 -- bias and header of the coming pass from these moments.
 // mode 3: after the fused convert-and-pack pass -- the same for the next iteration; keep the fit.
 //         In both, `hdr` is the plan's own header array.
-__global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr) {
+// mode 4: only add up the moments of every segment and write (N, S1, S2) to mom_out.
+// ext_mom (may be null): (N, S1, S2) per segment that replace the plan's own sums in the fit (the sums
+//         of a layer that is spread over several plans); the non-finite count stays the plan's own.
+__global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr,
+                                                          const double* __restrict__ ext_mom,
+                                                          double* __restrict__ mom_out) {
     __shared__ double s_a[FIT_THREADS / 32], s_b[FIT_THREADS / 32];
     __shared__ unsigned long long s_n[FIT_THREADS / 32];
     __shared__ double s_lg[3];
@@ -125,7 +130,12 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     unsigned long long nf = 0;
 #pragma unroll
     for (int w = 0; w < FIT_THREADS / 32; ++w) { S1 += s_a[w]; S2 += s_b[w]; nf += s_n[w]; }
-    const double N = (double)((unsigned long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * (unsigned long long)p.U - nf);
+    double N = (double)((unsigned long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * (unsigned long long)p.U - nf);
+    if (mode == 4) {
+        if (tid == 0) { mom_out[3 * seg] = N; mom_out[3 * seg + 1] = S1; mom_out[3 * seg + 2] = S2; }
+        return;
+    }
+    if (ext_mom) { N = ext_mom[3 * seg]; S1 = ext_mom[3 * seg + 1]; S2 = ext_mom[3 * seg + 2]; }
 
     // beta = clamp(R^-1(rho), 0.3, 2.0), rho = N S2 / S1^2; R is strictly decreasing in beta, and
     // the tables hold log R and log G at log2(beta) = T0 + i * H.
@@ -420,7 +430,9 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
     co3_prof_begin(pl, CO3_K_FIT, st);
     if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.red_k, pl->dev.S), RED_THREADS, 0, st>>>(pl->dev, mode == 1);
-    fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr);
+    const double* ext = (pl->use_ext_mom && mode != 4) ? pl->ext_mom : nullptr;
+    if (mode != 4) pl->use_ext_mom = false;                // imported moments serve one fit
+    fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out);
     co3_prof_end(pl, CO3_K_FIT, st, pl->dev.red_k > 0 ? 2 : 1);
     return cudaGetLastError();
 }

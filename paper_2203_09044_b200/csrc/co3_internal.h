@@ -138,6 +138,9 @@ struct co3_plan {
     bool ev_conv_recorded;          // a convert pass that read d_grad has been recorded
     int tiled_state;                // co3_tiled_*: 0 idle, 1 begun, 2 statistics tiles seen, 3 convert tiles seen
     int tiled_users;                // users converted so far in this tiled iteration
+    double* ext_mom;                // [S][3] moments handed in by co3_moments_import
+    bool use_ext_mom;               // ... and not yet consumed by a fit
+    double* mom_out;                // co3_moments_export: where the reduction-only fit launch writes
     bool record_conv;               // co3_encode records ev_conv after its last pass over the gradient
     void* allocs[128];
     int n_allocs;

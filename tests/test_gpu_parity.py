@@ -524,6 +524,91 @@ def test_host_iterations_back_to_back_overlap_their_copies(binding, oracle):
 
 
 # ---- full sizes, in the launch configuration the benchmark times ---------------------------
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("world", [2, 3])
+def test_slices_of_d_with_pooled_moments_equal_the_whole(binding, oracle, mode, world):
+    """The gradient cut into `world` slices of d, one plan per slice (as one GPU per slice would hold
+    them), run phase by phase on this GPU with the slices' moment tables added between the phases
+    (what the all-reduce does): payload, side information, headers, memory and average of the
+    slices, put end to end, are those of the oracle on the whole gradient."""
+    from paper_2203_09044_b200 import inputs, sharded
+    wl = inputs.workload(1, d=150_000, n_users=3)
+    U, d, off = wl.n_users, wl.d, wl.seg_offsets
+    orc = oracle.OracleCO3(d, U, 4, 3, off, gamma=wl.gamma, mode=mode)
+    ranks = [sharded.ShardedPlan(d, U, 4, 3, off, r, world, gamma=wl.gamma, bias_mode=mode) for r in range(world)]
+    assert sum(len(sp.layout.seg_ids) for sp in ranks) > len(off) - 1      # some layer spans a cut
+    outs = [sp.plan.alloc_outputs() for sp in ranks]
+    m_gpu = [torch.zeros((U, sp.plan.ld), dtype=torch.float32, device="cuda") for sp in ranks]
+    m_cpu = np.zeros((U, wl.ld), np.float32)
+    for t in range(3):
+        g = wl.gradient(t, device="cuda")
+        gs = []
+        for sp in ranks:
+            x = torch.zeros((U, sp.plan.ld), dtype=torch.float32, device="cuda")
+            x[:, :sp.plan.d] = g[:, sp.layout.lo:sp.layout.hi]
+            gs.append(x)
+        need = [sp.begin() for sp in ranks]
+        assert need == [t == 0 or mode == 0] * world
+        pooled = None
+        if need[0]:
+            pooled = sum(sp.statistics(gs[r], m_gpu[r]) for r, sp in enumerate(ranks))
+        pooled = sum(sp.convert(gs[r], m_gpu[r], pooled) for r, sp in enumerate(ranks))
+        for r, sp in enumerate(ranks):
+            sp.finish(pooled, outs[r])
+        ro = orc.encode(g.cpu().numpy(), m_cpu)
+        assert np.array_equal(pooled.cpu().numpy()[:, 0], ro.moments[:, 0]), f"t={t} pooled counts"
+        np.testing.assert_allclose(pooled.cpu().numpy()[:, 1:], ro.moments[:, 1:], rtol=1e-12)
+        m_all = np.concatenate([m.cpu().numpy()[:, :sp.plan.d] for m, sp in zip(m_gpu, ranks)], axis=1)
+        assert np.array_equal(_bits(m_all), _bits(m_cpu[:, :d])), f"t={t} residual"
+        for r, sp in enumerate(ranks):
+            hdr = binding.hdr_to_numpy(outs[r]["hdr"])
+            assert np.array_equal(hdr, ro.hdr[sp.layout.seg_ids]), f"t={t} header of slice {r}"
+        cos = [o["chunk_off"].cpu().numpy().view(np.uint32) for o in outs]
+        pays = [o["bitstream"].cpu().numpy().view(np.uint32) for o in outs]
+        for u in range(U):
+            words = np.concatenate([pays[r][u, :int(cos[r][u, -1])] for r in range(world)])
+            assert int(ro.chunk_off[u, -1]) == len(words)
+            assert np.array_equal(words, ro.payload[u, :len(words)]), f"t={t} payload of user {u}"
+            base, offs = 0, []
+            for r in range(world):
+                offs.append(cos[r][u, :-1].astype(np.int64) + base)
+                base += int(cos[r][u, -1])
+            assert np.array_equal(np.concatenate(offs), ro.chunk_off[u, :-1]), f"t={t} chunk offsets"
+        sb = np.concatenate([o["sub_bits"].cpu().numpy().view(np.uint16)[:, :sp.plan.n_sub]
+                             for o, sp in zip(outs, ranks)], axis=1)
+        assert np.array_equal(sb, ro.sub_bits[:, :sb.shape[1]]), f"t={t} sub_bits"
+        ub = sum(o["user_bits"].cpu().numpy().view(np.uint64) for o in outs)
+        assert np.array_equal(ub, ro.user_bits), f"t={t} user_bits"
+        avg = np.concatenate([sp.decode_aggregate(outs[r]).cpu().numpy()[:sp.plan.d] for r, sp in enumerate(ranks)])
+        rc, avg_o, _ = orc.decode_aggregate(ro.payload, ro.sub_bits, ro.chunk_off, ro.hdr)
+        assert rc == oracle.OK and np.array_equal(_bits(avg), _bits(avg_o)), f"t={t} averaged gradient"
+        for sp in ranks:
+            assert sp.plan.status()[0] == 0
+
+
+def test_moments_calls_are_refused_outside_their_places(binding):
+    plan = binding.Plan(10_000, 2, 4, 3)
+    mom = torch.zeros((1, 3), dtype=torch.float64, device="cuda")
+    with pytest.raises(binding.Co3Error):
+        plan.moments_export(mom)                                  # no tiled iteration open
+    assert plan.tiled_begin()
+    with pytest.raises(binding.Co3Error):
+        plan.moments_import(mom)                                  # before any statistics tile
+    g = torch.randn((2, plan.ld), device="cuda") * 1e-3
+    m = torch.zeros_like(g)
+    plan.tiled_statistics(g, m, 0, 1)
+    plan.tiled_statistics(g, m, 1, 1)
+    own = plan.moments_export().cpu().numpy()
+    assert own[0, 0] == 2 * 10_000 and own[0, 1] > 0 and own[0, 2] > 0
+    plan.tiled_convert(g, m, 0, 1)
+    with pytest.raises(binding.Co3Error):
+        plan.moments_export(mom)                                  # a user is still to be converted
+    plan.tiled_convert(g, m, 1, 1)
+    out = plan.alloc_outputs()
+    plan.tiled_finish(out)                                        # without an import: the plan's own sums
+    assert plan.status()[0] == 0
+
+
 @pytest.mark.slow
 def test_config0_full(binding, oracle):
     from paper_2203_09044_b200 import inputs
