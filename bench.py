@@ -330,6 +330,80 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sliced(args):
+    """--slices: the SAME total workload (configuration 1) cut into slices of d, one per rank, with the
+    all-reduce of the per-layer moment sums between the phases (strong scaling; not the default arm)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2203_09044_b200 import binding, inputs, sharded
+
+    binding.lib()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    if "RANK" in os.environ:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    wl = inputs.workload(1, n_users=args.users)
+    U, d = wl.n_users, wl.d
+    lay = sharded.SliceLayout(d, wl.seg_offsets, rank, world)
+    ld = inputs.aligned_ld(lay.hi - lay.lo)
+    sp = sharded.ShardedPlan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, rank, world, ld=ld, gamma=wl.gamma)
+    out = sp.plan.alloc_outputs()
+    residual = torch.zeros((U, ld), dtype=torch.float32, device="cuda")
+    pool = []
+    for t in range(POOL):                               # every rank draws the whole batch and keeps its slice
+        g = wl.gradient(t, device="cuda")
+        x = torch.zeros((U, ld), dtype=torch.float32, device="cuda")
+        x[:, :lay.hi - lay.lo] = g[:, lay.lo:lay.hi]
+        pool.append(x)
+        del g
+    torch.cuda.synchronize()
+
+    def step(t):
+        sp.encode(pool[t % POOL], residual, out)
+        sp.decode_aggregate(out)
+
+    def barrier():
+        if dist.is_initialized():
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        step(t)
+    barrier()
+    assert sp.plan.status(clear=True)[0] == 0
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    launches0 = sp.plan.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    e0.record()
+    for t in range(args.steps):
+        step(args.warmup + t)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    launches = sp.plan.launch_count() - launches0
+    assert sp.plan.status()[0] == 0
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": 4.0 * d * U * args.steps / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "configs[1] cut into %d slices of d (one per rank), moment sums all-reduced "
+                                   "twice at t = 0 and once per iteration after" % world,
+                       "d": d, "n_users": U, "slice_of_rank_0": [lay.lo, lay.hi], "row_stride": ld,
+                       "launch": "every step launched eagerly (the all-reduce sits between the phases)",
+                       "l2": "%d MB of gradient+memory read per step and rank, %d batches cycled"
+                             % (8 * U * (lay.hi - lay.lo) // 1000000, POOL)},
+            "clocks": clocks, "gpu_launches": launches}), flush=True)
+    if dist.is_initialized():
+        barrier()
+        dist.destroy_process_group()
+
+
 def oracle_sample_step(orc, wl, g, m):
     """One CO3 iteration of the oracle (encode + decode-aggregate) on host arrays."""
     r = orc.encode(g, m)
@@ -451,6 +525,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
     ap.add_argument("--mode", default="lagged", choices=["lagged", "current", "code-lagged"],
                     help="bias/code mode of the plan (default: lagged bias, the benchmark configuration)")
+    ap.add_argument("--slices", action="store_true",
+                    help="cut the one workload into slices of d, one per rank (strong scaling), instead of replicas")
     ap.add_argument("--oracle-worker", default=None, help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.oracle_worker:
@@ -460,6 +536,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.slices:
+        run_sliced(args)
     else:
         run_ours(args)
 

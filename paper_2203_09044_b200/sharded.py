@@ -50,22 +50,32 @@ class SliceLayout:
                 self.seg_ids.append(s)
                 self.local_offsets.append(b - self.lo)
 
+        self._index = {}                                # seg_ids as an index tensor, per device
+
+    def _ids(self, device):
+        import torch
+        key = str(device)
+        if key not in self._index:
+            self._index[key] = torch.as_tensor(self.seg_ids, dtype=torch.int64, device=device)
+        return self._index[key]
+
     def to_global(self, local):
         """[S_local][3] -> [n_segments][3], zero where this slice has no part of the segment."""
         import torch
         g = torch.zeros((self.n_segments, 3), dtype=local.dtype, device=local.device)
-        g[torch.as_tensor(self.seg_ids, device=local.device)] = local
+        g.index_copy_(0, self._ids(local.device), local)
         return g
 
     def to_local(self, glob):
-        import torch
-        return glob[torch.as_tensor(self.seg_ids, device=glob.device)].contiguous()
+        return glob.index_select(0, self._ids(glob.device))
 
 
 def all_reduce_sum(glob, group=None):
-    """Sum of the ranks' moment tables, in place (NCCL for CUDA tensors, gloo for CPU ones)."""
+    """Sum of the ranks' moment tables, in place (NCCL for CUDA tensors, gloo for CPU ones).  Without
+    a process group there is one slice and nothing to add."""
     import torch.distributed as dist
-    dist.all_reduce(glob, op=dist.ReduceOp.SUM, group=group)
+    if dist.is_available() and dist.is_initialized():
+        dist.all_reduce(glob, op=dist.ReduceOp.SUM, group=group)
     return glob
 
 
