@@ -254,6 +254,25 @@ def test_ragged_segments_and_tiny_inputs(binding, oracle):
         run_case(binding, oracle, d, 2, 4, 3, off, grads)
 
 
+@pytest.mark.slow
+@pytest.mark.parametrize("U,d", [(1, 5_000_123), (2, 5_000_123), (4, 2_600_077), (8, 1_300_031), (16, 1_300_031), (6, 700_001)])
+def test_many_chunks_per_block_with_tiny_layers_between_large_ones(binding, oracle, U, d):
+    """Enough chunks that every block of the decoders works through several of them with all its
+    teams, and layers of 1, 5 and 130 elements between the large ones (the table changes, and with it
+    the whole block synchronises, in the middle of a block's share)."""
+    a, b = d // 5, (7 * d) // 10
+    off = [0, a, a + 5, a + 135, b, b + 1, d]
+    gen = torch.Generator().manual_seed(1000 + U)
+    ld = (d + 3) // 4 * 4
+    grads = []
+    for t in range(2):
+        g = torch.zeros((U, ld))
+        g[:, :d] = torch.randn((U, d), generator=gen) * (1e-2 if t == 0 else 3e-3)
+        g[:, a:a + 135] *= 50.0                              # the tiny layers get their own scale
+        grads.append(g.cuda())
+    run_case(binding, oracle, d, U, 4, 3, off, grads)
+
+
 def test_degenerate_values(binding, oracle):
     """All-zero gradient, a constant segment, huge and subnormal values, signed zeros, ties."""
     d = 6000
