@@ -160,15 +160,37 @@ def measure(wl, iters, warm, pool, rule=0, mode=None):
     for t in range(1, warm):
         step(t)
     torch.cuda.synchronize()
-    plan.profile_enable(None, max_records=2 * iters + 8)
     e0.record()
     for t in range(iters):
         step(warm + t)
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / iters
+    # the per-kernel breakdown comes from a second set of iterations: an event pair around every
+    # launch costs a few microseconds, which the figure above should not carry
+    plan.profile_enable(None, max_records=2 * iters + 8)
+    for t in range(iters):
+        step(warm + iters + t)
+    torch.cuda.synchronize()
     prof = {k: v[0] / iters for k, v in plan.profile_collect().items() if v[1]}
     plan.profile_enable([], 0)
+    # a steady-state iteration has no host decision in it: the same steps replayed from one CUDA graph
+    graph_ms = None
+    if mode in (None, binding.BIAS_LAGGED, binding.BIAS_CURRENT, binding.CODE_LAGGED):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):
+            for t in range(pool):
+                step(t)
+        graph.replay()
+        torch.cuda.synchronize()
+        reps = max(1, (iters + pool - 1) // pool)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        graph_ms = e0.elapsed_time(e1) / (reps * pool)
+        del graph
     flags, nonfinite = plan.status(clear=True)
     code_bits = float(out["user_bits"].sum().item()) / (U * d)
     container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
@@ -185,7 +207,7 @@ def measure(wl, iters, warm, pool, rule=0, mode=None):
                + prof.get("code_enc", 0.0),
                fit_ms=prof.get("fit", 0.0), decode_ms=prof.get("decode", 0.0) + prof.get("code_dec", 0.0),
                code_bits=code_bits, container_bits=container_bits, flags=flags,
-               l2_resident=8.0 * U * d * pool < L2_BYTES)
+               l2_resident=8.0 * U * d * pool < L2_BYTES, graph_ms=graph_ms)
     plan.close()
     del out, residual, grads
     torch.cuda.empty_cache()
@@ -230,6 +252,8 @@ def row(r, peak):
     note = []
     if r["l2_resident"]:
         note.append("inputs fit L2, launch-bound")
+    if r.get("graph_ms"):
+        note.append("%.4f ms from a CUDA graph" % r["graph_ms"])
     if r["flags"]:
         note.append("flags=%d" % r["flags"])
     if r.get("tiled"):
