@@ -628,6 +628,30 @@ def test_moments_calls_are_refused_outside_their_places(binding):
     assert plan.status()[0] == 0
 
 
+def test_moments_export_of_a_very_long_segment(binding):
+    """A segment with more than 2^15 (user, chunk) pairs is summed in slices first; the exported sums
+    are those of a plain fp64 sum over the inputs, and exactly the ones the fit then reports."""
+    U, d = 64, 2_200_000
+    plan = binding.Plan(d, U, 3, 2)
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    g = torch.randn((U, plan.ld), generator=gen, device="cuda") * 2e-3
+    g[:, d:] = 0
+    m = torch.zeros_like(g)
+    assert plan.tiled_begin()
+    plan.tiled_statistics(g, m, 0, U)
+    mom = plan.moments_export().cpu().numpy()
+    a = g[:, :d].double()
+    assert mom[0, 0] == U * d
+    np.testing.assert_allclose(mom[0, 1:], [float(a.abs().sum()), float((a * a).sum())], rtol=1e-12)
+    plan.tiled_convert(g, m, 0, U)
+    mom2 = plan.moments_export().cpu().numpy()
+    out = plan.alloc_outputs()
+    plan.tiled_finish(out)
+    beta, alpha, N, S1, S2 = plan.get_fit(0)
+    assert (N, S1, S2) == tuple(mom2[0]) and plan.status()[0] == 0
+    np.testing.assert_allclose(mom2[0], mom[0], rtol=1e-12)          # same a = g + gamma * 0 in both passes
+
+
 @pytest.mark.slow
 def test_config0_full(binding, oracle):
     from paper_2203_09044_b200 import inputs
