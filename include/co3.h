@@ -118,7 +118,12 @@ typedef struct {
  * the host, allocates all device scratch on the current device and builds there, once, the
  * Huffman code (Sec. III (ii)) of every (shape, scale) pair a header can name, so that an
  * iteration only selects codes.  The iteration counter
- * starts at 0 (memory m_0 = 0 is the caller's zero-filled `residual`). */
+ * starts at 0 (memory m_0 = 0 is the caller's zero-filled `residual`).
+ * Every call that takes a stream only enqueues work on it (kernels, memsets, device-to-device copies)
+ * and never waits for the device, so a steady-state iteration (t >= 1 with CO3_BIAS_LAGGED or
+ * CO3_CODE_LAGGED, any t with CO3_BIAS_CURRENT; tracing off) may be recorded by stream capture and
+ * replayed as a CUDA graph: the kernel sequence does not depend on t.  Iteration 0 of the lagged modes
+ * runs an extra statistics pass and must be run, not replayed, first. */
 int co3_plan_create(co3_plan** out, const co3_config* cfg);
 void co3_plan_destroy(co3_plan* plan);
 
