@@ -123,7 +123,8 @@ typedef struct {
  * and never waits for the device, so a steady-state iteration (t >= 1 with CO3_BIAS_LAGGED or
  * CO3_CODE_LAGGED, any t with CO3_BIAS_CURRENT; tracing off) may be recorded by stream capture and
  * replayed as a CUDA graph: the kernel sequence does not depend on t.  Iteration 0 of the lagged modes
- * runs an extra statistics pass and must be run, not replayed, first. */
+ * runs an extra statistics pass and must be run, not replayed, first.  (The iteration counter that
+ * co3_state_export reports counts calls, not replays of a graph that recorded one.) */
 int co3_plan_create(co3_plan** out, const co3_config* cfg);
 void co3_plan_destroy(co3_plan* plan);
 
