@@ -54,8 +54,6 @@ struct TablesT {                                  // per-segment decoder tables 
     uint32_t long_first;                          // first 16-bit window it covers
     uint32_t long_n;                              // number of windows it covers
 };
-using Tables = TablesT<CO3_LUT_SMALL_BITS>;
-using TablesWide = TablesT<CO3_LUT_BITS>;
 
 __device__ __forceinline__ uint32_t keep_up_to(uint32_t e, uint32_t bits) { return (e & 0xFFu) > bits ? 0u : e; }
 
@@ -573,7 +571,7 @@ SmallVariant small_variant(int U) {
         case 4: return {decode_small_u_kernel<4, 12, 4>, 4, smem_a_bytes<4, 12>(U)};
         case 2: return {decode_small_u_kernel<3, 12, 2>, 3, smem_a_bytes<3, 12>(U)};
         case 1: return {decode_small_u_kernel<2, 12, 1>, 2, smem_a_bytes<2, 12>(U)};
-        default: return {decode_small_u_kernel<1, 11, 0>, 1, smem_a_bytes<1, 11>(U)};
+        default: return {decode_small_u_kernel<1, CO3_LUT_SMALL_BITS, 0>, 1, smem_a_bytes<1, CO3_LUT_SMALL_BITS>(U)};
     }
 }
 
