@@ -285,9 +285,12 @@ __device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co
     s.gsrc = g;
     s.staged = nwords <= CO3_STAGE_WORDS;
     if (s.staged) {
-        const uint4* gv = reinterpret_cast<const uint4*>(g);
-        uint4* sv = reinterpret_cast<uint4*>(stage);
-        for (uint32_t i = lane; i < nwords / 4; i += 32) sv[i] = __ldg(gv + i);
+        // asynchronous 16-byte copies: all of a lane's (up to eight) are in flight together, and the
+        // side information below is fetched while they are; waited for at the end
+        const uint32_t sdst = (uint32_t)__cvta_generic_to_shared(stage);
+        for (uint32_t i = lane; i < nwords / 4; i += 32)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sdst + 16u * i), "l"(g + 4u * i) : "memory");
+        asm volatile("cp.async.commit_group;\n" ::: "memory");
     }
     s.nwords = nwords;
     const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
@@ -309,6 +312,7 @@ __device__ __forceinline__ void open_stream(Stream& s, const Co3Dev& p, const Co
         bad = true;
         s.bitpos = nwords * 32u;
     }
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     __syncwarp();
 }
 
