@@ -34,7 +34,7 @@ CONVERT_TIMED_EVERY = 4          # the convert launches of the timed region that
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel on the full 8-user
 # workload (mean of three launches of the one-pass ncu capture summarised in
 # profiles/dram_traffic_config1_8users.md); it grows in proportion with the number of users
-CONVERT_DRAM_TRAFFIC_BYTES_8_USERS = 1109.8e6
+CONVERT_DRAM_TRAFFIC_BYTES_8_USERS = 1109.5e6
 
 
 def measured_peaks():
