@@ -5,7 +5,10 @@ A step is one CO3 iteration of Algorithm 1 over one batch of synthetic gradients
 (error-feedback add, float conversion, residual update, histogram and moments, GenNorm fit,
 Huffman code build, bit packing) followed by co3_decode_aggregate (code rebuild from the header,
 decode of all users, average).  The workload is the 8-user ResNet-18-sized configuration
-(d = 11,173,962 per user, 62 layers, 8-bit format, gamma = 0.9, lagged bias).
+(d = 11,173,962 per user, 62 layers, 8-bit format, gamma = 0.9).  `value` is measured with the bias of
+every iteration taken from that iteration's own moments, as Algorithm 1 prints it (one extra read pass);
+the same steps with the bias lagging one iteration behind (no extra pass) are timed beside it and
+reported as `lagged_bias`.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -31,10 +34,18 @@ POOL = 4                      # distinct gradient batches cycled through (each >
 # algorithmic bytes per user-element of the fused convert pass: read g, m (8), write m (4), symbol (1)
 CONVERT_BYTES_PER_ELEMENT = 13.0
 CONVERT_TIMED_EVERY = 4          # the convert launches of the timed region that carry an event pair
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel on the full 8-user
-# workload (mean of three launches of the one-pass ncu capture summarised in
-# profiles/dram_traffic_config1_8users.md); it grows in proportion with the number of users
-CONVERT_DRAM_TRAFFIC_BYTES_8_USERS = 1109.5e6
+SUSTAINED_MS = 2000.0             # device time of the sustained leg
+
+
+def convert_dram_traffic(n_users):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the convert kernel, from the figures of
+    the one-pass ncu capture on the full 8-user workload that are kept beside its summary; the traffic
+    grows in proportion with the number of users.  None if the file is missing."""
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic_config1_8users.json")))
+        return float(rec["convert_dram_bytes_per_launch"]) * n_users / float(rec["n_users"])
+    except Exception:
+        return None
 
 
 def measured_peaks():
@@ -93,8 +104,8 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2)
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return {"sm_mhz": statistics.median(self.samples), "sm_min_mhz": min(self.samples),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 def physical_gpu_index(local_rank):
@@ -191,29 +202,41 @@ def run_ours(args):
             per_step_launches = plan.launch_count() - n0
             graphs.append(gr)
         barrier()
-    plan.profile_enable(["convert"], max_records=args.steps)
-    plan.profile_stride(1 if graphs else CONVERT_TIMED_EVERY)
-    sampler = ClockSampler(physical_gpu_index(local_rank))
-    launches0 = plan.launch_count()
-    replays = 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    sampler.start()
-    e0.record()
-    for t in range(args.steps):
-        if graphs is None or t % CONVERT_TIMED_EVERY == 0:
-            step(args.warmup + t)
-        else:
-            graphs[(args.warmup + t) % POOL].replay()
-            replays += 1
-    e1.record()
-    barrier()
-    clocks = sampler.stop()
-    elapsed_ms = e0.elapsed_time(e1)
-    launches = plan.launch_count() - launches0 + replays * per_step_launches
-    conv_ms, conv_n = plan.profile_collect()["convert"]
-    flags, _ = plan.status(clear=True)
-    assert flags == 0, f"status flags {flags} in the timed region"
+
+    def timed_loop(n_steps, first_t):
+        """n_steps steps between two events, the convert launch of every eager step event-timed, NVML
+        clock samples taken meanwhile.  Returns (ms, launches, convert ms, convert launches timed, clocks)."""
+        plan.profile_enable(["convert"], max_records=n_steps)
+        plan.profile_stride(1 if graphs else CONVERT_TIMED_EVERY)
+        sampler = ClockSampler(physical_gpu_index(local_rank))
+        launches0 = plan.launch_count()
+        replays = 0
+        barrier()
+        sampler.start()
+        e0.record()
+        for t in range(n_steps):
+            if graphs is None or t % CONVERT_TIMED_EVERY == 0:
+                step(first_t + t)
+            else:
+                graphs[(first_t + t) % POOL].replay()
+                replays += 1
+        e1.record()
+        barrier()
+        clk = sampler.stop()
+        ms = e0.elapsed_time(e1)
+        n_launch = plan.launch_count() - launches0 + replays * per_step_launches
+        c_ms, c_n = plan.profile_collect()["convert"]
+        f, _ = plan.status(clear=True)
+        assert f == 0, f"status flags {f} in the timed region"
+        return ms, n_launch, c_ms, c_n, clk
+
+    elapsed_ms, launches, conv_ms, conv_n, clocks = timed_loop(args.steps, args.warmup)
+    # ---- sustained leg: the same loop for about two seconds of device time --------------------
+    # (a timed region of a few milliseconds is a burst figure and meets at most one clock sample)
+    sus_steps = max(args.steps, int(SUSTAINED_MS / max(elapsed_ms / args.steps, 1e-3)) + 1)
+    sus_ms, _, sus_conv_ms, sus_conv_n, sus_clocks = timed_loop(sus_steps, args.warmup + args.steps)
+    sus_ms = max_over_ranks(sus_ms, world, "cuda")
     code_bits = float(out["user_bits"].sum().item()) / (U * d)
     container_bits = (32.0 * float(out["chunk_off"][:, -1].sum().item()) + 16.0 * U * plan.n_sub
                       + 32.0 * U * (plan.n_chunks + 1) + 32.0 * plan.S) / (U * d)
@@ -229,6 +252,43 @@ def run_ours(args):
     breakdown = {k: {"ms_per_step": v[0] / nb, "launches_per_step": v[1] / nb}
                  for k, v in plan.profile_collect().items() if v[1]}
     plan.profile_enable([], 0)
+
+    # ---- the other bias mode, timed the same way (K steps, eager) ------------------------------
+    other = {"current": "lagged", "lagged": "current"}.get(args.mode)
+    other_rec = None
+    if other is not None:
+        plan_o = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
+                              bias_mode={"lagged": binding.BIAS_LAGGED, "current": binding.BIAS_CURRENT}[other],
+                              ld=wl.ld)
+        res_o = torch.zeros_like(residual)
+        for t in range(args.warmup):
+            plan_o.encode(pool[t % POOL], res_o, out)
+            plan_o.decode_aggregate(out)
+        gr_o = []
+        for i in range(POOL if not args.no_graph else 0):
+            g_o = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_o, capture_error_mode="thread_local"):
+                plan_o.encode(pool[i], res_o, out)
+                plan_o.decode_aggregate(out)
+            gr_o.append(g_o)
+        barrier()
+        e0.record()
+        for t in range(args.steps):
+            if gr_o:
+                gr_o[t % POOL].replay()
+            else:
+                plan_o.encode(pool[t % POOL], res_o, out)
+                plan_o.decode_aggregate(out)
+        e1.record()
+        barrier()
+        o_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+        assert plan_o.status(clear=True)[0] == 0
+        other_rec = {"bias_mode": other, "ms_per_step": o_ms / args.steps,
+                     "value": job_throughput_gbs(world, 4.0 * d * U, args.steps, o_ms), "unit": UNIT,
+                     "launch": "replayed from one-step CUDA graphs" if gr_o else "launched eagerly"}
+        del gr_o
+        plan_o.close()
+        del res_o
 
     # ---- the same steps replayed from a CUDA graph (one graph = one pass over the gradient pool) --
     # All steps from one graph, no eager step in between: what the loop costs without any launch gap.
@@ -279,7 +339,9 @@ def run_ours(args):
     conv_bytes = CONVERT_BYTES_PER_ELEMENT if args.mode != "code-lagged" else 12.0 + code_bits / 8.0
     achieved = conv_bytes * U * d / (conv_avg_ms * 1e-3) / 1e9
     # all passes of one iteration, E4M3: 13 + 1.9 (encode) + 0.87 (decode) per user-element + the average
-    step_bytes = ((15.9 if args.mode != "code-lagged" else 12.0 + 4.0 * code_bits / 8.0) * U + 4.0) * d
+    # (the statistics pass of the current-moments bias reads g and m once more: + 8)
+    per_ue = {"lagged": 15.9, "current": 23.9, "code-lagged": 12.0 + 4.0 * code_bits / 8.0}[args.mode]
+    step_bytes = (per_ue * U + 4.0) * d
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -306,7 +368,8 @@ def run_ours(args):
                                "ef_kernel<convert+pack> (EF-add/convert/residual/histogram/moments/codeword packing)",
                      "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
-                     "traffic": CONVERT_DRAM_TRAFFIC_BYTES_8_USERS * U / 8.0 if args.mode != "code-lagged" else None,
+                     "traffic": convert_dram_traffic(U) if args.mode != "code-lagged" else None,
+                     "traffic_source": "profiles/dram_traffic_config1_8users.json (one-pass ncu capture, scaled by users)",
                      "algorithmic_bytes_per_launch": conv_bytes * U * d,
                      "avg_launch_ms": conv_avg_ms, "launches_timed": conv_n,
                      "timing": "cudaEvent pair around the convert launch of every %d-th step, on the launching "
@@ -317,7 +380,17 @@ def run_ours(args):
                            "achieved_GBps": step_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9,
                            "frac_of_peak": step_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9 / peak},
         "kernels": breakdown,
+        "kernels_note": "a separate eager pass with every kernel class traced: each traced launch carries two "
+                        "event records, so the classes add up to a few per cent more than ms_per_step",
+        "sustained": {"steps": sus_steps, "ms_per_step": sus_ms / sus_steps,
+                      "value": job_throughput_gbs(world, in_bytes, sus_steps, sus_ms), "unit": UNIT,
+                      "device_seconds": sus_ms * 1e-3, "clocks": sus_clocks,
+                      "roofline": {"achieved": conv_bytes * U * d / (sus_conv_ms / max(sus_conv_n, 1) * 1e-3) / 1e9,
+                                   "frac": conv_bytes * U * d / (sus_conv_ms / max(sus_conv_n, 1) * 1e-3) / 1e9 / peak,
+                                   "avg_launch_ms": sus_conv_ms / max(sus_conv_n, 1), "launches_timed": sus_conv_n}},
     }
+    if other_rec is not None:
+        result["lagged_bias" if other == "lagged" else "current_bias"] = other_rec
     if graph_ms is not None:
         result["graph_replay"] = {"ms_per_step": graph_ms, "value": job_throughput_gbs(1, in_bytes, 1, graph_ms),
                                   "unit": UNIT, "note": "the same steps replayed from one captured CUDA graph"}
@@ -523,8 +596,9 @@ def main():
                     help="override the number of simulated users (profiling a smaller case); default 8")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
-    ap.add_argument("--mode", default="lagged", choices=["lagged", "current", "code-lagged"],
-                    help="bias/code mode of the plan (default: lagged bias, the benchmark configuration)")
+    ap.add_argument("--mode", default="current", choices=["lagged", "current", "code-lagged"],
+                    help="bias/code mode behind `value` (default: current, the bias of Algorithm 1 as printed; "
+                         "the lagged bias is timed beside it)")
     ap.add_argument("--slices", action="store_true",
                     help="cut the one workload into slices of d, one per rank (strong scaling), instead of replicas")
     ap.add_argument("--oracle-worker", default=None, help=argparse.SUPPRESS)

@@ -12,8 +12,10 @@
  *
  * Conventions
  *  - Every pointer marked "device" is CUDA device memory owned by the caller; "host" is host
- *    memory.  The plan owns its scratch, tables and status word; no call after co3_plan_create
- *    allocates memory.
+ *    memory.  The plan owns its scratch, tables, status word, and the two copy streams and four
+ *    events of co3_iteration_host; no call after co3_plan_create allocates device memory or creates
+ *    a stream or an event (co3_profile_enable creates the events it is asked for; the inspection
+ *    hooks co3_debug_* use temporary host memory).
  *  - co3_encode / co3_decode_aggregate only enqueue work on `cuda_stream` (a cudaStream_t cast
  *    to void*, NULL = default stream) and return without synchronising.  Calls on one plan must
  *    be issued on one stream (or be ordered by the caller).
@@ -56,8 +58,15 @@ extern "C" {
 #define CO3_FLAG_NONFINITE 4u
 #define CO3_FLAG_TIMEOUT 8u  /* a bounded wait between thread blocks ran out (should never happen) */
 
-#define CO3_BIAS_CURRENT 0 /* b_t from the moments of g_t + gamma m_{t-1} itself: one extra read pass */
-#define CO3_BIAS_LAGGED 1  /* that pass at t = 0 only; b_t (t >= 1) from the fit of iteration t-1      */
+/* CO3_BIAS_CURRENT is Algorithm 1 as printed: the bias b_t is chosen "at each time t" for the
+ * distribution of g_t + gamma m_{t-1} itself (Sec. III (i), Eq. "exp bias"), which costs one extra
+ * read pass over gradient and memory per iteration.
+ * CO3_BIAS_LAGGED is NOT Algorithm 1's per-iteration bias: that pass runs at t = 0 only, and b_t for
+ * t >= 1 is the rule applied to the fit of iteration t-1 (whose moments ride along with its conversion
+ * pass); the code of iteration t is still designed from iteration t's own fit.  It relies on the fitted
+ * model drifting slowly from one iteration to the next. */
+#define CO3_BIAS_CURRENT 0
+#define CO3_BIAS_LAGGED 1
 /* Not in the paper's Algorithm 1, which fits "at each time t": bias AND code model of iteration
  * t >= 1 come from the fit of iteration t-1, so the whole header of an iteration is known before its
  * gradient is seen and conversion and packing are one pass over the data (the symbols never go to
@@ -252,11 +261,11 @@ int co3_state_header(co3_plan* plan, int32_t import, co3_seg_header* next_header
 #define CO3_K_STATS 0        /* moments of g + gamma m (t = 0, or every t in CURRENT mode) */
 #define CO3_K_FIT 1          /* GenNorm fit, bias, header                                   */
 #define CO3_K_CONVERT 2      /* fused EF-add / convert / residual / histogram / moments      */
-#define CO3_K_CODE_ENC 3     /* (unused: codes are built once at plan creation)              */
+#define CO3_K_CODE_ENC 3     /* CO3_CODE_EMPIRICAL only: code build from the histogram (model codes are built once, at plan creation) */
 #define CO3_K_ENC_LEN 4      /* (unused: the lengths are taken inside the packing kernel)    */
 #define CO3_K_ENC_SCAN 5     /* chunk offsets (CO3_CODE_LAGGED only)                         */
 #define CO3_K_ENC_PACK 6     /* lengths + offsets + bit packing (CO3_CODE_LAGGED: concatenation) */
-#define CO3_K_CODE_DEC 7     /* (unused: codes are built once at plan creation)              */
+#define CO3_K_CODE_DEC 7     /* CO3_CODE_EMPIRICAL only: decoder tables from the received code lengths */
 #define CO3_K_DECODE 8       /* decode + aggregate                                           */
 #define CO3_NUM_KERNELS 9
 int co3_profile_enable(co3_plan* plan, uint32_t kernel_mask, int32_t max_records);
@@ -278,10 +287,36 @@ int co3_debug_symbols(co3_plan* plan, uint8_t* symbols, void* cuda_stream);
 int co3_debug_hist(co3_plan* plan, uint64_t* hist);
 int co3_debug_code(co3_plan* plan, const co3_seg_header* hdr, uint8_t* lengths, uint32_t* codewords);
 
+/* Test hook: from now on every fit of this plan takes (beta, alpha) of segment l from fit[2l], fit[2l+1]
+ * (host, [n_segments][2]; alpha = 0 means the degenerate all-zero segment) instead of solving the moment
+ * equations; bias and header follow from them by the usual rules, the moments reported by co3_get_fit
+ * stay the plan's own.  NULL switches it off.  A harness uses it to feed another implementation's fit
+ * and so tell a header that differs by a rounding of the fit from a fault further down.  Synchronises. */
+int co3_set_fit_override(co3_plan* plan, const double* fit);
+
+/* Test hook for the bounded waits of the encoder.  The thread blocks of co3_encode's packing kernel
+ * learn their chunk's place from the sizes that the blocks of the earlier chunks publish; each such wait
+ * polls a limited number of times and then gives up, raises CO3_FLAG_TIMEOUT and writes no payload.
+ * This call runs that kernel over the symbols of the last co3_encode with the block of (user 0, chunk 0)
+ * left out and the limit set to spin_limit polls (1 .. 2^20), so that the waits for that chunk's size run
+ * out: afterwards co3_status reports CO3_FLAG_TIMEOUT, the chunks of user 0 after the first are not
+ * written, and the device is as usable as before.  Needs a plan that keeps symbols (not
+ * CO3_CODE_LAGGED, not CO3_CODE_EMPIRICAL), at least one encoded iteration and at least two chunks. */
+int co3_debug_encode_stalled(co3_plan* plan, uint32_t* bitstream, uint16_t* sub_bits, uint32_t* chunk_off,
+                             uint64_t* user_bits, const co3_seg_header* hdr, int32_t spin_limit,
+                             void* cuda_stream);
+
 /* Host only, no GPU needed: integer model weights of the quantised GenNorm source for header
  * indices (ibeta in [-14, 8], ir in [-96, 31]), one per symbol byte, 2^(1+E+M) entries.  The
  * Huffman code of a segment is built from exactly these numbers (Sec. III (ii)). */
 int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint32_t* weights);
+
+/* Host only.  Users and parameter server rebuild every code from the header alone (Algorithm 1 lines 9
+ * and 13), i.e. from these weights, which each side computes with its own math library (lgamma, pow,
+ * exp): the two sides agree when they run the same build of this library against the same libm.  This
+ * is a 64-bit FNV-1a digest of the whole weight table of a format (all 23 x 128 index pairs); exchange
+ * and compare it once before the first iteration.  0: unsupported format or out of memory. */
+uint64_t co3_model_checksum(co3_format fmt);
 
 /* Host only: the table behind CO3_RULE_OPT, 23 x 8 int16: for shape index ibeta + 14 and residue
  * rho = round(8 log2 alpha) mod 8, the ir (congruent to rho) of least expected squared conversion

@@ -26,7 +26,8 @@ EXPORTS = [
     "co3_moments_static", "co3_state_header", "co3_decode_aggregate_update",
     "co3_bias_opt_table", "co3_grid_distortion", "co3_encode_empirical", "co3_decode_aggregate_empirical",
     "co3_profile_stride", "co3_tiled_begin", "co3_tiled_statistics", "co3_tiled_convert", "co3_tiled_finish",
-    "co3_moments_export", "co3_moments_import",
+    "co3_moments_export", "co3_moments_import", "co3_set_fit_override", "co3_debug_encode_stalled",
+    "co3_model_checksum",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -130,6 +131,12 @@ def lib():
     L.co3_bias_opt_table.argtypes = [Format, vp]
     L.co3_grid_distortion.restype = C.c_double
     L.co3_grid_distortion.argtypes = [Format, C.c_int32, C.c_int32]
+    L.co3_set_fit_override.restype = C.c_int
+    L.co3_set_fit_override.argtypes = [vp, vp]
+    L.co3_debug_encode_stalled.restype = C.c_int
+    L.co3_debug_encode_stalled.argtypes = [vp] * 6 + [C.c_int32, vp]
+    L.co3_model_checksum.restype = C.c_uint64
+    L.co3_model_checksum.argtypes = [Format]
     L.co3_strerror.restype = C.c_char_p
     L.co3_strerror.argtypes = [C.c_int]
     _lib = L
@@ -143,6 +150,11 @@ def model_weights(exp_bits, mant_bits, ibeta, ir):
     if rc != OK:
         raise Co3Error(rc, "co3_model_weights")
     return w
+
+
+def model_checksum(exp_bits, mant_bits):
+    """Host only: digest of the whole model-weight table of a format (0: unsupported format)."""
+    return int(lib().co3_model_checksum(Format(exp_bits, mant_bits)))
 
 
 def bias_opt_table(exp_bits, mant_bits):
@@ -378,6 +390,27 @@ class Plan:
         if rc != OK:
             raise Co3Error(rc, "co3_get_fit")
         return tuple(x.value for x in v)        # beta, alpha, N, S1, S2
+
+    def set_fit_override(self, fit=None):
+        """Test hook: every later fit takes (beta, alpha) per segment from `fit` ([S][2] float64);
+        None switches it off."""
+        if fit is None:
+            rc = lib().co3_set_fit_override(self.handle, None)
+        else:
+            f = np.ascontiguousarray(fit, np.float64)
+            assert f.shape == (self.S, 2)
+            rc = lib().co3_set_fit_override(self.handle, f.ctypes.data)
+        if rc != OK:
+            raise Co3Error(rc, "co3_set_fit_override")
+
+    def debug_encode_stalled(self, out, spin_limit=1000, stream=None):
+        """Test hook: the packing kernel once more with the block of (user 0, chunk 0) left out, so that
+        the bounded waits for that chunk's size run out after spin_limit polls (FLAG_TIMEOUT)."""
+        rc = lib().co3_debug_encode_stalled(self.handle, _ptr(out["bitstream"]), _ptr(out["sub_bits"]),
+                                            _ptr(out["chunk_off"]), _ptr(out["user_bits"]), _ptr(out["hdr"]),
+                                            int(spin_limit), self._stream(stream))
+        if rc != OK:
+            raise Co3Error(rc, "co3_debug_encode_stalled")
 
     def state_export(self):
         it = C.c_int64()

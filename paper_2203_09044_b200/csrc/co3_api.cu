@@ -2,6 +2,7 @@
 // Algorithm 1 (lines 8-10 at the users: co3_encode; lines 13-14 at the server:
 // co3_decode_aggregate).  Everything is enqueued on the caller's stream; nothing here allocates
 // after co3_plan_create and nothing synchronises except the inspection calls.
+#include <mutex>
 #include <new>
 #include <stdlib.h>
 #include <string.h>
@@ -47,7 +48,29 @@ int alloc_codebook(co3_plan* pl, Co3CodeBook& cb, size_t R, int ncand) {
 
 inline cudaStream_t as_stream(void* s) { return (cudaStream_t)s; }
 
-bool g_kernels_ready = false;
+// cudaFuncSetAttribute applies to the current device: one flag per device, set under a lock
+constexpr int MAX_DEVICES = 64;
+bool g_kernels_ready[MAX_DEVICES];
+std::mutex g_kernels_mutex;
+
+cudaError_t setup_kernels_once(int device) {
+    std::lock_guard<std::mutex> lock(g_kernels_mutex);
+    if (device >= 0 && device < MAX_DEVICES && g_kernels_ready[device]) return cudaSuccess;
+    cudaError_t e = co3_setup_kernels();
+    if (e == cudaSuccess) e = co3_setup_decode_kernels();
+    if (e == cudaSuccess && device >= 0 && device < MAX_DEVICES) g_kernels_ready[device] = true;
+    return e;
+}
+
+cudaError_t create_host_pipe(co3_plan* pl) {      // co3_iteration_host: copy streams and ordering events
+    cudaError_t e = cudaStreamCreateWithFlags(&pl->s_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&pl->s_out, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&pl->ev_h2d, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&pl->ev_conv, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&pl->ev_dec, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&pl->ev_d2h, cudaEventDisableTiming);
+    return e;
+}
 
 }  // namespace
 
@@ -121,10 +144,12 @@ extern "C" int64_t co3_launch_count(const co3_plan* pl) { return pl ? pl->launch
 extern "C" void co3_plan_destroy(co3_plan* pl) {
     if (!pl) return;
     free_events(pl);
-    if (pl->host_pipe_ready) {
-        cudaStreamDestroy(pl->s_in); cudaStreamDestroy(pl->s_out);
-        cudaEventDestroy(pl->ev_h2d); cudaEventDestroy(pl->ev_conv); cudaEventDestroy(pl->ev_dec); cudaEventDestroy(pl->ev_d2h);
-    }
+    if (pl->s_in) cudaStreamDestroy(pl->s_in);
+    if (pl->s_out) cudaStreamDestroy(pl->s_out);
+    if (pl->ev_h2d) cudaEventDestroy(pl->ev_h2d);
+    if (pl->ev_conv) cudaEventDestroy(pl->ev_conv);
+    if (pl->ev_dec) cudaEventDestroy(pl->ev_dec);
+    if (pl->ev_d2h) cudaEventDestroy(pl->ev_d2h);
     for (int i = 0; i < pl->n_allocs; ++i) cudaFree(pl->allocs[i]);
     free(pl->h_seg_off);
     delete pl;
@@ -260,6 +285,8 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         }
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
         a |= dev_alloc(pl, &pl->ext_mom, (size_t)S * 3);
+        a |= dev_alloc(pl, &pl->fit_ovr, (size_t)S * 2);
+        dv.spin_limit = 1 << 20;
         int16_t* d_opt = nullptr;
         const int16_t* h_opt = co3_host_bias_opt_table(E, M);
         a |= dev_alloc(pl, &d_opt, (size_t)CO3_NIBETA * 8);
@@ -305,11 +332,9 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             dv.ticket = reinterpret_cast<unsigned int*>(dv.hist + (size_t)dv.hist_copies * S * CO3_MAXSYM);
             if (e == cudaSuccess && dv.sym) e = cudaMemset(dv.sym, 0, (size_t)dv.U * (size_t)dv.sld);
             if (e == cudaSuccess) e = cudaMemset(dv.hdr_cur, 0, sizeof(co3_seg_header) * (size_t)S);
-            if (e == cudaSuccess && !g_kernels_ready) {
-                e = co3_setup_kernels();
-                if (e == cudaSuccess) e = co3_setup_decode_kernels();
-                g_kernels_ready = (e == cudaSuccess);
-            }
+            if (e == cudaSuccess) e = setup_kernels_once(pl->device);
+            if (e == cudaSuccess) e = create_host_pipe(pl);
+            pl->host_pipe_ready = (e == cudaSuccess);
             if (e != cudaSuccess) { (void)cudaGetLastError(); rc = CO3_ECUDA; }
             dv.chunks = d_chunks; dv.groups = d_groups; dv.seg_off = d_seg_off;
             dv.seg_chunk0 = d_seg_chunk0; dv.wtab = d_wtab; dv.logr_tab = d_logr;
@@ -509,15 +534,7 @@ extern "C" int co3_iteration_host(co3_plan* pl, const float* h_grad, float* d_gr
     // back (PCIe is full duplex).  d_grad is free as soon as the convert pass of the previous call
     // has read it; everything else is ordered through the caller's stream, which at the end of the
     // call also waits for the copy of the average, so synchronising it is still all the caller does.
-    if (!pl->host_pipe_ready) {
-        CO3_TRY(cudaStreamCreateWithFlags(&pl->s_in, cudaStreamNonBlocking));
-        CO3_TRY(cudaStreamCreateWithFlags(&pl->s_out, cudaStreamNonBlocking));
-        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_h2d, cudaEventDisableTiming));
-        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_conv, cudaEventDisableTiming));
-        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_dec, cudaEventDisableTiming));
-        CO3_TRY(cudaEventCreateWithFlags(&pl->ev_d2h, cudaEventDisableTiming));
-        pl->host_pipe_ready = true;
-    }
+    if (!pl->host_pipe_ready) return CO3_ECUDA;       // (its streams and events are made by co3_plan_create)
     if (pl->ev_conv_recorded) CO3_TRY(cudaStreamWaitEvent(pl->s_in, pl->ev_conv, 0));
     CO3_TRY(cudaMemcpyAsync(d_grad, h_grad, sizeof(float) * (size_t)pl->dev.U * (size_t)pl->dev.ld,
                             cudaMemcpyHostToDevice, pl->s_in));
@@ -600,6 +617,32 @@ extern "C" int co3_state_header(co3_plan* pl, int32_t import, co3_seg_header* ne
     } else {
         CO3_TRY(cudaMemcpy(next_header, pl->dev.hdr_cur, bytes, cudaMemcpyDeviceToHost));
     }
+    return CO3_OK;
+}
+
+extern "C" int co3_set_fit_override(co3_plan* pl, const double* fit) {
+    if (!pl) return CO3_EINVAL;
+    CO3_TRY(cudaStreamSynchronize(pl->last_stream));
+    pl->use_fit_ovr = false;
+    if (!fit) return CO3_OK;
+    for (int l = 0; l < pl->dev.S; ++l)
+        if (!(fit[2 * l] > 0.0) || !(fit[2 * l + 1] >= 0.0) || !(fit[2 * l + 1] < 1e300)) return CO3_EINVAL;
+    CO3_TRY(cudaMemcpy(pl->fit_ovr, fit, sizeof(double) * 2 * (size_t)pl->dev.S, cudaMemcpyHostToDevice));
+    pl->use_fit_ovr = true;
+    return CO3_OK;
+}
+
+extern "C" int co3_debug_encode_stalled(co3_plan* pl, uint32_t* bitstream, uint16_t* sub_bits, uint32_t* chunk_off,
+                                        uint64_t* user_bits, const co3_seg_header* hdr, int32_t spin_limit,
+                                        void* cuda_stream) {
+    if (!pl || !bitstream || !sub_bits || !chunk_off || !user_bits || !hdr) return CO3_EINVAL;
+    if ((uintptr_t)bitstream & 15 || spin_limit < 1 || spin_limit > (1 << 20)) return CO3_EINVAL;
+    if (!pl->dev.sym || pl->cfg.bias_mode == CO3_CODE_EMPIRICAL || pl->iteration < 1) return CO3_EINVAL;
+    if (pl->dev.n_chunks * (int64_t)pl->dev.U < 2) return CO3_EINVAL;
+    cudaStream_t st = as_stream(cuda_stream);
+    pl->last_stream = st;
+    CO3_TRY(co3_launch_encode_stalled(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits,
+                                      spin_limit, st));
     return CO3_OK;
 }
 

@@ -143,11 +143,11 @@ __device__ __forceinline__ void put_piece(uint32_t* s_buf, uint32_t pos, unsigne
 // CO3_FLAG_TIMEOUT and the block writes nothing.
 constexpr uint32_t ST_VALID = 0x80000000u;
 constexpr int GRP_SHIFT = 6, GRP_SIZE = 1 << GRP_SHIFT;
-constexpr int SPIN_LIMIT = 1 << 20;          // polls of a word in L2: about a second, then give up
+// (the polls of a word in L2 are limited by Co3Dev::spin_limit: 2^20 of them take about a second)
 
-__device__ __forceinline__ uint32_t wait_count(const uint32_t* st, bool& timeout) {
+__device__ __forceinline__ uint32_t wait_count(const uint32_t* st, int spin_limit, bool& timeout) {
     const volatile uint32_t* v = st;
-    for (int k = 0; k < SPIN_LIMIT; ++k) {
+    for (int k = 0; k < spin_limit; ++k) {
         const uint32_t w = *v;
         if (w & ST_VALID) return w & ~ST_VALID;
     }
@@ -155,9 +155,10 @@ __device__ __forceinline__ uint32_t wait_count(const uint32_t* st, bool& timeout
     return 0;
 }
 // waits until `expect` chunks have arrived in the group; returns words << 32 | bits
-__device__ __forceinline__ unsigned long long wait_group(const unsigned long long* grp, uint32_t expect, bool& timeout) {
+__device__ __forceinline__ unsigned long long wait_group(const unsigned long long* grp, uint32_t expect, int spin_limit,
+                                                         bool& timeout) {
     const volatile unsigned long long* v = grp;
-    for (int k = 0; k < SPIN_LIMIT; ++k) {
+    for (int k = 0; k < spin_limit; ++k) {
         const unsigned long long w = *v;
         if ((w >> 56) == (unsigned long long)expect) return w & ((1ull << 56) - 1);
     }
@@ -168,7 +169,7 @@ __device__ __forceinline__ unsigned long long wait_group(const unsigned long lon
 __global__ void __launch_bounds__(ENC_THREADS, 20)
 enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __restrict__ sub_bits,
                   uint32_t* __restrict__ chunk_off, unsigned long long* __restrict__ user_bits,
-                  uint32_t* __restrict__ bitstream) {
+                  uint32_t* __restrict__ bitstream, uint32_t n_items) {
     __shared__ __align__(16) uint8_t s_len[CO3_MAXSYM];
     __shared__ __align__(16) uint32_t s_enc[CO3_MAXSYM];            // codeword | length << 16
     __shared__ __align__(16) uint32_t s_buf[BUF_WORDS + 4];         // image of the chunk
@@ -178,6 +179,7 @@ enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __
     if (tid == 0) s_item = atomicAdd(p.enc_ticket, 1u);
     __syncthreads();
     const uint32_t item = s_item;
+    if (item >= n_items) return;                      // (only a launch that did not start the tickets at 0 gets here)
     bool bad = false;
     Item it;
     open_item(it, p, tid, item);
@@ -257,9 +259,9 @@ enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __
     bool timeout = false;
     uint32_t sum = 0;
     for (uint32_t i = tid; i < grp; i += ENC_THREADS)
-        sum += (uint32_t)(wait_group(p.enc_grp + (size_t)it.u * p.n_grp + i, GRP_SIZE, timeout) >> 32);
+        sum += (uint32_t)(wait_group(p.enc_grp + (size_t)it.u * p.n_grp + i, GRP_SIZE, p.spin_limit, timeout) >> 32);
     if ((uint32_t)tid < (it.c & (GRP_SIZE - 1)))
-        sum += wait_count(p.enc_st + (size_t)it.u * p.n_chunks + ((size_t)grp << GRP_SHIFT) + tid, timeout);
+        sum += wait_count(p.enc_st + (size_t)it.u * p.n_chunks + ((size_t)grp << GRP_SHIFT) + tid, p.spin_limit, timeout);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     if (lane == 0) s_sum[warp] = sum;
@@ -280,7 +282,7 @@ enc_single_kernel(Co3Dev p, const co3_seg_header* __restrict__ hdr, uint16_t* __
         unsigned long long ub = 0;
         for (uint32_t i = lane; i <= grp; i += 32) {
             const uint32_t expect = (i < grp) ? (uint32_t)GRP_SIZE : (it.c & (GRP_SIZE - 1)) + 1u;
-            ub += wait_group(p.enc_grp + (size_t)it.u * p.n_grp + i, expect, t2) & 0xFFFFFFFFull;
+            ub += wait_group(p.enc_grp + (size_t)it.u * p.n_grp + i, expect, p.spin_limit, t2) & 0xFFFFFFFFull;
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ub += __shfl_xor_sync(0xffffffffu, ub, o);
@@ -384,7 +386,27 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
     const unsigned items = (unsigned)(p.n_chunks * (int64_t)p.U);
     // (tickets, published counts and group totals were cleared by the fit kernel that ran before)
     co3_prof_begin(pl, CO3_K_ENC_PACK, st);
-    enc_single_kernel<<<items, ENC_THREADS, 0, st>>>(p, hdr, sub_bits, chunk_off, user_bits, bitstream);
+    enc_single_kernel<<<items, ENC_THREADS, 0, st>>>(p, hdr, sub_bits, chunk_off, user_bits, bitstream, items);
     co3_prof_end(pl, CO3_K_ENC_PACK, st, 1);
+    return cudaGetLastError();
+}
+
+// Test hook behind co3_debug_encode_stalled: the same kernel over the symbols of the last iteration,
+// but the tickets start at 1 and one block fewer is launched, so item 0 (user 0, chunk 0) is never
+// claimed and never publishes its size.  Every block that needs that size polls spin_limit times, gives
+// up, raises CO3_FLAG_TIMEOUT and writes no payload; nothing waits without a limit.
+cudaError_t co3_launch_encode_stalled(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
+                                      uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
+                                      int spin_limit, cudaStream_t st) {
+    Co3Dev p = pl->dev;
+    const unsigned items = (unsigned)(p.n_chunks * (int64_t)p.U);
+    if (items < 2) return cudaErrorInvalidValue;
+    p.spin_limit = spin_limit;
+    cudaError_t e = cudaMemsetAsync(p.enc_grp, 0, pl->enc_sync_bytes, st);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(p.enc_ticket, 1, 1, st);       // low byte of the zeroed ticket: the first ticket drawn is 1
+    if (e != cudaSuccess) return e;
+    enc_single_kernel<<<items - 1, ENC_THREADS, 0, st>>>(p, hdr, sub_bits, chunk_off, user_bits, bitstream, items);
+    pl->launches += 1;
     return cudaGetLastError();
 }

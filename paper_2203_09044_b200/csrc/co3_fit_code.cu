@@ -31,7 +31,7 @@ constexpr int RED_THREADS = 256;
 __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int clear_enc_sync) {
     __shared__ double s_a[RED_THREADS / 32], s_b[RED_THREADS / 32];
     __shared__ unsigned long long s_n[RED_THREADS / 32];
-    const int seg = blockIdx.y, slice = blockIdx.x, tid = threadIdx.x;
+    const int seg = blockIdx.x, slice = blockIdx.y, tid = threadIdx.x;   // (the x extent has no 65535 limit)
     if (clear_enc_sync) {                              // (see fit_kernel: here the many blocks share that job)
         const size_t nb = (size_t)gridDim.x * gridDim.y, b = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
         for (size_t i = b * RED_THREADS + tid; i < p.enc_sync_words64; i += nb * RED_THREADS) p.enc_grp[i] = 0ull;
@@ -78,9 +78,12 @@ __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int c
 // mode 4: only add up the moments of every segment and write (N, S1, S2) to mom_out.
 // ext_mom (may be null): (N, S1, S2) per segment that replace the plan's own sums in the fit (the sums
 //         of a layer that is spread over several plans); the non-finite count stays the plan's own.
+// fit_ovr (may be null): (beta, alpha) per segment that replace the solve (test hook: a harness feeds
+//         another implementation's fit to tell a rounding of the fit from a fault further down).
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr,
                                                           const double* __restrict__ ext_mom,
-                                                          double* __restrict__ mom_out) {
+                                                          double* __restrict__ mom_out,
+                                                          const double* __restrict__ fit_ovr) {
     __shared__ double s_a[FIT_THREADS / 32], s_b[FIT_THREADS / 32];
     __shared__ unsigned long long s_n[FIT_THREADS / 32];
     __shared__ double s_lg[3];
@@ -146,7 +149,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     __syncthreads();
     if (tid == 0) {
         s_state = 0; s_coarse = 0; s_fine = 0;
-        if (!(N > 0.0) || !(S1 > 0.0)) { s_state = 2; s_t = 0.0; }          // beta = 1, alpha = 0
+        if (fit_ovr) { s_state = fit_ovr[2 * seg + 1] > 0.0 ? 3 : 2; s_t = 0.0; }   // given; alpha = 0: as below
+        else if (!(N > 0.0) || !(S1 > 0.0)) { s_state = 2; s_t = 0.0; }     // beta = 1, alpha = 0
         else {
             s_target = s_lg[0] + s_lg[1] - 2.0 * s_lg[2];
             if (s_target >= tab[0]) { s_state = 1; s_t = T0; s_fine = 0; }
@@ -191,15 +195,18 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     } else if (s_state == 1) {
         beta = (t == T0) ? 0.3 : 2.0;
         log_g = tabg[s_fine];
+    } else if (s_state == 3) {
+        beta = fit_ovr[2 * seg];
+        log_g = 0.0;
     } else {
         beta = 1.0;
         log_g = 0.0;
     }
     const double log2e = 1.4426950408889634;
     // alpha = (S1 / N) * G(beta); its base-2 logarithm without forming alpha first
-    const double log2_alpha = (s_state == 2) ? 0.0 : (s_lg[2] - s_lg[0] + log_g) * log2e;
+    const double log2_alpha = (s_state == 2) ? 0.0 : (s_state == 3 ? log2(fit_ovr[2 * seg + 1]) : (s_lg[2] - s_lg[0] + log_g) * log2e);
     const bool has_alpha = s_state != 2;
-    const double alpha = has_alpha ? exp2(log2_alpha) : 0.0;
+    const double alpha = has_alpha ? (s_state == 3 ? fit_ovr[2 * seg + 1] : exp2(log2_alpha)) : 0.0;
     int b_rule = p.b_lo;
     if (has_alpha && alpha > 0.0) {
         if (p.bias_rule == CO3_RULE_OPT) {
@@ -429,10 +436,11 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
     co3_prof_begin(pl, CO3_K_FIT, st);
-    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.red_k, pl->dev.S), RED_THREADS, 0, st>>>(pl->dev, mode == 1);
+    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1);
     const double* ext = (pl->use_ext_mom && mode != 4) ? pl->ext_mom : nullptr;
     if (mode != 4) pl->use_ext_mom = false;                // imported moments serve one fit
-    fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out);
+    fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out,
+                                                  (pl->use_fit_ovr && mode != 4) ? pl->fit_ovr : nullptr);
     co3_prof_end(pl, CO3_K_FIT, st, pl->dev.red_k > 0 ? 2 : 1);
     return cudaGetLastError();
 }

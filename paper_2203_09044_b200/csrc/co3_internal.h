@@ -114,6 +114,7 @@ struct Co3Dev {
     unsigned int* enc_ticket;     // ... item ticket (the three live in one allocation, cleared per launch)
     int64_t n_grp;
     size_t enc_sync_words64;      // size of that allocation in 64-bit words
+    int spin_limit;               // polls after which a wait between thread blocks gives up (CO3_FLAG_TIMEOUT)
     uint32_t* flags;              // sticky status flags
     unsigned long long* nonfinite_total;
 };
@@ -141,6 +142,8 @@ struct co3_plan {
     double* ext_mom;                // [S][3] moments handed in by co3_moments_import
     bool use_ext_mom;               // ... and not yet consumed by a fit
     double* mom_out;                // co3_moments_export: where the reduction-only fit launch writes
+    double* fit_ovr;                // [S][2] (beta, alpha) handed in by co3_set_fit_override
+    bool use_fit_ovr;               // ... and in force until it is cleared
     bool record_conv;               // co3_encode records ev_conv after its last pass over the gradient
     void* allocs[128];
     int n_allocs;
@@ -203,6 +206,9 @@ cudaError_t co3_launch_encode(co3_plan* pl, const co3_seg_header* hdr, uint32_t*
 cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
                               const uint32_t* chunk_off, const co3_seg_header* hdr, float* avg,
                               float* weights, float step, cudaStream_t st);
+cudaError_t co3_launch_encode_stalled(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
+                                      uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
+                                      int spin_limit, cudaStream_t st);
 cudaError_t co3_setup_kernels(void);
 cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_t st);
 

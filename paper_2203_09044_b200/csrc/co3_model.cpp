@@ -232,6 +232,17 @@ extern "C" int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint
     return CO3_OK;
 }
 
+extern "C" uint64_t co3_model_checksum(co3_format fmt) {
+    if (!co3_host_fmt_ok(fmt)) return 0;
+    const uint32_t* t = co3_host_weight_table(fmt.exp_bits, fmt.mant_bits);
+    if (!t) return 0;
+    const size_t n = (size_t)CO3_NIBETA * CO3_NIR * ((size_t)1 << (fmt.exp_bits + fmt.mant_bits));
+    uint64_t h = 0xcbf29ce484222325ull;              // FNV-1a over the table's words, byte by byte, low byte first
+    for (size_t i = 0; i < n; ++i)
+        for (int b = 0; b < 4; ++b) { h ^= (t[i] >> (8 * b)) & 0xFFu; h *= 0x100000001b3ull; }
+    return h ? h : 1;
+}
+
 extern "C" int64_t co3_partition(int64_t d, int32_t n_segments, const int64_t* seg_offsets,
                                  int32_t* chunk_seg, int64_t* chunk_start, int64_t* chunk_end,
                                  int64_t* sub_base, int64_t* n_sub) {

@@ -377,6 +377,80 @@ def test_decode_with_fused_model_update(binding, oracle, U, E, M):
     assert plan.status()[0] == 0
 
 
+def test_fit_override_gives_the_oracles_header_from_the_oracles_fit(binding, oracle):
+    """Test hook co3_set_fit_override: with the oracle's (beta, alpha) handed in, bias and header come
+    out as the oracle's for those numbers, whatever the plan's own moments are; switched off, the
+    plan fits its own moments again."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=90_000, n_users=3)
+    b = binding
+    plan = b.Plan(wl.d, wl.n_users, 4, 3, wl.seg_offsets, gamma=wl.gamma, bias_mode=b.BIAS_CURRENT)
+    out = plan.alloc_outputs()
+    m = torch.zeros((wl.n_users, plan.ld), dtype=torch.float32, device="cuda")
+    g = wl.gradient(0, device="cuda")
+    rng = np.random.default_rng(5)
+    fit = np.stack([rng.uniform(0.3, 2.0, plan.S), 10.0 ** rng.uniform(-6, 1, plan.S)], axis=1)
+    fit[3] = (1.0, 0.0)                                      # a segment declared all-zero
+    plan.set_fit_override(fit)
+    plan.encode(g, m, out)
+    hdr = b.hdr_to_numpy(out["hdr"])
+    for l in range(plan.S):
+        beta, alpha = float(fit[l, 0]), float(fit[l, 1])
+        bias = oracle.bias(beta, alpha, 4, 3)
+        assert tuple(hdr[l]) == (bias,) + tuple(oracle.header(beta, alpha, bias)), l
+        assert plan.get_fit(l)[:2] == (beta, alpha)
+    plan.set_fit_override(None)
+    m.zero_()
+    plan2 = b.Plan(wl.d, wl.n_users, 4, 3, wl.seg_offsets, gamma=wl.gamma, bias_mode=b.BIAS_CURRENT)
+    out2 = plan2.alloc_outputs()
+    m2 = torch.zeros_like(m)
+    plan.encode(g, m, out)
+    plan2.encode(g, m2, out2)
+    assert torch.equal(out["hdr"], out2["hdr"]) and torch.equal(out["chunk_off"], out2["chunk_off"])
+    for u in range(wl.n_users):                              # (beyond a row's payload lies the first call's)
+        n = int(out["chunk_off"][u, -1])
+        assert torch.equal(out["bitstream"][u, :n], out2["bitstream"][u, :n])
+    with pytest.raises(b.Co3Error):
+        plan.set_fit_override(np.full((plan.S, 2), -1.0))
+
+
+def test_bounded_waits_of_the_encoder_run_out_and_report(binding):
+    """Failure detection without a fault: the packing kernel runs with the block of (user 0, chunk 0)
+    left out, so nothing publishes that chunk's size; the blocks that need it poll 1000 times, give
+    up and return.  The flag is raised, the later chunks are not written, and the same plan encodes
+    and decodes normally afterwards."""
+    b = binding
+    d, U = 3 * 4096, 1
+    plan = b.Plan(d, U, 4, 3, None, gamma=0.9)
+    out = plan.alloc_outputs()
+    m = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    g = torch.randn((U, plan.ld), generator=gen, device="cuda") * 1e-3
+    plan.encode(g, m, out)
+    assert plan.status()[0] == 0
+    good = {k: v.clone() for k, v in out.items()}
+    out["bitstream"].fill_(0x5A5A5A5A)
+    plan.debug_encode_stalled(out, spin_limit=1000)
+    flags, _ = plan.status(clear=True)
+    assert flags & b.FLAG_TIMEOUT
+    pay = out["bitstream"].view(-1)
+    assert bool((pay == 0x5A5A5A5A).all())                   # chunk 0 was left out, the others gave up
+    assert torch.equal(out["sub_bits"][0, 32:], good["sub_bits"][0, 32:])   # lengths do not depend on the waits
+    with pytest.raises(b.Co3Error):
+        plan.debug_encode_stalled(out, spin_limit=0)
+    # the device and the plan are as usable as before
+    m.zero_()
+    plan2 = b.Plan(d, U, 4, 3, None, gamma=0.9)
+    out2 = plan2.alloc_outputs()
+    plan2.encode(g, torch.zeros_like(m), out2)
+    plan.state_import(0, np.zeros(plan.S, np.int32))
+    plan.encode(g, m, out)
+    assert plan.status()[0] == 0
+    n = int(out["chunk_off"][0, -1])
+    assert torch.equal(out["bitstream"][0, :n], good["bitstream"][0, :n])
+    assert torch.equal(plan.decode_aggregate(out), plan2.decode_aggregate(out2))
+
+
 def test_decoder_depends_only_on_the_stream(binding, oracle):
     """A second plan that never encoded anything (the parameter server) decodes the outputs."""
     from paper_2203_09044_b200 import inputs
@@ -678,21 +752,25 @@ def test_config1_full_other_modes_two_iterations(binding, oracle, mode, rule):
 
 
 @pytest.mark.slow
-def test_config2_full_one_iteration(binding, oracle):
-    """16 users x d = 14,728,266 in 16 segments with odd offsets, E3M2 (the U > 8 decode path)."""
+def test_config2_full_two_iterations(binding, oracle):
+    """16 users x d = 14,728,266 in 16 segments with odd offsets, E3M2 (the U > 8 decode path).  The
+    second iteration runs on the carried memory with the bias of the first one's fit (Algorithm 1
+    lines 8 and 10 feed iteration t + 1)."""
     from paper_2203_09044_b200 import inputs
     wl = inputs.workload(2)
-    run_case(binding, oracle, wl.d, wl.n_users, 3, 2, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+    run_case(binding, oracle, wl.d, wl.n_users, 3, 2, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma)
 
 
 @pytest.mark.slow
-def test_config3_full_one_iteration(binding, oracle):
-    """4 users x d = 124,439,808 heavy-tailed with outliers, E4M3: the shape estimate clamps at 0.3."""
+def test_config3_full_two_iterations(binding, oracle):
+    """4 users x d = 124,439,808 heavy-tailed with outliers, E4M3: the shape estimate clamps at 0.3.
+    Two iterations, so that the sliced moment reduction of a very long segment also runs on carried
+    state (no statistics pass, non-zero memory, lagged bias)."""
     from paper_2203_09044_b200 import inputs
     wl = inputs.workload(3)
-    plan, orc, out, res = run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 1),
+    plan, orc, out, res = run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 2),
                                    gamma=wl.gamma)
-    assert res[0][0].fit[0, 0] == 0.3
+    assert res[0][0].fit[0, 0] == 0.3 and res[1][0].fit[0, 0] == 0.3
 
 
 # ---- the size / users / shape / format sweep (a subset the oracle can follow) ----------------
@@ -712,6 +790,33 @@ def test_sweep_d_2p20_8_users(binding, oracle, beta, E, M):
     from paper_2203_09044_b200 import inputs
     wl = inputs.sweep_cell(1 << 20, 8, beta, E, M)
     run_case(binding, oracle, wl.d, 8, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("U", [1, 8, 64])
+def test_sweep_d_2p20_laplace_shape(binding, oracle, U, E, M):
+    """d = 2^20 with 1, 8 and 64 users at beta = 1.0, two iterations (the second on carried state)."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 20, U, 1.0, E, M)
+    run_case(binding, oracle, wl.d, U, E, M, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("E,M", FORMATS)
+def test_sweep_d_2p24_8_users(binding, oracle, E, M):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 24, 8, 1.0, E, M)
+    run_case(binding, oracle, wl.d, 8, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+def test_sweep_d_2p24_64_users_fp4(binding, oracle):
+    """The one U = 64 cell above 2^16 that the oracle can follow in about two minutes: 4096 chunks of 64
+    streams each, so every block of the many-user decoder walks dozens of chunks."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 24, 64, 1.0, 1, 2)
+    run_case(binding, oracle, wl.d, 64, 1, 2, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
 
 
 @pytest.mark.slow

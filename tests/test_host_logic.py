@@ -79,6 +79,21 @@ def test_model_weight_table_identical_to_oracle(binding, oracle, E, M):
         binding.model_weights(E, M, 9, 0)
 
 
+def test_model_checksum_is_the_digest_of_the_weight_table(binding):
+    """What two hosts compare before the first iteration: FNV-1a over all 23 x 128 rows of non-negative
+    magnitudes, recomputed here from co3_model_weights."""
+    for E, M in [(1, 2), (3, 2), (4, 3)]:
+        J = 1 << (E + M)
+        h = 0xcbf29ce484222325
+        for ib in range(-14, 9):
+            for ir in range(-96, 32):
+                for byte in binding.model_weights(E, M, ib, ir)[:J].astype("<u4").tobytes():
+                    h = ((h ^ byte) * 0x100000001b3) & 0xFFFFFFFFFFFFFFFF
+        assert binding.model_checksum(E, M) == h != 0
+    assert binding.model_checksum(5, 3) == 0
+    assert len({binding.model_checksum(E, M) for E, M in [(1, 2), (3, 2), (4, 3)]}) == 3
+
+
 def test_partition_identical_to_oracle(binding, oracle):
     from paper_2203_09044_b200 import inputs
     cases = [(10000, [0, 10000]), (9000, [0, 5, 5, 4101, 8192, 9000]), (130, [0, 1, 130]),

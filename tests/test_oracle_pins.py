@@ -446,6 +446,33 @@ def test_stream_roundtrip_and_accounting(oracle, E, M):
             l = int(part.chunk_seg[c])
             s, e = int(part.chunk_start[c]), int(part.chunk_end[c])
             assert cb == int(r.lens[l][r.sym[u, s:e]].astype(np.int64).sum())
+            # the whole chunk, written out again here from the (length, codeword) table alone: codewords
+            # back to back, each one root bit first, stream bit p = bit (p & 31) of word (p >> 5)
+            want = np.zeros(cb, np.uint8)
+            p = 0
+            for sym in r.sym[u, s:e]:
+                L, cw = int(r.lens[l][sym]), int(r.codes[l][sym])
+                for i in range(L):
+                    want[p + i] = (cw >> (L - 1 - i)) & 1
+                p += L
+            assert p == cb and np.array_equal(allbits[:cb], want)
+            # and read back the same way: walk the bits, match the only codeword that fits (prefix code)
+            by_code = {(int(r.lens[l][x]), int(r.codes[l][x])): x for x in range(2 << (E + M))}
+            got_syms, acc, n = [], 0, 0
+            for bit in allbits[:cb]:
+                acc, n = (acc << 1) | int(bit), n + 1
+                assert n <= 16
+                if (n, acc) in by_code:
+                    got_syms.append(by_code[(n, acc)])
+                    acc, n = 0, 0
+            assert n == 0 and np.array_equal(np.array(got_syms, r.sym.dtype), r.sym[u, s:e])
+            # sub-chunk lengths: the bits of the symbols between the row's multiples of 128
+            k = k0
+            for a0 in range(s - s % 128, e, 128):
+                lo_, hi_ = max(a0, s), min(a0 + 128, e)
+                assert int(r.sub_bits[u, k]) == int(r.lens[l][r.sym[u, lo_:hi_]].astype(np.int64).sum())
+                k += 1
+            assert k == k1
             bits += cb
         assert bits == r.user_bits[u]
     # user_bits = sum over segments of hist * len when there is one user
