@@ -27,7 +27,7 @@ EXPORTS = [
     "co3_bias_opt_table", "co3_grid_distortion", "co3_encode_empirical", "co3_decode_aggregate_empirical",
     "co3_profile_stride", "co3_tiled_begin", "co3_tiled_statistics", "co3_tiled_convert", "co3_tiled_finish",
     "co3_moments_export", "co3_moments_import", "co3_set_fit_override", "co3_debug_encode_stalled",
-    "co3_model_checksum",
+    "co3_model_checksum", "co3_balanced_split",
 ]
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
@@ -137,6 +137,8 @@ def lib():
     L.co3_debug_encode_stalled.argtypes = [vp] * 6 + [C.c_int32, vp]
     L.co3_model_checksum.restype = C.c_uint64
     L.co3_model_checksum.argtypes = [Format]
+    L.co3_balanced_split.restype = C.c_int
+    L.co3_balanced_split.argtypes = [vp, vp, C.c_int64, C.c_int32, C.c_int32, vp]
     L.co3_strerror.restype = C.c_char_p
     L.co3_strerror.argtypes = [C.c_int]
     _lib = L
@@ -155,6 +157,17 @@ def model_weights(exp_bits, mant_bits, ibeta, ir):
 def model_checksum(exp_bits, mant_bits):
     """Host only: digest of the whole model-weight table of a format (0: unsupported format)."""
     return int(lib().co3_model_checksum(Format(exp_bits, mant_bits)))
+
+
+def balanced_split(cost, seg, teams, max_blocks):
+    """Host only: cuts (max_blocks + 1 int32) and the number of blocks in use (co3_balanced_split)."""
+    c = np.ascontiguousarray(cost, np.float64)
+    g = np.ascontiguousarray(seg, np.int32)
+    part = np.zeros(max_blocks + 1, np.int32)
+    nb = lib().co3_balanced_split(c.ctypes.data, g.ctypes.data, len(c), int(teams), int(max_blocks), part.ctypes.data)
+    if nb < 0:
+        raise Co3Error(EINVAL, "co3_balanced_split")
+    return part, nb
 
 
 def bias_opt_table(exp_bits, mant_bits):

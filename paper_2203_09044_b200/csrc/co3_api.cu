@@ -336,6 +336,20 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             if (e == cudaSuccess) e = create_host_pipe(pl);
             pl->host_pipe_ready = (e == cudaSuccess);
             if (e != cudaSuccess) { (void)cudaGetLastError(); rc = CO3_ECUDA; }
+            if (e == cudaSuccess) {                  // the decoder's work split (needs the kernels' attributes set)
+                const int max_blocks = co3_decode_max_blocks(dv.U, pl->num_sms);
+                int32_t* h_part = (int32_t*)malloc(sizeof(int32_t) * (size_t)(max_blocks + 1));
+                int32_t* d_part = nullptr;
+                if (!h_part || dev_alloc(pl, &d_part, (size_t)max_blocks + 1) != CO3_OK) rc = CO3_ENOMEM;
+                else {
+                    dv.dec_blocks = co3_decode_partition(h_chunks, nc, h_groups, n_groups, dv.U, max_blocks, h_part);
+                    e = cudaMemcpy(d_part, h_part, sizeof(int32_t) * (size_t)(max_blocks + 1), cudaMemcpyHostToDevice);
+                    dv.dec_part = d_part;
+                    if (dv.dec_blocks < 1) rc = CO3_ENOMEM;
+                    if (e != cudaSuccess) { (void)cudaGetLastError(); rc = CO3_ECUDA; }
+                }
+                free(h_part);
+            }
             dv.chunks = d_chunks; dv.groups = d_groups; dv.seg_off = d_seg_off;
             dv.seg_chunk0 = d_seg_chunk0; dv.wtab = d_wtab; dv.logr_tab = d_logr;
             if (rc == CO3_OK) {                      // Huffman codes of all model rows, once

@@ -35,8 +35,9 @@ namespace {
 
 constexpr int NW = CO3_THREADS / 32;              // warps = concurrent streams per block
 constexpr int PADW = 33;                          // row stride of the transposed accumulator
-// A lane never reads more than 128 * 16 bits past the start of its sub-chunk, so with this much
-// slack after the staged words the staged reader needs no bounds checks.
+// A lane never reads more than 128 * 16 bits (plus the three words its reader holds ahead) past the
+// start of its sub-chunk, so with this much slack after the staged words the staged reader needs no
+// bounds checks.
 constexpr int STAGE_PAD = 72;
 constexpr int STAGE_ROW = CO3_STAGE_WORDS + STAGE_PAD;
 static_assert(STAGE_ROW % 4 == 0, "stage rows must keep 16-byte alignment");
@@ -120,7 +121,8 @@ __device__ __forceinline__ uint32_t decode_long(uint32_t window, const T& t, boo
 }
 
 // LSB-first bit reader over staged words: the stream sits at bits [0, nb) of hi:lo and the bits above
-// are zero; rp is the shared-space byte address of the next word.  A refill is checked once per PAIR
+// are zero; nw is the word after those, already loaded (a refill takes it and loads the one after, so
+// that no refill waits for shared memory), and rp the shared-space byte address of the word after nw.  A refill is checked once per PAIR
 // of symbols: with nb >= 32 two codewords (at most 16 bits each) can be taken without looking at nb,
 // and one more word then always fits.  (With 32 lanes a per-symbol refill branch would be taken on
 // nearly every step, so its cost is paid per step, not per refill.)
@@ -130,13 +132,15 @@ struct Reader {
     uint32_t lo, hi;
     uint32_t nb;
     uint32_t rp;
+    uint32_t nw;                                  // the word before rp: fetched one refill before it is used
 };
 
 __device__ __forceinline__ uint32_t reader_bits(const Reader& r) { return r.nb & 0xFFu; }
 
 __device__ __forceinline__ void refill(Reader& r) {
     if (reader_bits(r) < 32u) {                               // then hi holds no bit
-        const uint32_t w = lds32(r.rp);
+        const uint32_t w = r.nw;
+        r.nw = lds32(r.rp);                                   // not needed before the next refill
         r.lo |= __funnelshift_l(0u, w, r.nb);                 // w << nb
         r.hi = __funnelshift_l(w, 0u, r.nb);                  // w >> (32 - nb), 0 for nb = 0
         r.nb += 32u;
@@ -151,7 +155,20 @@ __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint
     r.lo = (uint32_t)v;
     r.hi = (uint32_t)(v >> 32);
     r.nb = 64u - sh;
-    r.rp += 8;
+    r.nw = lds32(r.rp + 8);
+    r.rp += 12;
+}
+
+template <int OFF>
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.u32 [%0+%2], %1;" ::"r"(addr), "r"(v), "n"(OFF) : "memory");
+}
+// What a decoded symbol does to its cell: added (several users meet there) or stored (one user: the
+// cell is this lane's alone and holds the whole table entry until the read-out).
+template <int OFF, bool STORE>
+__device__ __forceinline__ void put_cell(uint32_t addr, uint32_t v) {
+    if (STORE) sts32<OFF>(addr, v);
+    else red_add<OFF>(addr, v);
 }
 
 // One symbol, fast form: look up, consume, add to the accumulator row at byte offset OFF, return
@@ -159,18 +176,18 @@ __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint
 // consumed, nothing is added), so every later look-up of the group sees the same window and returns 0
 // too, and the caller tests only the group's LAST entry.
 // PACKED: add the whole entry (length byte included); else add the signed magnitude.
-template <int OFF, bool PACKED, int BITS>
+template <int OFF, bool PACKED, int BITS, bool STORE = false>
 __device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr) {
     const uint32_t e = lds32(lut_addr + ((r.lo & ((1u << BITS) - 1u)) << 2));
     r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= e;                                    // the low byte counts
-    red_add<OFF>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
+    put_cell<OFF, STORE>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
     return e;
 }
 
 // One symbol with the test for a long codeword (group tails, and groups that met a long codeword).
-template <bool PACKED, class T>
+template <bool PACKED, class T, bool STORE = false>
 __device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr, uint32_t acc_addr,
                                                     const T& t, bool& bad) {
     uint32_t e = lds32(lut_addr + ((r.lo & ((1u << T::bits) - 1u)) << 2));
@@ -178,44 +195,45 @@ __device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr
     r.lo = __funnelshift_r(r.lo, r.hi, e);
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= e;                                    // the low byte counts
-    red_add<0>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
+    put_cell<0, STORE>(acc_addr, PACKED ? e : (uint32_t)((int32_t)e >> 8));
 }
 
 // A group of four whose fast pass stopped at a long codeword after `done` good symbols: the reader
 // stands exactly at that codeword, so the rest of the group is decoded with the checked step.
 // Rare (about one symbol in a thousand is longer than the table).  Inlined, so that the reader stays
 // in registers (its address is never taken); the long-codeword search itself is out of line.
-template <bool PACKED, class T>
+// (ROW: words between the cells of consecutive symbols of a lane)
+template <bool PACKED, class T, bool STORE = false, int ROW = PADW>
 __device__ __forceinline__ void finish_group(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int done,
                                              const T& t, bool& bad) {
 #pragma unroll 1
     for (int k = done; k < 4; ++k) {
         refill(r);
-        decode_step_checked<PACKED>(r, lut_addr, acc_addr + (uint32_t)k * (PADW * 4), t, bad);
+        decode_step_checked<PACKED, T, STORE>(r, lut_addr, acc_addr + (uint32_t)k * (ROW * 4), t, bad);
     }
 }
 
-template <bool PACKED, class T>
+template <bool PACKED, class T, bool STORE = false, int ROW = PADW>
 __device__ __forceinline__ void decode_run(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int n,
                                            const T& t, bool& bad) {
     int i = 0;
     for (; i + 4 <= n; i += 4) {
         refill(r);
-        const uint32_t e0 = decode_step<0, PACKED, T::bits>(r, lut_addr, acc_addr);
-        const uint32_t e1 = decode_step<PADW * 4, PACKED, T::bits>(r, lut_addr, acc_addr);
+        const uint32_t e0 = decode_step<0, PACKED, T::bits, STORE>(r, lut_addr, acc_addr);
+        const uint32_t e1 = decode_step<ROW * 4, PACKED, T::bits, STORE>(r, lut_addr, acc_addr);
         refill(r);
-        const uint32_t e2 = decode_step<PADW * 8, PACKED, T::bits>(r, lut_addr, acc_addr);
-        const uint32_t e3 = decode_step<PADW * 12, PACKED, T::bits>(r, lut_addr, acc_addr);
+        const uint32_t e2 = decode_step<ROW * 8, PACKED, T::bits, STORE>(r, lut_addr, acc_addr);
+        const uint32_t e3 = decode_step<ROW * 12, PACKED, T::bits, STORE>(r, lut_addr, acc_addr);
         if ((e3 & 0xFFu) == 0u) {
             const int done = ((e0 & 0xFFu) != 0u) + ((e1 & 0xFFu) != 0u) + ((e2 & 0xFFu) != 0u);
-            finish_group<PACKED>(r, lut_addr, acc_addr, done, t, bad);
+            finish_group<PACKED, T, STORE, ROW>(r, lut_addr, acc_addr, done, t, bad);
         }
-        acc_addr += PADW * 16;
+        acc_addr += ROW * 16;
     }
     for (; i < n; ++i) {
         refill(r);
-        decode_step_checked<PACKED>(r, lut_addr, acc_addr, t, bad);
-        acc_addr += PADW * 4;
+        decode_step_checked<PACKED, T, STORE>(r, lut_addr, acc_addr, t, bad);
+        acc_addr += ROW * 4;
     }
 }
 
@@ -239,7 +257,7 @@ __device__ void slow_init(SlowReader& r, const uint32_t* src, uint32_t nwords, u
     r.nb += 32;
     r.wp++;
 }
-template <bool PACKED, class T>
+template <bool PACKED, class T, bool STORE = false, int ROW = PADW>
 __device__ void slow_run(SlowReader& r, const T& t, const uint32_t* src, uint32_t nwords, int32_t* acc,
                          int n, bool& bad) {
     for (int i = 0; i < n; ++i) {
@@ -249,8 +267,9 @@ __device__ void slow_run(SlowReader& r, const T& t, const uint32_t* src, uint32_
         const uint32_t len = e & 0xFFu;
         r.buf >>= len;
         r.nb -= (int)len;
-        atomicAdd(acc, PACKED ? (int32_t)e : ((int32_t)e >> 8));
-        acc += PADW;
+        if (STORE) *acc = PACKED ? (int32_t)e : ((int32_t)e >> 8);
+        else atomicAdd(acc, PACKED ? (int32_t)e : ((int32_t)e >> 8));
+        acc += ROW;
         if (r.nb < 32) {
             r.buf |= (unsigned long long)fetch_checked(src, nwords, r.wp) << r.nb;
             r.nb += 32;
@@ -391,8 +410,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(acc0);
     const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[warp]);
     const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
-    const int64_t per = (p.n_groups + gridDim.x - 1) / gridDim.x;
-    const int64_t g0 = (int64_t)blockIdx.x * per, g1 = min(p.n_groups, g0 + per);
+    const int64_t g0 = p.dec_part[blockIdx.x], g1 = p.dec_part[blockIdx.x + 1];
     const float fu = (float)U;
     const float inv_u = (U & (U - 1)) == 0 ? 1.0f / fu : 0.0f;
     bool bad = false;
@@ -418,7 +436,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
             s.active = false; s.staged = true; s.nwords = 0; s.bitpos = 0; s.sub_len_bits = 0;
             s.i_lo = 0; s.i_hi = 0; s.gsrc = nullptr;
             Reader r;
-            r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr;
+            r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr; r.nw = 0;
             SlowReader sr;
             sr.buf = 0; sr.nb = 0; sr.wp = 0;
             long long my_tb = 0;                   // bounds of this warp's own chunk (used when all_mine)
@@ -467,12 +485,97 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                 }
             }
             if (mine && s.active) {
-                const uint32_t endpos = s.staged ? ((r.rp - stage_addr) << 3) - reader_bits(r)
+                const uint32_t endpos = s.staged ? ((r.rp - stage_addr - 4u) << 3) - reader_bits(r)
                                                  : sr.wp * 32u - (uint32_t)sr.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
             }
         }
         gi = ge;
+    }
+    if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
+}
+
+// ---- U = 1: nothing to add up, every warp on its own ------------------------------------------
+// One user: a chunk is one stream, and the average is the stream's values themselves.  A block is 32
+// independent warps that share the table; a warp stages its stream, decodes eight symbols per lane at a
+// time into a tile of its own (a plain store of the table entry: the cell is the lane's alone), and
+// writes the tile out transposed, 32 bytes of consecutive elements per sub-chunk and store.  No
+// barrier between warps except where the segment (the table) changes.  The tile rows are 36 words
+// apart: lane s stores symbol i at word 36 i + s (banks s + 4 i: distinct over the lanes), and the
+// read-out lane (i, s) = (lane % 8, 4 k + lane / 8) loads word 36 i + s (banks 4 i + s: distinct).
+constexpr int ONE_WARPS = 32, ONE_QB = 8, ONE_ROW = 36, BITS_ONE = 13;
+struct SmemOne {
+    TablesT<BITS_ONE> t;
+    alignas(16) uint32_t stage[ONE_WARPS][STAGE_ROW];
+    alignas(16) int32_t tile[ONE_WARPS][ONE_QB * ONE_ROW];
+};
+static_assert(sizeof(SmemOne) <= 227 * 1024, "one block per SM must fit its shared memory");
+
+__global__ void __launch_bounds__(ONE_WARPS * 32, 1)
+decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16_t* __restrict__ sub_bits,
+                  const uint32_t* __restrict__ chunk_off, const co3_seg_header* __restrict__ hdr,
+                  float* __restrict__ avg, float* __restrict__ weights, float step) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    SmemOne& sm = *reinterpret_cast<SmemOne*>(s_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(sm.stage[warp]);
+    int32_t* tile = sm.tile[warp];
+    const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile);
+    const int64_t c0 = p.dec_part[blockIdx.x], c1 = p.dec_part[blockIdx.x + 1];
+    bool bad = false;
+    int64_t ci = c0;
+    while (ci < c1) {                              // one trip per run of chunks of one segment
+        const int seg = p.chunks[ci].seg;
+        int64_t ce = ci + 1;
+        while (ce < c1 && p.chunks[ce].seg == seg) ++ce;
+        __syncthreads();                           // every warp is past its last look-up in the old tables
+        load_tables(sm.t, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, ONE_WARPS * 32);
+        __syncthreads();
+        const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
+        for (int64_t c = ci + warp; c < ce; c += ONE_WARPS) {
+            const Co3Chunk cd = p.chunks[c];
+            Stream s;
+            open_stream(s, p, cd, c, 0, bitstream, sub_bits, chunk_off, sm.stage[warp], lane, bad);
+            Reader r;
+            r.lo = 0; r.hi = 0; r.nb = 0; r.rp = stage_addr; r.nw = 0;
+            SlowReader sr;
+            sr.buf = 0; sr.nb = 0; sr.wp = 0;
+            if (s.active) {
+                if (s.staged) reader_init(r, stage_addr, s.bitpos);
+                else slow_init(sr, s.gsrc, s.nwords, s.bitpos);
+            }
+            const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+            const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+            const int ri = lane & (ONE_QB - 1), rs = lane >> 3;          // read-out: symbol in the batch, sub-chunk in the four
+#pragma unroll 1
+            for (int b = 0; b < CO3_SUB / ONE_QB; ++b) {
+                if (s.active) {
+                    const int a = max(s.i_lo, b * ONE_QB), z = min(s.i_hi, (b + 1) * ONE_QB);
+                    if (z > a) {
+                        const int cell = (a - b * ONE_QB) * ONE_ROW + lane;
+                        if (s.staged) decode_run<true, TablesT<BITS_ONE>, true, ONE_ROW>(r, lut_addr, tile_addr + 4u * (uint32_t)cell, z - a, sm.t, bad);
+                        else slow_run<true, TablesT<BITS_ONE>, true, ONE_ROW>(sr, sm.t, s.gsrc, s.nwords, tile + cell, z - a, bad);
+                    }
+                }
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < 32 / 4; ++k) {
+                    const int sc = 4 * k + rs;
+                    const int e = sc * CO3_SUB + b * ONE_QB + ri;
+                    const int32_t v = tile[ri * ONE_ROW + sc];
+                    if (e >= lo && e < hi) put_out(avg, weights, step, tb + e, __fmul_rn((float)(v >> 8), scale));
+                }
+                __syncwarp();                      // the tile is written again by the next batch
+            }
+            if (s.active) {
+                const uint32_t endpos = s.staged ? ((r.rp - stage_addr - 4u) << 3) - reader_bits(r)
+                                                 : sr.wp * 32u - (uint32_t)sr.nb;
+                if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
+            }
+            __syncwarp();                          // the stage is reused by this warp's next chunk
+        }
+        ci = ce;
     }
     if (bad) atomicOr(p.flags, CO3_FLAG_CORRUPT);
 }
@@ -504,8 +607,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
     const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(tm.acc);
     const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[warp]);
-    const int64_t per = (p.n_chunks + gridDim.x - 1) / gridDim.x;
-    const int64_t c0 = (int64_t)blockIdx.x * per, c1 = min(p.n_chunks, c0 + per);
+    const int64_t c0 = p.dec_part[blockIdx.x], c1 = p.dec_part[blockIdx.x + 1];
     const float fu = (float)p.U;
     const float inv_u = (p.U & (p.U - 1)) == 0 ? 1.0f / fu : 0.0f;
     bool bad = false;
@@ -531,7 +633,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                         Reader r;
                         reader_init(r, stage_addr, s.bitpos);
                         decode_run<false>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, s.i_hi - s.i_lo, sm.t, bad);
-                        endpos = ((r.rp - stage_addr) << 3) - reader_bits(r);
+                        endpos = ((r.rp - stage_addr - 4u) << 3) - reader_bits(r);
                     } else {
                         SlowReader sr;
                         slow_init(sr, s.gsrc, s.nwords, s.bitpos);
@@ -593,8 +695,55 @@ cudaError_t co3_setup_decode_kernels(void) {
         cudaError_t e = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
         if (e != cudaSuccess) return e;
     }
+    cudaError_t e1 = cudaFuncSetAttribute(decode_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmemOne));
+    if (e1 != cudaSuccess) return e1;
     return cudaFuncSetAttribute(decode_large_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)sizeof(SmemB));
+}
+
+// Blocks the decoder of a plan with U users can keep resident: one block of several teams per SM, or
+// (user counts that do not divide 8) as many one-team blocks as fit.
+int co3_decode_max_blocks(int U, int num_sms) {
+    if (U > NW || U == 1) return num_sms;
+    const SmallVariant v = small_variant(U);
+    int bpsm = 1;
+    if (v.teams == 1) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bpsm, v.fn, CO3_THREADS, v.smem) != cudaSuccess) (void)cudaGetLastError();
+        if (bpsm < 1) bpsm = 1;
+    }
+    return num_sms * bpsm;
+}
+
+// The decoder's work items (groups of chunks for U <= 8, chunks above) with their segment and a cost
+// in team-rounds (1 = a chunk whose longest sub-chunk is full), split over the blocks by
+// co3_host_balanced_split.
+int co3_decode_partition(const Co3Chunk* chunks, int64_t n_chunks, const Co3Group* groups, int64_t n_groups, int U,
+                         int max_blocks, int32_t* part) {
+    const bool by_group = U <= NW && U > 1;        // one user: chunks, taken by 32 independent warps
+    const int teams = U == 1 ? ONE_WARPS : (by_group ? small_variant(U).teams : TEAMS_B);
+    const int64_t n = by_group ? n_groups : n_chunks;
+    double* w = (double*)malloc(sizeof(double) * (size_t)n);
+    int32_t* seg = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+    int blocks = -1;
+    if (w && seg) {
+        for (int64_t i = 0; i < n; ++i) {
+            int longest = 0;
+            if (by_group) {
+                seg[i] = groups[i].seg;
+                for (int k = 0; k < groups[i].count; ++k) {
+                    const int len = chunks[groups[i].chunk0 + k].len;
+                    longest = longest > len ? longest : len;
+                }
+            } else {
+                seg[i] = chunks[i].seg;
+                longest = chunks[i].len;
+            }
+            w[i] = 0.04 + (longest >= CO3_SUB ? 1.0 : (double)longest / CO3_SUB);
+        }
+        blocks = co3_host_balanced_split(w, seg, n, teams, max_blocks, 0.08, part);
+    }
+    free(w); free(seg);
+    return blocks;
 }
 
 cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uint16_t* sub_bits,
@@ -603,19 +752,13 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
     Co3Dev p = pl->dev;
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) { p.cb = pl->cb_emp; p.code_by_segment = 1; }
     co3_prof_begin(pl, CO3_K_DECODE, st);
-    if (p.U <= NW) {
+    if (p.U == 1) {
+        decode_one_kernel<<<p.dec_blocks, ONE_WARPS * 32, sizeof(SmemOne), st>>>(p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
+    } else if (p.U <= NW) {
         const SmallVariant v = small_variant(p.U);
-        int bpsm = 1;
-        if (v.teams == 1) {
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bpsm, v.fn, CO3_THREADS, v.smem);
-            if (bpsm < 1) bpsm = 1;
-        }
-        const int64_t grid = (int64_t)pl->num_sms * bpsm;
-        v.fn<<<(int)(p.n_groups < grid ? p.n_groups : grid), v.teams * CO3_THREADS, v.smem, st>>>(
-            p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
+        v.fn<<<p.dec_blocks, v.teams * CO3_THREADS, v.smem, st>>>(p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     } else {
-        const int64_t grid = pl->num_sms;                    // one block of four teams per SM
-        decode_large_u_kernel<<<(int)(p.n_chunks < grid ? p.n_chunks : grid), TEAMS_B * CO3_THREADS, sizeof(SmemB), st>>>(
+        decode_large_u_kernel<<<p.dec_blocks, TEAMS_B * CO3_THREADS, sizeof(SmemB), st>>>(
             p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     }
     co3_prof_end(pl, CO3_K_DECODE, st, 1);

@@ -81,6 +81,8 @@ struct Co3Dev {
     float gamma;
     const Co3Chunk* chunks;       // [n_chunks]
     const Co3Group* groups;       // [n_groups]
+    const int32_t* dec_part;      // [dec_blocks + 1] decoder: block b takes the groups (U <= 8) or chunks (U > 8)
+    int dec_blocks;               //     dec_part[b] .. dec_part[b+1] - 1; a partition balanced on the host
     const int64_t* seg_off;       // [S+1]
     const int32_t* seg_chunk0;    // [S+1] first chunk of each segment
     uint8_t* sym;                 // [U][sld] internal symbols (co3_sym_internal)
@@ -209,6 +211,13 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
 cudaError_t co3_launch_encode_stalled(co3_plan* pl, const co3_seg_header* hdr, uint32_t* bitstream,
                                       uint16_t* sub_bits, uint32_t* chunk_off, unsigned long long* user_bits,
                                       int spin_limit, cudaStream_t st);
+// Decoder work split (host): fills part[0 .. n_blocks] for at most max_blocks blocks, returns n_blocks.
+// teams: teams per block of the decoder that will run; items are groups (U <= 8) or chunks (U > 8).
+int co3_decode_partition(const Co3Chunk* chunks, int64_t n_chunks, const Co3Group* groups, int64_t n_groups, int U,
+                         int max_blocks, int32_t* part);
+int co3_decode_max_blocks(int U, int num_sms);
+int co3_host_balanced_split(const double* w, const int32_t* seg, int64_t n, int teams, int max_blocks, double run_cost,
+                            int32_t* part);
 cudaError_t co3_setup_kernels(void);
 cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_t st);
 

@@ -232,6 +232,60 @@ extern "C" int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint
     return CO3_OK;
 }
 
+// Contiguous split of n work items over at most max_blocks thread blocks for kernels whose blocks walk
+// their items run by run of one segment, the block's `teams` teams taking every teams-th item of a run
+// and all of them meeting where the segment changes.  A run then costs its most loaded team's items
+// plus run_cost (the change of tables), and a block's rounds are the sum over its runs.  Equal item
+// counts per block would let a block whose range a segment boundary cuts into, say, 10 + 9 items take
+// six team-rounds where its neighbours take five, and every block waits for the slowest.  Rounds alone
+// would pack full rounds into fewer blocks than there are SMs, though, and a block whose teams are all
+// busy is bound by the throughput of its SM, i.e. by its total work: a block's cost is therefore the
+// mean of its rounds and of its work per team.  The cuts are placed so that the largest block cost is
+// as small as a contiguous split allows (bisection on that bound, greedy fill).  part[0 .. max_blocks]
+// receives the cuts; returns the blocks in use.
+int co3_host_balanced_split(const double* w, const int32_t* seg, int64_t n, int teams, int max_blocks, double run_cost,
+                            int32_t* part) {
+    if (!w || !seg || !part || n < 1 || n > 0x7FFFFFFFLL || teams < 1 || teams > 32 || max_blocks < 1) return -1;
+    auto blocks_needed = [&](double bound, int32_t* cuts) {
+        int64_t blocks = 0, i = 0;
+        while (i < n) {
+            if (cuts && blocks < max_blocks) cuts[blocks] = (int32_t)i;
+            double closed = run_cost, team_sum[32] = {0}, run_max = w[i];     // a block takes at least one item
+            double work = w[i];
+            int cur = seg[i], pos = 1;
+            team_sum[0] = w[i];
+            ++i;
+            while (i < n) {
+                const bool new_run = seg[i] != cur;
+                const double c2 = new_run ? closed + run_max + run_cost : closed;
+                const int p2 = new_run ? 0 : pos;
+                const double t2 = (new_run ? 0.0 : team_sum[p2 % teams]) + w[i];
+                const double r2 = new_run ? t2 : (run_max > t2 ? run_max : t2);
+                if (0.5 * (c2 + r2) + 0.5 * (work + w[i]) / teams > bound) break;
+                if (new_run) { for (int t = 0; t < teams; ++t) team_sum[t] = 0.0; cur = seg[i]; }
+                closed = c2; run_max = r2; team_sum[p2 % teams] = t2; pos = p2 + 1; work += w[i];
+                ++i;
+            }
+            ++blocks;
+        }
+        return blocks;
+    };
+    double lo = 0.0, hi = 0.0;
+    for (int64_t i = 0; i < n; ++i) hi += w[i] + run_cost;
+    for (int it = 0; it < 60; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (blocks_needed(mid, nullptr) <= max_blocks) hi = mid; else lo = mid;
+    }
+    const int64_t blocks = blocks_needed(hi, part);
+    for (int64_t b = blocks; b <= max_blocks; ++b) part[b] = (int32_t)n;
+    return (int)blocks;
+}
+
+extern "C" int co3_balanced_split(const double* cost, const int32_t* seg, int64_t n, int32_t teams, int32_t max_blocks,
+                                  int32_t* part) {
+    return co3_host_balanced_split(cost, seg, n, teams, max_blocks, 0.08, part);
+}
+
 extern "C" uint64_t co3_model_checksum(co3_format fmt) {
     if (!co3_host_fmt_ok(fmt)) return 0;
     const uint32_t* t = co3_host_weight_table(fmt.exp_bits, fmt.mant_bits);
