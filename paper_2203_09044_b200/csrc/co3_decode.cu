@@ -15,7 +15,8 @@
 // as shift amount (only its low five bits count), the bit buffer is topped up once per pair of
 // symbols, and four symbols are decoded per loop trip with immediate accumulator offsets.
 //
-// Two kernels.  U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
+// Three kernels.  U = 1 has nothing to add up: 24 independent warps per block, each transposing its
+// own stream through a small tile.  2 <= U <= 8 keeps one stream per warp and walks the chunk in quarters of 32 symbols
 // per sub-chunk (small double-buffered accumulator, several chunks per group when U < 8); the
 // whole table entries are accumulated (the length bytes of at most 8 users cannot carry into
 // the magnitude) and the magnitude sum is taken out with one shift at the end.  U > 8 keeps a
@@ -496,14 +497,13 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
 }
 
 // ---- U = 1: nothing to add up, every warp on its own ------------------------------------------
-// One user: a chunk is one stream, and the average is the stream's values themselves.  A block is 32
-// independent warps that share the table; a warp stages its stream, decodes eight symbols per lane at a
+// One user: a chunk is one stream, and the average is the stream's values themselves.  A block is 24
+// independent warps that share the table; a warp stages its stream, decodes 32 symbols per lane at a
 // time into a tile of its own (a plain store of the table entry: the cell is the lane's alone), and
-// writes the tile out transposed, 32 bytes of consecutive elements per sub-chunk and store.  No
-// barrier between warps except where the segment (the table) changes.  The tile rows are 36 words
-// apart: lane s stores symbol i at word 36 i + s (banks s + 4 i: distinct over the lanes), and the
-// read-out lane (i, s) = (lane % 8, 4 k + lane / 8) loads word 36 i + s (banks 4 i + s: distinct).
-constexpr int ONE_WARPS = 32, ONE_QB = 8, ONE_ROW = 36, BITS_ONE = 13;
+// writes the tile out transposed, one 128-byte line of consecutive elements per store.  No barrier
+// between warps except where the segment (the table) changes.  Lane s stores symbol i at word
+// 33 i + s, the read-out lane i loads word 33 i + s of sub-chunk s: both free of bank conflicts.
+constexpr int ONE_WARPS = 24, ONE_QB = 32, ONE_ROW = PADW, BITS_ONE = 12;
 struct SmemOne {
     TablesT<BITS_ONE> t;
     alignas(16) uint32_t stage[ONE_WARPS][STAGE_ROW];
@@ -511,6 +511,7 @@ struct SmemOne {
 };
 static_assert(sizeof(SmemOne) <= 227 * 1024, "one block per SM must fit its shared memory");
 
+template <bool UPDATE>
 __global__ void __launch_bounds__(ONE_WARPS * 32, 1)
 decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16_t* __restrict__ sub_bits,
                   const uint32_t* __restrict__ chunk_off, const co3_seg_header* __restrict__ hdr,
@@ -547,7 +548,9 @@ decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16
             }
             const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
             const int lo = (int)(cd.start - tb), hi = lo + cd.len;
-            const int ri = lane & (ONE_QB - 1), rs = lane >> 3;          // read-out: symbol in the batch, sub-chunk in the four
+            const bool whole = lo == 0 && hi == CO3_TILE;
+            float* out = avg + tb + lane;           // element `lane` of the batch, sub-chunk 0
+            float* wout = UPDATE ? weights + tb + lane : nullptr;
 #pragma unroll 1
             for (int b = 0; b < CO3_SUB / ONE_QB; ++b) {
                 if (s.active) {
@@ -559,13 +562,26 @@ decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16
                     }
                 }
                 __syncwarp();
-#pragma unroll
-                for (int k = 0; k < 32 / 4; ++k) {
-                    const int sc = 4 * k + rs;
-                    const int e = sc * CO3_SUB + b * ONE_QB + ri;
-                    const int32_t v = tile[ri * ONE_ROW + sc];
-                    if (e >= lo && e < hi) put_out(avg, weights, step, tb + e, __fmul_rn((float)(v >> 8), scale));
+                const int32_t* col = tile + lane * ONE_ROW;    // this lane's symbol of the batch, sub-chunk by sub-chunk
+                if (whole) {
+#pragma unroll 8
+                    for (int sc = 0; sc < 32; ++sc) {
+                        const float v = __fmul_rn((float)(col[sc] >> 8), scale);
+                        out[sc * CO3_SUB] = v;
+                        if (UPDATE) wout[sc * CO3_SUB] = __fadd_rn(wout[sc * CO3_SUB], __fmul_rn(step, v));
+                    }
+                } else {
+                    for (int sc = 0; sc < 32; ++sc) {
+                        const int e = sc * CO3_SUB + b * ONE_QB + lane;
+                        if (e >= lo && e < hi) {
+                            const float v = __fmul_rn((float)(col[sc] >> 8), scale);
+                            out[sc * CO3_SUB] = v;
+                            if (UPDATE) wout[sc * CO3_SUB] = __fadd_rn(wout[sc * CO3_SUB], __fmul_rn(step, v));
+                        }
+                    }
                 }
+                out += ONE_QB;
+                if (UPDATE) wout += ONE_QB;
                 __syncwarp();                      // the tile is written again by the next batch
             }
             if (s.active) {
@@ -676,7 +692,6 @@ SmallVariant small_variant(int U) {
         case 8: return {decode_small_u_kernel<4, 13, 8>, 4, smem_a_bytes<4, 13>(U)};
         case 4: return {decode_small_u_kernel<4, 12, 4>, 4, smem_a_bytes<4, 12>(U)};
         case 2: return {decode_small_u_kernel<3, 12, 2>, 3, smem_a_bytes<3, 12>(U)};
-        case 1: return {decode_small_u_kernel<2, 12, 1>, 2, smem_a_bytes<2, 12>(U)};
         default: return {decode_small_u_kernel<1, CO3_LUT_SMALL_BITS, 0>, 1, smem_a_bytes<1, CO3_LUT_SMALL_BITS>(U)};
     }
 }
@@ -695,7 +710,8 @@ cudaError_t co3_setup_decode_kernels(void) {
         cudaError_t e = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
         if (e != cudaSuccess) return e;
     }
-    cudaError_t e1 = cudaFuncSetAttribute(decode_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmemOne));
+    cudaError_t e1 = cudaFuncSetAttribute(decode_one_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmemOne));
+    if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(decode_one_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SmemOne));
     if (e1 != cudaSuccess) return e1;
     return cudaFuncSetAttribute(decode_large_u_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)sizeof(SmemB));
@@ -753,7 +769,8 @@ cudaError_t co3_launch_decode(co3_plan* pl, const uint32_t* bitstream, const uin
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) { p.cb = pl->cb_emp; p.code_by_segment = 1; }
     co3_prof_begin(pl, CO3_K_DECODE, st);
     if (p.U == 1) {
-        decode_one_kernel<<<p.dec_blocks, ONE_WARPS * 32, sizeof(SmemOne), st>>>(p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
+        if (weights) decode_one_kernel<true><<<p.dec_blocks, ONE_WARPS * 32, sizeof(SmemOne), st>>>(p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
+        else decode_one_kernel<false><<<p.dec_blocks, ONE_WARPS * 32, sizeof(SmemOne), st>>>(p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
     } else if (p.U <= NW) {
         const SmallVariant v = small_variant(p.U);
         v.fn<<<p.dec_blocks, v.teams * CO3_THREADS, v.smem, st>>>(p, bitstream, sub_bits, chunk_off, hdr, avg, weights, step);
