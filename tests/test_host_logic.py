@@ -94,6 +94,46 @@ def test_model_checksum_is_the_digest_of_the_weight_table(binding):
     assert len({binding.model_checksum(E, M) for E, M in [(1, 2), (3, 2), (4, 3)]}) == 3
 
 
+def _block_cost(w, seg, a, z, teams):
+    """Cost of the items a .. z-1 in one block, as co3_balanced_split defines it."""
+    rounds, work, i = 0.0, float(np.sum(w[a:z])), a
+    while i < z:
+        j = i
+        while j < z and seg[j] == seg[i]:
+            j += 1
+        rounds += max(float(np.sum(w[i + t:j:teams])) for t in range(teams)) + 0.08
+        i = j
+    return 0.5 * rounds + 0.5 * work / teams
+
+
+def test_balanced_split_of_the_decoders_work(binding):
+    """The cuts cover the items in order, use at most max_blocks blocks, and their largest block cost
+    is the least any contiguous split reaches (brute force on small cases); on the ResNet-18 layer mix
+    it beats equal item counts per block."""
+    import itertools
+    from paper_2203_09044_b200 import inputs
+    rng = np.random.default_rng(3)
+    for n, blocks, teams in ((9, 3, 2), (11, 4, 4), (7, 7, 1), (10, 2, 3), (5, 8, 4)):
+        w = rng.choice([0.04 + 1.0, 0.04 + 0.5, 0.04 + 0.1], n)
+        seg = np.sort(rng.integers(0, 3, n)).astype(np.int32)
+        part, nb = binding.balanced_split(w, seg, teams, blocks)
+        assert part[0] == 0 and part[nb] == n and np.all(np.diff(part[:nb + 1]) > 0) and np.all(part[nb:] == n)
+        got = max(_block_cost(w, seg, part[b], part[b + 1], teams) for b in range(nb))
+        best = min(max(_block_cost(w, seg, a, z, teams) for a, z in zip((0,) + cuts, cuts + (n,)))
+                   for k in range(0, min(blocks, n)) for cuts in itertools.combinations(range(1, n), k))
+        assert got <= best + 1e-9, (n, blocks, teams, got, best)
+    wl = inputs.workload(1)
+    seg, st, en, _, _ = binding.partition(wl.d, wl.seg_offsets)
+    w = 0.04 + np.minimum(en - st, 128) / 128.0
+    part, nb = binding.balanced_split(w, seg, 4, 148)
+    balanced = max(_block_cost(w, seg, part[b], part[b + 1], 4) for b in range(nb))
+    per = -(-len(seg) // 148)
+    equal = max(_block_cost(w, seg, a, min(a + per, len(seg)), 4) for a in range(0, len(seg), per))
+    assert 140 <= nb <= 148 and balanced < 0.9 * equal, (nb, balanced, equal)
+    with pytest.raises(binding.Co3Error):
+        binding.balanced_split(w, seg, 33, 148)
+
+
 def test_partition_identical_to_oracle(binding, oracle):
     from paper_2203_09044_b200 import inputs
     cases = [(10000, [0, 10000]), (9000, [0, 5, 5, 4101, 8192, 9000]), (130, [0, 1, 130]),
