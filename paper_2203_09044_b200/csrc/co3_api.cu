@@ -48,6 +48,88 @@ int alloc_codebook(co3_plan* pl, Co3CodeBook& cb, size_t R, int ncand) {
 
 inline cudaStream_t as_stream(void* s) { return (cudaStream_t)s; }
 
+// The code tables of all model rows are a pure function of the format (148 MB for E4M3), so the plans
+// of one device and format share one copy: built by the first plan, freed with the last.
+struct SharedBook {
+    int device, E, M, refs;
+    Co3CodeBook cb;
+    void* allocs[16];
+    int n_allocs;
+};
+constexpr int MAX_BOOKS = 32;
+SharedBook g_books[MAX_BOOKS];
+std::mutex g_books_mutex;
+
+template <typename T>
+bool book_alloc(SharedBook& b, T** out, size_t count) {
+    void* ptr = nullptr;
+    if (b.n_allocs >= 16 || cudaMalloc(&ptr, (count ? count : 1) * sizeof(T)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    b.allocs[b.n_allocs++] = ptr;
+    *out = (T*)ptr;
+    return true;
+}
+
+void book_free(SharedBook& b) {
+    for (int i = 0; i < b.n_allocs; ++i) cudaFree(b.allocs[i]);
+    b = SharedBook{};
+}
+
+// Takes a reference to the book of (pl->device, format), building it with the plan's own configuration
+// if it does not exist yet (the plan's static tables must already be on the device).
+int book_acquire(co3_plan* pl) {
+    std::lock_guard<std::mutex> lock(g_books_mutex);
+    const int E = pl->dev.E, M = pl->dev.M;
+    SharedBook* slot = nullptr;
+    for (SharedBook& b : g_books) {
+        if (b.refs > 0 && b.device == pl->device && b.E == E && b.M == M) {
+            ++b.refs;
+            pl->dev.cb = b.cb;
+            pl->book = &b;
+            return CO3_OK;
+        }
+        if (b.refs == 0 && !slot) slot = &b;
+    }
+    if (!slot) return CO3_ENOMEM;
+    SharedBook& b = *slot;
+    b = SharedBook{};
+    Co3CodeBook& cb = b.cb;
+    const size_t R = CO3_NROWS;
+    cb.ncand = CO3_NCAND;
+    cb.long_stride = 16 * pl->dev.nsym < CO3_LONG_CACHE ? CO3_LONG_CACHE : 16 * pl->dev.nsym;
+    bool ok = book_alloc(b, &cb.cand_len, R * (size_t)cb.ncand * CO3_MAXSYM) && book_alloc(b, &cb.cand_max, R * (size_t)cb.ncand) &&
+              book_alloc(b, &cb.len8, R * CO3_MAXSYM) && book_alloc(b, &cb.len_pub, R * CO3_MAXSYM) &&
+              book_alloc(b, &cb.enc, R * CO3_MAXSYM) && book_alloc(b, &cb.code_msb, R * CO3_MAXSYM) &&
+              book_alloc(b, &cb.lut, R * CO3_LUT_SIZE) && book_alloc(b, &cb.lut_long, R * (size_t)cb.long_stride) &&
+              book_alloc(b, &cb.first, R * (CO3_MAXLEN + 1)) && book_alloc(b, &cb.count, R * (CO3_MAXLEN + 1)) &&
+              book_alloc(b, &cb.offs, R * (CO3_MAXLEN + 1)) && book_alloc(b, &cb.perm, R * CO3_MAXSYM) &&
+              book_alloc(b, &cb.ksign, (size_t)CO3_MAXSYM);
+    if (!ok) { book_free(b); return CO3_ENOMEM; }
+    pl->dev.cb = cb;
+    if (co3_build_codebook(pl, 0) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+        (void)cudaGetLastError();
+        book_free(b);
+        return CO3_ECUDA;
+    }
+    cudaFree(cb.cand_len); cudaFree(cb.cand_max);        // build scratch (the first two allocations)
+    b.allocs[0] = b.allocs[1] = nullptr;
+    b.cb.cand_len = nullptr; b.cb.cand_max = nullptr;
+    pl->dev.cb = b.cb;
+    b.device = pl->device; b.E = E; b.M = M; b.refs = 1;
+    pl->book = &b;
+    return CO3_OK;
+}
+
+void book_release(co3_plan* pl) {
+    if (!pl->book) return;
+    std::lock_guard<std::mutex> lock(g_books_mutex);
+    SharedBook& b = *static_cast<SharedBook*>(pl->book);
+    if (--b.refs == 0) book_free(b);
+    pl->book = nullptr;
+}
+
 // cudaFuncSetAttribute applies to the current device: one flag per device, set under a lock
 constexpr int MAX_DEVICES = 64;
 bool g_kernels_ready[MAX_DEVICES];
@@ -150,6 +232,7 @@ extern "C" void co3_plan_destroy(co3_plan* pl) {
     if (pl->ev_conv) cudaEventDestroy(pl->ev_conv);
     if (pl->ev_dec) cudaEventDestroy(pl->ev_dec);
     if (pl->ev_d2h) cudaEventDestroy(pl->ev_d2h);
+    book_release(pl);
     for (int i = 0; i < pl->n_allocs; ++i) cudaFree(pl->allocs[i]);
     free(pl->h_seg_off);
     delete pl;
@@ -308,7 +391,6 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
         }
         a |= dev_alloc(pl, &dv.flags, 1);
         a |= dev_alloc(pl, &dv.nonfinite_total, 1);
-        a |= alloc_codebook(pl, dv.cb, CO3_NROWS, CO3_NCAND);
         if (cfg->bias_mode == CO3_CODE_EMPIRICAL) a |= alloc_codebook(pl, pl->cb_emp, (size_t)S, CO3_NCAND_HIST);
         if (a) rc = CO3_ENOMEM;
         if (rc == CO3_OK) {
@@ -352,12 +434,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             }
             dv.chunks = d_chunks; dv.groups = d_groups; dv.seg_off = d_seg_off;
             dv.seg_chunk0 = d_seg_chunk0; dv.wtab = d_wtab; dv.logr_tab = d_logr;
-            if (rc == CO3_OK) {                      // Huffman codes of all model rows, once
-                if (co3_build_codebook(pl, 0) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
-                    (void)cudaGetLastError();
-                    rc = CO3_ECUDA;
-                }
-            }
+            if (rc == CO3_OK) rc = book_acquire(pl);  // Huffman codes of all model rows: built once per device and format
         }
     }
     free(h_chunks); free(h_seg); free(h_start); free(h_end); free(h_sub); free(h_seg_chunk0); free(h_groups);

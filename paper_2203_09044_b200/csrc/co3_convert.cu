@@ -165,7 +165,12 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
     if (item >= n_items) return;
     __syncthreads();                                  // both tickets read before slot 0 is reused
 
-    auto make_ctx = [&](uint32_t it, const Co3Chunk& cd) {
+    // The statistics pass walks the items from the last one down: it ends where the convert pass that
+    // follows it begins, and begins where the previous iteration's convert pass ended, so both meet
+    // part of their input (what the 126 MB L2 still holds of gradient and memory) without going to HBM.
+    auto phys = [&](uint32_t t) { return (!CONVERT && t < n_items) ? n_items - 1u - t : t; };
+    auto make_ctx = [&](uint32_t t, const Co3Chunk& cd) {
+        const uint32_t it = phys(t);
         const uint32_t ul = it / n_chunks, uu = ul + (uint32_t)p.u_base;
         ItemCtx x;
         const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
@@ -195,13 +200,13 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
         cp_async_commit();
     };
 
-    ItemCtx cur = make_ctx(item, p.chunks[item % n_chunks]);
+    ItemCtx cur = make_ctx(item, p.chunks[phys(item) % n_chunks]);
     issue(cur, true, 0);
     issue(cur, true, 1);
     issue(cur, true, 2);
     bool has_nxt = nitem < n_items;
     ItemCtx nxt = cur;
-    if (has_nxt) nxt = make_ctx(nitem, p.chunks[nitem % n_chunks]);
+    if (has_nxt) nxt = make_ctx(nitem, p.chunks[phys(nitem) % n_chunks]);
 
     // the code table of an item's segment is fetched while the previous item is converted
     auto enc_entry = [&](int seg) {
@@ -249,7 +254,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
             // 0..2 of the next one, each into the slot the consumer has just left
             if (r == 0) issue(cur, true, 3);
             else issue(nxt, has_nxt, r - 1);
-            if (r == 2 && tid == 0 && claim < n_items) claim_cd = p.chunks[claim % n_chunks];
+            if (r == 2 && tid == 0 && claim < n_items) claim_cd = p.chunks[phys(claim) % n_chunks];
             cp_async_wait<STAGES - 1>();              // this step's copies have landed
             const uint32_t slot = r * SLOT_BYTES;
             const int e0 = 4 * tid + VSTRIDE * r;
@@ -357,7 +362,8 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
             uint32_t tn = 0;
 #pragma unroll
             for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
-            p.part_s1[item_base + item] = t1; p.part_s2[item_base + item] = t2; p.part_nf[item_base + item] = tn;
+            const uint32_t pi = item_base + phys(item);
+            p.part_s1[pi] = t1; p.part_s2[pi] = t2; p.part_nf[pi] = tn;
         }
         // When the block leaves the segment (or ends) its histogram goes to global memory; the next
         // item counts in the other copy, and this copy is not touched again before a later barrier.

@@ -128,6 +128,7 @@ struct co3_plan {
     int64_t worst_case_words;
     int device;
     int num_sms;
+    void* book;                     // the shared code tables of (device, format) this plan holds a reference to
     Co3CodeBook cb_emp;             // empirical-histogram code: S rows (else unallocated)
     uint8_t* emp_lens;              // ... the caller's length table during co3_encode_empirical
     const uint8_t* emp_lens_in;     // ... and during co3_decode_aggregate_empirical

@@ -451,6 +451,35 @@ def test_bounded_waits_of_the_encoder_run_out_and_report(binding):
     assert torch.equal(plan.decode_aggregate(out), plan2.decode_aggregate(out2))
 
 
+def test_plans_of_one_format_share_their_code_tables(binding):
+    """The code tables of all model rows (148 MB for E4M3) exist once per device and format: a second
+    plan costs far less device memory than the first, and outlives the first."""
+    from paper_2203_09044_b200 import inputs
+    b = binding
+    wl = inputs.workload(1, d=50_000, n_users=2)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    p1 = b.Plan(wl.d, wl.n_users, 4, 3, wl.seg_offsets, gamma=wl.gamma)
+    free1 = torch.cuda.mem_get_info()[0]
+    p2 = b.Plan(wl.d, wl.n_users, 4, 3, wl.seg_offsets, gamma=wl.gamma)
+    free2 = torch.cuda.mem_get_info()[0]
+    assert free1 - free2 < 40 << 20 and (free0 - free1 > 100 << 20 or free0 - free1 < 40 << 20)   # (an earlier test's plan may still hold the tables)
+    g = wl.gradient(0, device="cuda")
+    outs = []
+    for p in (p1, p2):
+        out = p.alloc_outputs()
+        p.encode(g, torch.zeros((wl.n_users, p.ld), device="cuda"), out)
+        outs.append(out)
+    assert torch.equal(outs[0]["bitstream"], outs[1]["bitstream"])
+    avg1 = p1.decode_aggregate(outs[0]).clone()
+    p1.close()
+    out = p2.alloc_outputs()
+    p2.state_import(0, np.zeros(p2.S, np.int32))
+    p2.encode(g, torch.zeros((wl.n_users, p2.ld), device="cuda"), out)
+    assert torch.equal(out["bitstream"], outs[0]["bitstream"]) and torch.equal(p2.decode_aggregate(out), avg1)
+    assert p2.status()[0] == 0
+
+
 def test_decoder_depends_only_on_the_stream(binding, oracle):
     """A second plan that never encoded anything (the parameter server) decodes the outputs."""
     from paper_2203_09044_b200 import inputs
