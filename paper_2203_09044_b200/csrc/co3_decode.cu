@@ -47,10 +47,13 @@ static_assert(STAGE_ROW % 4 == 0, "stage rows must keep 16-byte alignment");
 // windows), so the head of the second table that fits here nearly always holds all of them.
 constexpr int LONG_CACHE = CO3_LONG_CACHE;
 
+// (The primary table itself is a static __shared__ array of each kernel, so that its address is a
+// constant of the load instruction and a look-up is mask, load; `lut` points to it for the rare paths.)
 template <int BITS>
 struct TablesT {                                  // per-segment decoder tables in shared memory
     static constexpr int bits = BITS;
-    alignas(16) uint32_t lut[1 << BITS];
+    static_assert(BITS <= 14, "two codewords of the primary table must fit the 30 bits a refill guarantees");
+    uint32_t* lut;
     alignas(16) uint32_t long_cache[LONG_CACHE];  // the row's second table from the first codeword longer than BITS
     const uint32_t* lut_long;                     // the rest of it (global memory)
     uint32_t long_first;                          // first 16-bit window it covers
@@ -62,9 +65,10 @@ __device__ __forceinline__ uint32_t keep_up_to(uint32_t e, uint32_t bits) { retu
 // The stored table has 2^13 entries indexed by the next 13 stream bits (first bit lowest); its first
 // 2^BITS entries are the table for BITS index bits once the entries of longer codewords are blanked.
 template <int BITS>
-__device__ void load_tables(TablesT<BITS>& t, const Co3CodeBook& cb, int row, int tid, int nthreads) {
+__device__ void load_tables(TablesT<BITS>& t, uint32_t* s_lut, const Co3CodeBook& cb, int row, int tid, int nthreads) {
     const uint4* lut = reinterpret_cast<const uint4*>(cb.lut + (size_t)row * CO3_LUT_SIZE);
-    uint4* dst = reinterpret_cast<uint4*>(t.lut);
+    uint4* dst = reinterpret_cast<uint4*>(s_lut);
+    if (tid == 0) t.lut = s_lut;
     for (int i = tid; i < (1 << BITS) / 4; i += nthreads) {
         uint4 v = __ldg(lut + i);
         if (BITS < CO3_LUT_BITS) {
@@ -121,14 +125,19 @@ __device__ __forceinline__ uint32_t decode_long(uint32_t window, const T& t, boo
     return e;
 }
 
-// LSB-first bit reader over staged words: the stream sits at bits [0, nb) of hi:lo and the bits above
-// are zero; nw is the word after those, already loaded (a refill takes it and loads the one after, so
-// that no refill waits for shared memory), and rp the shared-space byte address of the word after nw.  A refill is checked once per PAIR
-// of symbols: with nb >= 32 two codewords (at most 16 bits each) can be taken without looking at nb,
-// and one more word then always fits.  (With 32 lanes a per-symbol refill branch would be taken on
-// nearly every step, so its cost is paid per step, not per refill.)
+// LSB-first bit reader over staged words.  The window hi:lo holds the stream SHIFTED LEFT BY TWO: the
+// next stream bits sit at bits [2, nb) and the bits above are zero, so that `lo & (mask << 2)` is at
+// once the byte offset of the table entry (bits 0 and 1 hold leftovers of consumed codewords, which
+// the mask drops).  nb therefore counts the stream bits in the window plus two.  nw is the word after
+// those, already loaded (a refill takes it and loads the one after, so that no refill waits for
+// shared memory), and rp the shared-space byte address of the word after nw.  A refill is checked once
+// per PAIR of symbols: with nb >= 32 the window holds at least 30 stream bits, which two codewords of
+// the primary table (at most 14 bits each) or one of any length (16) never exceed, and with nb < 32
+// one more word always fits.  (With 32 lanes a per-symbol refill branch would be taken on nearly every
+// step, so its cost is paid per step, not per refill.)
 // nb is kept in the low byte of its register only: a step subtracts the whole table entry (length in
-// the low byte, which never borrows because nb >= length), and the shifts look at five bits.
+// the low byte, which never borrows because nb >= length + 2), and the shifts look at five bits (a
+// refill finds 2 <= nb <= 31).
 struct Reader {
     uint32_t lo, hi;
     uint32_t nb;
@@ -143,7 +152,7 @@ __device__ __forceinline__ void refill(Reader& r) {
         const uint32_t w = r.nw;
         r.nw = lds32(r.rp);                                   // not needed before the next refill
         r.lo |= __funnelshift_l(0u, w, r.nb);                 // w << nb
-        r.hi = __funnelshift_l(w, 0u, r.nb);                  // w >> (32 - nb), 0 for nb = 0
+        r.hi = __funnelshift_l(w, 0u, r.nb);                  // w >> (32 - nb)
         r.nb += 32u;
         r.rp += 4;
     }
@@ -152,13 +161,19 @@ __device__ __forceinline__ void refill(Reader& r) {
 __device__ __forceinline__ void reader_init(Reader& r, uint32_t stage_addr, uint32_t bitpos) {
     r.rp = stage_addr + ((bitpos >> 5) << 2);
     const uint32_t sh = bitpos & 31u;
-    const unsigned long long v = (((unsigned long long)lds32(r.rp + 4) << 32) | lds32(r.rp)) >> sh;
-    r.lo = (uint32_t)v;
-    r.hi = (uint32_t)(v >> 32);
-    r.nb = 64u - sh;
-    r.nw = lds32(r.rp + 8);
-    r.rp += 12;
+    const uint32_t w0 = lds32(r.rp) >> sh;                    // the 32 - sh bits left of the first word
+    r.lo = w0 << 2;
+    r.hi = w0 >> 30;
+    r.nb = 34u - sh;
+    r.nw = lds32(r.rp + 4);
+    r.rp += 8;
 }
+// stream bits consumed since bit 0 of the staged words
+__device__ __forceinline__ uint32_t reader_pos(const Reader& r, uint32_t stage_addr) {
+    return ((r.rp - stage_addr - 4u) << 3) + 2u - reader_bits(r);
+}
+// the next 30 stream bits, unshifted (for the second table)
+__device__ __forceinline__ uint32_t reader_window(const Reader& r) { return __funnelshift_r(r.lo, r.hi, 2); }
 
 template <int OFF>
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
@@ -178,8 +193,8 @@ __device__ __forceinline__ void put_cell(uint32_t addr, uint32_t v) {
 // too, and the caller tests only the group's LAST entry.
 // PACKED: add the whole entry (length byte included); else add the signed magnitude.
 template <int OFF, bool PACKED, int BITS, bool STORE = false>
-__device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, uint32_t acc_addr) {
-    const uint32_t e = lds32(lut_addr + ((r.lo & ((1u << BITS) - 1u)) << 2));
+__device__ __forceinline__ uint32_t decode_step(Reader& r, const unsigned char* lut, uint32_t acc_addr) {
+    const uint32_t e = *reinterpret_cast<const uint32_t*>(lut + (r.lo & (((1u << BITS) - 1u) << 2)));
     r.lo = __funnelshift_r(r.lo, r.hi, e);        // shift by the length: low five bits of e
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= e;                                    // the low byte counts
@@ -189,10 +204,10 @@ __device__ __forceinline__ uint32_t decode_step(Reader& r, uint32_t lut_addr, ui
 
 // One symbol with the test for a long codeword (group tails, and groups that met a long codeword).
 template <bool PACKED, class T, bool STORE = false>
-__device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr, uint32_t acc_addr,
+__device__ __forceinline__ void decode_step_checked(Reader& r, const unsigned char* lut, uint32_t acc_addr,
                                                     const T& t, bool& bad) {
-    uint32_t e = lds32(lut_addr + ((r.lo & ((1u << T::bits) - 1u)) << 2));
-    if ((e & 0xFFu) == 0u) e = decode_long(r.lo, t, bad);
+    uint32_t e = *reinterpret_cast<const uint32_t*>(lut + (r.lo & (((1u << T::bits) - 1u) << 2)));
+    if ((e & 0xFFu) == 0u) e = decode_long(reader_window(r), t, bad);
     r.lo = __funnelshift_r(r.lo, r.hi, e);
     r.hi = __funnelshift_r(r.hi, 0u, e);
     r.nb -= e;                                    // the low byte counts
@@ -205,7 +220,7 @@ __device__ __forceinline__ void decode_step_checked(Reader& r, uint32_t lut_addr
 // in registers (its address is never taken); the long-codeword search itself is out of line.
 // (ROW: words between the cells of consecutive symbols of a lane)
 template <bool PACKED, class T, bool STORE = false, int ROW = PADW>
-__device__ __forceinline__ void finish_group(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int done,
+__device__ __forceinline__ void finish_group(Reader& r, const unsigned char* lut_addr, uint32_t acc_addr, int done,
                                              const T& t, bool& bad) {
 #pragma unroll 1
     for (int k = done; k < 4; ++k) {
@@ -215,7 +230,7 @@ __device__ __forceinline__ void finish_group(Reader& r, uint32_t lut_addr, uint3
 }
 
 template <bool PACKED, class T, bool STORE = false, int ROW = PADW>
-__device__ __forceinline__ void decode_run(Reader& r, uint32_t lut_addr, uint32_t acc_addr, int n,
+__device__ __forceinline__ void decode_run(Reader& r, const unsigned char* lut_addr, uint32_t acc_addr, int n,
                                            const T& t, bool& bad) {
     int i = 0;
     for (; i + 4 <= n; i += 4) {
@@ -407,7 +422,8 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     int32_t* acc0 = reinterpret_cast<int32_t*>(team_raw + sizeof(TeamHead));
     const int cpg = NW / U;                        // chunks per group (>= 1)
     const int accw = acc_words_a(U);               // words per accumulator buffer
-    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(tabs.lut);
+    __shared__ __align__(16) uint32_t s_lut[1 << BITS];
+    const unsigned char* lut_addr = reinterpret_cast<const unsigned char*>(s_lut);
     const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(acc0);
     const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[warp]);
     const int ci = warp / U, us = warp - ci * U;   // this warp's chunk-in-group and user
@@ -426,7 +442,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
         int64_t ge = gi + 1;
         while (ge < g1 && p.groups[ge].seg == seg) ++ge;
         __syncthreads();                           // every team is past its last look-up in the old tables
-        load_tables(tabs, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, TEAMS * CO3_THREADS);
+        load_tables(tabs, s_lut, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, TEAMS * CO3_THREADS);
         __syncthreads();                           // (and the first zeroing)
         const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
         for (int64_t g = gi + team; g < ge; g += TEAMS, ++opened) {
@@ -486,8 +502,7 @@ decode_small_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                 }
             }
             if (mine && s.active) {
-                const uint32_t endpos = s.staged ? ((r.rp - stage_addr - 4u) << 3) - reader_bits(r)
-                                                 : sr.wp * 32u - (uint32_t)sr.nb;
+                const uint32_t endpos = s.staged ? reader_pos(r, stage_addr) : sr.wp * 32u - (uint32_t)sr.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
             }
         }
@@ -509,7 +524,7 @@ struct SmemOne {
     alignas(16) uint32_t stage[ONE_WARPS][STAGE_ROW];
     alignas(16) int32_t tile[ONE_WARPS][ONE_QB * ONE_ROW];
 };
-static_assert(sizeof(SmemOne) <= 227 * 1024, "one block per SM must fit its shared memory");
+static_assert(sizeof(SmemOne) + (4u << BITS_ONE) <= 227 * 1024, "one block per SM must fit its shared memory");
 
 template <bool UPDATE>
 __global__ void __launch_bounds__(ONE_WARPS * 32, 1)
@@ -519,7 +534,8 @@ decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16
     extern __shared__ __align__(16) unsigned char s_raw[];
     SmemOne& sm = *reinterpret_cast<SmemOne*>(s_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    __shared__ __align__(16) uint32_t s_lut[1 << BITS_ONE];
+    const unsigned char* lut_addr = reinterpret_cast<const unsigned char*>(s_lut);
     const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(sm.stage[warp]);
     int32_t* tile = sm.tile[warp];
     const uint32_t tile_addr = (uint32_t)__cvta_generic_to_shared(tile);
@@ -531,7 +547,7 @@ decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16
         int64_t ce = ci + 1;
         while (ce < c1 && p.chunks[ce].seg == seg) ++ce;
         __syncthreads();                           // every warp is past its last look-up in the old tables
-        load_tables(sm.t, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, ONE_WARPS * 32);
+        load_tables(sm.t, s_lut, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, ONE_WARPS * 32);
         __syncthreads();
         const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
         for (int64_t c = ci + warp; c < ce; c += ONE_WARPS) {
@@ -585,8 +601,7 @@ decode_one_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream, const uint16
                 __syncwarp();                      // the tile is written again by the next batch
             }
             if (s.active) {
-                const uint32_t endpos = s.staged ? ((r.rp - stage_addr - 4u) << 3) - reader_bits(r)
-                                                 : sr.wp * 32u - (uint32_t)sr.nb;
+                const uint32_t endpos = s.staged ? reader_pos(r, stage_addr) : sr.wp * 32u - (uint32_t)sr.nb;
                 if (endpos - s.bitpos != s.sub_len_bits || endpos > s.nwords * 32u) bad = true;
             }
             __syncwarp();                          // the stage is reused by this warp's next chunk
@@ -608,7 +623,7 @@ struct SmemB {
     TablesT<BITS_B> t;
     TeamB team[TEAMS_B];
 };
-static_assert(sizeof(SmemB) <= 227 * 1024, "one block per SM must fit its shared memory");
+static_assert(sizeof(SmemB) + (4u << BITS_B) <= 227 * 1024, "one block per SM must fit its shared memory");
 
 __global__ void __launch_bounds__(TEAMS_B * CO3_THREADS, 1)
 decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
@@ -620,7 +635,8 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
     const int tid = threadIdx.x, lane = tid & 31;
     const int team = tid / CO3_THREADS, ttid = tid - team * CO3_THREADS, warp = ttid >> 5;
     TeamB& tm = sm.team[team];
-    const uint32_t lut_addr = (uint32_t)__cvta_generic_to_shared(sm.t.lut);
+    __shared__ __align__(16) uint32_t s_lut[1 << BITS_B];
+    const unsigned char* lut_addr = reinterpret_cast<const unsigned char*>(s_lut);
     const uint32_t acc_addr0 = (uint32_t)__cvta_generic_to_shared(tm.acc);
     const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(tm.stage[warp]);
     const int64_t c0 = p.dec_part[blockIdx.x], c1 = p.dec_part[blockIdx.x + 1];
@@ -634,7 +650,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
         int64_t ce = ci + 1;
         while (ce < c1 && p.chunks[ce].seg == seg) ++ce;
         __syncthreads();                           // every team is past its last look-up in the old tables
-        load_tables(sm.t, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, TEAMS_B * CO3_THREADS);
+        load_tables(sm.t, s_lut, p.cb, p.code_by_segment ? seg : co3_row_of(hdr[seg], &bad), tid, TEAMS_B * CO3_THREADS);
         __syncthreads();                           // (and the first zeroing)
         const float scale = pow2_clamped((int)hdr[seg].bias + p.cF);
         for (int64_t c = ci + team; c < ce; c += TEAMS_B) {
@@ -649,7 +665,7 @@ decode_large_u_kernel(Co3Dev p, const uint32_t* __restrict__ bitstream,
                         Reader r;
                         reader_init(r, stage_addr, s.bitpos);
                         decode_run<false>(r, lut_addr, acc_addr0 + 4u * (uint32_t)row0, s.i_hi - s.i_lo, sm.t, bad);
-                        endpos = ((r.rp - stage_addr - 4u) << 3) - reader_bits(r);
+                        endpos = reader_pos(r, stage_addr);
                     } else {
                         SlowReader sr;
                         slow_init(sr, s.gsrc, s.nwords, s.bitpos);
@@ -683,16 +699,17 @@ typedef void (*SmallKernel)(Co3Dev, const uint32_t*, const uint16_t*, const uint
 struct SmallVariant {
     SmallKernel fn;
     int teams;
-    size_t smem;
+    size_t smem;                                  // dynamic shared memory
+    size_t smem_static;                           // the primary table
 };
 // The widest table and the most teams that fit the shared memory of an SM (227 KB per block); user
 // counts that do not divide 8 leave warps idle and keep the plain one-team blocks, four per SM.
 SmallVariant small_variant(int U) {
     switch (U) {
-        case 8: return {decode_small_u_kernel<4, 13, 8>, 4, smem_a_bytes<4, 13>(U)};
-        case 4: return {decode_small_u_kernel<4, 12, 4>, 4, smem_a_bytes<4, 12>(U)};
-        case 2: return {decode_small_u_kernel<3, 12, 2>, 3, smem_a_bytes<3, 12>(U)};
-        default: return {decode_small_u_kernel<1, CO3_LUT_SMALL_BITS, 0>, 1, smem_a_bytes<1, CO3_LUT_SMALL_BITS>(U)};
+        case 8: return {decode_small_u_kernel<4, 13, 8>, 4, smem_a_bytes<4, 13>(U), 4u << 13};
+        case 4: return {decode_small_u_kernel<4, 12, 4>, 4, smem_a_bytes<4, 12>(U), 4u << 12};
+        case 2: return {decode_small_u_kernel<3, 12, 2>, 3, smem_a_bytes<3, 12>(U), 4u << 12};
+        default: return {decode_small_u_kernel<1, CO3_LUT_SMALL_BITS, 0>, 1, smem_a_bytes<1, CO3_LUT_SMALL_BITS>(U), 4u << CO3_LUT_SMALL_BITS};
     }
 }
 
@@ -706,7 +723,7 @@ cudaError_t co3_setup_decode_kernels(void) {
             const SmallVariant v2 = small_variant(U2);
             if (v2.fn == v.fn && v2.smem > need) need = v2.smem;
         }
-        if (need > 227u * 1024u) return cudaErrorInvalidConfiguration;
+        if (need + v.smem_static > 227u * 1024u) return cudaErrorInvalidConfiguration;
         cudaError_t e = cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
         if (e != cudaSuccess) return e;
     }
