@@ -234,7 +234,7 @@ def run_ours(args):
     elapsed_ms, launches, conv_ms, conv_n, clocks = timed_loop(args.steps, args.warmup)
     # ---- sustained leg: the same loop for about two seconds of device time --------------------
     # (a timed region of a few milliseconds is a burst figure and meets at most one clock sample)
-    sus_steps = max(args.steps, int(SUSTAINED_MS / max(elapsed_ms / args.steps, 1e-3)) + 1)
+    sus_steps = args.steps if args.short else max(args.steps, int(SUSTAINED_MS / max(elapsed_ms / args.steps, 1e-3)) + 1)
     sus_ms, _, sus_conv_ms, sus_conv_n, sus_clocks = timed_loop(sus_steps, args.warmup + args.steps)
     sus_ms = max_over_ranks(sus_ms, world, "cuda")
     code_bits = float(out["user_bits"].sum().item()) / (U * d)
@@ -254,7 +254,7 @@ def run_ours(args):
     plan.profile_enable([], 0)
 
     # ---- the other bias mode, timed the same way (K steps, eager) ------------------------------
-    other = {"current": "lagged", "lagged": "current"}.get(args.mode)
+    other = None if args.short else {"current": "lagged", "lagged": "current"}.get(args.mode)
     other_rec = None
     if other is not None:
         plan_o = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
@@ -596,6 +596,8 @@ def main():
                     help="override the number of simulated users (profiling a smaller case); default 8")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay leg")
+    ap.add_argument("--short", action="store_true",
+                    help="profiling runs: the sustained leg repeats only --steps steps, the other bias mode is not timed")
     ap.add_argument("--mode", default="current", choices=["lagged", "current", "code-lagged"],
                     help="bias/code mode behind `value` (default: current, the bias of Algorithm 1 as printed; "
                          "the lagged bias is timed beside it)")
