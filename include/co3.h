@@ -124,9 +124,11 @@ typedef struct {
 
 /* Algorithm 1 line 2 and Table I: fixes d, U, the format, the layers, gamma.  Validates the
  * configuration, computes the static chunk partition, builds the GenNorm model-weight table on
- * the host, allocates all device scratch on the current device and builds there, once, the
- * Huffman code (Sec. III (ii)) of every (shape, scale) pair a header can name, so that an
- * iteration only selects codes.  The iteration counter
+ * the host, allocates all device scratch on the current device and builds there the Huffman code
+ * (Sec. III (ii)) of every (shape, scale) pair a header can name, so that an iteration only selects
+ * codes.  Those code tables depend on the format alone: the plans of one device and format share one
+ * copy, built by the first of them and freed with the last (plan creation and destruction take a
+ * process-wide lock for that).  The iteration counter
  * starts at 0 (memory m_0 = 0 is the caller's zero-filled `residual`).
  * Every call that takes a stream only enqueues work on it (kernels, memsets, device-to-device copies)
  * and never waits for the device, so a steady-state iteration (t >= 1 with CO3_BIAS_LAGGED or
