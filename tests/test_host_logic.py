@@ -179,3 +179,17 @@ def test_optimal_bias_table_is_identical_in_library_and_oracle(binding, oracle, 
             a, b = binding.grid_distortion(E, M, ib, ir), oracle.distortion(E, M, ib, ir)
             assert a > 0 and abs(a - b) <= 1e-9 * b
     assert binding.grid_distortion(E, M, 9, 0) < 0 and binding.grid_distortion(E, M, 0, 32) < 0
+
+
+def test_bench_reads_the_convert_traffic_from_the_profile_record():
+    """roofline.traffic of the bench line comes from the figures kept beside the ncu summary, scaled
+    by the number of users; algorithmic bytes of the convert pass are 13 per user-element."""
+    import json
+    import sys
+    sys.path.insert(0, ROOT)
+    import bench
+    rec = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic_config1_8users.json")))
+    assert bench.convert_dram_traffic(8) == rec["convert_dram_bytes_per_launch"]
+    assert bench.convert_dram_traffic(2) == rec["convert_dram_bytes_per_launch"] / 4
+    algorithmic = bench.CONVERT_BYTES_PER_ELEMENT * 8 * 11_173_962
+    assert 0.9 * algorithmic < rec["convert_dram_bytes_per_launch"] < 1.05 * algorithmic
