@@ -333,15 +333,16 @@ int64_t co3_partition(int64_t d, int32_t n_segments, const int64_t* seg_offsets,
                       int32_t* chunk_seg, int64_t* chunk_start, int64_t* chunk_end,
                       int64_t* sub_base, int64_t* n_sub);
 
-/* Host only: how co3_plan_create splits the decoder's work over its thread blocks.  n items in order,
- * each with a cost (host, double) and a segment number (host, int32); a block takes a contiguous range and
- * walks it run by run of one segment, its `teams` (1..32) teams taking every teams-th item of a run and
- * meeting where the segment changes, so a run takes as long as its most loaded team's items plus a fixed
- * 0.08 for the change of code tables; the cost of a block is the mean of that time summed over its runs
- * and of its total item cost divided by `teams` (what binds when all its teams are busy).  part (host,
- * max_blocks + 1 entries) receives cuts that minimise the largest block cost over all contiguous splits
- * into at most max_blocks blocks: block b takes items
- * part[b] .. part[b+1] - 1.  Returns the number of blocks in use, or a negative value for bad arguments. */
+/* Host only: how co3_plan_create splits the work of the multi-user decoders over their thread blocks.
+ * n items in order, each with a cost (host, double; 1 = a full chunk) and a segment number (host, int32);
+ * a block takes a contiguous range and walks it run by run of one segment, its `teams` (1..32) teams
+ * taking every teams-th item of a run and meeting where the segment changes.  The time of a run is
+ * modelled as the mean of the cost of its most loaded team and of its total cost / teams (what binds
+ * when all teams are busy), plus a fixed 0.04 for the change of code tables; a block takes the sum over
+ * its runs.  part (host, max_blocks + 1 entries) receives cuts whose largest block time is the least
+ * that a contiguous split into at most max_blocks blocks reaches, with the work spread over all
+ * min(max_blocks, n) blocks in proportion within that bound: block b takes items part[b] .. part[b+1] - 1.
+ * Returns the number of blocks in use, or a negative value for bad arguments. */
 int co3_balanced_split(const double* cost, const int32_t* seg, int64_t n, int32_t teams, int32_t max_blocks,
                        int32_t* part);
 

@@ -234,50 +234,86 @@ extern "C" int co3_model_weights(co3_format fmt, int32_t ibeta, int32_t ir, uint
 
 // Contiguous split of n work items over at most max_blocks thread blocks for kernels whose blocks walk
 // their items run by run of one segment, the block's `teams` teams taking every teams-th item of a run
-// and all of them meeting where the segment changes.  A run then costs its most loaded team's items
-// plus run_cost (the change of tables), and a block's rounds are the sum over its runs.  Equal item
-// counts per block would let a block whose range a segment boundary cuts into, say, 10 + 9 items take
-// six team-rounds where its neighbours take five, and every block waits for the slowest.  Rounds alone
-// would pack full rounds into fewer blocks than there are SMs, though, and a block whose teams are all
-// busy is bound by the throughput of its SM, i.e. by its total work: a block's cost is therefore the
-// mean of its rounds and of its work per team.  The cuts are placed so that the largest block cost is
-// as small as a contiguous split allows (bisection on that bound, greedy fill).  part[0 .. max_blocks]
+// and all of them meeting where the segment changes.  A run lasts at least as long as its most loaded
+// team needs, and a block whose teams are all busy is bound by the throughput of its SM, i.e. by its
+// total work; the time of a run is modelled as the mean of the two (its most loaded team's items, and
+// its total / teams) plus run_cost / 2 for the change of tables, and a block takes the sum over its
+// runs.  (Per-block cycle counts taken with clock64 on the 62-layer ResNet-18 workload, 8 users, 4
+// teams: 20 full chunks in one run 166 k, 19 in one run 145-160 k, 10 + 1 + 2 + 5 chunks in four runs
+// of which two are tiny layers 170 k.  A model that takes the larger of 0.45 x the team's items and the
+// total / teams fits those counts a little better and gave a kernel 2 % slower on that workload, 3 %
+// faster with four users: within what the choice of cuts can move.)  Equal item counts per block let a
+// block with a few tiny layers in its range, or one that a layer boundary cuts into 10 + 9, take a
+// round more than its neighbours, and every block waits for the slowest; the cuts are therefore placed
+// so that the largest block cost is as small as a contiguous split allows (bisection on that bound),
+// and within that bound the work is spread over all the blocks in proportion.  part[0 .. max_blocks]
 // receives the cuts; returns the blocks in use.
 int co3_host_balanced_split(const double* w, const int32_t* seg, int64_t n, int teams, int max_blocks, double run_cost,
                             int32_t* part) {
     if (!w || !seg || !part || n < 1 || n > 0x7FFFFFFFLL || teams < 1 || teams > 32 || max_blocks < 1) return -1;
-    auto blocks_needed = [&](double bound, int32_t* cuts) {
-        int64_t blocks = 0, i = 0;
+    auto run_time = [&](double team_max, double work) {
+        return 0.5 * team_max + 0.5 * work / teams + 0.5 * run_cost;
+    };
+    // furthest end (exclusive) of a block that starts at item `from` and costs at most `bound`
+    auto reach = [&](int64_t from, double bound) {
+        int64_t i = from;
+        double closed = 0.0, team_sum[32] = {0}, run_max = w[i], run_work = w[i];   // a block takes at least one item
+        int cur = seg[i], pos = 1;
+        team_sum[0] = w[i];
+        ++i;
         while (i < n) {
-            if (cuts && blocks < max_blocks) cuts[blocks] = (int32_t)i;
-            double closed = run_cost, team_sum[32] = {0}, run_max = w[i];     // a block takes at least one item
-            double work = w[i];
-            int cur = seg[i], pos = 1;
-            team_sum[0] = w[i];
+            const bool new_run = seg[i] != cur;
+            const double c2 = new_run ? closed + run_time(run_max, run_work) : closed;
+            const int p2 = new_run ? 0 : pos;
+            const double t2 = (new_run ? 0.0 : team_sum[p2 % teams]) + w[i];
+            const double m2 = new_run ? t2 : (run_max > t2 ? run_max : t2);
+            const double k2 = (new_run ? 0.0 : run_work) + w[i];
+            if (c2 + run_time(m2, k2) > bound) break;
+            if (new_run) { for (int t = 0; t < teams; ++t) team_sum[t] = 0.0; cur = seg[i]; }
+            closed = c2; run_max = m2; run_work = k2; team_sum[p2 % teams] = t2; pos = p2 + 1;
             ++i;
-            while (i < n) {
-                const bool new_run = seg[i] != cur;
-                const double c2 = new_run ? closed + run_max + run_cost : closed;
-                const int p2 = new_run ? 0 : pos;
-                const double t2 = (new_run ? 0.0 : team_sum[p2 % teams]) + w[i];
-                const double r2 = new_run ? t2 : (run_max > t2 ? run_max : t2);
-                if (0.5 * (c2 + r2) + 0.5 * (work + w[i]) / teams > bound) break;
-                if (new_run) { for (int t = 0; t < teams; ++t) team_sum[t] = 0.0; cur = seg[i]; }
-                closed = c2; run_max = r2; team_sum[p2 % teams] = t2; pos = p2 + 1; work += w[i];
-                ++i;
-            }
-            ++blocks;
         }
+        return i;
+    };
+    auto blocks_needed = [&](double bound) {
+        int64_t blocks = 0;
+        for (int64_t i = 0; i < n; i = reach(i, bound)) ++blocks;
         return blocks;
     };
     double lo = 0.0, hi = 0.0;
     for (int64_t i = 0; i < n; ++i) hi += w[i] + run_cost;
     for (int it = 0; it < 60; ++it) {
         const double mid = 0.5 * (lo + hi);
-        if (blocks_needed(mid, nullptr) <= max_blocks) hi = mid; else lo = mid;
+        if (blocks_needed(mid) <= max_blocks) hi = mid; else lo = mid;
     }
-    const int64_t blocks = blocks_needed(hi, part);
+    // Within the bound found, spread the items over ALL the blocks: the greedy fill would leave the last
+    // blocks empty, and a block with less work is never slower.  need[i] = blocks a greedy fill needs for
+    // the items i .. n-1; a cut at i before block b is admissible if the rest still fits the blocks left.
+    const int64_t blocks = max_blocks < n ? max_blocks : n;
+    int32_t* need = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n + 1));
+    double* pre = (double*)malloc(sizeof(double) * (size_t)(n + 1));
+    if (!need || !pre) { free(need); free(pre); return -1; }
+    {   // backwards: need[i] = 1 + need[reach(i)], computed with a moving window of block starts
+        need[n] = 0;
+        for (int64_t i = n - 1; i >= 0; --i) need[i] = 1 + need[reach(i, hi)];
+        pre[0] = 0.0;
+        for (int64_t i = 0; i < n; ++i) pre[i + 1] = pre[i] + w[i];
+    }
+    int64_t at = 0;
+    for (int64_t b = 0; b < blocks; ++b) {
+        part[b] = (int32_t)at;
+        if (at >= n) continue;
+        const int64_t far = reach(at, hi);                  // the block may end anywhere in (at, far]
+        const double target = pre[n] * (double)(b + 1) / (double)blocks;
+        int64_t end = at + 1;
+        while (end < far && pre[end] < target) ++end;       // proportional share of the work ...
+        while (end < far && need[end] > blocks - b - 1) ++end;   // ... unless the rest would not fit
+        if (n - end < blocks - b - 1) end = n - (blocks - b - 1) > at ? n - (blocks - b - 1) : at + 1;   // leave an item for every later block
+        at = end;
+    }
     for (int64_t b = blocks; b <= max_blocks; ++b) part[b] = (int32_t)n;
+    part[blocks] = (int32_t)n;
+    free(need); free(pre);
     return (int)blocks;
 }
 
