@@ -2,8 +2,9 @@
 
 The arithmetic lives in co3_oracle.c; this file only sequences the steps of Algorithm 1
 (lines 8-10 at the users, lines 13-14 at the parameter server) and keeps the state that the
-method carries between iterations (the bias for the next iteration in LAGGED mode).  The
-memory m^(u) is the caller's array and is updated in place.
+method carries between iterations (the bias for the next iteration in LAGGED mode).  The one
+exception is the model update of line 14 (decode_aggregate_update), two numpy float32 operations
+written out here.  The memory m^(u) is the caller's array and is updated in place.
 """
 import ctypes as C
 import numpy as np
