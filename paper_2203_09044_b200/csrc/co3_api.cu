@@ -476,13 +476,16 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
         pl->iteration++;
         return CO3_OK;
     }
-    if (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) {
+    // Bias from the current moments: the fit after the statistics pass also gives the header (the convert
+    // pass would hand the next fit the same sums), so there is one fit per iteration in both modes.
+    const bool current = pl->cfg.bias_mode == CO3_BIAS_CURRENT;
+    if (pl->iteration == 0 || current) {
         CO3_TRY(co3_launch_stats(pl, grad, residual, 0, pl->dev.U, st));
-        CO3_TRY(co3_launch_fit(pl, 0, hdr, st));
+        CO3_TRY(co3_launch_fit(pl, current ? 5 : 0, hdr, st));
     }
     CO3_TRY(co3_launch_convert(pl, grad, residual, 0, pl->dev.U, true, st));
     if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));   // the gradient buffer is free from here on
-    CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
+    if (!current) CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) CO3_TRY(co3_build_hist_codes(pl, pl->emp_lens, st));
     CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;

@@ -76,6 +76,10 @@ __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int c
 // mode 3: after the fused convert-and-pack pass -- the same for the next iteration; keep the fit.
 //         In both, `hdr` is the plan's own header array.
 // mode 4: only add up the moments of every segment and write (N, S1, S2) to mom_out.
+// mode 5: after the stats pass when the bias comes from the current iteration's own moments: the bias for
+//         the coming convert pass AND the header of this iteration (the convert pass sums the same
+//         a = g + gamma m item by item in the same order, so a second fit after it would reproduce these
+//         numbers bit for bit); keeps the fit and prepares the encoder like mode 1.
 // ext_mom (may be null): (N, S1, S2) per segment that replace the plan's own sums in the fit (the sums
 //         of a layer that is spread over several plans); the non-finite count stays the plan's own.
 // fit_ovr (may be null): (beta, alpha) per segment that replace the solve (test hook: a harness feeds
@@ -91,7 +95,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     __shared__ int s_state, s_coarse, s_fine;
 
     const int seg = blockIdx.x, tid = threadIdx.x;
-    if (mode == 1 && p.red_k == 0) {
+    if ((mode == 1 || mode == 5) && p.red_k == 0) {
         // side job: the single-pass encode that follows this launch wants its tickets, published
         // counts and group totals at zero
         unsigned long long* z = p.enc_grp;
@@ -436,7 +440,7 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
     co3_prof_begin(pl, CO3_K_FIT, st);
-    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1);
+    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1 || mode == 5);
     const double* ext = (pl->use_ext_mom && mode != 4) ? pl->ext_mom : nullptr;
     if (mode != 4) pl->use_ext_mom = false;                // imported moments serve one fit
     fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out,
