@@ -833,10 +833,31 @@ def test_sweep_d_2p20_laplace_shape(binding, oracle, U, E, M):
 
 @pytest.mark.slow
 @pytest.mark.parametrize("E,M", FORMATS)
-def test_sweep_d_2p24_8_users(binding, oracle, E, M):
+@pytest.mark.parametrize("beta", [0.5, 1.0, 2.0])
+def test_sweep_d_2p24_8_users(binding, oracle, beta, E, M):
     from paper_2203_09044_b200 import inputs
-    wl = inputs.sweep_cell(1 << 24, 8, 1.0, E, M)
+    wl = inputs.sweep_cell(1 << 24, 8, beta, E, M)
     run_case(binding, oracle, wl.d, 8, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("beta", [0.5, 1.0, 2.0])
+def test_sweep_d_2p24_single_user_all_shapes(binding, oracle, beta, E, M):
+    """One user: the decoder of its own (24 independent warps per block), 4096 chunks."""
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 24, 1, beta, E, M)
+    run_case(binding, oracle, wl.d, 1, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("E,M", FORMATS)
+@pytest.mark.parametrize("beta", [0.5, 2.0])
+@pytest.mark.parametrize("U", [1, 64])
+def test_sweep_d_2p20_other_shapes(binding, oracle, U, beta, E, M):
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.sweep_cell(1 << 20, U, beta, E, M)
+    run_case(binding, oracle, wl.d, U, E, M, wl.seg_offsets, _grads(wl, 1), gamma=wl.gamma)
 
 
 @pytest.mark.slow
