@@ -127,13 +127,15 @@ __device__ __forceinline__ void or_piece(uint32_t* img, uint32_t pos, unsigned l
     if (w2) atomicOr(&img[wi + 2], w2);
 }
 
-// MODE 0: statistics only.  MODE 1: convert, symbols to memory.  MODE 2: convert and pack.
+// MODE 1: convert, symbols to memory.  MODE 2: convert and pack.  (The statistics pass has a kernel of
+// its own, below.)
 template <int M, int MODE>
 __global__ void __launch_bounds__(CO3_THREADS, 4)
 ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t* __restrict__ sub_bits) {
-    constexpr bool CONVERT = MODE >= 1, PACK = MODE == 2;
+    static_assert(MODE == 1 || MODE == 2, "the statistics pass is stats_kernel");
+    constexpr bool PACK = MODE == 2;
     extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS] (+ PackSmem)
-    __shared__ uint32_t s_hist[2][CONVERT ? CO3_THREADS / 32 : 1][CO3_MAXSYM];   // [item parity][warp][symbol]
+    __shared__ uint32_t s_hist[2][CO3_THREADS / 32][CO3_MAXSYM];   // [item parity][warp][symbol]
     __shared__ double s_red[2][2][CO3_THREADS / 32];
     __shared__ uint32_t s_rednf[2][CO3_THREADS / 32];
     __shared__ uint32_t s_ticket[2];
@@ -155,8 +157,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
         s_ticket[0] = atomicAdd(p.ticket, 1u);
         s_ticket[1] = atomicAdd(p.ticket, 1u);
     }
-    if (CONVERT)
-        for (int i = tid; i < 2 * (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0][0])[i] = 0;
+    for (int i = tid; i < 2 * (CO3_THREADS / 32) * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0][0])[i] = 0;
     PackSmem& pk = *reinterpret_cast<PackSmem*>(s_ring + STAGES * 2 * CO3_THREADS);
     if (PACK)
         for (int i = tid; i < (CO3_THREADS / 32) * SLOT_W; i += CO3_THREADS) (&pk.slot[0][0])[i] = 0;
@@ -165,13 +166,8 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
     if (item >= n_items) return;
     __syncthreads();                                  // both tickets read before slot 0 is reused
 
-    // The statistics pass walks the items from the last one down: it ends where the convert pass that
-    // follows it begins, and begins where the previous iteration's convert pass ended, so both meet
-    // part of their input (what the 126 MB L2 still holds of gradient and memory) without going to HBM.
-    auto phys = [&](uint32_t t) { return (!CONVERT && t < n_items) ? n_items - 1u - t : t; };
     auto make_ctx = [&](uint32_t t, const Co3Chunk& cd) {
-        const uint32_t it = phys(t);
-        const uint32_t ul = it / n_chunks, uu = ul + (uint32_t)p.u_base;
+        const uint32_t ul = t / n_chunks, uu = ul + (uint32_t)p.u_base;
         ItemCtx x;
         const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
         x.gp = g + (size_t)ul * p.ld + tb + 4 * tid;
@@ -200,13 +196,13 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
         cp_async_commit();
     };
 
-    ItemCtx cur = make_ctx(item, p.chunks[phys(item) % n_chunks]);
+    ItemCtx cur = make_ctx(item, p.chunks[item % n_chunks]);
     issue(cur, true, 0);
     issue(cur, true, 1);
     issue(cur, true, 2);
     bool has_nxt = nitem < n_items;
     ItemCtx nxt = cur;
-    if (has_nxt) nxt = make_ctx(nitem, p.chunks[phys(nitem) % n_chunks]);
+    if (has_nxt) nxt = make_ctx(nitem, p.chunks[nitem % n_chunks]);
 
     // the code table of an item's segment is fetched while the previous item is converted
     auto enc_entry = [&](int seg) {
@@ -229,7 +225,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
         uint32_t claim = n_items;
         Co3Chunk claim_cd;
         if (tid == 0 && has_nxt) claim = atomicAdd(p.ticket, 1u);
-        if (CONVERT && cur.seg != cur_seg) {
+        if (cur.seg != cur_seg) {
             cur_seg = cur.seg;
             const int lambda = p.bias_cur[cur.seg] + p.cF;
             q.top = __fmul_rn((float)p.Kmax, pow2f(lambda));
@@ -254,7 +250,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
             // 0..2 of the next one, each into the slot the consumer has just left
             if (r == 0) issue(cur, true, 3);
             else issue(nxt, has_nxt, r - 1);
-            if (r == 2 && tid == 0 && claim < n_items) claim_cd = p.chunks[phys(claim) % n_chunks];
+            if (r == 2 && tid == 0 && claim < n_items) claim_cd = p.chunks[claim % n_chunks];
             cp_async_wait<STAGES - 1>();              // this step's copies have landed
             const uint32_t slot = r * SLOT_BYTES;
             const int e0 = 4 * tid + VSTRIDE * r;
@@ -269,17 +265,15 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
                 uint32_t so[4], en[4] = {0u, 0u, 0u, 0u};
                 if (full) {
                     ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
-                    if (CONVERT) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            quantize<M>(a[e], q, so[e], mo[e]);
-                            atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
-                            if (PACK) en[e] = enc_tab[so[e]];
-                        }
-                        *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
-                        if (!PACK)
-                            *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
+                    for (int e = 0; e < 4; ++e) {
+                        quantize<M>(a[e], q, so[e], mo[e]);
+                        atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
+                        if (PACK) en[e] = enc_tab[so[e]];
                     }
+                    *reinterpret_cast<float4*>(cur.mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+                    if (!PACK)
+                        *reinterpret_cast<uint32_t*>(cur.sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
                 } else {                              // a vector on the chunk's edge: element by element
                     const bool in0 = e0 >= cur.lo && e0 < cur.hi, in1 = e0 + 1 >= cur.lo && e0 + 1 < cur.hi;
                     const bool in2 = e0 + 2 >= cur.lo && e0 + 2 < cur.hi, in3 = e0 + 3 >= cur.lo && e0 + 3 < cur.hi;
@@ -289,16 +283,14 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
                     if (!in2) { gv.z = 0.0f; mv.z = 0.0f; }
                     if (!in3) { gv.w = 0.0f; mv.w = 0.0f; }
                     ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
-                    if (CONVERT) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            if (in[e]) {
-                                quantize<M>(a[e], q, so[e], mo[e]);
-                                atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
-                                cur.mp[VSTRIDE * r + e] = mo[e];
-                                if (PACK) en[e] = enc_tab[so[e]];
-                                else cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
-                            }
+                    for (int e = 0; e < 4; ++e) {
+                        if (in[e]) {
+                            quantize<M>(a[e], q, so[e], mo[e]);
+                            atomicAdd(&s_hist[hpar][warp][so[e]], 1u);
+                            cur.mp[VSTRIDE * r + e] = mo[e];
+                            if (PACK) en[e] = enc_tab[so[e]];
+                            else cur.sp[VSTRIDE * r + e] = (uint8_t)so[e];
                         }
                     }
                 }
@@ -362,14 +354,14 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
             uint32_t tn = 0;
 #pragma unroll
             for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[par][0][w]; t2 += s_red[par][1][w]; tn += s_rednf[par][w]; }
-            const uint32_t pi = item_base + phys(item);
+            const uint32_t pi = item_base + item;
             p.part_s1[pi] = t1; p.part_s2[pi] = t2; p.part_nf[pi] = tn;
         }
         // When the block leaves the segment (or ends) its histogram goes to global memory; the next
         // item counts in the other copy, and this copy is not touched again before a later barrier.
         // (Flushing after every item instead costs a single-segment E4M3 gradient 30 % of the pass:
         // all blocks then hammer the same 256 counters.)
-        if (CONVERT && (!has_nxt || nxt.seg != cur.seg)) {
+        if (!has_nxt || nxt.seg != cur.seg) {
             if (tid < p.nsym) {
                 unsigned long long tot = 0;
 #pragma unroll
@@ -387,6 +379,93 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
         par ^= 1;
     }
     cp_async_wait<0>();
+}
+
+// Statistics pass (the bias of Algorithm 1 line 8 taken from the moments of g_t + gamma m_{t-1}
+// themselves, before they are converted): nothing is written but three numbers per item, so a plain
+// grid does it -- one block per item, all of a thread's eight 128-bit loads in flight at once, five
+// blocks per SM so that nobody waits for the reduction at the end.  The block scheduler hands the
+// items out in order, which keeps the sweep of a streaming read.  The loads are marked evict-first
+// (read once: 117 -> 110 us on 8 x 11.2 M elements), except those of the items the convert pass will
+// take first, which ask to stay in L2.  The items are walked from the last one down, so the pass ends
+// with exactly those, and begins where the previous iteration's convert pass ended.
+// A thread takes the same elements in the same order as in the convert pass and the partial sums are
+// combined in the same order, so both passes give the same bits.
+constexpr uint32_t STATS_KEEP_ITEMS = (32u << 20) / (2 * sizeof(float) * CO3_TILE);   // 32 MB of g and m
+
+__device__ __forceinline__ float4 ld_keep(const float4* ptr, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr), "l"(policy));
+    return v;
+}
+
+__global__ void __launch_bounds__(CO3_THREADS, 4)
+stats_kernel(Co3Dev p, const float* __restrict__ g, const float* __restrict__ m) {
+    __shared__ double s_red[2][CO3_THREADS / 32];
+    __shared__ uint32_t s_rednf[CO3_THREADS / 32];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t n_chunks = (uint32_t)p.n_chunks;
+    const uint32_t it = gridDim.x - 1u - blockIdx.x;          // item: user (of this launch) x chunk
+    const uint32_t ul = it / n_chunks, uu = ul + (uint32_t)p.u_base;
+    const Co3Chunk cd = p.chunks[it - ul * n_chunks];
+    const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+    const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+    const bool whole = cd.len == CO3_TILE;
+    constexpr int VSTRIDE = 4 * CO3_THREADS;
+    const float4* gp = reinterpret_cast<const float4*>(g + (size_t)ul * p.ld + tb + 4 * tid);
+    const float4* mp = reinterpret_cast<const float4*>(m + (size_t)uu * p.ld + tb + 4 * tid);
+    const bool keep = it < STATS_KEEP_ITEMS;
+    uint64_t keep_policy = 0;
+    if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep_policy));
+    float4 gv[STEPS], mv[STEPS];
+#pragma unroll
+    for (int r = 0; r < STEPS; ++r) {
+        const int e0 = 4 * tid + VSTRIDE * r;
+        gv[r] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        mv[r] = gv[r];
+        if (whole || (e0 < hi && e0 + 4 > lo)) {
+            if (keep) {
+                gv[r] = ld_keep(gp + (VSTRIDE / 4) * r, keep_policy);
+                mv[r] = ld_keep(mp + (VSTRIDE / 4) * r, keep_policy);
+            } else {
+                gv[r] = __ldcs(gp + (VSTRIDE / 4) * r);
+                mv[r] = __ldcs(mp + (VSTRIDE / 4) * r);
+            }
+        }
+    }
+    double s1 = 0.0, s2 = 0.0;
+    uint32_t nf = 0;
+#pragma unroll
+    for (int r = 0; r < STEPS; ++r) {
+        const int e0 = 4 * tid + VSTRIDE * r;
+        if (!whole && !(e0 >= lo && e0 + 4 <= hi)) {          // a vector on the chunk's edge, or outside it
+            if (e0 + 4 <= lo || e0 >= hi) continue;
+            if (e0 < lo || e0 >= hi) { gv[r].x = 0.0f; mv[r].x = 0.0f; }   // elements of the neighbouring chunk count as 0
+            if (e0 + 1 < lo || e0 + 1 >= hi) { gv[r].y = 0.0f; mv[r].y = 0.0f; }
+            if (e0 + 2 < lo || e0 + 2 >= hi) { gv[r].z = 0.0f; mv[r].z = 0.0f; }
+            if (e0 + 3 < lo || e0 + 3 >= hi) { gv[r].w = 0.0f; mv[r].w = 0.0f; }
+        }
+        float a[4];
+        ef_add4(gv[r], mv[r], p.gamma, a, s1, s2, nf);
+    }
+    // lanes, then warps, in the order of the convert pass
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        s1 += __shfl_down_sync(0xffffffffu, s1, o);
+        s2 += __shfl_down_sync(0xffffffffu, s2, o);
+        nf += __shfl_down_sync(0xffffffffu, nf, o);
+    }
+    if (lane == 0) { s_red[0][warp] = s1; s_red[1][warp] = s2; s_rednf[warp] = nf; }
+    __syncthreads();
+    if (tid == 0) {
+        double t1 = 0.0, t2 = 0.0;
+        uint32_t tn = 0;
+#pragma unroll
+        for (int w = 0; w < CO3_THREADS / 32; ++w) { t1 += s_red[0][w]; t2 += s_red[1][w]; tn += s_rednf[w]; }
+        const uint32_t pi = n_chunks * (uint32_t)p.u_base + it;
+        p.part_s1[pi] = t1; p.part_s2[pi] = t2; p.part_nf[pi] = tn;
+    }
 }
 
 // Inspection: copy the stored symbols to a caller buffer [U][d] in the public form.
@@ -434,15 +513,11 @@ cudaError_t co3_launch_symbol_export(co3_plan* pl, uint8_t* symbols, cudaStream_
 
 // u_base / u_count: the users this launch covers (g is then the gradient of those users only).
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u_base, int u_count, cudaStream_t st) {
-    ef_fn fn = pick_kernel<0>(pl->dev.M);
-    if (!pl->grid_stats) pl->grid_stats = ef_grid(pl, fn, RING_BYTES);
-    cudaError_t e = cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
-    if (e != cudaSuccess) return e;
     Co3Dev p = pl->dev;
     p.u_base = u_base; p.u_count = u_count;
-    const int64_t items = p.n_chunks * (int64_t)u_count;
+    const int64_t items = p.n_chunks * (int64_t)u_count;       // below 2^31 (checked when the plan is made)
     co3_prof_begin(pl, CO3_K_STATS, st);
-    fn<<<(int)(items < pl->grid_stats ? items : pl->grid_stats), CO3_THREADS, RING_BYTES, st>>>(p, g, const_cast<float*>(m), nullptr);
+    stats_kernel<<<(unsigned)items, CO3_THREADS, 0, st>>>(p, g, m);
     co3_prof_end(pl, CO3_K_STATS, st, 1);
     return cudaGetLastError();
 }

@@ -133,7 +133,7 @@ struct co3_plan {
     uint8_t* emp_lens;              // ... the caller's length table during co3_encode_empirical
     const uint8_t* emp_lens_in;     // ... and during co3_decode_aggregate_empirical
     size_t enc_sync_bytes;          // size of the enc_grp / enc_st / enc_ticket allocation
-    int grid_stats, grid_convert;   // launch grids (fixed per plan: they define the reduction order)
+    int grid_convert;               // launch grid of the convert pass (fixed per plan)
     cudaStream_t last_stream;
     // co3_iteration_host: copy streams and the events that order them against the caller's stream
     cudaStream_t s_in, s_out;
