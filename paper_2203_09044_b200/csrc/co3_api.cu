@@ -479,11 +479,12 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
     // Bias from the current moments: the fit after the statistics pass also gives the header (the convert
     // pass would hand the next fit the same sums), so there is one fit per iteration in both modes.
     const bool current = pl->cfg.bias_mode == CO3_BIAS_CURRENT;
-    if (pl->iteration == 0 || current) {
+    const bool with_stats = pl->iteration == 0 || current;
+    if (with_stats) {
         CO3_TRY(co3_launch_stats(pl, grad, residual, 0, pl->dev.U, st));
-        CO3_TRY(co3_launch_fit(pl, current ? 5 : 0, hdr, st));
+        CO3_TRY(co3_launch_fit(pl, current ? 5 : 0, hdr, st, true));   // also zeroes the convert pass's histogram and ticket
     }
-    CO3_TRY(co3_launch_convert(pl, grad, residual, 0, pl->dev.U, true, st));
+    CO3_TRY(co3_launch_convert(pl, grad, residual, 0, pl->dev.U, true, st, with_stats));
     if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));   // the gradient buffer is free from here on
     if (!current) CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
     if (pl->cfg.bias_mode == CO3_CODE_EMPIRICAL) CO3_TRY(co3_build_hist_codes(pl, pl->emp_lens, st));

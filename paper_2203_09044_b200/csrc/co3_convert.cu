@@ -523,11 +523,14 @@ cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u
 }
 
 // first: this launch starts the iteration's histogram (later tiles of the same iteration add to it)
+// cleared: the fit kernel launched just before has zeroed the histogram and the ticket
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, int u_base, int u_count, bool first,
-                               cudaStream_t st) {
+                               cudaStream_t st, bool cleared) {
     // one memset clears the histogram and the item ticket that follows it in the same allocation
-    cudaError_t e = first ? cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st)
-                          : cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
+    cudaError_t e = cudaSuccess;
+    if (cleared) {}
+    else if (first) e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st);
+    else e = cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
     ef_fn fn = pick_kernel<1>(pl->dev.M);
     if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn, RING_BYTES);

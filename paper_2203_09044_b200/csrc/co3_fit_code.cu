@@ -84,10 +84,12 @@ __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int c
 //         of a layer that is spread over several plans); the non-finite count stays the plan's own.
 // fit_ovr (may be null): (beta, alpha) per segment that replace the solve (test hook: a harness feeds
 //         another implementation's fit to tell a rounding of the fit from a fault further down).
+// clear_hist: the convert pass is the next launch; its histogram and item ticket are zeroed here
+//         (a memset of its own between the two kernels costs the step two microseconds).
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr,
                                                           const double* __restrict__ ext_mom,
                                                           double* __restrict__ mom_out,
-                                                          const double* __restrict__ fit_ovr) {
+                                                          const double* __restrict__ fit_ovr, int clear_hist) {
     __shared__ double s_a[FIT_THREADS / 32], s_b[FIT_THREADS / 32];
     __shared__ unsigned long long s_n[FIT_THREADS / 32];
     __shared__ double s_lg[3];
@@ -100,6 +102,11 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         // counts and group totals at zero
         unsigned long long* z = p.enc_grp;
         for (size_t i = (size_t)blockIdx.x * FIT_THREADS + tid; i < p.enc_sync_words64; i += (size_t)gridDim.x * FIT_THREADS) z[i] = 0ull;
+    }
+    if (clear_hist) {
+        for (int h = 0; h < p.hist_copies; ++h)
+            for (int i = tid; i < CO3_MAXSYM; i += FIT_THREADS) p.hist[((size_t)h * p.S + seg) * CO3_MAXSYM + i] = 0ull;
+        if (seg == 0 && tid == 0) *p.ticket = 0u;
     }
     const int c0 = p.seg_chunk0[seg], c1 = p.seg_chunk0[seg + 1];
     // fixed order: thread t takes the (user, chunk) pairs t, t + 512, ... of the segment, all loads
@@ -438,13 +445,13 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 
 }  // namespace
 
-cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st) {
+cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist) {
     co3_prof_begin(pl, CO3_K_FIT, st);
     if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1 || mode == 5);
     const double* ext = (pl->use_ext_mom && mode != 4) ? pl->ext_mom : nullptr;
     if (mode != 4) pl->use_ext_mom = false;                // imported moments serve one fit
     fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out,
-                                                  (pl->use_fit_ovr && mode != 4) ? pl->fit_ovr : nullptr);
+                                                  (pl->use_fit_ovr && mode != 4) ? pl->fit_ovr : nullptr, clear_hist ? 1 : 0);
     co3_prof_end(pl, CO3_K_FIT, st, pl->dev.red_k > 0 ? 2 : 1);
     return cudaGetLastError();
 }

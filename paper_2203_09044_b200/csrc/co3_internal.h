@@ -193,11 +193,11 @@ const int16_t* co3_host_bias_opt_table(int E, int M);   // [NIBETA][8], cached p
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u_base, int u_count, cudaStream_t st);
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, int u_base, int u_count, bool first,
-                               cudaStream_t st);
+                               cudaStream_t st, bool cleared = false);
 cudaError_t co3_launch_convert_pack(co3_plan* pl, const float* g, float* m, uint16_t* sub_bits, cudaStream_t st);
 cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint16_t* sub_bits, uint32_t* chunk_off,
                                    unsigned long long* user_bits, cudaStream_t st);
-cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st);
+cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist = false);
 cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st);
 // empirical-histogram code: S codes from this iteration's histogram (lengths also to code_lens, device
 // [S][2^B]), or the tables of the codes whose lengths are given
