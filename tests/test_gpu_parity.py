@@ -254,6 +254,40 @@ def test_ragged_segments_and_tiny_inputs(binding, oracle):
         run_case(binding, oracle, d, 2, 4, 3, off, grads)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_random_plans(binding, oracle, seed):
+    """Plans drawn at random: size, segment cuts (tiny, empty and chunk-straddling layers), user count,
+    format, bias mode and rule, memory weight, row padding, per-layer scales spread over ten binades,
+    a few exact zeros and large outliers.  Three iterations each, everything compared."""
+    rng = np.random.default_rng(9000 + seed)
+    d = int(rng.choice([rng.integers(1, 300), rng.integers(300, 9000), rng.integers(9000, 70_000)]))
+    U = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 12, 16, 17, 33]))
+    E, M = FORMATS[int(rng.integers(0, 3))]
+    mode = int(rng.choice([0, 1, 1, 2, 3]))
+    rule = int(rng.integers(0, 2))
+    gamma = float(rng.choice([0.0, 0.5, 0.9, 1.0]))
+    n_cut = int(rng.integers(0, min(12, d)))
+    cuts = np.sort(rng.integers(0, d + 1, size=n_cut))               # repeated cuts = empty layers
+    if n_cut and rng.random() < 0.5:
+        cuts[rng.integers(0, n_cut)] = min(d, 4096 * int(rng.integers(0, d // 4096 + 1)))   # a cut on the chunk grid
+        cuts = np.sort(cuts)
+    off = [0] + [int(c) for c in cuts] + [d]
+    ld = (d + 3) // 4 * 4 + 4 * int(rng.integers(0, 3)) * int(rng.integers(0, 40))
+    gen = torch.Generator().manual_seed(9000 + seed)
+    scales = torch.tensor(np.exp2(rng.uniform(-16, -6, size=len(off) - 1)), dtype=torch.float32)
+    grads = []
+    for t in range(3):
+        g = torch.zeros((U, ld))
+        x = torch.randn((U, d), generator=gen)
+        for l in range(len(off) - 1):
+            x[:, off[l]:off[l + 1]] *= scales[l] * (1.0 + 0.3 * t)
+        x[torch.rand((U, d), generator=gen) < 0.01] = 0.0
+        x[torch.rand((U, d), generator=gen) < 0.002] *= 300.0
+        g[:, :d] = x
+        grads.append(g.cuda())
+    run_case(binding, oracle, d, U, E, M, off, grads, gamma=gamma, mode=mode, rule=rule)
+
+
 @pytest.mark.slow
 @pytest.mark.parametrize("U,d", [(1, 5_000_123), (2, 5_000_123), (4, 2_600_077), (8, 1_300_031), (16, 1_300_031), (6, 700_001)])
 def test_many_chunks_per_block_with_tiny_layers_between_large_ones(binding, oracle, U, d):
