@@ -57,6 +57,9 @@ extern "C" {
 #define CO3_FLAG_CORRUPT 2u
 #define CO3_FLAG_NONFINITE 4u
 #define CO3_FLAG_TIMEOUT 8u  /* a bounded wait between thread blocks ran out (should never happen) */
+#define CO3_FLAG_INEXACT 16u /* CO3_BIAS_CURRENT only: more than 4096 elements of one iteration lay some 2^20 times
+                                beyond the largest value of their layer's format AND that layer's bias changed: those
+                                elements were converted at the previous iteration's bias (see co3_encode) */
 
 /* CO3_BIAS_CURRENT is Algorithm 1 as printed: the bias b_t is chosen "at each time t" for the
  * distribution of g_t + gamma m_{t-1} itself (Sec. III (i), Eq. "exp bias"), which costs one extra
@@ -264,7 +267,7 @@ int co3_state_header(co3_plan* plan, int32_t import, co3_seg_header* next_header
 #define CO3_K_FIT 1          /* GenNorm fit, bias, header                                   */
 #define CO3_K_CONVERT 2      /* fused EF-add / convert / residual / histogram / moments      */
 #define CO3_K_CODE_ENC 3     /* CO3_CODE_EMPIRICAL only: code build from the histogram (model codes are built once, at plan creation) */
-#define CO3_K_ENC_LEN 4      /* (unused: the lengths are taken inside the packing kernel)    */
+#define CO3_K_RECONVERT 4    /* CO3_BIAS_CURRENT, t >= 1: layers whose bias differs from the guess, converted again */
 #define CO3_K_ENC_SCAN 5     /* chunk offsets (CO3_CODE_LAGGED only)                         */
 #define CO3_K_ENC_PACK 6     /* lengths + offsets + bit packing (CO3_CODE_LAGGED: concatenation) */
 #define CO3_K_CODE_DEC 7     /* CO3_CODE_EMPIRICAL only: decoder tables from the received code lengths */

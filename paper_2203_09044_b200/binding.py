@@ -17,6 +17,7 @@ FLAG_CAPACITY, FLAG_CORRUPT, FLAG_NONFINITE = 1, 2, 4
 BIAS_CURRENT, BIAS_LAGGED, CODE_LAGGED, CODE_EMPIRICAL = 0, 1, 2, 3
 RULE_POLY, RULE_OPT = 0, 1
 FLAG_TIMEOUT = 8
+FLAG_INEXACT = 16
 
 EXPORTS = [
     "co3_plan_create", "co3_plan_destroy", "co3_sizes", "co3_encode", "co3_decode_aggregate",
@@ -32,7 +33,7 @@ EXPORTS = [
 ELIMIT = -7
 STATIC_MAX_ELEMENTS = 1 << 29
 
-KERNEL_NAMES = ["stats", "fit", "convert", "code_enc", "enc_len", "enc_scan", "enc_pack", "code_dec",
+KERNEL_NAMES = ["stats", "fit", "convert", "code_enc", "reconvert", "enc_scan", "enc_pack", "code_dec",
                 "decode"]
 
 

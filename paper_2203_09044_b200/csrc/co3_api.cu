@@ -260,6 +260,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
     if (!pl) return CO3_ENOMEM;
     memset(pl, 0, sizeof(*pl));
     pl->cfg = *cfg;
+    { const char* e = getenv("CO3_TWO_PASS"); pl->two_pass_current = e && e[0] == '1'; }
     pl->h_seg_off = (int64_t*)malloc(sizeof(int64_t) * (size_t)(S + 1));
     if (!pl->h_seg_off) { delete pl; return CO3_ENOMEM; }
     if (cfg->seg_offsets) memcpy(pl->h_seg_off, cfg->seg_offsets, sizeof(int64_t) * (size_t)(S + 1));
@@ -367,6 +368,10 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             }
         }
         a |= dev_alloc(pl, &dv.bias_cur, (size_t)S);
+        a |= dev_alloc(pl, &dv.spec, 4);
+        a |= dev_alloc(pl, &dv.redo_seg, (size_t)S);
+        a |= dev_alloc(pl, &dv.redo_old, (size_t)S);
+        a |= dev_alloc(pl, &dv.side, (size_t)CO3_SIDE_CAP);
         a |= dev_alloc(pl, &pl->ext_mom, (size_t)S * 3);
         a |= dev_alloc(pl, &pl->fit_ovr, (size_t)S * 2);
         dv.spin_limit = 1 << 20;
@@ -409,6 +414,7 @@ extern "C" int co3_plan_create(co3_plan** out, const co3_config* cfg) {
             if (e == cudaSuccess) e = cudaMemset(dv.flags, 0, sizeof(uint32_t));
             if (e == cudaSuccess) e = cudaMemset(dv.nonfinite_total, 0, sizeof(unsigned long long));
             if (e == cudaSuccess) e = cudaMemset(dv.bias_cur, 0, sizeof(int32_t) * (size_t)S);
+            if (e == cudaSuccess) e = cudaMemset(dv.spec, 0, sizeof(int32_t) * 4);
             if (e == cudaSuccess) e = cudaMemset(dv.fit, 0, sizeof(double) * (size_t)S * 5);
             if (e == cudaSuccess) e = cudaMemset(dv.hist, 0, sizeof(unsigned long long) * ((size_t)dv.hist_copies * S * CO3_MAXSYM + 1));
             dv.ticket = reinterpret_cast<unsigned int*>(dv.hist + (size_t)dv.hist_copies * S * CO3_MAXSYM);
@@ -479,6 +485,19 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
     // Bias from the current moments: the fit after the statistics pass also gives the header (the convert
     // pass would hand the next fit the same sums), so there is one fit per iteration in both modes.
     const bool current = pl->cfg.bias_mode == CO3_BIAS_CURRENT;
+    if (current && pl->iteration > 0 && !pl->two_pass_current) {
+        // The bias of this iteration comes from this iteration's own moments, and those ride along with
+        // the convert pass: convert under the previous iteration's bias, fit, and convert again only
+        // the layers whose bias came out different (co3_launch_reconvert) -- the results are those of
+        // the statistics-pass-first order, bit for bit, at the cost of the lagged bias.
+        CO3_TRY(co3_launch_convert(pl, grad, residual, 0, pl->dev.U, true, st, false, true));
+        if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));
+        CO3_TRY(co3_launch_fit(pl, 6, hdr, st));
+        CO3_TRY(co3_launch_reconvert(pl, residual, st));
+        CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
+        pl->iteration++;
+        return CO3_OK;
+    }
     const bool with_stats = pl->iteration == 0 || current;
     if (with_stats) {
         CO3_TRY(co3_launch_stats(pl, grad, residual, 0, pl->dev.U, st));

@@ -41,6 +41,7 @@ struct QParams {                 // per segment
     float top;                   // K_max * 2^lambda: largest grid value (grid value = K * 2^lambda)
     uint32_t low_bits;           // bits of 2^(lambda + M): below it the quantum stays 2^lambda
     uint32_t e0;                 // exponent field of 1.5 * 2^(lambda + 23): lambda + 150
+    uint32_t far_bits;           // conversion under a guessed bias: bits of 2^(23 - M) * top (capped at those of Inf)
 };
 
 __device__ __forceinline__ float pow2f(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
@@ -75,20 +76,48 @@ __device__ __forceinline__ void quantize(float a, const QParams& q, uint32_t& sy
     m_new = __fsub_rn(a, __uint_as_float(__float_as_uint(r) | sb));
 }
 
+// a from its grid value and its new memory (exact for every element that is not on the side list; qv = 0
+// leaves a itself, sign of zero included).
+__device__ __forceinline__ float rebuild_a(float qv, float m_new) { return qv == 0.0f ? m_new : __fadd_rn(qv, m_new); }
+
+// Conversion under a guessed bias: an element that the re-conversion pass could not rebuild bit for bit
+// from its symbol and its new memory is kept on the side.  Only an element far beyond the largest grid
+// value `top` can be one: below top, q is a rounding of a at a quantum of at least ulp(a), so a - q is a
+// multiple of ulp(a) no larger than a, hence exact; and a - top is exact while |a| < 2^24 * (lowest
+// set bit of top), which 2^(23 - M) * top stays below.  Everything at or above that bound goes on the list.
+__device__ __noinline__ void side_push(int32_t* spec, Co3Side* side, uint32_t item, uint32_t pos, uint32_t a_bits) {
+    const int k = atomicAdd(spec + 2, 1);
+    if (k < CO3_SIDE_CAP) {
+        Co3Side e;
+        e.item = item; e.pos = pos; e.a_bits = a_bits; e.pad_ = 0;
+        side[k] = e;
+    } else {
+        spec[3] = 1;
+    }
+}
+
 // a = g + gamma m for the four elements of a vector; moments of the finite ones; NaN/Inf are
 // counted and replaced by 0 (so they are coded as +0 and their memory is reset to 0).
+// far_bits: 0x7F800000, or (FAR) the bound above which a finite element goes on the side list as well.
+template <bool FAR = false>
 __device__ __forceinline__ void ef_add4(const float4& gv, const float4& mv, float gamma, float a[4],
-                                        double& s1, double& s2, uint32_t& nf) {
+                                        double& s1, double& s2, uint32_t& nf, uint32_t far_bits = 0x7F800000u,
+                                        int32_t* spec = nullptr, Co3Side* side = nullptr, uint32_t item = 0, uint32_t pos0 = 0,
+                                        uint32_t in_mask = 15u) {
     a[0] = __fadd_rn(gv.x, __fmul_rn(gamma, mv.x));
     a[1] = __fadd_rn(gv.y, __fmul_rn(gamma, mv.y));
     a[2] = __fadd_rn(gv.z, __fmul_rn(gamma, mv.z));
     a[3] = __fadd_rn(gv.w, __fmul_rn(gamma, mv.w));
     const uint32_t big = max(max(__float_as_uint(a[0]) & 0x7FFFFFFFu, __float_as_uint(a[1]) & 0x7FFFFFFFu),
                              max(__float_as_uint(a[2]) & 0x7FFFFFFFu, __float_as_uint(a[3]) & 0x7FFFFFFFu));
-    if (big >= 0x7F800000u) {                 // rare: some element is NaN or Inf
+    if (big >= (FAR ? far_bits : 0x7F800000u)) {   // rare: some element is NaN or Inf (or far out)
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if ((__float_as_uint(a[e]) & 0x7FFFFFFFu) >= 0x7F800000u) { a[e] = 0.0f; ++nf; }
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t ab = __float_as_uint(a[e]) & 0x7FFFFFFFu;
+            if (ab >= 0x7F800000u) { a[e] = 0.0f; ++nf; }
+            else if (FAR && ab >= far_bits && ((in_mask >> e) & 1u))
+                side_push(spec, side, item, pos0 + e, __float_as_uint(a[e]));
+        }
     }
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -127,13 +156,15 @@ __device__ __forceinline__ void or_piece(uint32_t* img, uint32_t pos, unsigned l
     if (w2) atomicOr(&img[wi + 2], w2);
 }
 
-// MODE 1: convert, symbols to memory.  MODE 2: convert and pack.  (The statistics pass has a kernel of
-// its own, below.)
+// MODE 1: convert, symbols to memory.  MODE 2: convert and pack.  MODE 3: as 1 under a GUESSED bias (that
+// of the previous iteration, while the bias of this one is still to come out of this very pass's moments):
+// the elements that could not be rebuilt from what is stored are kept, see reconvert_kernel.  (The
+// statistics pass has a kernel of its own, below.)
 template <int M, int MODE>
 __global__ void __launch_bounds__(CO3_THREADS, 4)
 ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t* __restrict__ sub_bits) {
-    static_assert(MODE == 1 || MODE == 2, "the statistics pass is stats_kernel");
-    constexpr bool PACK = MODE == 2;
+    static_assert(MODE == 1 || MODE == 2 || MODE == 3, "the statistics pass is stats_kernel");
+    constexpr bool PACK = MODE == 2, GUESS = MODE == 3;
     extern __shared__ __align__(16) float4 s_ring[];            // [STAGES][2][CO3_THREADS] (+ PackSmem)
     __shared__ uint32_t s_hist[2][CO3_THREADS / 32][CO3_MAXSYM];   // [item parity][warp][symbol]
     __shared__ double s_red[2][2][CO3_THREADS / 32];
@@ -217,7 +248,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
     int cur_seg = -1, par = 0, hpar = 0;
     unsigned long long* hist_copy = p.hist + (size_t)(blockIdx.x % (unsigned)p.hist_copies) * p.S * CO3_MAXSYM;
     QParams q;
-    q.top = 0.0f; q.low_bits = 0; q.e0 = 0;
+    q.top = 0.0f; q.low_bits = 0; q.e0 = 0; q.far_bits = 0x7F800000u;
 
     while (true) {
         // thread 0 claims the item after next now, fetches its chunk descriptor half-way through the
@@ -231,6 +262,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
             q.top = __fmul_rn((float)p.Kmax, pow2f(lambda));
             q.low_bits = __float_as_uint(pow2f(lambda + M));
             q.e0 = (uint32_t)(lambda + 150);
+            q.far_bits = min(__float_as_uint(q.top) + ((23u - M) << 23), 0x7F800000u);   // top < 2^100: no overflow into the sign
         }
         uint32_t enc_next = 0;                        // PACK: my entry of the next item's code table
         if (PACK && has_nxt) enc_next = enc_entry(nxt.seg);
@@ -264,7 +296,8 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
                 float a[4], mo[4];
                 uint32_t so[4], en[4] = {0u, 0u, 0u, 0u};
                 if (full) {
-                    ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
+                    if (GUESS) ef_add4<true>(gv, mv, p.gamma, a, s1, s2, nf, q.far_bits, p.spec, p.side, item, (uint32_t)e0, 15u);
+                    else ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         quantize<M>(a[e], q, so[e], mo[e]);
@@ -282,7 +315,9 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
                     if (!in1) { gv.y = 0.0f; mv.y = 0.0f; }
                     if (!in2) { gv.z = 0.0f; mv.z = 0.0f; }
                     if (!in3) { gv.w = 0.0f; mv.w = 0.0f; }
-                    ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
+                    if (GUESS) ef_add4<true>(gv, mv, p.gamma, a, s1, s2, nf, q.far_bits, p.spec, p.side, item, (uint32_t)e0,
+                                             (uint32_t)in0 | ((uint32_t)in1 << 1) | ((uint32_t)in2 << 2) | ((uint32_t)in3 << 3));
+                    else ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if (in[e]) {
@@ -468,6 +503,127 @@ stats_kernel(Co3Dev p, const float* __restrict__ g, const float* __restrict__ m)
     }
 }
 
+// Bias from the current moments WITHOUT a statistics pass in every iteration.  The convert pass runs
+// under a guess (the previous iteration's bias), the fit that follows it finds the bias of this
+// iteration from the pass's own moments -- the same sums, in the same order, that a statistics pass
+// would have handed it -- and lists the layers where the two differ.  Those layers (usually none, and
+// if any, small ones whose fit is noisy) are converted again here: a = g + gamma m is rebuilt from
+// what the first conversion stored, a = q + m' (exact: the residual identity of Algorithm 1 line 10
+// read backwards; the few elements so far out that it does not hold were kept on a side list by the
+// convert pass), and quantised at the right bias: symbols, memory and histogram are then bit for bit
+// what the statistics-pass-first order of Algorithm 1 line 8 gives.
+// Grid: a few blocks per SM; a block that finds the list empty returns at once.  The last block to
+// finish applies the side list and clears the counters for the next iteration.
+template <int M>
+__global__ void __launch_bounds__(CO3_THREADS)
+reconvert_kernel(Co3Dev p, float* __restrict__ m) {
+    __shared__ uint32_t s_hist[2][CO3_MAXSYM];        // symbols taken out of the layer's histogram, symbols put in
+    __shared__ int s_last;
+    const int tid = threadIdx.x;
+    const int n = p.spec[0];
+    if (n == 0) {                                     // every guess was right
+        if (blockIdx.x == 0 && tid == 0) { p.spec[2] = 0; p.spec[3] = 0; }
+        return;
+    }
+    constexpr int VSTRIDE = 4 * CO3_THREADS;
+    auto params_of = [&](int lam) {
+        QParams q;
+        q.top = __fmul_rn((float)p.Kmax, pow2f(lam));
+        q.low_bits = __float_as_uint(pow2f(lam + M));
+        q.e0 = (uint32_t)(lam + 150);
+        q.far_bits = 0x7F800000u;
+        return q;
+    };
+    for (int k = 0; k < n; ++k) {
+        const int seg = p.redo_seg[k];
+        const int c0 = p.seg_chunk0[seg], nck = p.seg_chunk0[seg + 1] - c0;
+        const int64_t n_it = (int64_t)nck * p.U;
+        if ((int64_t)blockIdx.x >= n_it) continue;    // (uniform in the block)
+        const QParams q = params_of(p.bias_cur[seg] + p.cF);
+        const float quantum_old = pow2f(p.redo_old[k] + p.cF);
+        for (int i = tid; i < 2 * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
+        __syncthreads();
+        for (int64_t it = blockIdx.x; it < n_it; it += gridDim.x) {
+            const int u = (int)(it / nck);
+            const Co3Chunk cd = p.chunks[c0 + (int)(it - (int64_t)u * nck)];
+            const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
+            const int lo = (int)(cd.start - tb), hi = lo + cd.len;
+            float* mp = m + (size_t)u * p.ld + tb + 4 * tid;
+            uint8_t* sp = p.sym + (size_t)u * p.sld + tb + 4 * tid;
+#pragma unroll
+            for (int r = 0; r < STEPS; ++r) {
+                const int e0 = 4 * tid + VSTRIDE * r;
+                if (e0 >= hi || e0 + 4 <= lo) continue;
+                if (e0 >= lo && e0 + 4 <= hi) {
+                    const uint32_t sw = *reinterpret_cast<const uint32_t*>(sp + VSTRIDE * r);
+                    const float4 mv = *reinterpret_cast<const float4*>(mp + VSTRIDE * r);
+                    const float mold[4] = {mv.x, mv.y, mv.z, mv.w};
+                    uint32_t so[4];
+                    float mo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t sy = (sw >> (8 * e)) & 0xFFu;
+                        const float qv = __fmul_rn((float)co3_ksigned_internal((int)sy, M), quantum_old);   // exact
+                        quantize<M>(rebuild_a(qv, mold[e]), q, so[e], mo[e]);
+                        atomicAdd(&s_hist[0][sy], 1u);
+                        atomicAdd(&s_hist[1][so[e]], 1u);
+                    }
+                    *reinterpret_cast<float4*>(mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
+                    *reinterpret_cast<uint32_t*>(sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
+                } else {                              // a vector on the chunk's edge: element by element
+                    for (int e = 0; e < 4; ++e) {
+                        if (e0 + e < lo || e0 + e >= hi) continue;
+                        const uint32_t sy = sp[VSTRIDE * r + e];
+                        const float qv = __fmul_rn((float)co3_ksigned_internal((int)sy, M), quantum_old);
+                        uint32_t so;
+                        float mo;
+                        quantize<M>(rebuild_a(qv, mp[VSTRIDE * r + e]), q, so, mo);
+                        atomicAdd(&s_hist[0][sy], 1u);
+                        atomicAdd(&s_hist[1][so], 1u);
+                        mp[VSTRIDE * r + e] = mo;
+                        sp[VSTRIDE * r + e] = (uint8_t)so;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        for (int i = tid; i < CO3_MAXSYM; i += CO3_THREADS)   // (into copy 0: the copies are summed when the histogram is read)
+            if (s_hist[0][i] != s_hist[1][i])
+                atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + i], (unsigned long long)s_hist[1][i] - (unsigned long long)s_hist[0][i]);
+        __syncthreads();
+    }
+    // the last block to get here: side list, then the counters
+    __threadfence();
+    if (tid == 0) s_last = atomicAdd(p.spec + 1, 1) == (int)gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const int n_side = min(p.spec[2], CO3_SIDE_CAP);
+    for (int j = tid; j < n_side; j += CO3_THREADS) {
+        const Co3Side e = p.side[j];
+        const uint32_t user = e.item / (uint32_t)p.n_chunks;
+        const Co3Chunk cd = p.chunks[e.item - user * (uint32_t)p.n_chunks];
+        const int64_t i = (cd.start & ~(int64_t)(CO3_TILE - 1)) + e.pos;      // element index in the user's row
+        const int seg = cd.seg;
+        bool listed = false;
+        for (int k = 0; k < n; ++k) listed |= p.redo_seg[k] == seg;
+        if (!listed) continue;                        // its layer kept the guess: what is stored is right
+        const QParams q = params_of(p.bias_cur[seg] + p.cF);
+        uint32_t so;
+        float mo;
+        quantize<M>(__uint_as_float(e.a_bits), q, so, mo);
+        uint8_t* sp = p.sym + (size_t)user * p.sld + i;
+        atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + *sp], ~0ull);      // minus one: the symbol that the rebuilt value gave
+        atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + so], 1ull);
+        *sp = (uint8_t)so;
+        m[(size_t)user * p.ld + i] = mo;
+    }
+    if (tid == 0) {
+        if (p.spec[3]) atomicOr(p.flags, CO3_FLAG_INEXACT);   // more far-out elements than the list holds, and a wrong guess
+        p.spec[0] = 0; p.spec[1] = 0; p.spec[2] = 0; p.spec[3] = 0;
+    }
+}
+
 // Inspection: copy the stored symbols to a caller buffer [U][d] in the public form.
 __global__ void symbol_export_kernel(Co3Dev p, uint8_t* __restrict__ out) {
     const int64_t n = (int64_t)p.U * p.d;
@@ -525,21 +681,40 @@ cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u
 // first: this launch starts the iteration's histogram (later tiles of the same iteration add to it)
 // cleared: the fit kernel launched just before has zeroed the histogram and the ticket
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, int u_base, int u_count, bool first,
-                               cudaStream_t st, bool cleared) {
+                               cudaStream_t st, bool cleared, bool check_guess) {
     // one memset clears the histogram and the item ticket that follows it in the same allocation
     cudaError_t e = cudaSuccess;
     if (cleared) {}
     else if (first) e = cudaMemsetAsync(pl->dev.hist, 0, sizeof(unsigned long long) * ((size_t)pl->dev.hist_copies * pl->dev.S * CO3_MAXSYM + 1), st);
     else e = cudaMemsetAsync(pl->dev.ticket, 0, sizeof(unsigned int), st);
     if (e != cudaSuccess) return e;
-    ef_fn fn = pick_kernel<1>(pl->dev.M);
-    if (!pl->grid_convert) pl->grid_convert = ef_grid(pl, fn, RING_BYTES);
+    ef_fn fn = check_guess ? pick_kernel<3>(pl->dev.M) : pick_kernel<1>(pl->dev.M);
+    int& grid = check_guess ? pl->grid_convert_spec : pl->grid_convert;
+    if (!grid) grid = ef_grid(pl, fn, RING_BYTES);
     Co3Dev p = pl->dev;
     p.u_base = u_base; p.u_count = u_count;
     const int64_t items = p.n_chunks * (int64_t)u_count;
     co3_prof_begin(pl, CO3_K_CONVERT, st);
-    fn<<<(int)(items < pl->grid_convert ? items : pl->grid_convert), CO3_THREADS, RING_BYTES, st>>>(p, g, m, nullptr);
+    fn<<<(int)(items < grid ? items : grid), CO3_THREADS, RING_BYTES, st>>>(p, g, m, nullptr);
     co3_prof_end(pl, CO3_K_CONVERT, st, 1);
+    return cudaGetLastError();
+}
+
+typedef void (*reconv_fn)(Co3Dev, float*);
+cudaError_t co3_launch_reconvert(co3_plan* pl, float* m, cudaStream_t st) {
+    reconv_fn fn;
+    switch (pl->dev.M) {
+        case 1: fn = reconvert_kernel<1>; break;
+        case 2: fn = reconvert_kernel<2>; break;
+        case 3: fn = reconvert_kernel<3>; break;
+        case 4: fn = reconvert_kernel<4>; break;
+        case 5: fn = reconvert_kernel<5>; break;
+        default: fn = reconvert_kernel<6>; break;
+    }
+    const int64_t items = pl->dev.n_chunks * (int64_t)pl->dev.U, grid = (int64_t)pl->num_sms * 4;
+    co3_prof_begin(pl, CO3_K_RECONVERT, st);
+    fn<<<(int)(items < grid ? items : grid), CO3_THREADS, 0, st>>>(pl->dev, m);
+    co3_prof_end(pl, CO3_K_RECONVERT, st, 1);
     return cudaGetLastError();
 }
 

@@ -80,6 +80,11 @@ __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int c
 //         the coming convert pass AND the header of this iteration (the convert pass sums the same
 //         a = g + gamma m item by item in the same order, so a second fit after it would reproduce these
 //         numbers bit for bit); keeps the fit and prepares the encoder like mode 1.
+// mode 6: after a convert pass that ran under a GUESSED bias (bias_cur, the previous iteration's) although the
+//         bias is to come from this iteration's own moments: bias and header from these moments as in mode 5;
+//         a layer whose bias differs from the guess is put on the list of layers to convert again,
+//         and bias_cur takes the bias found (the re-conversion's target and
+//         the next iteration's guess).
 // ext_mom (may be null): (N, S1, S2) per segment that replace the plan's own sums in the fit (the sums
 //         of a layer that is spread over several plans); the non-finite count stays the plan's own.
 // fit_ovr (may be null): (beta, alpha) per segment that replace the solve (test hook: a harness feeds
@@ -97,7 +102,7 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     __shared__ int s_state, s_coarse, s_fine;
 
     const int seg = blockIdx.x, tid = threadIdx.x;
-    if ((mode == 1 || mode == 5) && p.red_k == 0) {
+    if ((mode == 1 || mode == 5 || mode == 6) && p.red_k == 0) {
         // side job: the single-pass encode that follows this launch wants its tickets, published
         // counts and group totals at zero
         unsigned long long* z = p.enc_grp;
@@ -252,6 +257,11 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     co3_seg_header h;
     h.bias = (int8_t)b_used; h.ibeta = (int8_t)(int)x; h.ir = (int16_t)(int)y;
     hdr[seg] = h;
+    if (mode == 6 && b_rule != p.bias_cur[seg]) {
+        const int k = atomicAdd(p.spec, 1);
+        p.redo_seg[k] = seg;
+        p.redo_old[k] = p.bias_cur[seg];
+    }
     p.bias_cur[seg] = b_rule;
     if (mode == 2) return;
     double* f = p.fit + 5 * (size_t)seg;
@@ -447,7 +457,7 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 
 cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist) {
     co3_prof_begin(pl, CO3_K_FIT, st);
-    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1 || mode == 5);
+    if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1 || mode == 5 || mode == 6);
     const double* ext = (pl->use_ext_mom && mode != 4) ? pl->ext_mom : nullptr;
     if (mode != 4) pl->use_ext_mom = false;                // imported moments serve one fit
     fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out,

@@ -71,6 +71,16 @@ struct Co3CodeBook {
     int32_t* ksign;      // [256]           signed integer magnitude of each symbol
 };
 
+// Bias from the current moments without a statistics pass (see co3_encode): an element whose
+// a = g + gamma m cannot be rebuilt bit for bit from its symbol and its new memory is kept here.
+struct Co3Side {
+    uint32_t item;                // user * n_chunks + chunk
+    uint32_t pos;                 // element within the chunk's tile
+    uint32_t a_bits;
+    uint32_t pad_;
+};
+constexpr int CO3_SIDE_CAP = 4096;
+
 // Everything the kernels need, passed by value.
 struct Co3Dev {
     int E, M, nm, nsym, J, cF, b_lo, b_hi;
@@ -97,6 +107,10 @@ struct Co3Dev {
     double* red_s1;               //      fit_reduce_kernel ([S][red_k] each) -- plans with very long segments
     double* red_s2;
     unsigned long long* red_nf;
+    int32_t* spec;                // [4] layers to convert again | blocks done | side entries | side list overflowed
+    int32_t* redo_seg;            // [S] the layers whose bias turned out different from the guess ...
+    int32_t* redo_old;            // [S] ... and the guess they were converted with
+    Co3Side* side;                // [CO3_SIDE_CAP]
     int32_t* bias_cur;            // [S] bias used by the next convert pass
     int bias_rule;                // CO3_RULE_POLY or CO3_RULE_OPT
     const int16_t* bias_opt_tab;  // [NIBETA][8] best ir per (shape index, round(8 log2 alpha) mod 8)
@@ -134,6 +148,8 @@ struct co3_plan {
     const uint8_t* emp_lens_in;     // ... and during co3_decode_aggregate_empirical
     size_t enc_sync_bytes;          // size of the enc_grp / enc_st / enc_ticket allocation
     int grid_convert;               // launch grid of the convert pass (fixed per plan)
+    int grid_convert_spec;          // ... of its variant that checks the guess (current-moments bias, t >= 1)
+    bool two_pass_current;          // current-moments bias with a statistics pass in every iteration (CO3_TWO_PASS=1)
     cudaStream_t last_stream;
     // co3_iteration_host: copy streams and the events that order them against the caller's stream
     cudaStream_t s_in, s_out;
@@ -193,7 +209,8 @@ const int16_t* co3_host_bias_opt_table(int E, int M);   // [NIBETA][8], cached p
 // kernel launchers (each returns a cudaError_t from the launch)
 cudaError_t co3_launch_stats(co3_plan* pl, const float* g, const float* m, int u_base, int u_count, cudaStream_t st);
 cudaError_t co3_launch_convert(co3_plan* pl, const float* g, float* m, int u_base, int u_count, bool first,
-                               cudaStream_t st, bool cleared = false);
+                               cudaStream_t st, bool cleared = false, bool check_guess = false);
+cudaError_t co3_launch_reconvert(co3_plan* pl, float* m, cudaStream_t st);
 cudaError_t co3_launch_convert_pack(co3_plan* pl, const float* g, float* m, uint16_t* sub_bits, cudaStream_t st);
 cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint16_t* sub_bits, uint32_t* chunk_off,
                                    unsigned long long* user_bits, cudaStream_t st);
@@ -238,6 +255,13 @@ __host__ __device__ inline int co3_row_of(const co3_seg_header h, bool* bad) {
 // signs) are then neighbours, so table look-ups of a warp spread over distinct shared-memory banks.
 __host__ __device__ inline int co3_sym_internal(int sym, int nm) { return ((sym & ((1 << nm) - 1)) << 1) | (sym >> nm); }
 __host__ __device__ inline int co3_sym_public(int isym, int nm) { return ((isym & 1) << nm) | (isym >> 1); }
+
+// The same from the internal symbol form (magnitude code << 1 | sign).
+__host__ __device__ inline int32_t co3_ksigned_internal(int isym, int M) {
+    const int j = isym >> 1, e = j >> M, f = j & ((1 << M) - 1);
+    const int32_t k = (e == 0) ? f : (((1 << M) + f) << (e - 1));
+    return (isym & 1) ? -k : k;
+}
 
 // Signed integer magnitude of a symbol byte: K(j) = f (e = 0) or (2^M + f) << (e - 1).
 __host__ __device__ inline int32_t co3_ksigned(int sym, int M, int nm) {

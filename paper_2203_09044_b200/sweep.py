@@ -203,7 +203,7 @@ def measure(wl, iters, warm, pool, rule=0, mode=None):
                name=wl.name, d=d, U=U, S=plan.S, fmt="E%dM%d" % (wl.exp_bits, wl.mant_bits), beta=wl.beta,
                ms=ms, first_ms=first_ms, gbs=4.0 * U * d / (ms * 1e-3) / 1e9,
                convert_ms=prof.get("convert", 0.0),
-               encode_ms=prof.get("enc_len", 0.0) + prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0)
+               encode_ms=prof.get("enc_scan", 0.0) + prof.get("enc_pack", 0.0)
                + prof.get("code_enc", 0.0),
                fit_ms=prof.get("fit", 0.0), decode_ms=prof.get("decode", 0.0) + prof.get("code_dec", 0.0),
                code_bits=code_bits, container_bits=container_bits, flags=flags,
