@@ -492,7 +492,7 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
         // the statistics-pass-first order, bit for bit, at the cost of the lagged bias.
         CO3_TRY(co3_launch_convert(pl, grad, residual, 0, pl->dev.U, true, st, false, true));
         if (pl->record_conv) CO3_TRY(cudaEventRecord(pl->ev_conv, st));
-        CO3_TRY(co3_launch_fit(pl, 6, hdr, st));
+        CO3_TRY(co3_launch_fit(pl, 6, hdr, st, false, residual));
         CO3_TRY(co3_launch_reconvert(pl, residual, st));
         CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
         pl->iteration++;

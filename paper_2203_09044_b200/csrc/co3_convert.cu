@@ -31,20 +31,12 @@
 // bit count.  No block barrier is involved.  Where a sub-chunk lands in the user's payload depends
 // on all earlier ones, so a scan and a concatenation pass follow (co3_encode.cu).
 #include "co3_internal.h"
+#include "co3_quant.cuh"
 
 namespace {
 
 constexpr int STEPS = CO3_TILE / (4 * CO3_THREADS);   // vectors per thread per item (4)
 constexpr int STAGES = 4;                             // ring depth of the asynchronous copies
-
-struct QParams {                 // per segment
-    float top;                   // K_max * 2^lambda: largest grid value (grid value = K * 2^lambda)
-    uint32_t low_bits;           // bits of 2^(lambda + M): below it the quantum stays 2^lambda
-    uint32_t e0;                 // exponent field of 1.5 * 2^(lambda + 23): lambda + 150
-    uint32_t far_bits;           // conversion under a guessed bias: bits of 2^(23 - M) * top (capped at those of Inf)
-};
-
-__device__ __forceinline__ float pow2f(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_dst), "l"(gsrc) : "memory");
@@ -52,33 +44,6 @@ __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-
-// Q_fp on one finite element, branch-free.  |a| (clamped to the top grid value) is rounded to
-// nearest even at the quantum 2^qe of its binade -- or the subnormal quantum 2^lambda, whichever
-// is larger -- by adding 1.5 * 2^(qe+23): the sum t holds n = |a| / 2^qe rounded, as an integer, in
-// its low mantissa bits, and subtracting the constant again gives the rounded value r.  The
-// magnitude code is j = ((qe - lambda) << M) + n for every binade (n < 2^(M+1) below the second
-// binade, where it is the code itself; 2^M <= n <= 2^(M+1) above, where it carries the mantissa
-// and, on a carry, the next exponent).
-template <int M>
-__device__ __forceinline__ void quantize(float a, const QParams& q, uint32_t& sym, float& m_new) {
-    const uint32_t ab = __float_as_uint(a);
-    const float axc = fminf(fabsf(a), q.top);
-    // exponent field of max(|a|, 2^(lambda+M)), moved up by 23 - M binades, plus the 1.5
-    const uint32_t mb = (max(__float_as_uint(axc), q.low_bits) & 0x7F800000u) + (((23u - M) << 23) | 0x400000u);
-    const float magic = __uint_as_float(mb);
-    const float t = __fadd_rn(axc, magic);
-    const float r = __fsub_rn(t, magic);      // multiple of 2^qe, <= top
-    const uint32_t tb = __float_as_uint(t);
-    const uint32_t j = (((tb >> 23) - q.e0) << M) + (tb & 0x3FFFFFu);
-    const uint32_t sb = (r != 0.0f) ? (ab & 0x80000000u) : 0u;  // "-0" is never emitted
-    sym = (j << 1) | (sb >> 31);                                 // internal form: code << 1 | sign
-    m_new = __fsub_rn(a, __uint_as_float(__float_as_uint(r) | sb));
-}
-
-// a from its grid value and its new memory (exact for every element that is not on the side list; qv = 0
-// leaves a itself, sign of zero included).
-__device__ __forceinline__ float rebuild_a(float qv, float m_new) { return qv == 0.0f ? m_new : __fadd_rn(qv, m_new); }
 
 // Conversion under a guessed bias: an element that the re-conversion pass could not rebuild bit for bit
 // from its symbol and its new memory is kept on the side.  Only an element far beyond the largest grid
@@ -525,72 +490,11 @@ reconvert_kernel(Co3Dev p, float* __restrict__ m) {
         if (blockIdx.x == 0 && tid == 0) { p.spec[2] = 0; p.spec[3] = 0; }
         return;
     }
-    constexpr int VSTRIDE = 4 * CO3_THREADS;
-    auto params_of = [&](int lam) {
-        QParams q;
-        q.top = __fmul_rn((float)p.Kmax, pow2f(lam));
-        q.low_bits = __float_as_uint(pow2f(lam + M));
-        q.e0 = (uint32_t)(lam + 150);
-        q.far_bits = 0x7F800000u;
-        return q;
-    };
     for (int k = 0; k < n; ++k) {
         const int seg = p.redo_seg[k];
         const int c0 = p.seg_chunk0[seg], nck = p.seg_chunk0[seg + 1] - c0;
-        const int64_t n_it = (int64_t)nck * p.U;
-        if ((int64_t)blockIdx.x >= n_it) continue;    // (uniform in the block)
-        const QParams q = params_of(p.bias_cur[seg] + p.cF);
-        const float quantum_old = pow2f(p.redo_old[k] + p.cF);
-        for (int i = tid; i < 2 * CO3_MAXSYM; i += CO3_THREADS) (&s_hist[0][0])[i] = 0;
-        __syncthreads();
-        for (int64_t it = blockIdx.x; it < n_it; it += gridDim.x) {
-            const int u = (int)(it / nck);
-            const Co3Chunk cd = p.chunks[c0 + (int)(it - (int64_t)u * nck)];
-            const int64_t tb = cd.start & ~(int64_t)(CO3_TILE - 1);
-            const int lo = (int)(cd.start - tb), hi = lo + cd.len;
-            float* mp = m + (size_t)u * p.ld + tb + 4 * tid;
-            uint8_t* sp = p.sym + (size_t)u * p.sld + tb + 4 * tid;
-#pragma unroll
-            for (int r = 0; r < STEPS; ++r) {
-                const int e0 = 4 * tid + VSTRIDE * r;
-                if (e0 >= hi || e0 + 4 <= lo) continue;
-                if (e0 >= lo && e0 + 4 <= hi) {
-                    const uint32_t sw = *reinterpret_cast<const uint32_t*>(sp + VSTRIDE * r);
-                    const float4 mv = *reinterpret_cast<const float4*>(mp + VSTRIDE * r);
-                    const float mold[4] = {mv.x, mv.y, mv.z, mv.w};
-                    uint32_t so[4];
-                    float mo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint32_t sy = (sw >> (8 * e)) & 0xFFu;
-                        const float qv = __fmul_rn((float)co3_ksigned_internal((int)sy, M), quantum_old);   // exact
-                        quantize<M>(rebuild_a(qv, mold[e]), q, so[e], mo[e]);
-                        atomicAdd(&s_hist[0][sy], 1u);
-                        atomicAdd(&s_hist[1][so[e]], 1u);
-                    }
-                    *reinterpret_cast<float4*>(mp + VSTRIDE * r) = make_float4(mo[0], mo[1], mo[2], mo[3]);
-                    *reinterpret_cast<uint32_t*>(sp + VSTRIDE * r) = so[0] | (so[1] << 8) | (so[2] << 16) | (so[3] << 24);
-                } else {                              // a vector on the chunk's edge: element by element
-                    for (int e = 0; e < 4; ++e) {
-                        if (e0 + e < lo || e0 + e >= hi) continue;
-                        const uint32_t sy = sp[VSTRIDE * r + e];
-                        const float qv = __fmul_rn((float)co3_ksigned_internal((int)sy, M), quantum_old);
-                        uint32_t so;
-                        float mo;
-                        quantize<M>(rebuild_a(qv, mp[VSTRIDE * r + e]), q, so, mo);
-                        atomicAdd(&s_hist[0][sy], 1u);
-                        atomicAdd(&s_hist[1][so], 1u);
-                        mp[VSTRIDE * r + e] = mo;
-                        sp[VSTRIDE * r + e] = (uint8_t)so;
-                    }
-                }
-            }
-        }
-        __syncthreads();
-        for (int i = tid; i < CO3_MAXSYM; i += CO3_THREADS)   // (into copy 0: the copies are summed when the histogram is read)
-            if (s_hist[0][i] != s_hist[1][i])
-                atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + i], (unsigned long long)s_hist[1][i] - (unsigned long long)s_hist[0][i]);
-        __syncthreads();
+        if ((int64_t)blockIdx.x >= (int64_t)nck * p.U) continue;    // (uniform in the block)
+        redo_items<M>(p, m, seg, c0, nck, p.redo_old[k], p.bias_cur[seg], blockIdx.x, gridDim.x, tid, CO3_THREADS, s_hist);
     }
     // the last block to get here: side list, then the counters
     __threadfence();
@@ -608,7 +512,7 @@ reconvert_kernel(Co3Dev p, float* __restrict__ m) {
         bool listed = false;
         for (int k = 0; k < n; ++k) listed |= p.redo_seg[k] == seg;
         if (!listed) continue;                        // its layer kept the guess: what is stored is right
-        const QParams q = params_of(p.bias_cur[seg] + p.cF);
+        const QParams q = make_qparams<M>(p.Kmax, p.bias_cur[seg] + p.cF);
         uint32_t so;
         float mo;
         quantize<M>(__uint_as_float(e.a_bits), q, so, mo);

@@ -13,11 +13,13 @@
 // lgamma evaluation; the depth limit of the code is resolved by building every weight-floor
 // candidate in its own block.
 #include "co3_internal.h"
+#include "co3_quant.cuh"
 
 namespace {
 
 constexpr int FIT_THREADS = 512;   // reduction width
 constexpr int FIT_SEARCH = 128;    // = FIT_GRID / 64: one coarse table interval per searching thread
+constexpr long long FIT_REDO_MAX = 8192;   // user-elements of a layer that the fit's own block converts again (mode 6)
 
 __device__ __forceinline__ double poly_bias(double b) {
     const double b2 = b * b;
@@ -94,12 +96,15 @@ __global__ void __launch_bounds__(RED_THREADS) fit_reduce_kernel(Co3Dev p, int c
 __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co3_seg_header* hdr,
                                                           const double* __restrict__ ext_mom,
                                                           double* __restrict__ mom_out,
-                                                          const double* __restrict__ fit_ovr, int clear_hist) {
+                                                          const double* __restrict__ fit_ovr, int clear_hist,
+                                                          float* __restrict__ residual) {
     __shared__ double s_a[FIT_THREADS / 32], s_b[FIT_THREADS / 32];
     __shared__ unsigned long long s_n[FIT_THREADS / 32];
     __shared__ double s_lg[3];
     __shared__ double s_target, s_t;        // log rho; log2(beta)
     __shared__ int s_state, s_coarse, s_fine;
+    __shared__ int s_redo_old;              // mode 6: the guess this layer was converted with, if this block converts it again
+    __shared__ uint32_t s_rh[2][CO3_MAXSYM];
 
     const int seg = blockIdx.x, tid = threadIdx.x;
     if ((mode == 1 || mode == 5 || mode == 6) && p.red_k == 0) {
@@ -186,8 +191,9 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         }
         __syncthreads();
     }
-    if (tid != 0) return;
-
+    constexpr int NO_REDO = -(1 << 30);
+    if (tid == 0) s_redo_old = NO_REDO;
+    if (tid == 0) [&]() {                   // the solve, by one thread
     double t = s_t, beta, log_g;
     if (s_state == 0) {
         // inverse cubic (Lagrange) interpolation of log2(beta) as a function of log R through the
@@ -258,9 +264,13 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     h.bias = (int8_t)b_used; h.ibeta = (int8_t)(int)x; h.ir = (int16_t)(int)y;
     hdr[seg] = h;
     if (mode == 6 && b_rule != p.bias_cur[seg]) {
-        const int k = atomicAdd(p.spec, 1);
-        p.redo_seg[k] = seg;
-        p.redo_old[k] = p.bias_cur[seg];
+        // a small layer is converted again by this very block (below); a large one by the pass that follows
+        if ((long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * p.U <= FIT_REDO_MAX) s_redo_old = p.bias_cur[seg];
+        else {
+            const int k = atomicAdd(p.spec, 1);
+            p.redo_seg[k] = seg;
+            p.redo_old[k] = p.bias_cur[seg];
+        }
     }
     p.bias_cur[seg] = b_rule;
     if (mode == 2) return;
@@ -269,6 +279,21 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     if (nf) {
         atomicAdd(p.nonfinite_total, nf);
         atomicOr(p.flags, CO3_FLAG_NONFINITE);
+    }
+    }();
+    if (mode != 6) return;
+    __syncthreads();
+    if (s_redo_old == NO_REDO) return;
+    // mode 6, a small layer whose bias differs from the guess: converted again here (the layers that keep
+    // the convert pass busy for microseconds go on the list instead, for all SMs to share)
+    const int b_new = p.bias_cur[seg];      // (written by thread 0 before the barrier)
+    switch (p.M) {
+        case 1: redo_small<1>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
+        case 2: redo_small<2>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
+        case 3: redo_small<3>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
+        case 4: redo_small<4>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
+        case 5: redo_small<5>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
+        default: redo_small<6>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
     }
 }
 
@@ -455,13 +480,13 @@ __global__ void __launch_bounds__(CO3_MAXSYM) code_finalize_kernel(Co3Dev p, Co3
 
 }  // namespace
 
-cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist) {
+cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist, float* residual) {
     co3_prof_begin(pl, CO3_K_FIT, st);
     if (pl->dev.red_k > 0) fit_reduce_kernel<<<dim3(pl->dev.S, pl->dev.red_k), RED_THREADS, 0, st>>>(pl->dev, mode == 1 || mode == 5 || mode == 6);
     const double* ext = (pl->use_ext_mom && mode != 4) ? pl->ext_mom : nullptr;
     if (mode != 4) pl->use_ext_mom = false;                // imported moments serve one fit
     fit_kernel<<<pl->dev.S, FIT_THREADS, 0, st>>>(pl->dev, mode, hdr, ext, pl->mom_out,
-                                                  (pl->use_fit_ovr && mode != 4) ? pl->fit_ovr : nullptr, clear_hist ? 1 : 0);
+                                                  (pl->use_fit_ovr && mode != 4) ? pl->fit_ovr : nullptr, clear_hist ? 1 : 0, residual);
     co3_prof_end(pl, CO3_K_FIT, st, pl->dev.red_k > 0 ? 2 : 1);
     return cudaGetLastError();
 }

@@ -214,7 +214,8 @@ cudaError_t co3_launch_reconvert(co3_plan* pl, float* m, cudaStream_t st);
 cudaError_t co3_launch_convert_pack(co3_plan* pl, const float* g, float* m, uint16_t* sub_bits, cudaStream_t st);
 cudaError_t co3_launch_scan_gather(co3_plan* pl, uint32_t* bitstream, const uint16_t* sub_bits, uint32_t* chunk_off,
                                    unsigned long long* user_bits, cudaStream_t st);
-cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist = false);
+cudaError_t co3_launch_fit(co3_plan* pl, int mode, co3_seg_header* hdr, cudaStream_t st, bool clear_hist = false,
+                           float* residual = nullptr);   // residual: mode 6 only
 cudaError_t co3_build_codebook(co3_plan* pl, cudaStream_t st);
 // empirical-histogram code: S codes from this iteration's histogram (lengths also to code_lens, device
 // [S][2^B]), or the tables of the codes whose lengths are given
