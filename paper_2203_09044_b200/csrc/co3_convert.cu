@@ -507,20 +507,9 @@ reconvert_kernel(Co3Dev p, float* __restrict__ m) {
         const Co3Side e = p.side[j];
         const uint32_t user = e.item / (uint32_t)p.n_chunks;
         const Co3Chunk cd = p.chunks[e.item - user * (uint32_t)p.n_chunks];
-        const int64_t i = (cd.start & ~(int64_t)(CO3_TILE - 1)) + e.pos;      // element index in the user's row
-        const int seg = cd.seg;
         bool listed = false;
-        for (int k = 0; k < n; ++k) listed |= p.redo_seg[k] == seg;
-        if (!listed) continue;                        // its layer kept the guess: what is stored is right
-        const QParams q = make_qparams<M>(p.Kmax, p.bias_cur[seg] + p.cF);
-        uint32_t so;
-        float mo;
-        quantize<M>(__uint_as_float(e.a_bits), q, so, mo);
-        uint8_t* sp = p.sym + (size_t)user * p.sld + i;
-        atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + *sp], ~0ull);      // minus one: the symbol that the rebuilt value gave
-        atomicAdd(&p.hist[(size_t)seg * CO3_MAXSYM + so], 1ull);
-        *sp = (uint8_t)so;
-        m[(size_t)user * p.ld + i] = mo;
+        for (int k = 0; k < n; ++k) listed |= p.redo_seg[k] == cd.seg;
+        if (listed) redo_side_entry<M>(p, m, e, cd, user);   // (a layer that kept the guess: what is stored is right)
     }
     if (tid == 0) {
         if (p.spec[3]) atomicOr(p.flags, CO3_FLAG_INEXACT);   // more far-out elements than the list holds, and a wrong guess

@@ -288,12 +288,12 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     // the convert pass busy for microseconds go on the list instead, for all SMs to share)
     const int b_new = p.bias_cur[seg];      // (written by thread 0 before the barrier)
     switch (p.M) {
-        case 1: redo_small<1>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
-        case 2: redo_small<2>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
-        case 3: redo_small<3>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
-        case 4: redo_small<4>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
-        case 5: redo_small<5>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
-        default: redo_small<6>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); break;
+        case 1: redo_small<1>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); redo_side_of_layer<1>(p, residual, seg, tid, FIT_THREADS); break;
+        case 2: redo_small<2>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); redo_side_of_layer<2>(p, residual, seg, tid, FIT_THREADS); break;
+        case 3: redo_small<3>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); redo_side_of_layer<3>(p, residual, seg, tid, FIT_THREADS); break;
+        case 4: redo_small<4>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); redo_side_of_layer<4>(p, residual, seg, tid, FIT_THREADS); break;
+        case 5: redo_small<5>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); redo_side_of_layer<5>(p, residual, seg, tid, FIT_THREADS); break;
+        default: redo_small<6>(p, residual, seg, c0, nck, s_redo_old, b_new, tid, FIT_THREADS, s_rh); redo_side_of_layer<6>(p, residual, seg, tid, FIT_THREADS); break;
     }
 }
 

@@ -141,3 +141,33 @@ __device__ void redo_small(const Co3Dev& p, float* __restrict__ m, int seg, int 
     }
     redo_flush(p, seg, tid, nthreads, s_hist);
 }
+
+// An element of the side list whose layer has been converted again: the value the convert pass kept is
+// converted in place of the rebuilt one, and the histogram follows.
+template <int M>
+__device__ __forceinline__ void redo_side_entry(const Co3Dev& p, float* __restrict__ m, const Co3Side& e, const Co3Chunk& cd,
+                                                uint32_t user) {
+    const int64_t i = (cd.start & ~(int64_t)(CO3_TILE - 1)) + e.pos;       // element index in the user's row
+    const QParams q = make_qparams<M>(p.Kmax, p.bias_cur[cd.seg] + p.cF);
+    uint32_t so;
+    float mo;
+    quantize<M>(__uint_as_float(e.a_bits), q, so, mo);
+    uint8_t* sp = p.sym + (size_t)user * p.sld + i;
+    atomicAdd(&p.hist[(size_t)cd.seg * CO3_MAXSYM + *sp], ~0ull);          // minus one: the symbol that the rebuilt value gave
+    atomicAdd(&p.hist[(size_t)cd.seg * CO3_MAXSYM + so], 1ull);
+    *sp = (uint8_t)so;
+    m[(size_t)user * p.ld + i] = mo;
+}
+
+// The side-list entries of layer `seg`, after that layer has been converted again by this block.
+template <int M>
+__device__ void redo_side_of_layer(const Co3Dev& p, float* __restrict__ m, int seg, int tid, int nthreads) {
+    const int n_side = min(p.spec[2], CO3_SIDE_CAP);
+    for (int j = tid; j < n_side; j += nthreads) {
+        const Co3Side e = p.side[j];
+        const uint32_t user = e.item / (uint32_t)p.n_chunks;
+        const Co3Chunk cd = p.chunks[e.item - user * (uint32_t)p.n_chunks];
+        if (cd.seg == seg) redo_side_entry<M>(p, m, e, cd, user);
+    }
+    if (tid == 0 && p.spec[3]) atomicOr(p.flags, CO3_FLAG_INEXACT);        // the list did not hold them all
+}

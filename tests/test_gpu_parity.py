@@ -288,6 +288,118 @@ def test_random_plans(binding, oracle, seed):
     run_case(binding, oracle, d, U, E, M, off, grads, gamma=gamma, mode=mode, rule=rule)
 
 
+def _scaled_grads(U, d, ld, off, scales_per_iter, seed, far=None, neg_zero=False):
+    """Gaussian gradients whose scale changes from iteration to iteration (scales_per_iter[t][layer]);
+    far = (layer, count, value): that many elements of the layer set to +-value in every ODD iteration (so
+    that they arrive under a bias that was fitted without them)."""
+    gen = torch.Generator().manual_seed(seed)
+    grads = []
+    for t, sc in enumerate(scales_per_iter):
+        g = torch.zeros((U, ld))
+        x = torch.randn((U, d), generator=gen)
+        for l in range(len(off) - 1):
+            x[:, off[l]:off[l + 1]] *= sc[l]
+        if far is not None and t % 2 == 1:
+            l, count, value = far
+            idx = torch.randint(off[l], off[l + 1], (U, count), generator=gen)
+            sign = torch.where(torch.rand((U, count), generator=gen) < 0.5, -1.0, 1.0)
+            x.scatter_(1, idx, sign * value)
+        if neg_zero:
+            x[:, ::7] = -0.0
+        g[:, :d] = x
+        grads.append(g.cuda())
+    return grads
+
+
+@pytest.mark.parametrize("E,M", FORMATS)
+def test_current_bias_when_the_guess_is_wrong(binding, oracle, E, M):
+    """Bias from the current moments, t >= 1: the convert pass runs under the previous iteration's bias and
+    the layers whose bias comes out different are converted again from what was stored.  Here every
+    layer's scale jumps by factors of 4 to 64 between iterations, so every guess is wrong: large layers
+    (the re-conversion pass), small ones (the fit's own block), a layer of one element, an empty one,
+    chunk-straddling ones; exact zeros of both signs ride along."""
+    d, U = 70_000, 3
+    off = [0, 1, 65, 65, 5000, 9000, 30_000, 30_100, d]
+    ld = (d + 3) // 4 * 4 + 8
+    L = len(off) - 1
+    scales = [[1e-3 * 4.0 ** ((t * (l + 1)) % 4) for l in range(L)] for t in range(5)]
+    grads = _scaled_grads(U, d, ld, off, scales, seed=77, neg_zero=True)
+    for gamma in (0.0, 0.9):
+        plan, orc, out, res = run_case(binding, oracle, d, U, E, M, off, grads, gamma=gamma, mode=0)
+        biases = np.stack([r.hdr[:, 0] for r, _ in res])
+        assert (np.diff(biases, axis=0) != 0).sum() >= 2 * (L - 1), "the biases were meant to move"
+        assert plan.status()[0] == 0
+
+
+def test_current_bias_with_elements_far_beyond_the_format(binding, oracle):
+    """Elements some 2^20 times the largest grid value cannot be rebuilt from symbol and memory (their
+    residual is rounded); the convert pass keeps them on a side list and the re-conversion takes them
+    from there.  NaN and Inf in the same layers."""
+    d, U = 40_000, 2
+    off = [0, 100, 20_000, d]
+    ld = d
+    scales = [[1e-3, 1e-3, 1e-3 * 16.0 ** (t % 2)] for t in range(4)]
+    for layer in (0, 1):                                   # a small layer (the fit's block) and a large one (the pass)
+        grads = _scaled_grads(U, d, ld, off, scales, seed=78 + layer, far=(layer, 40, 3e9))
+        for g in grads:
+            g[0, off[layer] + 3] = float("nan")
+            g[1, off[layer] + 5] = float("-inf")
+        plan, orc, out, res = run_case(binding, oracle, d, U, 4, 3, off, grads, gamma=0.9, mode=0)
+        flags = plan.status()[0]
+        assert flags & binding.FLAG_NONFINITE and not (flags & binding.FLAG_INEXACT)
+
+
+def test_current_bias_side_list_overflow_is_reported(binding):
+    """More far-out elements in one iteration than the side list holds (in a layer whose bias they change):
+    CO3_FLAG_INEXACT.  With fewer of them than the list holds nothing is raised."""
+    b = binding
+    d, U = 60_000, 2
+    off = [0, 30_000, d]
+    for moving, count in ((False, 1500), (True, 6000)):
+        scales = [[1e-3, 1e-3] for t in range(3)]
+        grads = _scaled_grads(U, d, d, off, scales, seed=80, far=(1, count, 3e9))
+        plan = b.Plan(d, U, 4, 3, off, gamma=0.0, bias_mode=b.BIAS_CURRENT)
+        out = plan.alloc_outputs()
+        m = torch.zeros((U, plan.ld), dtype=torch.float32, device="cuda")
+        for g in grads:
+            plan.encode(g, m, out)
+        flags = plan.status()[0]
+        assert bool(flags & b.FLAG_INEXACT) == moving, (moving, flags)
+        plan.close()
+
+
+def test_current_bias_two_implementations_agree(binding, monkeypatch):
+    """CO3_TWO_PASS=1 keeps the statistics pass in every iteration (Algorithm 1 line 8 in its printed order);
+    the default runs it at t = 0 only and repairs wrong guesses.  Same bits."""
+    b = binding
+    from paper_2203_09044_b200 import inputs
+    wl = inputs.workload(1, d=400_000, n_users=4)
+    outs = []
+    for two_pass in ("0", "1"):
+        monkeypatch.setenv("CO3_TWO_PASS", two_pass)
+        plan = b.Plan(wl.d, wl.n_users, 4, 3, wl.seg_offsets, gamma=wl.gamma, bias_mode=b.BIAS_CURRENT, ld=wl.ld)
+        out = plan.alloc_outputs()
+        m = torch.zeros((wl.n_users, plan.ld), dtype=torch.float32, device="cuda")
+        rec = []
+        for t in range(5):
+            g = wl.gradient(t, device="cuda") * (1.0 if t % 2 == 0 else 5.0)
+            plan.encode(g, m, out)
+            n = out["chunk_off"][:, -1].cpu().numpy()
+            rec.append((out["hdr"].clone(), out["chunk_off"].clone(), m.clone(), plan.debug_symbols().clone(),
+                        [out["bitstream"][u, :int(n[u])].clone() for u in range(wl.n_users)], plan.debug_hist().copy(),
+                        plan.decode_aggregate(out).clone()))
+        assert plan.status()[0] == 0
+        outs.append(rec)
+        plan.close()
+    for t, (x, y) in enumerate(zip(*outs)):
+        assert torch.equal(x[0], y[0]) and torch.equal(x[1], y[1]), f"t={t} header / offsets"
+        assert torch.equal(x[2].view(torch.int32), y[2].view(torch.int32)), f"t={t} residual"
+        assert torch.equal(x[3], y[3]), f"t={t} symbols"
+        assert all(torch.equal(p, q) for p, q in zip(x[4], y[4])), f"t={t} payload"
+        assert np.array_equal(x[5], y[5]), f"t={t} histogram"
+        assert torch.equal(x[6].view(torch.int32), y[6].view(torch.int32)), f"t={t} average"
+
+
 @pytest.mark.slow
 @pytest.mark.parametrize("U,d", [(1, 5_000_123), (2, 5_000_123), (4, 2_600_077), (8, 1_300_031), (16, 1_300_031), (6, 700_001)])
 def test_many_chunks_per_block_with_tiny_layers_between_large_ones(binding, oracle, U, d):
