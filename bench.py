@@ -6,9 +6,11 @@ A step is one CO3 iteration of Algorithm 1 over one batch of synthetic gradients
 Huffman code build, bit packing) followed by co3_decode_aggregate (code rebuild from the header,
 decode of all users, average).  The workload is the 8-user ResNet-18-sized configuration
 (d = 11,173,962 per user, 62 layers, 8-bit format, gamma = 0.9).  `value` is measured with the bias of
-every iteration taken from that iteration's own moments, as Algorithm 1 prints it (one extra read pass);
-the same steps with the bias lagging one iteration behind (no extra pass) are timed beside it and
-reported as `lagged_bias`.
+every iteration taken from that iteration's own moments, as Algorithm 1 prints it; the library gets those
+results without a statistics pass in every iteration (it converts under the previous bias and converts
+again the layers whose bias changed).  The same steps with that pass in every iteration
+(`current_two_pass`, the same bits) and with the bias lagging one iteration behind (`lagged_bias`)
+are timed beside it.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -256,10 +258,19 @@ def run_ours(args):
     # ---- the other bias mode, timed the same way (K steps, eager) ------------------------------
     other = None if args.short else {"current": "lagged", "lagged": "current"}.get(args.mode)
     other_rec = None
-    if other is not None:
-        plan_o = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
-                              bias_mode={"lagged": binding.BIAS_LAGGED, "current": binding.BIAS_CURRENT}[other],
-                              ld=wl.ld)
+    two_pass_rec = None
+
+    def timed_other(other, two_pass):
+        """K steps of another bias mode (or of the current-moments bias in its two-pass form: a statistics pass
+        in every iteration, CO3_TWO_PASS=1 when the plan is made), graph-replayed like the main loop."""
+        if two_pass:
+            os.environ["CO3_TWO_PASS"] = "1"
+        try:
+            plan_o = binding.Plan(d, U, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
+                                  bias_mode={"lagged": binding.BIAS_LAGGED, "current": binding.BIAS_CURRENT}[other],
+                                  ld=wl.ld)
+        finally:
+            os.environ.pop("CO3_TWO_PASS", None)
         res_o = torch.zeros_like(residual)
         for t in range(args.warmup):
             plan_o.encode(pool[t % POOL], res_o, out)
@@ -283,12 +294,21 @@ def run_ours(args):
         barrier()
         o_ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
         assert plan_o.status(clear=True)[0] == 0
-        other_rec = {"bias_mode": other, "ms_per_step": o_ms / args.steps,
-                     "value": job_throughput_gbs(world, 4.0 * d * U, args.steps, o_ms), "unit": UNIT,
-                     "launch": "replayed from one-step CUDA graphs" if gr_o else "launched eagerly"}
+        rec = {"bias_mode": other, "ms_per_step": o_ms / args.steps,
+               "value": job_throughput_gbs(world, 4.0 * d * U, args.steps, o_ms), "unit": UNIT,
+               "launch": "replayed from one-step CUDA graphs" if gr_o else "launched eagerly"}
+        if two_pass:
+            rec["note"] = ("a statistics pass in every iteration (Algorithm 1 line 8 in its printed order); the same "
+                           "bits as `value`, whose iterations convert under the previous bias and convert again "
+                           "only the layers whose bias changed")
         del gr_o
         plan_o.close()
         del res_o
+        return rec
+
+    if other is not None:
+        other_rec = timed_other(other, False)
+        two_pass_rec = timed_other("current", True)
 
     # ---- the same steps replayed from a CUDA graph (one graph = one pass over the gradient pool) --
     # All steps from one graph, no eager step in between: what the loop costs without any launch gap.
@@ -339,8 +359,9 @@ def run_ours(args):
     conv_bytes = CONVERT_BYTES_PER_ELEMENT if args.mode != "code-lagged" else 12.0 + code_bits / 8.0
     achieved = conv_bytes * U * d / (conv_avg_ms * 1e-3) / 1e9
     # all passes of one iteration, E4M3: 13 + 1.9 (encode) + 0.87 (decode) per user-element + the average
-    # (the statistics pass of the current-moments bias reads g and m once more: + 8)
-    per_ue = {"lagged": 15.9, "current": 23.9, "code-lagged": 12.0 + 4.0 * code_bits / 8.0}[args.mode]
+    # (the current-moments bias pays a statistics pass at t = 0 only: later iterations run the lagged-bias
+    # passes and convert again the layers whose bias changed -- on this workload five of 64-128 elements)
+    per_ue = {"lagged": 15.9, "current": 15.9, "code-lagged": 12.0 + 4.0 * code_bits / 8.0}[args.mode]
     step_bytes = (per_ue * U + 4.0) * d
 
     result = {
@@ -349,7 +370,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": "configs[1]: %d users x ResNet-18 (10-class head) gradient, d=11173962, "
                                "62 layers, iid GenNorm(beta=0.8) per layer, E4M3, gamma=0.9, %s" % (
-                                   U, {"lagged": "lagged bias", "current": "bias from the current moments",
+                                   U, {"lagged": "lagged bias", "current": "bias from the current moments (Algorithm 1 as printed)",
                                        "code-lagged": "lagged bias and code (single-pass encode)"}[args.mode]),
                    "d": d, "n_users": U, "n_segments": plan.S, "format": "E4M3", "gamma": wl.gamma,
                    "bias_mode": args.mode, "replicas": world, "row_stride": plan.ld,
@@ -391,6 +412,8 @@ def run_ours(args):
     }
     if other_rec is not None:
         result["lagged_bias" if other == "lagged" else "current_bias"] = other_rec
+    if two_pass_rec is not None:
+        result["current_two_pass"] = two_pass_rec
     if graph_ms is not None:
         result["graph_replay"] = {"ms_per_step": graph_ms, "value": job_throughput_gbs(1, in_bytes, 1, graph_ms),
                                   "unit": UNIT, "note": "the same steps replayed from one captured CUDA graph"}

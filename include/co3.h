@@ -57,13 +57,23 @@ extern "C" {
 #define CO3_FLAG_CORRUPT 2u
 #define CO3_FLAG_NONFINITE 4u
 #define CO3_FLAG_TIMEOUT 8u  /* a bounded wait between thread blocks ran out (should never happen) */
-#define CO3_FLAG_INEXACT 16u /* CO3_BIAS_CURRENT only: more than 4096 elements of one iteration lay some 2^20 times
-                                beyond the largest value of their layer's format AND that layer's bias changed: those
-                                elements were converted at the previous iteration's bias (see co3_encode) */
+#define CO3_FLAG_INEXACT 16u /* CO3_BIAS_CURRENT only: in one iteration more than 4096 elements lay at least 2^(23-M)
+                                times beyond the largest value that the PREVIOUS iteration's bias of their layer could
+                                represent, and a layer's bias changed: some of them were converted at the previous
+                                bias (see the note on CO3_BIAS_CURRENT) */
 
 /* CO3_BIAS_CURRENT is Algorithm 1 as printed: the bias b_t is chosen "at each time t" for the
- * distribution of g_t + gamma m_{t-1} itself (Sec. III (i), Eq. "exp bias"), which costs one extra
- * read pass over gradient and memory per iteration.
+ * distribution of g_t + gamma m_{t-1} itself (Sec. III (i), Eq. "exp bias").  Taken literally that is an
+ * extra read pass over gradient and memory in front of every conversion.  co3_encode runs that pass at
+ * t = 0 only.  For t >= 1 it converts under the bias of iteration t-1, takes the moments of
+ * g_t + gamma m_{t-1} from that same pass (the same sums in the same order), derives b_t from them, and
+ * converts again -- from the stored symbol and memory, g + gamma m = q + m' exactly -- only the layers
+ * whose b_t differs from the bias they were converted with.  Symbols, memory, histogram, header and
+ * payload are bit for bit those of the two-pass order (the environment variable CO3_TWO_PASS=1, read
+ * when a plan is made, keeps the statistics pass in every iteration; a test compares the two).  An
+ * element so far beyond the format's range under the previous bias that q + m' would not give it back
+ * is kept on a side list of 4096 entries and converted from there; should an iteration have more of
+ * them, CO3_FLAG_INEXACT is raised.  The co3_tiled_* calls keep the two-pass order.
  * CO3_BIAS_LAGGED is NOT Algorithm 1's per-iteration bias: that pass runs at t = 0 only, and b_t for
  * t >= 1 is the rule applied to the fit of iteration t-1 (whose moments ride along with its conversion
  * pass); the code of iteration t is still designed from iteration t's own fit.  It relies on the fitted
@@ -135,8 +145,8 @@ typedef struct {
  * starts at 0 (memory m_0 = 0 is the caller's zero-filled `residual`).
  * Every call that takes a stream only enqueues work on it (kernels, memsets, device-to-device copies)
  * and never waits for the device, so a steady-state iteration (t >= 1 with CO3_BIAS_LAGGED or
- * CO3_CODE_LAGGED, any t with CO3_BIAS_CURRENT; tracing off) may be recorded by stream capture and
- * replayed as a CUDA graph: the kernel sequence does not depend on t.  Iteration 0 of the lagged modes
+ * CO3_CODE_LAGGED or CO3_BIAS_CURRENT; tracing off) may be recorded by stream capture and
+ * replayed as a CUDA graph: the kernel sequence does not depend on t.  Iteration 0
  * runs an extra statistics pass and must be run, not replayed, first.  (The iteration counter that
  * co3_state_export reports counts calls, not replays of a graph that recorded one.) */
 int co3_plan_create(co3_plan** out, const co3_config* cfg);

@@ -916,13 +916,15 @@ def test_config1_full_two_iterations(binding, oracle):
 
 
 @pytest.mark.slow
-@pytest.mark.parametrize("mode,rule", [(2, 0), (3, 0), (1, 1)])
+@pytest.mark.parametrize("mode,rule", [(0, 0), (2, 0), (3, 0), (1, 1)])
 def test_config1_full_other_modes_two_iterations(binding, oracle, mode, rule):
-    """Configuration 1 at full size in the fully lagged-code mode, the empirical-histogram mode and
-    with the L2-optimal bias rule (two iterations each: the second one runs on carried state)."""
+    """Configuration 1 at full size with the bias from the current moments (three iterations: the second
+    and third convert under the previous bias and repair the layers whose bias changed), in the fully
+    lagged-code mode, the empirical-histogram mode and with the L2-optimal bias rule (two iterations
+    each: the second one runs on carried state)."""
     from paper_2203_09044_b200 import inputs
     wl = inputs.workload(1).align_rows()
-    run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 2), gamma=wl.gamma,
+    run_case(binding, oracle, wl.d, wl.n_users, 4, 3, wl.seg_offsets, _grads(wl, 3 if mode == 0 else 2), gamma=wl.gamma,
              mode=mode, rule=rule)
 
 
