@@ -726,15 +726,19 @@ def test_iteration_in_tiles_of_users(binding, oracle, mode, tile):
     assert L.co3_tiled_finish(fresh.handle, *ptrs, None) == binding.EINVAL
 
 
-def test_steady_state_iteration_replays_from_a_cuda_graph(binding, oracle):
+@pytest.mark.parametrize("mode", [1, 0])
+def test_steady_state_iteration_replays_from_a_cuda_graph(binding, oracle, mode):
     """After the first iteration (which has the extra statistics pass) an iteration is a fixed
     sequence of memsets and kernels on one stream with no host decision in it, so it can be captured
     once in a CUDA graph and replayed: the replays, fed through the captured input buffer, must be
-    the oracle's iterations bit for bit (state carried in device memory: residual, bias, tickets)."""
+    the oracle's iterations bit for bit (state carried in device memory: residual, bias, tickets).
+    With the bias from the current moments (mode 0) the layers whose bias changed are found and
+    converted again on the device; the gradients' scale moves between the replays so that some are."""
     from paper_2203_09044_b200 import inputs
     wl = inputs.workload(1, d=120_000, n_users=3)
-    plan = binding.Plan(wl.d, 3, 4, 3, wl.seg_offsets)
-    orc = oracle.OracleCO3(wl.d, 3, 4, 3, wl.seg_offsets, cap_words=plan.cap_words)
+    plan = binding.Plan(wl.d, 3, 4, 3, wl.seg_offsets, bias_mode=mode)
+    orc = oracle.OracleCO3(wl.d, 3, 4, 3, wl.seg_offsets, cap_words=plan.cap_words, mode=mode)
+    scale = (1.0, 1.0, 6.0, 0.5)
     out = plan.alloc_outputs()
     m = torch.zeros((3, plan.ld), device="cuda")
     m_cpu = np.zeros((3, plan.ld), np.float32)
@@ -748,10 +752,10 @@ def test_steady_state_iteration_replays_from_a_cuda_graph(binding, oracle):
         plan.encode(g_static, m, out)
         plan.decode_aggregate(out)
     for t in range(1, 4):
-        g_static.copy_(wl.gradient(t))
+        g_static.copy_(wl.gradient(t) * scale[t])
         graph.replay()
         torch.cuda.synchronize()
-        r = orc.encode(wl.gradient(t).numpy(), m_cpu)
+        r = orc.encode((wl.gradient(t) * scale[t]).numpy(), m_cpu)
         rc, avg_o, _ = orc.decode_aggregate(r.payload, r.sub_bits, r.chunk_off, r.hdr)
         assert rc == oracle.OK
         assert np.array_equal(b_hdr(binding, out), r.hdr), f"t={t} header"
