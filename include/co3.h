@@ -57,7 +57,7 @@ extern "C" {
 #define CO3_FLAG_CORRUPT 2u
 #define CO3_FLAG_NONFINITE 4u
 #define CO3_FLAG_TIMEOUT 8u  /* a bounded wait between thread blocks ran out (should never happen) */
-#define CO3_FLAG_INEXACT 16u /* CO3_BIAS_CURRENT only: in one iteration more than 4096 elements lay at least 2^(23-M)
+#define CO3_FLAG_INEXACT 16u /* CO3_BIAS_CURRENT only: in one iteration more than 65536 elements lay at least 2^(23-M)
                                 times beyond the largest value that the PREVIOUS iteration's bias of their layer could
                                 represent, and a layer's bias changed: some of them were converted at the previous
                                 bias (see the note on CO3_BIAS_CURRENT) */
@@ -72,7 +72,7 @@ extern "C" {
  * payload are bit for bit those of the two-pass order (the environment variable CO3_TWO_PASS=1, read
  * when a plan is made, keeps the statistics pass in every iteration; a test compares the two).  An
  * element so far beyond the format's range under the previous bias that q + m' would not give it back
- * is kept on a side list of 4096 entries and converted from there; should an iteration have more of
+ * is kept on a side list of 65536 entries and converted from there; should an iteration have more of
  * them, CO3_FLAG_INEXACT is raised.  The co3_tiled_* calls keep the two-pass order.
  * CO3_BIAS_LAGGED is NOT Algorithm 1's per-iteration bias: that pass runs at t = 0 only, and b_t for
  * t >= 1 is the rule applied to the fit of iteration t-1 (whose moments ride along with its conversion

@@ -263,7 +263,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     co3_seg_header h;
     h.bias = (int8_t)b_used; h.ibeta = (int8_t)(int)x; h.ir = (int16_t)(int)y;
     hdr[seg] = h;
-    if (mode == 6 && b_rule != p.bias_cur[seg]) {
+    // (a layer of zeros converts to the same symbols and memory under every bias: nothing to repair)
+    if (mode == 6 && b_rule != p.bias_cur[seg] && S1 > 0.0) {
         // a small layer is converted again by this very block (below); a large one by the pass that follows
         if ((long long)(p.seg_off[seg + 1] - p.seg_off[seg]) * p.U <= FIT_REDO_MAX) s_redo_old = p.bias_cur[seg];
         else {
@@ -272,7 +273,11 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
             p.redo_old[k] = p.bias_cur[seg];
         }
     }
-    p.bias_cur[seg] = b_rule;
+    // Bias from the current moments: bias_cur is the next conversion's GUESS (and, for a layer that is
+    // converted again, the bias to convert it to).  After a layer of zeros the rule's bias is the lowest one,
+    // under which the first non-zero gradient would saturate beyond recovery; the highest one turns
+    // everything into zeros with the element itself as memory, from which any bias can be reached.
+    p.bias_cur[seg] = ((mode == 5 || mode == 6) && !(S1 > 0.0)) ? p.b_hi : b_rule;
     if (mode == 2) return;
     double* f = p.fit + 5 * (size_t)seg;
     f[0] = beta; f[1] = alpha; f[2] = N; f[3] = S1; f[4] = S2;

@@ -79,7 +79,7 @@ struct Co3Side {
     uint32_t a_bits;
     uint32_t pad_;
 };
-constexpr int CO3_SIDE_CAP = 4096;
+constexpr int CO3_SIDE_CAP = 65536;
 
 // Everything the kernels need, passed by value.
 struct Co3Dev {

@@ -349,13 +349,27 @@ def test_current_bias_with_elements_far_beyond_the_format(binding, oracle):
         assert flags & binding.FLAG_NONFINITE and not (flags & binding.FLAG_INEXACT)
 
 
+def test_current_bias_after_layers_of_zeros_and_of_tiny_values(binding, oracle):
+    """A layer that is all zeros (its bias is the lowest one) and then is not, a layer whose scale jumps
+    by 10^27 (every element lies far beyond what the previous bias could hold: thousands of side-list
+    entries), and back; next to a steady layer."""
+    d, U = 30_000, 3
+    off = [0, 5000, 10_000, 20_000, d]
+    scales = [[0.0, 1e-30, 1e-3, 1e-3], [0.0, 1e-3, 1e-3, 0.0], [1e-3, 1e-30, 1e-3, 0.0], [0.0, 3e-2, 1e-3, 1e-4],
+              [2e-3, 1e-3, 1e-3, 0.0]]
+    for E, M in ((4, 3), (1, 2)):
+        grads = _scaled_grads(U, d, d, off, scales, seed=81)
+        plan, orc, out, res = run_case(binding, oracle, d, U, E, M, off, grads, gamma=0.5, mode=0)
+        assert plan.status()[0] == 0
+
+
 def test_current_bias_side_list_overflow_is_reported(binding):
     """More far-out elements in one iteration than the side list holds (in a layer whose bias they change):
     CO3_FLAG_INEXACT.  With fewer of them than the list holds nothing is raised."""
     b = binding
-    d, U = 60_000, 2
+    d, U = 120_000, 2
     off = [0, 30_000, d]
-    for moving, count in ((False, 1500), (True, 6000)):
+    for moving, count in ((False, 1500), (True, 80_000)):
         scales = [[1e-3, 1e-3] for t in range(3)]
         grads = _scaled_grads(U, d, d, off, scales, seed=80, far=(1, count, 3e9))
         plan = b.Plan(d, U, 4, 3, off, gamma=0.0, bias_mode=b.BIAS_CURRENT)
