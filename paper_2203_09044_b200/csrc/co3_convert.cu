@@ -30,6 +30,12 @@
 // the sub-chunk's place in a staging buffer (64 words per sub-chunk) together with the sub-chunk's
 // bit count.  No block barrier is involved.  Where a sub-chunk lands in the user's payload depends
 // on all earlier ones, so a scan and a concatenation pass follow (co3_encode.cu).
+//
+// Fourth variant (bias from the current iteration's own moments, t >= 1): the pass runs under the
+// previous iteration's bias and only makes sure that every element could be converted again from what it
+// stores; reconvert_kernel below does that for the layers whose bias comes out different.  The
+// statistics pass that the printed order of Algorithm 1 puts in front of the conversion (stats_kernel)
+// then runs at t = 0 only.
 #include "co3_internal.h"
 #include "co3_quant.cuh"
 
