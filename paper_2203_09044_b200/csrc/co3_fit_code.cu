@@ -123,6 +123,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     // independent; then lanes, then warps.  (Plans with very long segments: the pairs were summed in
     // red_k slices by fit_reduce_kernel, and the slices are added here.)
     const int nck = c1 - c0, npairs = nck * p.U;
+    if (mode == 6 && tid < 2 && nck > 0)              // should this block convert its layer again: descriptor and side-list count on their way
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(tid == 0 ? (const void*)(p.chunks + c0) : (const void*)(p.spec + 2)));
     double a1 = 0.0, a2 = 0.0;
     unsigned long long an = 0;
     if (p.red_k > 0) {
