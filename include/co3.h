@@ -73,7 +73,7 @@ extern "C" {
  * when a plan is made, keeps the statistics pass in every iteration; a test compares the two).  An
  * element so far beyond the format's range under the previous bias that q + m' would not give it back
  * is kept on a side list of 65536 entries and converted from there; should an iteration have more of
- * them, CO3_FLAG_INEXACT is raised.  The co3_tiled_* calls keep the two-pass order.
+ * them, CO3_FLAG_INEXACT is raised.  The co3_tiled_* calls do the same (co3_tiled_finish repairs).
  * CO3_BIAS_LAGGED is NOT Algorithm 1's per-iteration bias: that pass runs at t = 0 only, and b_t for
  * t >= 1 is the rule applied to the fit of iteration t-1 (whose moments ride along with its conversion
  * pass); the code of iteration t is still designed from iteration t's own fit.  It relies on the fitted
@@ -176,7 +176,7 @@ int co3_encode(co3_plan* plan, const float* grad, float* residual, uint32_t* bit
  * at once (residual, payload and side information still cover all users and stay resident; only the
  * gradient buffer holds a tile and is refilled by the caller between calls):
  *   co3_tiled_begin       starts the iteration; *need_statistics = 1 if the bias has to come from a
- *                         statistics pass first (t = 0, or CO3_BIAS_CURRENT)
+ *                         statistics pass first (t = 0; with CO3_BIAS_CURRENT and CO3_TWO_PASS=1 every t)
  *   co3_tiled_statistics  (only then) once for every tile: grad_tile is [n_tile_users][ld] for the
  *                         users user0 .. user0 + n_tile_users - 1, residual the full [U][ld] array
  *   co3_tiled_convert     once for every tile, after all statistics calls: as co3_encode's convert

@@ -513,13 +513,19 @@ extern "C" int co3_encode(co3_plan* pl, const float* grad, float* residual, uint
 }
 
 // ---- one iteration in tiles of users (gradients that do not fit the device at once) -------------
+// A statistics pass in front of the conversion: at t = 0, and in every iteration of the current-moments bias
+// in its two-pass form; else that bias converts under the previous one and repairs (see co3_encode).
+static bool tiled_needs_statistics(const co3_plan* pl) {
+    return pl->iteration == 0 || (pl->cfg.bias_mode == CO3_BIAS_CURRENT && pl->two_pass_current);
+}
+
 extern "C" int co3_tiled_begin(co3_plan* pl, int32_t* need_statistics) {
     if (!pl || !need_statistics) return CO3_EINVAL;
     if (pl->cfg.bias_mode != CO3_BIAS_CURRENT && pl->cfg.bias_mode != CO3_BIAS_LAGGED) return CO3_EINVAL;
     pl->tiled_state = 1;
     pl->tiled_users = 0;
     pl->use_ext_mom = false;
-    *need_statistics = (pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT) ? 1 : 0;
+    *need_statistics = tiled_needs_statistics(pl) ? 1 : 0;
     return CO3_OK;
 }
 
@@ -544,13 +550,15 @@ extern "C" int co3_tiled_convert(co3_plan* pl, const float* grad_tile, float* re
                                  int32_t n_tile_users, void* cuda_stream) {
     if (!tile_args_ok(pl, grad_tile, residual, user0, n_tile_users)) return CO3_EINVAL;
     if (pl->tiled_state < 1) return CO3_EINVAL;
-    const bool need_stats = pl->iteration == 0 || pl->cfg.bias_mode == CO3_BIAS_CURRENT;
+    const bool need_stats = tiled_needs_statistics(pl);
+    const bool guess = pl->cfg.bias_mode == CO3_BIAS_CURRENT && !need_stats;
     if (pl->tiled_state == 1 && need_stats) return CO3_EINVAL;                 // the statistics tiles come first
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
     const bool first = pl->tiled_state != 3;
     if (first && need_stats) CO3_TRY(co3_launch_fit(pl, 0, nullptr, st));       // bias from the pooled statistics
-    CO3_TRY(co3_launch_convert(pl, grad_tile, residual, user0, n_tile_users, first, st));
+    CO3_TRY(co3_launch_convert(pl, grad_tile, residual, user0, n_tile_users, first, st, false, guess));
+    pl->tiled_residual = residual;
     pl->tiled_state = 3;
     pl->tiled_users += n_tile_users;
     return CO3_OK;
@@ -563,7 +571,12 @@ extern "C" int co3_tiled_finish(co3_plan* pl, uint32_t* bitstream, uint16_t* sub
     if (pl->tiled_state != 3 || pl->tiled_users != pl->dev.U) return CO3_EINVAL;   // every user exactly once
     cudaStream_t st = as_stream(cuda_stream);
     pl->last_stream = st;
-    CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
+    if (pl->cfg.bias_mode == CO3_BIAS_CURRENT && !tiled_needs_statistics(pl)) {
+        CO3_TRY(co3_launch_fit(pl, 6, hdr, st, false, pl->tiled_residual));     // the tiles were converted under the previous bias
+        CO3_TRY(co3_launch_reconvert(pl, pl->tiled_residual, st));
+    } else {
+        CO3_TRY(co3_launch_fit(pl, 1, hdr, st));
+    }
     CO3_TRY(co3_launch_encode(pl, hdr, bitstream, sub_bits, chunk_off, (unsigned long long*)user_bits, st));
     pl->iteration++;
     pl->tiled_state = 0;

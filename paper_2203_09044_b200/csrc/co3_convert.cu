@@ -267,7 +267,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
                 float a[4], mo[4];
                 uint32_t so[4], en[4] = {0u, 0u, 0u, 0u};
                 if (full) {
-                    if (GUESS) ef_add4<true>(gv, mv, p.gamma, a, s1, s2, nf, q.far_bits, p.spec, p.side, item, (uint32_t)e0, 15u);
+                    if (GUESS) ef_add4<true>(gv, mv, p.gamma, a, s1, s2, nf, q.far_bits, p.spec, p.side, item_base + item, (uint32_t)e0, 15u);
                     else ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -286,7 +286,7 @@ ef_kernel(Co3Dev p, const float* __restrict__ g, float* __restrict__ m, uint16_t
                     if (!in1) { gv.y = 0.0f; mv.y = 0.0f; }
                     if (!in2) { gv.z = 0.0f; mv.z = 0.0f; }
                     if (!in3) { gv.w = 0.0f; mv.w = 0.0f; }
-                    if (GUESS) ef_add4<true>(gv, mv, p.gamma, a, s1, s2, nf, q.far_bits, p.spec, p.side, item, (uint32_t)e0,
+                    if (GUESS) ef_add4<true>(gv, mv, p.gamma, a, s1, s2, nf, q.far_bits, p.spec, p.side, item_base + item, (uint32_t)e0,
                                              (uint32_t)in0 | ((uint32_t)in1 << 1) | ((uint32_t)in2 << 2) | ((uint32_t)in3 << 3));
                     else ef_add4(gv, mv, p.gamma, a, s1, s2, nf);
 #pragma unroll

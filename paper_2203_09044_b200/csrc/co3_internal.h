@@ -158,6 +158,7 @@ struct co3_plan {
     bool ev_conv_recorded;          // a convert pass that read d_grad has been recorded
     int tiled_state;                // co3_tiled_*: 0 idle, 1 begun, 2 statistics tiles seen, 3 convert tiles seen
     int tiled_users;                // users converted so far in this tiled iteration
+    float* tiled_residual;          // the residual array of its convert calls (the re-conversion in co3_tiled_finish needs it)
     double* ext_mom;                // [S][3] moments handed in by co3_moments_import
     bool use_ext_mom;               // ... and not yet consumed by a fit
     double* mom_out;                // co3_moments_export: where the reduction-only fit launch writes

@@ -4,8 +4,9 @@ Every rank holds its slice of every user's gradient and memory.  Conversion, cod
 averaging are local to a slice; the only exchange is the three moment sums per layer (entries,
 sum |a|, sum a^2 of a = g + gamma m, Sec. III (i)): a layer that spans several slices must be
 fitted to the sums over ALL its entries, so that every rank derives the same exponent bias and the
-same header for it.  That is one all-reduce of n_segments x 3 doubles after the statistics pass
-(t = 0, or when the bias comes from the current iteration) and one after the convert pass.
+same header for it.  That is one all-reduce of n_segments x 3 doubles after the convert pass, and at
+t = 0 one more after the statistics pass (with the bias from the current iteration's moments the later
+iterations convert under the previous bias and repair the layers whose bias changed after the fit).
 
 Slices are cut at multiples of 4096 elements, so the chunks of the slices together are exactly the
 chunks of the unsliced gradient: a user's payload is the slices' payloads one after the other, and
