@@ -103,6 +103,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     __shared__ double s_lg[3];
     __shared__ double s_target, s_t;        // log rho; log2(beta)
     __shared__ int s_state, s_coarse, s_fine;
+    __shared__ double s_ct[FIT_SEARCH + 1];  // log R at every 64th grid point (the coarse level of the search)
+    __shared__ double s_fx[68], s_fg[68];   // log R and log G around the bracket: grid points i0 - 1 .. i0 + 66
     __shared__ int s_redo_old;              // mode 6: the guess this layer was converted with, if this block converts it again
     __shared__ uint32_t s_rh[2][CO3_MAXSYM];
 
@@ -123,6 +125,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
     // independent; then lanes, then warps.  (Plans with very long segments: the pairs were summed in
     // red_k slices by fit_reduce_kernel, and the slices are added here.)
     const int nck = c1 - c0, npairs = nck * p.U;
+    // the coarse level of the search table: on its way while the partial sums are added up
+    if (tid <= FIT_SEARCH && mode != 4) s_ct[tid] = p.logr_tab[tid * (CO3_FIT_GRID / FIT_SEARCH)];
     if (mode == 6 && tid < 2 && nck > 0)              // should this block convert its layer again: descriptor and side-list count on their way
         asm volatile("prefetch.global.L2 [%0];" ::"l"(tid == 0 ? (const void*)(p.chunks + c0) : (const void*)(p.spec + 2)));
     double a1 = 0.0, a2 = 0.0;
@@ -176,8 +180,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         else if (!(N > 0.0) || !(S1 > 0.0)) { s_state = 2; s_t = 0.0; }     // beta = 1, alpha = 0
         else {
             s_target = s_lg[0] + s_lg[1] - 2.0 * s_lg[2];
-            if (s_target >= tab[0]) { s_state = 1; s_t = T0; s_fine = 0; }
-            else if (s_target <= tab[CO3_FIT_GRID]) { s_state = 1; s_t = 1.0; s_fine = CO3_FIT_GRID; }
+            if (s_target >= s_ct[0]) { s_state = 1; s_t = T0; s_fine = 0; }
+            else if (s_target <= s_ct[FIT_SEARCH]) { s_state = 1; s_t = 1.0; s_fine = CO3_FIT_GRID; }
         }
     }
     __syncthreads();
@@ -185,12 +189,17 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         // interval i with tab[i] > target >= tab[i+1]: coarse then fine, 64 entries each
         constexpr int STEP = CO3_FIT_GRID / FIT_SEARCH;        // 64
         const double target = s_target;
-        if (tid < FIT_SEARCH && tab[tid * STEP] > target && target >= tab[(tid + 1) * STEP]) s_coarse = tid;
+        if (tid < FIT_SEARCH && s_ct[tid] > target && target >= s_ct[tid + 1]) s_coarse = tid;
         __syncthreads();
-        if (tid < STEP) {
-            const int i = s_coarse * STEP + tid;
-            if (tab[i] > target && target >= tab[i + 1]) s_fine = i;
+        // one round of loads brings the bracket's 64 intervals and the nodes of both interpolations
+        const int i0 = s_coarse * STEP;
+        if (tid < 68) {
+            const int gi = min(max(i0 - 1 + tid, 0), CO3_FIT_GRID);
+            s_fx[tid] = tab[gi];
+            s_fg[tid] = tabg[gi];
         }
+        __syncthreads();
+        if (tid < STEP && s_fx[tid + 1] > target && target >= s_fx[tid + 2]) s_fine = i0 + tid;
         __syncthreads();
     }
     constexpr int NO_REDO = -(1 << 30);
@@ -204,7 +213,8 @@ __global__ void __launch_bounds__(FIT_THREADS) fit_kernel(Co3Dev p, int mode, co
         i = i < 1 ? 1 : (i > CO3_FIT_GRID - 2 ? CO3_FIT_GRID - 2 : i);
         const double target = s_target;
         double xs[4], gs[4], acc = 0.0;
-        for (int k = 0; k < 4; ++k) { xs[k] = tab[i - 1 + k]; gs[k] = tabg[i - 1 + k]; }
+        const int o = i - (s_coarse * (CO3_FIT_GRID / FIT_SEARCH));      // 0 .. 63 within the bracket (clamped at the table's ends)
+        for (int k = 0; k < 4; ++k) { xs[k] = s_fx[o + k]; gs[k] = s_fg[o + k]; }
         for (int a = 0; a < 4; ++a) {
             double term = T0 + H * (double)(i - 1 + a);
             for (int c = 0; c < 4; ++c)
