@@ -726,3 +726,44 @@ def test_empirical_histogram_code_mode(oracle):
     big = np.array([3 << 33, 1 << 33, 5, 0], np.uint64)
     ln, f = oracle.huffman_counts(big)
     assert list(ln) == [1, 2, 3, 3] and f == 1
+
+
+def test_conversion_can_be_undone_from_symbol_and_memory(oracle):
+    """Algorithm 1 line 10 read backwards: m' = a - q is exact (the residual identity), so a = q + m' gives the
+    corrected gradient back bit for bit and it can be converted again under another bias, unless |a| lies
+    some 2^(23 - M) times beyond the largest grid value (there a - q is rounded).  The library's
+    single-pass form of the current-moments bias rests on this; here it is checked on the oracle's own
+    conversion, for every format, across the grid's whole range, with both signs of zero."""
+    rng = np.random.default_rng(12)
+    for E, M in ((1, 2), (3, 2), (4, 3)):
+        for b1, b2 in ((0, 3), (-7, -9), (5, -20), (-30, 10)):
+            top = oracle.Kmax(E, M) * 2.0 ** (b1 + oracle.cF(E, M))
+            n = 20_000
+            mag = np.exp2(rng.uniform(np.log2(top) - 40.0, np.log2(top) + 22.5 - M, n))
+            a = (mag * rng.choice([-1.0, 1.0], n)).astype(np.float32)
+            a[:8] = np.float32([0.0, -0.0, top, -top, top * 1.0000001, np.float32(top) * np.float32(2.0 ** (22 - M)),
+                                1e-45, -1e-45])
+            g = a.reshape(1, n).copy()
+            a = a + np.float32(0.0)                                        # a = g + gamma * 0 (which turns -0 into +0)
+            m1 = np.zeros((1, n), np.float32)
+            s1 = np.zeros((1, n), np.uint8)
+            hist = np.zeros(1 << (1 + E + M), np.uint64)
+            oracle.convert(g, m1, s1, 0, n, 1.0, E, M, b1, hist)           # a = g + 1 * 0: the first conversion, bias b1
+            q1 = np.float32([oracle.grid_value(E, M, b1, int(s)) for s in s1[0]])
+            back = np.where(q1 == 0.0, m1[0], (q1 + m1[0]).astype(np.float32))
+            assert np.array_equal(back.view(np.uint32), a.view(np.uint32))
+            # ... and converting what came back under b2 is converting a under b2
+            m2a, s2a = np.zeros((1, n), np.float32), np.zeros((1, n), np.uint8)
+            oracle.convert(back.reshape(1, n).copy(), m2a, s2a, 0, n, 1.0, E, M, b2, hist)
+            m2b, s2b = np.zeros((1, n), np.float32), np.zeros((1, n), np.uint8)
+            oracle.convert(g, m2b, s2b, 0, n, 1.0, E, M, b2, hist)
+            assert np.array_equal(s2a, s2b) and np.array_equal(m2a.view(np.uint32), m2b.view(np.uint32))
+        # just beyond the bound the residual is rounded, and some elements do not come back
+        top = np.float32(oracle.Kmax(E, M) * 2.0 ** oracle.cF(E, M))
+        n = 4000
+        far = (np.float64(top) * np.exp2(rng.uniform(23.0 - M, 25.0, n))).astype(np.float32)
+        g = far.reshape(1, n).copy()
+        m1, s1 = np.zeros((1, n), np.float32), np.zeros((1, n), np.uint8)
+        oracle.convert(g, m1, s1, 0, n, 1.0, E, M, 0, np.zeros(1 << (1 + E + M), np.uint64))
+        assert np.all(s1 == (1 << (E + M)) - 1)                            # all saturated at the top code
+        assert np.count_nonzero((top + m1[0]).astype(np.float32) != far) > n // 10
