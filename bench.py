@@ -585,7 +585,10 @@ def run_reference(args):
     users = max(1, min(full.n_users, n // 65536, 8))
     d_s = max(4096, min(full.d, n // users))
     wl = inputs.workload(1, d=None if d_s >= full.d else d_s, n_users=users)
-    orc = co3_oracle.OracleCO3(wl.d, users, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma)
+    # the bias mode of this arm's config (`--mode`, default: from the current moments, as `value` is measured)
+    orc = co3_oracle.OracleCO3(wl.d, users, wl.exp_bits, wl.mant_bits, wl.seg_offsets, gamma=wl.gamma,
+                               mode={"current": co3_oracle.MODE_CURRENT, "lagged": co3_oracle.MODE_LAGGED,
+                                     "code-lagged": co3_oracle.MODE_LAGGED_CODE}[args.mode])
     grads = [wl.gradient(t).numpy() for t in range(2)]
     m = np.zeros_like(grads[0])
     for t in range(args.warmup):
